@@ -1,0 +1,212 @@
+/*
+ * lisa.h -- C ABI of the LiSA shared-layer attention library for NVIDIA B200 (sm_100a).
+ *
+ * LiSA (arXiv 2408.01890, Sec. 5.1) replaces a layer's Q K^T by
+ *     A_n = Integrate( Align(A_{n-1}), A_Delta ),   A_Delta = Q' K'^T / sqrt(r)      (Eq. 3-4)
+ * where A_{n-1} are the previous layer's pre-softmax scores (already scaled by
+ * 1/sqrt(d_k), Eq. 2), Align is a tiny FFN over the head axis applied at every
+ * (query, key) position, and Q', K' are low-rank (r << d_k) projections.  The
+ * layer then applies the causal softmax and multiplies by its own V (Eq. 1).
+ *
+ * Conventions that hold for every entry point
+ *   - Returns a lisa_status_t.  Never throws, never aborts.  Unless an entry
+ *     point says otherwise it allocates and frees no device memory and does not
+ *     synchronise: it validates on the host, then enqueues kernels on the
+ *     caller's stream.  On any error nothing is launched and outputs are untouched.
+ *   - All data pointers are DEVICE pointers owned by the caller, 16-byte
+ *     aligned, and must stay valid until the enqueued work has finished.
+ *     Descriptor structs and the `links` array are HOST memory, read only
+ *     during the call.
+ *   - Activations are [B, N, H, x] with x (d or r) contiguous; strides are in
+ *     elements.  Scores handed between decode layers are fp32 [B, Hq, L_cap].
+ *   - Grouped-query attention: query head h reads key/value head h / (Hq/Hkv).
+ *   - Scratch memory comes from the caller: ask lisa_workspace_bytes() for the
+ *     size and pass a buffer of at least that size (may be NULL when 0).
+ *   - Supported ranges: d in {32, 64, 128}; 1 <= r <= 32; Hq <= 64, Hq % Hkv == 0;
+ *     m <= 256; chain_len <= 8.  Outside them: LISA_ERR_UNSUPPORTED.
+ */
+#ifndef LISA_H_
+#define LISA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void* lisa_stream_t; /* a cudaStream_t (NULL = the default stream) */
+
+typedef enum lisa_status_t {
+    LISA_OK = 0,
+    LISA_ERR_INVALID_ARG = 1, /* NULL where data is required, bad size/stride/alignment, wrong struct_size */
+    LISA_ERR_UNSUPPORTED = 2, /* well-formed but outside the supported ranges above */
+    LISA_ERR_WORKSPACE = 3,   /* workspace missing or smaller than lisa_workspace_bytes() */
+    LISA_ERR_CUDA = 4,        /* a CUDA call failed; the code is kept for lisa_last_cuda_error() */
+    LISA_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (reported by lisa_check) */
+} lisa_status_t;
+
+typedef enum lisa_dtype_t { LISA_F32 = 0, LISA_BF16 = 1 } lisa_dtype_t;
+typedef enum lisa_act_t { LISA_ACT_NONE = 0, LISA_ACT_RELU = 1, LISA_ACT_SILU = 2 } lisa_act_t;
+
+/* Eq. 4's Integrate.  ADD: A_n = FFN(A_{n-1}) + A_Delta.  CONCAT (Sec. 5.1, "An overview of LiSA"):
+ * A_n = FFN([A_{n-1}; A_Delta]) with the two halves stacked on the head axis in that order, so W1 has
+ * 2*Hq rows.  PLUS: no FFN, A_n = A_{n-1} + A_Delta (the variant for models pre-trained with sharing). */
+typedef enum lisa_integrate_t { LISA_INTEGRATE_ADD = 0, LISA_INTEGRATE_CONCAT = 1, LISA_INTEGRATE_PLUS = 2 } lisa_integrate_t;
+
+typedef enum lisa_cache_kind_t { LISA_CACHE_STANDARD = 0, LISA_CACHE_SHARED = 1 } lisa_cache_kind_t;
+typedef enum lisa_op_t { LISA_OP_ANCHOR = 0, LISA_OP_SHARED_PREFILL = 1, LISA_OP_SHARED_DECODE = 2 } lisa_op_t;
+
+/* A strided view of an activation tensor [B, N, H, x]; x contiguous. */
+typedef struct lisa_tensor {
+    void* ptr;        /* device */
+    int32_t dtype;    /* lisa_dtype_t */
+    int32_t reserved; /* 0 */
+    int64_t stride_b; /* elements */
+    int64_t stride_n;
+    int64_t stride_h;
+} lisa_tensor;
+
+/* One shared layer ("link") of a chain: the difference-compensation operands (Eq. 3) and the
+ * attention-heads alignment FFN (Sec. 5.1).  Weights are row-major, row = input unit:
+ *   w1 [h_in, m]   h_in = Hq (ADD) or 2*Hq (CONCAT);  b1 [m] or NULL
+ *   w2 [m, Hq], b2 [Hq] or NULL                       (ffn_layers == 2)
+ *   ffn_layers == 1: y = W1^T x + b1 with m == Hq, no activation, w2/b2 ignored (the LiSA_SL variant)
+ *   integrate == PLUS: all four ignored.
+ * For a two-layer FFN: y = W2^T act(W1^T x + b1) + b2. */
+typedef struct lisa_link {
+    lisa_tensor qp; /* Q' [B, N, Hq, r]   (decode: [B, 1, Hq, r], the new token's) */
+    lisa_tensor kp; /* K' [B, N, Hkv, r]  (decode: ignored, K' is read from the cache) */
+    const void* w1;
+    const void* b1;
+    const void* w2;
+    const void* b2;
+    int32_t w_dtype; /* lisa_dtype_t of w1,b1,w2,b2 */
+    int32_t r;
+    int32_t m;
+    int32_t act;        /* lisa_act_t */
+    int32_t integrate;  /* lisa_integrate_t */
+    int32_t ffn_layers; /* 1 or 2 */
+} lisa_link;
+
+/* The cache of one layer (Sec. 2.2 "KV cache"; Sec. 5.2: a shared layer stores K_LR instead of K).
+ *   STANDARD: k = K   [B][Hkv][L_cap][d]
+ *   SHARED:   k = K'^T [B][Hkv][r][L_cap]   (position contiguous, so r needs no padding)
+ *   both:     v = V   [B][Hkv][L_cap][d]
+ * L_cap must be a multiple of 8.  Memory is the caller's; lisa_kvcache_bytes() gives the sizes. */
+typedef struct lisa_kvcache_layer {
+    int32_t kind;  /* lisa_cache_kind_t */
+    int32_t dtype; /* lisa_dtype_t */
+    int32_t B;
+    int32_t Hkv;
+    int32_t L_cap;
+    int32_t d;
+    int32_t r; /* SHARED only */
+    int32_t reserved;
+    void* k;
+    void* v;
+} lisa_kvcache_layer;
+
+/* ------------------------------------------------------------------------------------------------
+ * lisa_attn_anchor -- standard causal attention (Eq. 1-2), the layer whose scores a chain starts from.
+ * Prefill (cache == NULL): q [B,Nq,Hq,d], k, v [B,Nq,Hkv,d]; o[b,i,h,:] = sum_{j<=i} softmax_j(q_i.k_j/sqrt(d)) v_j.
+ * Decode  (cache != NULL, Nq == 1): the new token's q against a STANDARD cache that already holds the
+ *   new token's K and V.  The context length of sequence b is seq_lens[b] (device int32 [B]) with
+ *   1 <= seq_lens[b] <= L, or L for every sequence when seq_lens is NULL; L <= L_cap.
+ *   If out_scores != NULL the pre-softmax row q.k_j/sqrt(d), j < length, is written there in fp32 for
+ *   the following shared layer (entries beyond the length are left untouched).
+ * o has q's shape.  Workspace: lisa_workspace_bytes(LISA_OP_ANCHOR, args, &n). */
+typedef struct lisa_anchor_args {
+    size_t struct_size; /* sizeof(lisa_anchor_args) */
+    int32_t B, Nq, Hq, Hkv, d;
+    int32_t L; /* decode: context length (upper bound of seq_lens when those are given) */
+    lisa_tensor q, k, v, o;
+    const lisa_kvcache_layer* cache;
+    const int32_t* seq_lens;
+    float* out_scores; /* decode only; [B, Hq, >= length] */
+    int64_t scores_stride_b, scores_stride_h;
+    void* workspace;
+    size_t workspace_bytes;
+} lisa_anchor_args;
+lisa_status_t lisa_attn_anchor(const lisa_anchor_args* args, lisa_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * lisa_attn_shared_prefill -- a shared layer at chain depth c = chain_len over a whole prompt
+ * (Sec. 5.1, Eq. 3-4, then Eq. 1).  The N x N x Hq scores are never stored: they are recomputed tile by
+ * tile from the anchor's q0 [B,N,Hq,d], k0 [B,N,Hkv,d] and links[0..c-1] (links[c-1] is this layer's own,
+ * the earlier ones belong to the shared layers between the anchor and this one), masked causally AFTER
+ * the last link, soft-maxed and multiplied by this layer's v [B,N,Hkv,d].  o [B,N,Hq,d].
+ * chain_len == 0 degenerates to lisa_attn_anchor on (q0,k0,v). */
+typedef struct lisa_shared_prefill_args {
+    size_t struct_size;
+    int32_t B, N, Hq, Hkv, d, chain_len;
+    lisa_tensor q0, k0, v, o;
+    const lisa_link* links; /* host array [chain_len] */
+    void* workspace;
+    size_t workspace_bytes;
+} lisa_shared_prefill_args;
+lisa_status_t lisa_attn_shared_prefill(const lisa_shared_prefill_args* args, lisa_stream_t stream);
+
+/* The same call with every tensor, weight and `o` in HOST memory (dense [B,N,H,x] layout, strides
+ * ignored; workspace fields ignored).  Inputs are staged into `device_arena` (device memory of at least
+ * lisa_host_arena_bytes(), 256-byte aligned), the layer runs, `o` is copied back and the stream is
+ * synchronised before returning.  Pinned host memory makes the copies faster but is not required. */
+lisa_status_t lisa_attn_shared_prefill_host(const lisa_shared_prefill_args* host_args, void* device_arena,
+                                            size_t arena_bytes, lisa_stream_t stream);
+lisa_status_t lisa_host_arena_bytes(const lisa_shared_prefill_args* host_args, size_t* bytes);
+
+/* ------------------------------------------------------------------------------------------------
+ * lisa_attn_shared_decode -- one decode step of a shared layer (Sec. 5.2, decoding stage).
+ * prev_scores: the previous layer's fp32 score row [B,Hq,>=length]; link.qp the new token's Q' [B,1,Hq,r];
+ * cache: a SHARED layer already holding the new token's K' and V; length = seq_lens[b] (<= L) or L.
+ * For each cached position j < length: A[:,j] = Integrate(Align(prev[:,j]), q'.K'_j/sqrt(r)); then softmax
+ * over j and the product with V.  o [B,1,Hq,d].  out_scores (fp32 [B,Hq,>=length], may be NULL, must not
+ * alias prev_scores) receives A for the next shared layer. */
+typedef struct lisa_shared_decode_args {
+    size_t struct_size;
+    int32_t B, Hq, L;
+    int32_t reserved;
+    const float* prev_scores;
+    int64_t prev_stride_b, prev_stride_h;
+    lisa_link link;
+    const lisa_kvcache_layer* cache;
+    const int32_t* seq_lens; /* device int32 [B] or NULL */
+    lisa_tensor o;
+    float* out_scores;
+    int64_t scores_stride_b, scores_stride_h;
+    void* workspace;
+    size_t workspace_bytes;
+} lisa_shared_decode_args;
+lisa_status_t lisa_attn_shared_decode(const lisa_shared_decode_args* args, lisa_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * lisa_kvcache_append -- write n_new new positions into a layer's cache (Sec. 2.2; Sec. 5.2: "store K_LR
+ * instead of K").  k_or_kp: [B,n_new,Hkv,d] for a STANDARD layer, [B,n_new,Hkv,r] (K') for a SHARED one,
+ * which is stored transposed.  v: [B,n_new,Hkv,d].  Row t of sequence b lands at position
+ * seq_lens_before[b] + t (device int32 [B]; NULL = position 0).  Positions that would fall at or beyond
+ * L_cap are dropped and counted: lisa_check() then reports LISA_ERR_INVALID_ARG. */
+lisa_status_t lisa_kvcache_append(const lisa_kvcache_layer* layer, const lisa_tensor* k_or_kp, const lisa_tensor* v,
+                                  const int32_t* seq_lens_before, int32_t n_new, lisa_stream_t stream);
+
+/* Host-only helpers (no device work). */
+
+/* Bytes of the k and v buffers of a cache layer (fields k, v ignored).  For one SHARED layer with 2-byte
+ * elements, k_bytes is smaller than a STANDARD layer's by B*Hkv*L_cap*(d-r)*2, the saving of Sec. 5.2. */
+lisa_status_t lisa_kvcache_bytes(const lisa_kvcache_layer* layer, size_t* k_bytes, size_t* v_bytes);
+
+/* Scratch bytes the given call needs; `args` is the call's argument struct (data pointers are not read). */
+lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes);
+
+/* Synchronises `stream` and reports device-side conditions recorded since the last call: a dropped cache
+ * append (LISA_ERR_INVALID_ARG) or a bounded wait that ran out (LISA_ERR_TIMEOUT); LISA_ERR_CUDA if the
+ * stream itself reports an error. */
+lisa_status_t lisa_check(lisa_stream_t stream);
+
+int lisa_last_cuda_error(void);             /* the cudaError_t of the last LISA_ERR_CUDA on this thread, else 0 */
+const char* lisa_status_string(int status); /* static string */
+int lisa_version(void);                     /* major*1000 + minor */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LISA_H_ */

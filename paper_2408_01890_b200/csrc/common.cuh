@@ -1,0 +1,69 @@
+// Shared device/host helpers of the LiSA CUDA library: tensor views, element loads, status word.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lisa.h"
+
+namespace lisa {
+
+constexpr int kMaxHeads = 64;
+constexpr int kMaxHidden = 256;
+constexpr int kMaxChain = 8;
+constexpr int kMaxRank = 32;
+
+// Strided view of [B, N, H, x] passed by value to kernels.
+struct TView {
+    const void* ptr;
+    int64_t sb, sn, sh;
+    int32_t dtype;
+};
+
+inline TView make_view(const lisa_tensor& t) { return TView{t.ptr, t.stride_b, t.stride_n, t.stride_h, t.dtype}; }
+
+// Aligner FFN of one link, by value.
+struct LinkDev {
+    TView qp, kp;
+    const void *w1, *b1, *w2, *b2;
+    int32_t w_dtype, r, m, act, integrate, ffn_layers;
+};
+
+inline LinkDev make_link(const lisa_link& l) {
+    return LinkDev{make_view(l.qp), make_view(l.kp), l.w1, l.b1, l.w2, l.b2, l.w_dtype, l.r, l.m, l.act, l.integrate,
+                   l.ffn_layers};
+}
+
+__device__ __forceinline__ float ld_elem(const void* p, int64_t idx, int dtype) {
+    if (dtype == LISA_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[idx]);
+    return reinterpret_cast<const float*>(p)[idx];
+}
+
+__device__ __forceinline__ void st_elem(void* p, int64_t idx, int dtype, float v) {
+    if (dtype == LISA_BF16)
+        reinterpret_cast<__nv_bfloat16*>(p)[idx] = __float2bfloat16_rn(v);
+    else
+        reinterpret_cast<float*>(p)[idx] = v;
+}
+
+__device__ __forceinline__ float act_apply(float x, int act) {
+    if (act == LISA_ACT_RELU) return fmaxf(x, 0.f);
+    if (act == LISA_ACT_SILU) return x / (1.f + __expf(-x));
+    return x;
+}
+
+// Device status words (this device's copy): [0] cache appends dropped, [1] bounded waits that ran out.
+// Host function; returns the device address to hand to kernels, or nullptr if the lookup failed.
+int* status_words();
+
+// Host-side launchers implemented in the .cu files. Each returns the cudaError_t of its launches.
+cudaError_t launch_generic_prefill(const lisa_shared_prefill_args& a, cudaStream_t s);
+
+cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cudaStream_t s);
+cudaError_t launch_anchor_decode(const lisa_anchor_args& a, void* ws, cudaStream_t s);
+size_t decode_workspace(int B, int Hq, int d, int L);
+
+cudaError_t launch_kvcache_append(const lisa_kvcache_layer& c, const lisa_tensor& k, const lisa_tensor& v,
+                                  const int32_t* lens_before, int n_new, cudaStream_t s);
+
+}  // namespace lisa
