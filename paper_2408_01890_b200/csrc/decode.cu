@@ -1,0 +1,481 @@
+// Decode step of a shared layer (Sec. 5.2, decoding stage) and of a standard layer (Eq. 1-2, last row).
+//
+// Both are streaming scans over a cache, bound by HBM bandwidth.  Work is split over (sequence b,
+// chunk of 128 cached positions); a CTA handles ALL heads of its chunk because the aligner mixes heads:
+//   phase A  scores of the chunk for every head
+//            shared:   A[:,j] = W2^T act(W1^T prev[:,j] + b1) + b2 + q'.K'_j/sqrt(r)     (Eq. 3-4)
+//            standard: A[h,j] = q_h.K_j/sqrt(d)                                           (Eq. 2)
+//            and, if asked, the fp32 row handed to the next shared layer
+//   phase B  chunk-local softmax statistics (max, sum) per head and the partial product with V
+// A second kernel merges the per-chunk partials (m, l, o) into the output (split-K softmax).
+// K' is cached transposed ([r][L_cap], position contiguous) so that r = 21 needs no padding and every
+// load is a full 16-byte vector along the position axis; V rows are 256 contiguous bytes.
+#include "common.cuh"
+
+namespace lisa {
+namespace {
+
+constexpr int kChunk = 128;
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+
+struct DecodeParams {
+    int B, Hq, Hkv, d, L_cap, L_uniform, n_chunks;
+    const int32_t* seq_lens;
+    // shared layer
+    const float* prev;
+    int64_t prev_sb, prev_sh;
+    TView qp;
+    const void* kpT;
+    int r, m, act, integrate, ffn_layers, w_dtype;
+    const void *w1, *b1, *w2, *b2;
+    // standard layer
+    TView q;
+    const void* kcache;
+    // common
+    const void* vcache;
+    int cache_dtype;
+    float* out_scores;
+    int64_t sc_sb, sc_sh;
+    float *ws_m, *ws_l, *ws_o;
+    TView o;
+};
+
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+    f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+    f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+
+__device__ __forceinline__ float ldw(const void* p, int idx, int dtype) { return p ? ld_elem(p, idx, dtype) : 0.f; }
+
+// ---------------------------------------------------------------------------------------------
+// Phase B: s_s[h][kChunk] holds the chunk's scores (-inf beyond the sequence end). Produces the
+// chunk's (max, sum, unnormalised P.V) per head into the workspace.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void softmax_pv_chunk(const DecodeParams& p, float* s_s, int b, int chunk, int nrows) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int Hq = p.Hq, d = p.d, G = p.Hq / p.Hkv;
+    const size_t part = ((size_t)b * p.n_chunks + chunk) * Hq;
+    for (int h = warp; h < Hq; h += kWarps) {
+        float v[kChunk / 32];
+        float cmax = -INFINITY;
+#pragma unroll
+        for (int t = 0; t < kChunk / 32; ++t) {
+            v[t] = s_s[h * kChunk + lane + 32 * t];
+            cmax = fmaxf(cmax, v[t]);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, off));
+        float sum = 0.f;
+#pragma unroll
+        for (int t = 0; t < kChunk / 32; ++t) {
+            const float e = __expf(v[t] - cmax);
+            s_s[h * kChunk + lane + 32 * t] = e;
+            sum += e;
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        if (lane == 0) {
+            p.ws_m[part + h] = cmax;
+            p.ws_l[part + h] = sum;
+        }
+    }
+    __syncthreads();
+    const int j0 = chunk * kChunk;
+    if (p.cache_dtype == LISA_BF16) {
+        const int lpr = d / 8;          // lanes per V row (16 bytes each)
+        const int rstep = 32 / lpr;     // rows fetched by one warp-wide load
+        const int sub = lane % lpr, rsel = lane / lpr;
+        for (int h = warp; h < Hq; h += kWarps) {
+            const uint4* vbase = reinterpret_cast<const uint4*>(p.vcache) +
+                                 (((size_t)b * p.Hkv + h / G) * p.L_cap + j0) * lpr + sub;
+            const float* ps = s_s + h * kChunk;
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            int jj = rsel;
+            for (; jj + 7 * rstep < nrows; jj += 8 * rstep) {
+                uint4 raw[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) raw[u] = ld_stream16(vbase + (size_t)(jj + u * rstep) * lpr);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    float f[8];
+                    bf16x8_to_f32(raw[u], f);
+                    const float pj = ps[jj + u * rstep];
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) acc[t] = fmaf(pj, f[t], acc[t]);
+                }
+            }
+            for (; jj < nrows; jj += rstep) {
+                float f[8];
+                bf16x8_to_f32(ld_stream16(vbase + (size_t)jj * lpr), f);
+                const float pj = ps[jj];
+#pragma unroll
+                for (int t = 0; t < 8; ++t) acc[t] = fmaf(pj, f[t], acc[t]);
+            }
+            for (int off = lpr; off < 32; off <<= 1)
+#pragma unroll
+                for (int t = 0; t < 8; ++t) acc[t] += __shfl_xor_sync(0xffffffffu, acc[t], off);
+            if (rsel == 0) {
+                float4* dst = reinterpret_cast<float4*>(p.ws_o + (part + h) * d + sub * 8);
+                dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+            }
+        }
+    } else {
+        // fp32 cache: thread per output column
+        for (int e = tid; e < Hq * d; e += kThreads) {
+            const int h = e / d, x = e % d;
+            const float* vb = reinterpret_cast<const float*>(p.vcache) + (((size_t)b * p.Hkv + h / G) * p.L_cap + j0) * d + x;
+            float acc = 0.f;
+            for (int jj = 0; jj < nrows; ++jj) acc = fmaf(s_s[h * kChunk + jj], vb[(size_t)jj * d], acc);
+            p.ws_o[(part + h) * d + x] = acc;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Shared layer.  HQ_C/M_C > 0: compile-time sizes, aligner in registers (ADD, two layers, bf16 cache,
+// M_C % 8 == 0, HQ_C % 4 == 0).  HQ_C == 0: any supported mode and size, per-thread scratch arrays.
+// ---------------------------------------------------------------------------------------------
+template <int HQ_C, int M_C>
+__global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_kernel(const __grid_constant__ DecodeParams p) {
+    extern __shared__ __align__(16) float smem[];
+    const int b = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x;
+    const int L = p.seq_lens ? p.seq_lens[b] : p.L_uniform;
+    const int j0 = chunk * kChunk;
+    if (j0 >= L) return;
+    const int nrows = min(kChunk, L - j0);
+    const int Hq = HQ_C ? HQ_C : p.Hq;
+    const int m = M_C ? M_C : (p.integrate == LISA_INTEGRATE_PLUS ? 0 : p.m);
+    const int r = p.r, G = Hq / p.Hkv;
+    const int h_in = p.integrate == LISA_INTEGRATE_CONCAT ? 2 * Hq : Hq;
+
+    float* s_s = smem;                      // [Hq][kChunk]  delta, then scores, then exp
+    float* part_s = s_s + Hq * kChunk;      // [Hq][kChunk]  partial FFN output of the upper half
+    float* qp_s = part_s + Hq * kChunk;     // [Hq][kMaxRank]
+    float* w1_s = qp_s + Hq * kMaxRank;     // [h_in][m]
+    float* w2_s = w1_s + h_in * m;          // [m][Hq]
+    float* b1_s = w2_s + m * Hq;            // [m]
+    float* b2_s = b1_s + m;                 // [Hq]
+
+    for (int e = tid; e < Hq * r; e += kThreads) {
+        const int h = e / r, x = e % r;
+        qp_s[h * kMaxRank + x] = ld_elem(p.qp.ptr, b * p.qp.sb + h * p.qp.sh + x, p.qp.dtype);
+    }
+    if (p.integrate != LISA_INTEGRATE_PLUS) {
+        for (int e = tid; e < h_in * m; e += kThreads) w1_s[e] = ld_elem(p.w1, e, p.w_dtype);
+        for (int e = tid; e < m; e += kThreads) b1_s[e] = ldw(p.b1, e, p.w_dtype);
+        if (p.ffn_layers == 2) {
+            for (int e = tid; e < m * Hq; e += kThreads) w2_s[e] = ld_elem(p.w2, e, p.w_dtype);
+            for (int e = tid; e < Hq; e += kThreads) b2_s[e] = ldw(p.b2, e, p.w_dtype);
+        }
+    }
+    __syncthreads();
+
+    // A_Delta for the chunk (Eq. 3): unit = (head, 8 consecutive positions)
+    const float inv_sqrt_r = rsqrtf((float)r);
+    if (p.cache_dtype == LISA_BF16) {
+        for (int u = tid; u < Hq * (kChunk / 8); u += kThreads) {
+            const int h = u / (kChunk / 8), j8 = u % (kChunk / 8);
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            if (j0 + j8 * 8 < p.L_cap) {
+                const __nv_bfloat16* base = reinterpret_cast<const __nv_bfloat16*>(p.kpT) +
+                                            ((size_t)b * p.Hkv + h / G) * r * p.L_cap + j0 + j8 * 8;
+                for (int x = 0; x < r; ++x) {
+                    float f[8];
+                    bf16x8_to_f32(ld_stream16(base + (size_t)x * p.L_cap), f);
+                    const float qx = qp_s[h * kMaxRank + x];
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) acc[t] = fmaf(qx, f[t], acc[t]);
+                }
+            }
+            float4* dst = reinterpret_cast<float4*>(s_s + h * kChunk + j8 * 8);
+            dst[0] = make_float4(acc[0] * inv_sqrt_r, acc[1] * inv_sqrt_r, acc[2] * inv_sqrt_r, acc[3] * inv_sqrt_r);
+            dst[1] = make_float4(acc[4] * inv_sqrt_r, acc[5] * inv_sqrt_r, acc[6] * inv_sqrt_r, acc[7] * inv_sqrt_r);
+        }
+    } else {
+        for (int u = tid; u < Hq * kChunk; u += kThreads) {
+            const int h = u / kChunk, jj = u % kChunk;
+            float acc = 0.f;
+            if (jj < nrows) {
+                const float* base = reinterpret_cast<const float*>(p.kpT) + ((size_t)b * p.Hkv + h / G) * r * p.L_cap + j0 + jj;
+                for (int x = 0; x < r; ++x) acc = fmaf(qp_s[h * kMaxRank + x], base[(size_t)x * p.L_cap], acc);
+            }
+            s_s[u] = acc * inv_sqrt_r;
+        }
+    }
+    __syncthreads();
+
+    const int pos = tid & (kChunk - 1), half = tid / kChunk;
+    const bool valid = pos < nrows;
+    const float* prev = p.prev + b * p.prev_sb + j0 + pos;
+    float* outrow = p.out_scores ? p.out_scores + b * p.sc_sb + j0 + pos : nullptr;
+
+    if constexpr (HQ_C > 0) {
+        // ADD, two-layer FFN; the two halves of the CTA split the hidden units of each position
+        constexpr int MH = M_C / 2;
+        float a[HQ_C], y[HQ_C];
+#pragma unroll
+        for (int h = 0; h < HQ_C; ++h) {
+            a[h] = valid ? prev[h * p.prev_sh] : 0.f;
+            y[h] = 0.f;
+        }
+        const int u0 = half * MH;
+#pragma unroll 1
+        for (int ub = 0; ub < MH; ub += 4) {
+            float4 hacc = *reinterpret_cast<const float4*>(b1_s + u0 + ub);
+#pragma unroll
+            for (int h = 0; h < HQ_C; ++h) {
+                const float4 w = *reinterpret_cast<const float4*>(w1_s + h * M_C + u0 + ub);
+                hacc.x = fmaf(a[h], w.x, hacc.x); hacc.y = fmaf(a[h], w.y, hacc.y);
+                hacc.z = fmaf(a[h], w.z, hacc.z); hacc.w = fmaf(a[h], w.w, hacc.w);
+            }
+            const float hv[4] = {act_apply(hacc.x, p.act), act_apply(hacc.y, p.act), act_apply(hacc.z, p.act),
+                                 act_apply(hacc.w, p.act)};
+#pragma unroll
+            for (int uu = 0; uu < 4; ++uu) {
+                const float* wrow = w2_s + (u0 + ub + uu) * HQ_C;
+#pragma unroll
+                for (int g4 = 0; g4 < HQ_C / 4; ++g4) {
+                    const float4 w = *reinterpret_cast<const float4*>(wrow + g4 * 4);
+                    y[g4 * 4 + 0] = fmaf(hv[uu], w.x, y[g4 * 4 + 0]); y[g4 * 4 + 1] = fmaf(hv[uu], w.y, y[g4 * 4 + 1]);
+                    y[g4 * 4 + 2] = fmaf(hv[uu], w.z, y[g4 * 4 + 2]); y[g4 * 4 + 3] = fmaf(hv[uu], w.w, y[g4 * 4 + 3]);
+                }
+            }
+        }
+        if (half == 1) {
+#pragma unroll
+            for (int g = 0; g < HQ_C; ++g) part_s[g * kChunk + pos] = y[g];
+        }
+        __syncthreads();
+        if (half == 0) {
+#pragma unroll
+            for (int g = 0; g < HQ_C; ++g) {
+                const float sc = y[g] + part_s[g * kChunk + pos] + b2_s[g] + s_s[g * kChunk + pos];
+                s_s[g * kChunk + pos] = valid ? sc : -INFINITY;
+                if (valid && outrow) outrow[g * p.sc_sh] = sc;
+            }
+        }
+    } else {
+        if (half == 0) {
+            float a[kMaxHeads], dl[kMaxHeads], hid[kMaxHidden];
+            for (int h = 0; h < Hq; ++h) {
+                a[h] = valid ? prev[h * p.prev_sh] : 0.f;
+                dl[h] = s_s[h * kChunk + pos];
+            }
+            if (p.integrate == LISA_INTEGRATE_PLUS) {
+                for (int g = 0; g < Hq; ++g) a[g] += dl[g];
+            } else {
+                for (int u = 0; u < m; ++u) {
+                    float s = b1_s[u];
+                    for (int x = 0; x < Hq; ++x) s = fmaf(a[x], w1_s[x * m + u], s);
+                    if (p.integrate == LISA_INTEGRATE_CONCAT)
+                        for (int x = 0; x < Hq; ++x) s = fmaf(dl[x], w1_s[(Hq + x) * m + u], s);
+                    hid[u] = s;
+                }
+                if (p.ffn_layers == 1) {
+                    for (int g = 0; g < Hq; ++g) a[g] = hid[g];
+                } else {
+                    for (int u = 0; u < m; ++u) hid[u] = act_apply(hid[u], p.act);
+                    for (int g = 0; g < Hq; ++g) {
+                        float s = b2_s[g];
+                        for (int u = 0; u < m; ++u) s = fmaf(hid[u], w2_s[u * Hq + g], s);
+                        a[g] = s;
+                    }
+                }
+                if (p.integrate == LISA_INTEGRATE_ADD)
+                    for (int g = 0; g < Hq; ++g) a[g] += dl[g];
+            }
+            for (int g = 0; g < Hq; ++g) {
+                s_s[g * kChunk + pos] = valid ? a[g] : -INFINITY;
+                if (valid && outrow) outrow[g * p.sc_sh] = a[g];
+            }
+        }
+    }
+    __syncthreads();
+    softmax_pv_chunk(p, s_s, b, chunk, nrows);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Standard layer: scores from the K cache.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 2) anchor_decode_chunk_kernel(const __grid_constant__ DecodeParams p) {
+    extern __shared__ __align__(16) float smem[];
+    const int b = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int L = p.seq_lens ? p.seq_lens[b] : p.L_uniform;
+    const int j0 = chunk * kChunk;
+    if (j0 >= L) return;
+    const int nrows = min(kChunk, L - j0);
+    const int Hq = p.Hq, d = p.d, G = Hq / p.Hkv;
+    float* s_s = smem;               // [Hq][kChunk]
+    float* q_s = s_s + Hq * kChunk;  // [Hq][d]
+    for (int e = tid; e < Hq * d; e += kThreads) {
+        const int h = e / d, x = e % d;
+        q_s[e] = ld_elem(p.q.ptr, b * p.q.sb + h * p.q.sh + x, p.q.dtype);
+    }
+    __syncthreads();
+    const float inv_sqrt_d = rsqrtf((float)d);
+    if (p.cache_dtype == LISA_BF16) {
+        const int lpr = d / 8, rstep = 32 / lpr, sub = lane % lpr, rsel = lane / lpr;
+        for (int h = warp; h < Hq; h += kWarps) {
+            float qv[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) qv[t] = q_s[h * d + sub * 8 + t];
+            const uint4* kbase = reinterpret_cast<const uint4*>(p.kcache) +
+                                 (((size_t)b * p.Hkv + h / G) * p.L_cap + j0) * lpr + sub;
+            for (int jb = 0; jb < kChunk; jb += 4 * rstep) {
+                float dot[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int jj = jb + u * rstep + rsel;
+                    dot[u] = 0.f;
+                    if (jj < nrows) {
+                        float f[8];
+                        bf16x8_to_f32(ld_stream16(kbase + (size_t)jj * lpr), f);
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) dot[u] = fmaf(qv[t], f[t], dot[u]);
+                    }
+                }
+                for (int off = lpr >> 1; off > 0; off >>= 1)
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) dot[u] += __shfl_xor_sync(0xffffffffu, dot[u], off);
+                if (sub == 0) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int jj = jb + u * rstep + rsel;
+                        if (jj < kChunk) s_s[h * kChunk + jj] = jj < nrows ? dot[u] * inv_sqrt_d : -INFINITY;
+                    }
+                }
+            }
+        }
+    } else {
+        for (int u = tid; u < Hq * kChunk; u += kThreads) {
+            const int h = u / kChunk, jj = u % kChunk;
+            float acc = -INFINITY;
+            if (jj < nrows) {
+                const float* kr = reinterpret_cast<const float*>(p.kcache) + (((size_t)b * p.Hkv + h / G) * p.L_cap + j0 + jj) * d;
+                acc = 0.f;
+                for (int x = 0; x < d; ++x) acc = fmaf(q_s[h * d + x], kr[x], acc);
+                acc *= inv_sqrt_d;
+            }
+            s_s[u] = acc;
+        }
+    }
+    __syncthreads();
+    if (p.out_scores) {
+        for (int u = tid; u < Hq * kChunk; u += kThreads) {
+            const int h = u / kChunk, jj = u % kChunk;
+            if (jj < nrows) p.out_scores[b * p.sc_sb + h * p.sc_sh + j0 + jj] = s_s[u];
+        }
+    }
+    softmax_pv_chunk(p, s_s, b, chunk, nrows);
+}
+
+// Merge the per-chunk (m, l, o) partials of one (b, h): o = sum_c e^{m_c - M} o_c / sum_c e^{m_c - M} l_c.
+__global__ void decode_merge_kernel(const __grid_constant__ DecodeParams p) {
+    const int h = blockIdx.x, b = blockIdx.y, x = threadIdx.x;
+    const int L = p.seq_lens ? p.seq_lens[b] : p.L_uniform;
+    const int nc = (L + kChunk - 1) / kChunk;
+    const size_t base = (size_t)b * p.n_chunks * p.Hq + h;
+    float M = -INFINITY;
+    for (int c = 0; c < nc; ++c) M = fmaxf(M, p.ws_m[base + (size_t)c * p.Hq]);
+    float num = 0.f, den = 0.f;
+    for (int c = 0; c < nc; ++c) {
+        const float w = __expf(p.ws_m[base + (size_t)c * p.Hq] - M);
+        den = fmaf(w, p.ws_l[base + (size_t)c * p.Hq], den);
+        num = fmaf(w, p.ws_o[(base + (size_t)c * p.Hq) * p.d + x], num);
+    }
+    st_elem(const_cast<void*>(p.o.ptr), b * p.o.sb + h * p.o.sh + x, p.o.dtype, num / den);
+}
+
+void carve_workspace(DecodeParams& p, void* ws) {
+    const size_t n = (size_t)p.B * p.n_chunks * p.Hq;
+    const size_t npad = (n + 3) & ~(size_t)3;  // keeps the o partials 16-byte aligned
+    p.ws_m = reinterpret_cast<float*>(ws);
+    p.ws_l = p.ws_m + npad;
+    p.ws_o = p.ws_l + npad;
+}
+
+template <typename K>
+cudaError_t set_smem(K kernel, size_t smem) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+
+}  // namespace
+
+size_t decode_workspace(int B, int Hq, int d, int L) {
+    const size_t nc = (size_t)(L + kChunk - 1) / kChunk;
+    const size_t n = (size_t)B * nc * Hq;
+    const size_t npad = (n + 3) & ~(size_t)3;
+    size_t bytes = (2 * npad + n * d) * sizeof(float);
+    return (bytes + 255) & ~(size_t)255;
+}
+
+cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cudaStream_t s) {
+    const lisa_kvcache_layer& c = *a.cache;
+    DecodeParams p{};
+    p.B = a.B; p.Hq = a.Hq; p.Hkv = c.Hkv; p.d = c.d; p.L_cap = c.L_cap; p.L_uniform = a.L;
+    p.n_chunks = (a.L + kChunk - 1) / kChunk;
+    p.seq_lens = a.seq_lens;
+    p.prev = a.prev_scores; p.prev_sb = a.prev_stride_b; p.prev_sh = a.prev_stride_h;
+    p.qp = make_view(a.link.qp);
+    p.kpT = c.k; p.vcache = c.v; p.cache_dtype = c.dtype;
+    p.r = c.r; p.m = a.link.m; p.act = a.link.act; p.integrate = a.link.integrate; p.ffn_layers = a.link.ffn_layers;
+    p.w_dtype = a.link.w_dtype;
+    p.w1 = a.link.w1; p.b1 = a.link.b1; p.w2 = a.link.w2; p.b2 = a.link.b2;
+    p.out_scores = a.out_scores; p.sc_sb = a.scores_stride_b; p.sc_sh = a.scores_stride_h;
+    p.o = make_view(a.o);
+    carve_workspace(p, ws);
+    const int h_in = p.integrate == LISA_INTEGRATE_CONCAT ? 2 * p.Hq : p.Hq;
+    const int m = p.integrate == LISA_INTEGRATE_PLUS ? 0 : p.m;
+    const size_t smem = sizeof(float) * ((size_t)2 * p.Hq * kChunk + (size_t)p.Hq * kMaxRank + (size_t)h_in * m +
+                                         (size_t)m * p.Hq + m + p.Hq + 8);
+    dim3 grid(p.n_chunks, p.B);
+    const bool fast = p.integrate == LISA_INTEGRATE_ADD && p.ffn_layers == 2 && c.dtype == LISA_BF16;
+    cudaError_t e;
+    if (fast && p.Hq == 40 && p.m == 80) {
+        if ((e = set_smem(shared_decode_chunk_kernel<40, 80>, smem)) != cudaSuccess) return e;
+        shared_decode_chunk_kernel<40, 80><<<grid, kThreads, smem, s>>>(p);
+    } else if (fast && p.Hq == 32 && p.m == 64) {
+        if ((e = set_smem(shared_decode_chunk_kernel<32, 64>, smem)) != cudaSuccess) return e;
+        shared_decode_chunk_kernel<32, 64><<<grid, kThreads, smem, s>>>(p);
+    } else {
+        if ((e = set_smem(shared_decode_chunk_kernel<0, 0>, smem)) != cudaSuccess) return e;
+        shared_decode_chunk_kernel<0, 0><<<grid, kThreads, smem, s>>>(p);
+    }
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_anchor_decode(const lisa_anchor_args& a, void* ws, cudaStream_t s) {
+    const lisa_kvcache_layer& c = *a.cache;
+    DecodeParams p{};
+    p.B = a.B; p.Hq = a.Hq; p.Hkv = c.Hkv; p.d = c.d; p.L_cap = c.L_cap; p.L_uniform = a.L;
+    p.n_chunks = (a.L + kChunk - 1) / kChunk;
+    p.seq_lens = a.seq_lens;
+    p.q = make_view(a.q);
+    p.kcache = c.k; p.vcache = c.v; p.cache_dtype = c.dtype;
+    p.out_scores = a.out_scores; p.sc_sb = a.scores_stride_b; p.sc_sh = a.scores_stride_h;
+    p.o = make_view(a.o);
+    carve_workspace(p, ws);
+    const size_t smem = sizeof(float) * ((size_t)p.Hq * kChunk + (size_t)p.Hq * p.d);
+    cudaError_t e;
+    if ((e = set_smem(anchor_decode_chunk_kernel, smem)) != cudaSuccess) return e;
+    anchor_decode_chunk_kernel<<<dim3(p.n_chunks, p.B), kThreads, smem, s>>>(p);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace lisa
