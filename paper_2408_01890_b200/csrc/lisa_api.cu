@@ -1,0 +1,362 @@
+// C-ABI entry points: host-side validation and dispatch.  No arithmetic of the method lives here.
+#include <cstring>
+
+#include "common.cuh"
+
+namespace lisa {
+
+static __device__ int g_status[4];
+static thread_local int t_last_cuda_error = 0;
+
+int* status_words() {
+    static int* cached[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cached[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status) != cudaSuccess) return nullptr;
+        cached[dev] = reinterpret_cast<int*>(p);
+    }
+    return cached[dev];
+}
+
+namespace {
+
+lisa_status_t cuda_fail(cudaError_t e) {
+    t_last_cuda_error = (int)e;
+    return LISA_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool dtype_ok(int dt) { return dt == LISA_F32 || dt == LISA_BF16; }
+size_t esize(int dt) { return dt == LISA_BF16 ? 2 : 4; }
+
+lisa_status_t check_tensor(const lisa_tensor& t) {
+    if (!t.ptr || !dtype_ok(t.dtype) || !aligned16(t.ptr)) return LISA_ERR_INVALID_ARG;
+    return LISA_OK;
+}
+
+lisa_status_t check_dims(int B, int N, int Hq, int Hkv, int d) {
+    if (B < 1 || N < 1 || Hq < 1 || Hkv < 1 || d < 1) return LISA_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0) return LISA_ERR_INVALID_ARG;
+    if (Hq > kMaxHeads) return LISA_ERR_UNSUPPORTED;
+    if (d != 32 && d != 64 && d != 128) return LISA_ERR_UNSUPPORTED;
+    return LISA_OK;
+}
+
+lisa_status_t check_link(const lisa_link& l, int Hq, bool prefill) {
+    if (l.r < 1) return LISA_ERR_INVALID_ARG;
+    if (l.r > kMaxRank) return LISA_ERR_UNSUPPORTED;
+    if (l.integrate < LISA_INTEGRATE_ADD || l.integrate > LISA_INTEGRATE_PLUS) return LISA_ERR_INVALID_ARG;
+    lisa_status_t st = check_tensor(l.qp);
+    if (st != LISA_OK) return st;
+    if (prefill && (st = check_tensor(l.kp)) != LISA_OK) return st;
+    if (l.integrate == LISA_INTEGRATE_PLUS) return LISA_OK;
+    if (l.act < LISA_ACT_NONE || l.act > LISA_ACT_SILU) return LISA_ERR_INVALID_ARG;
+    if (l.ffn_layers != 1 && l.ffn_layers != 2) return LISA_ERR_INVALID_ARG;
+    if (!dtype_ok(l.w_dtype) || !l.w1 || l.m < 1) return LISA_ERR_INVALID_ARG;
+    if (l.m > kMaxHidden) return LISA_ERR_UNSUPPORTED;
+    if (l.ffn_layers == 2 && !l.w2) return LISA_ERR_INVALID_ARG;
+    if (l.ffn_layers == 1 && l.m != Hq) return LISA_ERR_INVALID_ARG;
+    return LISA_OK;
+}
+
+lisa_status_t check_cache(const lisa_kvcache_layer* c, int kind, bool need_ptrs) {
+    if (!c || c->kind != kind || !dtype_ok(c->dtype)) return LISA_ERR_INVALID_ARG;
+    if (c->B < 1 || c->Hkv < 1 || c->L_cap < 8 || c->L_cap % 8 != 0) return LISA_ERR_INVALID_ARG;
+    if (c->d != 32 && c->d != 64 && c->d != 128) return LISA_ERR_UNSUPPORTED;
+    if (kind == LISA_CACHE_SHARED) {
+        if (c->r < 1) return LISA_ERR_INVALID_ARG;
+        if (c->r > kMaxRank) return LISA_ERR_UNSUPPORTED;
+    }
+    if (need_ptrs && (!c->k || !c->v || !aligned16(c->k) || !aligned16(c->v))) return LISA_ERR_INVALID_ARG;
+    return LISA_OK;
+}
+
+lisa_status_t check_workspace(const void* ws, size_t have, size_t need) {
+    if (need == 0) return LISA_OK;
+    if (!ws || have < need || !aligned16(ws)) return LISA_ERR_WORKSPACE;
+    return LISA_OK;
+}
+
+lisa_status_t validate_prefill(const lisa_shared_prefill_args* a) {
+    if (!a || a->struct_size != sizeof(lisa_shared_prefill_args)) return LISA_ERR_INVALID_ARG;
+    lisa_status_t st = check_dims(a->B, a->N, a->Hq, a->Hkv, a->d);
+    if (st != LISA_OK) return st;
+    if (a->chain_len < 0) return LISA_ERR_INVALID_ARG;
+    if (a->chain_len > kMaxChain) return LISA_ERR_UNSUPPORTED;
+    if (a->chain_len > 0 && !a->links) return LISA_ERR_INVALID_ARG;
+    const lisa_tensor* ts[4] = {&a->q0, &a->k0, &a->v, &a->o};
+    for (const lisa_tensor* t : ts)
+        if ((st = check_tensor(*t)) != LISA_OK) return st;
+    for (int k = 0; k < a->chain_len; ++k)
+        if ((st = check_link(a->links[k], a->Hq, true)) != LISA_OK) return st;
+    return LISA_OK;
+}
+
+lisa_status_t validate_anchor_decode(const lisa_anchor_args* a) {
+    lisa_status_t st = check_cache(a->cache, LISA_CACHE_STANDARD, true);
+    if (st != LISA_OK) return st;
+    const lisa_kvcache_layer& c = *a->cache;
+    if (a->Nq != 1 || a->B > c.B || a->Hkv != c.Hkv || a->d != c.d) return LISA_ERR_INVALID_ARG;
+    if (a->L < 1 || a->L > c.L_cap) return LISA_ERR_INVALID_ARG;
+    if ((st = check_tensor(a->q)) != LISA_OK || (st = check_tensor(a->o)) != LISA_OK) return st;
+    return LISA_OK;
+}
+
+lisa_status_t validate_shared_decode(const lisa_shared_decode_args* a) {
+    if (!a || a->struct_size != sizeof(lisa_shared_decode_args)) return LISA_ERR_INVALID_ARG;
+    lisa_status_t st = check_cache(a->cache, LISA_CACHE_SHARED, true);
+    if (st != LISA_OK) return st;
+    const lisa_kvcache_layer& c = *a->cache;
+    if ((st = check_dims(a->B, 1, a->Hq, c.Hkv, c.d)) != LISA_OK) return st;
+    if (a->B > c.B || a->L < 1 || a->L > c.L_cap) return LISA_ERR_INVALID_ARG;
+    if (a->link.r != c.r) return LISA_ERR_INVALID_ARG;
+    if ((st = check_link(a->link, a->Hq, false)) != LISA_OK) return st;
+    if (!a->prev_scores || (reinterpret_cast<uintptr_t>(a->prev_scores) & 3u)) return LISA_ERR_INVALID_ARG;
+    if (a->out_scores && a->out_scores == a->prev_scores) return LISA_ERR_INVALID_ARG;
+    if ((st = check_tensor(a->o)) != LISA_OK) return st;
+    return LISA_OK;
+}
+
+}  // namespace
+}  // namespace lisa
+
+using namespace lisa;
+
+extern "C" {
+
+int lisa_version(void) { return 1000; }
+int lisa_last_cuda_error(void) { return t_last_cuda_error; }
+
+const char* lisa_status_string(int status) {
+    switch (status) {
+        case LISA_OK: return "ok";
+        case LISA_ERR_INVALID_ARG: return "invalid argument";
+        case LISA_ERR_UNSUPPORTED: return "unsupported shape or type";
+        case LISA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case LISA_ERR_CUDA: return "CUDA error";
+        case LISA_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+lisa_status_t lisa_kvcache_bytes(const lisa_kvcache_layer* layer, size_t* k_bytes, size_t* v_bytes) {
+    if (!layer || !k_bytes || !v_bytes) return LISA_ERR_INVALID_ARG;
+    lisa_status_t st = check_cache(layer, layer->kind, false);
+    if (st != LISA_OK) return st;
+    if (layer->kind != LISA_CACHE_STANDARD && layer->kind != LISA_CACHE_SHARED) return LISA_ERR_INVALID_ARG;
+    const size_t rows = (size_t)layer->B * layer->Hkv * layer->L_cap;
+    const size_t kw = layer->kind == LISA_CACHE_SHARED ? (size_t)layer->r : (size_t)layer->d;
+    *k_bytes = rows * kw * esize(layer->dtype);
+    *v_bytes = rows * (size_t)layer->d * esize(layer->dtype);
+    return LISA_OK;
+}
+
+lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes) {
+    if (!args || !bytes) return LISA_ERR_INVALID_ARG;
+    if (op == LISA_OP_ANCHOR) {
+        const lisa_anchor_args* a = static_cast<const lisa_anchor_args*>(args);
+        if (a->struct_size != sizeof(lisa_anchor_args)) return LISA_ERR_INVALID_ARG;
+        *bytes = a->cache ? decode_workspace(a->B, a->Hq, a->d, a->L) : 0;
+        return LISA_OK;
+    }
+    if (op == LISA_OP_SHARED_PREFILL) {
+        const lisa_shared_prefill_args* a = static_cast<const lisa_shared_prefill_args*>(args);
+        if (a->struct_size != sizeof(lisa_shared_prefill_args)) return LISA_ERR_INVALID_ARG;
+        *bytes = 0;
+        return LISA_OK;
+    }
+    if (op == LISA_OP_SHARED_DECODE) {
+        const lisa_shared_decode_args* a = static_cast<const lisa_shared_decode_args*>(args);
+        if (a->struct_size != sizeof(lisa_shared_decode_args) || !a->cache) return LISA_ERR_INVALID_ARG;
+        *bytes = decode_workspace(a->B, a->Hq, a->cache->d, a->L);
+        return LISA_OK;
+    }
+    return LISA_ERR_INVALID_ARG;
+}
+
+lisa_status_t lisa_attn_shared_prefill(const lisa_shared_prefill_args* a, lisa_stream_t stream) {
+    lisa_status_t st = validate_prefill(a);
+    if (st != LISA_OK) return st;
+    cudaError_t e = launch_generic_prefill(*a, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+}
+
+lisa_status_t lisa_attn_anchor(const lisa_anchor_args* a, lisa_stream_t stream) {
+    if (!a || a->struct_size != sizeof(lisa_anchor_args)) return LISA_ERR_INVALID_ARG;
+    lisa_status_t st = check_dims(a->B, a->Nq, a->Hq, a->Hkv, a->d);
+    if (st != LISA_OK) return st;
+    if (a->cache) {
+        if ((st = validate_anchor_decode(a)) != LISA_OK) return st;
+        const size_t need = decode_workspace(a->B, a->Hq, a->d, a->L);
+        if ((st = check_workspace(a->workspace, a->workspace_bytes, need)) != LISA_OK) return st;
+        cudaError_t e = launch_anchor_decode(*a, a->workspace, static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+    }
+    lisa_shared_prefill_args p;
+    std::memset(&p, 0, sizeof(p));
+    p.struct_size = sizeof(p);
+    p.B = a->B; p.N = a->Nq; p.Hq = a->Hq; p.Hkv = a->Hkv; p.d = a->d; p.chain_len = 0;
+    p.q0 = a->q; p.k0 = a->k; p.v = a->v; p.o = a->o;
+    p.workspace = a->workspace; p.workspace_bytes = a->workspace_bytes;
+    return lisa_attn_shared_prefill(&p, stream);
+}
+
+lisa_status_t lisa_attn_shared_decode(const lisa_shared_decode_args* a, lisa_stream_t stream) {
+    lisa_status_t st = validate_shared_decode(a);
+    if (st != LISA_OK) return st;
+    const size_t need = decode_workspace(a->B, a->Hq, a->cache->d, a->L);
+    if ((st = check_workspace(a->workspace, a->workspace_bytes, need)) != LISA_OK) return st;
+    cudaError_t e = launch_shared_decode(*a, a->workspace, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+}
+
+lisa_status_t lisa_kvcache_append(const lisa_kvcache_layer* layer, const lisa_tensor* k_or_kp, const lisa_tensor* v,
+                                  const int32_t* seq_lens_before, int32_t n_new, lisa_stream_t stream) {
+    if (!layer || !k_or_kp || !v || n_new < 1) return LISA_ERR_INVALID_ARG;
+    lisa_status_t st = check_cache(layer, layer->kind, true);
+    if (st != LISA_OK) return st;
+    if ((st = check_tensor(*k_or_kp)) != LISA_OK || (st = check_tensor(*v)) != LISA_OK) return st;
+    if (k_or_kp->dtype != layer->dtype || v->dtype != layer->dtype) return LISA_ERR_INVALID_ARG;
+    const int64_t vec = 16 / (int64_t)esize(layer->dtype);  // rows of d elements move as 16-byte vectors
+    auto rows_ok = [&](const lisa_tensor& t) { return t.stride_b % vec == 0 && t.stride_n % vec == 0 && t.stride_h % vec == 0; };
+    if (!rows_ok(*v)) return LISA_ERR_INVALID_ARG;
+    if (layer->kind == LISA_CACHE_STANDARD && !rows_ok(*k_or_kp)) return LISA_ERR_INVALID_ARG;
+    cudaError_t e = launch_kvcache_append(*layer, *k_or_kp, *v, seq_lens_before, n_new, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+}
+
+lisa_status_t lisa_check(lisa_stream_t stream) {
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    int* dev = status_words();
+    if (!dev) return cuda_fail(cudaErrorUnknown);
+    int host[4] = {0, 0, 0, 0};
+    if ((e = cudaMemcpy(host, dev, sizeof(host), cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(e);
+    if (host[0] || host[1]) {
+        if ((e = cudaMemset(dev, 0, sizeof(host))) != cudaSuccess) return cuda_fail(e);
+    }
+    if (host[1]) return LISA_ERR_TIMEOUT;
+    if (host[0]) return LISA_ERR_INVALID_ARG;
+    return LISA_OK;
+}
+
+// ---- host-memory variant: stage in, run, copy out -------------------------------------------------
+namespace {
+struct Arena {
+    char* base;
+    size_t off;
+    void* take(size_t bytes) {
+        void* p = base ? base + off : nullptr;
+        off += (bytes + 255) & ~(size_t)255;
+        return p;
+    }
+};
+
+// Lays the call's tensors out in the arena. With arena.base == nullptr only the size is computed.
+// dev receives device-side copies of the descriptors; h2d lists (dst, src, bytes) to copy.
+struct Copy { void* dst; const void* src; size_t bytes; };
+
+size_t plan_host_call(const lisa_shared_prefill_args& h, char* base, lisa_shared_prefill_args* dev, lisa_link* dlinks,
+                      Copy* copies, int* n_copies, size_t* o_bytes) {
+    Arena ar{base, 0};
+    int nc = 0;
+    auto dense = [&](const lisa_tensor& src, int H, int x, lisa_tensor* dst, bool copy_in) {
+        const size_t bytes = (size_t)h.B * h.N * H * x * esize(src.dtype);
+        void* p = ar.take(bytes);
+        if (dst) {
+            *dst = lisa_tensor{p, src.dtype, 0, (int64_t)h.N * H * x, (int64_t)H * x, (int64_t)x};
+            if (copy_in) copies[nc++] = Copy{p, src.ptr, bytes};
+        }
+        return bytes;
+    };
+    dense(h.q0, h.Hq, h.d, dev ? &dev->q0 : nullptr, true);
+    dense(h.k0, h.Hkv, h.d, dev ? &dev->k0 : nullptr, true);
+    dense(h.v, h.Hkv, h.d, dev ? &dev->v : nullptr, true);
+    const size_t ob = dense(h.o, h.Hq, h.d, dev ? &dev->o : nullptr, false);
+    if (o_bytes) *o_bytes = ob;
+    for (int k = 0; k < h.chain_len; ++k) {
+        const lisa_link& l = h.links[k];
+        lisa_link* dl = dlinks ? &dlinks[k] : nullptr;
+        if (dl) *dl = l;
+        dense(l.qp, h.Hq, l.r, dl ? &dl->qp : nullptr, true);
+        dense(l.kp, h.Hkv, l.r, dl ? &dl->kp : nullptr, true);
+        if (l.integrate == LISA_INTEGRATE_PLUS) continue;
+        const int h_in = l.integrate == LISA_INTEGRATE_CONCAT ? 2 * h.Hq : h.Hq;
+        const size_t ws = esize(l.w_dtype);
+        auto weight = [&](const void* src, size_t n, const void** dst) {
+            if (!src) return;
+            void* p = ar.take(n * ws);
+            if (dst) { *dst = p; copies[nc++] = Copy{p, src, n * ws}; }
+        };
+        weight(l.w1, (size_t)h_in * l.m, dl ? &dl->w1 : nullptr);
+        weight(l.b1, (size_t)l.m, dl ? &dl->b1 : nullptr);
+        if (l.ffn_layers == 2) {
+            weight(l.w2, (size_t)l.m * h.Hq, dl ? &dl->w2 : nullptr);
+            weight(l.b2, (size_t)h.Hq, dl ? &dl->b2 : nullptr);
+        }
+    }
+    if (n_copies) *n_copies = nc;
+    return ar.off;
+}
+
+lisa_status_t validate_host_args(const lisa_shared_prefill_args* a) {
+    if (!a || a->struct_size != sizeof(lisa_shared_prefill_args)) return LISA_ERR_INVALID_ARG;
+    lisa_status_t st = check_dims(a->B, a->N, a->Hq, a->Hkv, a->d);
+    if (st != LISA_OK) return st;
+    if (a->chain_len < 0 || (a->chain_len > 0 && !a->links)) return LISA_ERR_INVALID_ARG;
+    if (a->chain_len > kMaxChain) return LISA_ERR_UNSUPPORTED;
+    if (!a->q0.ptr || !a->k0.ptr || !a->v.ptr || !a->o.ptr) return LISA_ERR_INVALID_ARG;
+    if (!dtype_ok(a->q0.dtype) || !dtype_ok(a->k0.dtype) || !dtype_ok(a->v.dtype) || !dtype_ok(a->o.dtype))
+        return LISA_ERR_INVALID_ARG;
+    for (int k = 0; k < a->chain_len; ++k) {
+        const lisa_link& l = a->links[k];
+        if (!l.qp.ptr || !l.kp.ptr || !dtype_ok(l.qp.dtype) || !dtype_ok(l.kp.dtype)) return LISA_ERR_INVALID_ARG;
+        if (l.r < 1 || l.m < 0 || !dtype_ok(l.w_dtype)) return LISA_ERR_INVALID_ARG;
+        if (l.r > kMaxRank || l.m > kMaxHidden) return LISA_ERR_UNSUPPORTED;
+    }
+    return LISA_OK;
+}
+}  // namespace
+
+lisa_status_t lisa_host_arena_bytes(const lisa_shared_prefill_args* host_args, size_t* bytes) {
+    if (!bytes) return LISA_ERR_INVALID_ARG;
+    lisa_status_t st = validate_host_args(host_args);
+    if (st != LISA_OK) return st;
+    size_t ws = 0;
+    if ((st = lisa_workspace_bytes(LISA_OP_SHARED_PREFILL, host_args, &ws)) != LISA_OK) return st;
+    *bytes = plan_host_call(*host_args, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr) + ((ws + 255) & ~(size_t)255);
+    return LISA_OK;
+}
+
+lisa_status_t lisa_attn_shared_prefill_host(const lisa_shared_prefill_args* host_args, void* device_arena,
+                                            size_t arena_bytes, lisa_stream_t stream) {
+    size_t need = 0;
+    lisa_status_t st = lisa_host_arena_bytes(host_args, &need);
+    if (st != LISA_OK) return st;
+    if (!device_arena || arena_bytes < need || (reinterpret_cast<uintptr_t>(device_arena) & 255u)) return LISA_ERR_WORKSPACE;
+    lisa_shared_prefill_args dev = *host_args;
+    lisa_link dlinks[kMaxChain];
+    Copy copies[3 + 6 * kMaxChain];
+    int nc = 0;
+    size_t o_bytes = 0;
+    const size_t used = plan_host_call(*host_args, static_cast<char*>(device_arena), &dev, dlinks, copies, &nc, &o_bytes);
+    dev.links = dlinks;
+    size_t ws = 0;
+    lisa_workspace_bytes(LISA_OP_SHARED_PREFILL, host_args, &ws);
+    dev.workspace = ws ? static_cast<char*>(device_arena) + used : nullptr;
+    dev.workspace_bytes = ws;
+    if ((st = validate_prefill(&dev)) != LISA_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    for (int i = 0; i < nc; ++i)
+        if ((e = cudaMemcpyAsync(copies[i].dst, copies[i].src, copies[i].bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+            return cuda_fail(e);
+    if ((st = lisa_attn_shared_prefill(&dev, stream)) != LISA_OK) return st;
+    if ((e = cudaMemcpyAsync(host_args->o.ptr, dev.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
+    return LISA_OK;
+}
+
+}  // extern "C"
