@@ -90,21 +90,27 @@ def prefill_inputs(w: Workload, seed: int = 0, B=None, N=None):
     return t
 
 
-def decode_inputs(w: Workload, seed: int = 0, B=None, L=None):
+def decode_inputs(w: Workload, seed: int = 0, B=None, L=None, seqs=None):
     """Host tensors for one decode step of a shared layer and of a standard layer.
 
-    prev [B,Hq,L] fp32 score row; qp [B,Hq,r]; kp [B,L,Hkv,r]; v [B,L,Hkv,d]; aligner w1,w2;
-    and q0 [B,Hq,d], k [B,L,Hkv,d] for the standard-attention comparison.
+    prev [B,Hq,L] fp32 score row; qp [B,1,Hq,r]; kp [B,L,Hkv,r]; v [B,L,Hkv,d]; aligner w1,w2;
+    and q0 [B,1,Hq,d], k [B,L,Hkv,d] for the standard-attention comparison.  Every sequence has its own
+    streams, so `seqs` (a list of sequence indices) yields exactly those sequences of the full batch.
     """
     B = w.B if B is None else B
     L = w.N if L is None else L
+    seqs = list(range(B)) if seqs is None else list(seqs)
+
+    def per_seq(name, shape, dtype):
+        return torch.stack([as_dtype(normal("%s/%d" % (name, b), shape, seed), dtype) for b in seqs])
+
     t = {}
-    t["prev"] = torch.from_numpy(normal("prev", (B, w.Hq, L), seed))
-    t["qp"] = as_dtype(normal("qp", (B, w.Hq, w.r), seed), w.dtype)
-    t["kp"] = as_dtype(normal("kp", (B, L, w.Hkv, w.r), seed), w.dtype)
-    t["v"] = as_dtype(normal("v", (B, L, w.Hkv, w.d), seed), w.dtype)
+    t["prev"] = per_seq("prev", (w.Hq, L), "f32")
+    t["qp"] = per_seq("qp", (1, w.Hq, w.r), w.dtype)
+    t["kp"] = per_seq("kp", (L, w.Hkv, w.r), w.dtype)
+    t["v"] = per_seq("v", (L, w.Hkv, w.d), w.dtype)
     t["w1"] = as_dtype(normal("w1", (w.Hq, w.m), seed, std=w.Hq ** -0.5), w.dtype)
     t["w2"] = as_dtype(normal("w2", (w.m, w.Hq), seed, std=w.m ** -0.5), w.dtype)
-    t["q0"] = as_dtype(normal("q0", (B, w.Hq, w.d), seed), w.dtype)
-    t["k"] = as_dtype(normal("k", (B, L, w.Hkv, w.d), seed), w.dtype)
+    t["q0"] = per_seq("q0", (1, w.Hq, w.d), w.dtype)
+    t["k"] = per_seq("k", (L, w.Hkv, w.d), w.dtype)
     return t
