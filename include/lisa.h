@@ -202,6 +202,9 @@ lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes);
  * stream itself reports an error. */
 lisa_status_t lisa_check(lisa_stream_t stream);
 
+/* Number of kernels this library has enqueued so far in this process (all threads). */
+uint64_t lisa_kernel_launches(void);
+
 int lisa_last_cuda_error(void);             /* the cudaError_t of the last LISA_ERR_CUDA on this thread, else 0 */
 const char* lisa_status_string(int status); /* static string */
 int lisa_version(void);                     /* major*1000 + minor */

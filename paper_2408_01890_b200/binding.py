@@ -27,7 +27,7 @@ ACTS = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
 
 EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_host", "lisa_host_arena_bytes",
            "lisa_attn_shared_decode", "lisa_kvcache_append", "lisa_kvcache_bytes", "lisa_workspace_bytes", "lisa_check",
-           "lisa_last_cuda_error", "lisa_status_string", "lisa_version"]
+           "lisa_kernel_launches", "lisa_last_cuda_error", "lisa_status_string", "lisa_version"]
 
 
 class LisaError(RuntimeError):
@@ -100,6 +100,7 @@ def load():
         lib.lisa_kvcache_bytes.argtypes = [C.POINTER(CCacheLayer), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
         lib.lisa_workspace_bytes.argtypes = [C.c_int32, C.c_void_p, C.POINTER(C.c_size_t)]
         lib.lisa_check.argtypes = [C.c_void_p]
+        lib.lisa_kernel_launches.restype = C.c_uint64
         _lib = lib
     return _lib
 
@@ -289,3 +290,8 @@ def lisa_attn_shared_decode(prev_scores: torch.Tensor, link: Link, cache: KVCach
 def lisa_check() -> int:
     """Synchronises the current stream and returns the library's device-side status (0 = ok)."""
     return int(load().lisa_check(_stream()))
+
+
+def lisa_kernel_launches() -> int:
+    """Kernels the library has enqueued so far in this process."""
+    return int(load().lisa_kernel_launches())

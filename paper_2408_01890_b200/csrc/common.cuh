@@ -56,6 +56,9 @@ __device__ __forceinline__ float act_apply(float x, int act) {
 // Host function; returns the device address to hand to kernels, or nullptr if the lookup failed.
 int* status_words();
 
+// Adds n to the process-wide count of kernels enqueued by the library.
+void count_launches(int n);
+
 // Host-side launchers implemented in the .cu files. Each returns the cudaError_t of its launches.
 cudaError_t launch_generic_prefill(const lisa_shared_prefill_args& a, cudaStream_t s);
 

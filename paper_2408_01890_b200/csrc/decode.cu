@@ -455,6 +455,7 @@ cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cud
     }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, 0, s>>>(p);
+    count_launches(2);
     return cudaGetLastError();
 }
 
@@ -475,6 +476,7 @@ cudaError_t launch_anchor_decode(const lisa_anchor_args& a, void* ws, cudaStream
     anchor_decode_chunk_kernel<<<dim3(p.n_chunks, p.B), kThreads, smem, s>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, 0, s>>>(p);
+    count_launches(2);
     return cudaGetLastError();
 }
 

@@ -175,6 +175,7 @@ cudaError_t launch_generic_prefill(const lisa_shared_prefill_args& a, cudaStream
     if (e != cudaSuccess) return e;
     dim3 grid(a.N, a.B);
     generic_prefill_kernel<<<grid, kThreads, smem, s>>>(p);
+    count_launches(1);
     return cudaGetLastError();
 }
 

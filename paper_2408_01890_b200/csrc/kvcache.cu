@@ -81,6 +81,7 @@ cudaError_t launch_kvcache_append(const lisa_kvcache_layer& c, const lisa_tensor
         else
             append_kp_transposed_kernel<float><<<blocks_for(rows), threads, 0, s>>>(p);
     }
+    count_launches(2);
     return cudaGetLastError();
 }
 

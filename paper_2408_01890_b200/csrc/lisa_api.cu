@@ -1,4 +1,5 @@
 // C-ABI entry points: host-side validation and dispatch.  No arithmetic of the method lives here.
+#include <atomic>
 #include <cstring>
 
 #include "common.cuh"
@@ -7,6 +8,9 @@ namespace lisa {
 
 static __device__ int g_status[4];
 static thread_local int t_last_cuda_error = 0;
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
 int* status_words() {
     static int* cached[64] = {nullptr};
@@ -127,6 +131,7 @@ using namespace lisa;
 extern "C" {
 
 int lisa_version(void) { return 1000; }
+uint64_t lisa_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 int lisa_last_cuda_error(void) { return t_last_cuda_error; }
 
 const char* lisa_status_string(int status) {

@@ -114,3 +114,12 @@ def decode_inputs(w: Workload, seed: int = 0, B=None, L=None, seqs=None):
     t["q0"] = per_seq("q0", (1, w.Hq, w.d), w.dtype)
     t["k"] = per_seq("k", (L, w.Hkv, w.d), w.dtype)
     return t
+
+
+def device_normal(name: str, shape, seed: int = 0, dtype: str = "bf16", device="cuda") -> torch.Tensor:
+    """N(0,1) tensor drawn on the device from the stream keyed by (seed, name); for tensors too large to
+    draw on the host in reasonable time.  Whoever needs the same bytes on the host copies them back."""
+    g = torch.Generator(device=device)
+    g.manual_seed((int(seed) << 32) ^ zlib.crc32(name.encode()))
+    x = torch.randn(tuple(shape), generator=g, device=device, dtype=torch.float32)
+    return x.to(torch.bfloat16) if dtype == "bf16" else x
