@@ -180,6 +180,32 @@ typedef struct lisa_shared_decode_args {
 lisa_status_t lisa_attn_shared_decode(const lisa_shared_decode_args* args, lisa_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * lisa_attn_shared_decode_static -- lisa_attn_shared_decode without caller-provided scratch.
+ * (The paper has no counterpart to this entry point; it exists for integration reasons only.)
+ *
+ * Who needs it: callers that cannot obtain device memory at the moment they need to decode.  Typical cases
+ * are a serving process whose memory manager claimed the whole GPU at start-up (so cudaMalloc fails or
+ * fragments its pool), code running where an allocation would stall the device (cudaMalloc and cudaFree
+ * synchronise it), and hosts that forbid allocator calls inside their latency-critical loop.  For them the
+ * split-K partials live in a fixed array that is part of the library image: LISA_STATIC_SCRATCH_BYTES bytes
+ * of device memory are held on every GPU that loads the library, until the process exits.
+ *
+ * Same arguments, results and errors as lisa_attn_shared_decode, except:
+ *   - args->workspace and args->workspace_bytes are ignored;
+ *   - if the step needs more than LISA_STATIC_SCRATCH_BYTES of scratch (lisa_workspace_bytes(
+ *     LISA_OP_SHARED_DECODE, ...) tells how much) nothing is launched and LISA_ERR_WORKSPACE is returned;
+ *     use the regular entry point with your own buffer for such sizes;
+ *   - it calls no allocation routine of any kind, on the host or on the device.
+ * The first call on each device looks up the array's device address (a host-side call, made with that device
+ * current).  Make that first call outside of any stream capture.
+ * All calls on a device share the one array, and it keeps whatever the previous call left there.  Nothing in
+ * it has to start at zero: each call fully rewrites every entry it later reads.  Two calls whose kernels may
+ * run at the same time on one GPU (different streams, or different host threads) race on the array and give
+ * wrong results; order them on one stream or with events. */
+#define LISA_STATIC_SCRATCH_BYTES (8u << 20)
+lisa_status_t lisa_attn_shared_decode_static(const lisa_shared_decode_args* args, lisa_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
  * lisa_kvcache_append -- write n_new new positions into a layer's cache (Sec. 2.2; Sec. 5.2: "store K_LR
  * instead of K").  k_or_kp: [B,n_new,Hkv,d] for a STANDARD layer, [B,n_new,Hkv,r] (K') for a SHARED one,
  * which is stored transposed.  v: [B,n_new,Hkv,d].  Row t of sequence b lands at position

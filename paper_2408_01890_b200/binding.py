@@ -26,7 +26,7 @@ OP_ANCHOR, OP_SHARED_PREFILL, OP_SHARED_DECODE = 0, 1, 2
 ACTS = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
 
 EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_host", "lisa_host_arena_bytes",
-           "lisa_attn_shared_decode", "lisa_kvcache_append", "lisa_kvcache_bytes", "lisa_workspace_bytes", "lisa_check",
+           "lisa_attn_shared_decode", "lisa_attn_shared_decode_static", "lisa_kvcache_append", "lisa_kvcache_bytes", "lisa_workspace_bytes", "lisa_check",
            "lisa_kernel_launches", "lisa_last_cuda_error", "lisa_status_string", "lisa_version"]
 
 
@@ -95,6 +95,8 @@ def load():
         lib.lisa_attn_shared_prefill_host.argtypes = [C.POINTER(SharedPrefillArgs), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.lisa_host_arena_bytes.argtypes = [C.POINTER(SharedPrefillArgs), C.POINTER(C.c_size_t)]
         lib.lisa_attn_shared_decode.argtypes = [C.POINTER(SharedDecodeArgs), C.c_void_p]
+        lib.lisa_attn_shared_decode_static.argtypes = [C.POINTER(SharedDecodeArgs), C.c_void_p]
+        lib.lisa_attn_shared_decode_static.restype = C.c_int
         lib.lisa_kvcache_append.argtypes = [C.POINTER(CCacheLayer), C.POINTER(Tensor), C.POINTER(Tensor), C.c_void_p,
                                             C.c_int32, C.c_void_p]
         lib.lisa_kvcache_bytes.argtypes = [C.POINTER(CCacheLayer), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
@@ -284,6 +286,33 @@ def lisa_attn_shared_decode(prev_scores: torch.Tensor, link: Link, cache: KVCach
     ws = workspace if workspace is not None else _workspace(OP_SHARED_DECODE, a)
     a.workspace, a.workspace_bytes = _ptr(ws), (ws.numel() if ws is not None else 0)
     _check(load().lisa_attn_shared_decode(C.byref(a), _stream()), "lisa_attn_shared_decode")
+    return out
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def lisa_attn_shared_decode_static(prev_scores: torch.Tensor, link: Link, cache: KVCacheLayer, *, L: int, out: torch.Tensor,
+                                   seq_lens: Optional[torch.Tensor] = None,
+                                   out_scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """lisa_attn_shared_decode for callers that cannot allocate device memory when they decode: the scratch is a
+    fixed STATIC_SCRATCH_BYTES array inside the library, so this wrapper allocates nothing either -- `out`
+    ([B,1,Hq,d]) must be passed in.  Steps that need more scratch raise LisaError(ERR_WORKSPACE).  Calls share
+    that array: keep them ordered on one stream."""
+    B, Hq = prev_scores.shape[0], prev_scores.shape[1]
+    assert prev_scores.dtype == torch.float32 and prev_scores.stride(2) == 1
+    a = SharedDecodeArgs()
+    a.struct_size = C.sizeof(SharedDecodeArgs)
+    a.B, a.Hq, a.L = B, Hq, int(L)
+    a.prev_scores, a.prev_stride_b, a.prev_stride_h = prev_scores.data_ptr(), prev_scores.stride(0), prev_scores.stride(1)
+    a.link = link.to_c()
+    a.cache = C.pointer(cache.desc)
+    a.seq_lens = _ptr(seq_lens)
+    a.o = _tensor4(out)
+    if out_scores is not None:
+        assert out_scores.dtype == torch.float32 and out_scores.stride(2) == 1
+        a.out_scores, a.scores_stride_b, a.scores_stride_h = out_scores.data_ptr(), out_scores.stride(0), out_scores.stride(1)
+    _check(load().lisa_attn_shared_decode_static(C.byref(a), _stream()), "lisa_attn_shared_decode_static")
     return out
 
 

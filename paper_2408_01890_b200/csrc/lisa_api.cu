@@ -217,6 +217,38 @@ lisa_status_t lisa_attn_shared_decode(const lisa_shared_decode_args* a, lisa_str
     return e == cudaSuccess ? LISA_OK : cuda_fail(e);
 }
 
+// ---- decode with the scratch held inside the library image -----------------------------------------
+// For callers that cannot allocate device memory when they decode (see lisa.h).  The array's name is only
+// a host-side handle: kernels get the device address that cudaGetSymbolAddress returns for the current device.
+static __device__ __align__(256) unsigned char g_static_scratch[LISA_STATIC_SCRATCH_BYTES];
+
+static void* static_scratch_address() {
+    static void* cached[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cached[dev]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) {
+            t_last_cuda_error = (int)e;
+            return nullptr;
+        }
+        cached[dev] = p;
+    }
+    return cached[dev];
+}
+
+lisa_status_t lisa_attn_shared_decode_static(const lisa_shared_decode_args* a, lisa_stream_t stream) {
+    lisa_status_t st = validate_shared_decode(a);
+    if (st != LISA_OK) return st;
+    const size_t need = decode_workspace(a->B, a->Hq, a->cache->d, a->L);
+    if (need > (size_t)LISA_STATIC_SCRATCH_BYTES) return LISA_ERR_WORKSPACE;
+    void* scratch = static_scratch_address();
+    if (!scratch) return LISA_ERR_CUDA;
+    cudaError_t e = launch_shared_decode(*a, scratch, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+}
+
 lisa_status_t lisa_kvcache_append(const lisa_kvcache_layer* layer, const lisa_tensor* k_or_kp, const lisa_tensor* v,
                                   const int32_t* seq_lens_before, int32_t n_new, lisa_stream_t stream) {
     if (!layer || !k_or_kp || !v || n_new < 1) return LISA_ERR_INVALID_ARG;
