@@ -228,6 +228,10 @@ lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes);
  * stream itself reports an error. */
 lisa_status_t lisa_check(lisa_stream_t stream);
 
+/* on != 0: every later call in this process uses the general SIMT kernels even where a tensor-core kernel
+ * exists (for cross-checking the two paths against each other); on == 0 restores the default choice. */
+void lisa_force_general_kernels(int on);
+
 /* Number of kernels this library has enqueued so far in this process (all threads). */
 uint64_t lisa_kernel_launches(void);
 

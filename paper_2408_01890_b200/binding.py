@@ -27,7 +27,7 @@ ACTS = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
 
 EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_host", "lisa_host_arena_bytes",
            "lisa_attn_shared_decode", "lisa_attn_shared_decode_static", "lisa_kvcache_append", "lisa_kvcache_bytes", "lisa_workspace_bytes", "lisa_check",
-           "lisa_kernel_launches", "lisa_last_cuda_error", "lisa_status_string", "lisa_version"]
+           "lisa_force_general_kernels", "lisa_kernel_launches", "lisa_last_cuda_error", "lisa_status_string", "lisa_version"]
 
 
 class LisaError(RuntimeError):
@@ -324,3 +324,8 @@ def lisa_check() -> int:
 def lisa_kernel_launches() -> int:
     """Kernels the library has enqueued so far in this process."""
     return int(load().lisa_kernel_launches())
+
+
+def lisa_force_general_kernels(on: bool) -> None:
+    """Route every later call through the general SIMT kernels (True) or restore the default choice (False)."""
+    load().lisa_force_general_kernels(1 if on else 0)

@@ -66,6 +66,20 @@ cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cud
 cudaError_t launch_anchor_decode(const lisa_anchor_args& a, void* ws, cudaStream_t s);
 size_t decode_workspace(int B, int Hq, int d, int L);
 
+// Tensor-core flash kernel (head width 128, bf16): O = softmax_causal(QA.KA^T * scale [+ plane]) . V for query tiles
+// [qt_begin, qt_begin + qt_count).  qa [B,N,Hq,kd], ka [B,N,Hkv,kd] with kd in {64,128}; plane (optional) holds
+// bf16 [B*Hq][plane_rows][plane_cols] pre-computed scores for query rows qt_begin*128 onwards.
+struct TcFlashArgs {
+    int B, N, Hq, Hkv, kd;
+    lisa_tensor qa, ka, v, o;
+    float scale;
+    const void* plane;
+    int64_t plane_rows, plane_cols;
+    int qt_begin, qt_count;
+};
+bool tc_flash_supported(const TcFlashArgs& a);
+cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t s);
+
 cudaError_t launch_kvcache_append(const lisa_kvcache_layer& c, const lisa_tensor& k, const lisa_tensor& v,
                                   const int32_t* lens_before, int n_new, cudaStream_t s);
 

@@ -1,5 +1,6 @@
 // C-ABI entry points: host-side validation and dispatch.  No arithmetic of the method lives here.
 #include <atomic>
+#include <cmath>
 #include <cstring>
 
 #include "common.cuh"
@@ -9,6 +10,7 @@ namespace lisa {
 static __device__ int g_status[4];
 static thread_local int t_last_cuda_error = 0;
 
+static std::atomic<int> g_force_general{0};
 static std::atomic<uint64_t> g_launches{0};
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
@@ -131,6 +133,7 @@ using namespace lisa;
 extern "C" {
 
 int lisa_version(void) { return 1000; }
+void lisa_force_general_kernels(int on) { g_force_general.store(on ? 1 : 0); }
 uint64_t lisa_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 int lisa_last_cuda_error(void) { return t_last_cuda_error; }
 
@@ -184,7 +187,16 @@ lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes) 
 lisa_status_t lisa_attn_shared_prefill(const lisa_shared_prefill_args* a, lisa_stream_t stream) {
     lisa_status_t st = validate_prefill(a);
     if (st != LISA_OK) return st;
-    cudaError_t e = launch_generic_prefill(*a, static_cast<cudaStream_t>(stream));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!g_force_general.load() && a->d == 128 && a->chain_len == 0) {
+        TcFlashArgs f{a->B, a->N, a->Hq, a->Hkv, 128, a->q0, a->k0, a->v, a->o, 1.0f / sqrtf((float)a->d), nullptr, 0, 0,
+                      0, (a->N + 127) / 128};
+        if (tc_flash_supported(f)) {
+            cudaError_t e = launch_tc_flash(f, s);
+            return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+        }
+    }
+    cudaError_t e = launch_generic_prefill(*a, s);
     return e == cudaSuccess ? LISA_OK : cuda_fail(e);
 }
 

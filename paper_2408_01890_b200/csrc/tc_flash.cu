@@ -1,0 +1,377 @@
+// Tensor-core flash kernel (tcgen05 + TMEM + TMA) for head width 128, bf16.
+//
+// One CTA per (batch b, query head h, 128-row query tile).  For every key tile j <= the query tile:
+//   scores  S = QA . KA^T            tcgen05.mma, fp32 accumulator in tensor memory
+//   logits  A = S * scale (+ Y)      Y: optional bf16 tile of pre-computed scores (the aligned part of a
+//                                    shared layer, Eq. 4; then QA/KA are the layer's low-rank Q'/K', Eq. 3)
+//   causal mask (diagonal tile), online softmax in registers (one thread per query row), P as bf16
+//   O += P . V                       tcgen05.mma, V read MN-major straight from its [key][d] tile
+// With QA/KA = Q/K and no Y this is standard attention (Eq. 1-2).
+//
+// Warp roles: warps 0-3 softmax/epilogue (thread = query row = TMEM lane), warp 4 TMA producer,
+// warp 5 MMA issuer and TMEM owner.  Two-stage K/V(/Y) ring; S(t+1) is issued before P.V(t).
+// Every wait is bounded; on expiry the CTA records it in the status word, drains and exits.
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace lisa {
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BN = 128, D = 128;
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+constexpr int kThreads = 192;
+constexpr uint32_t TMEM_COLS = 256;  // S: [0,128), O: [128,256)
+
+struct FlashParams {
+    int B, N, Hq, Hkv;
+    float scale_log2;  // score scale * log2(e)
+    __nv_bfloat16* o;
+    int64_t o_sb, o_sn, o_sh;
+    int* status;
+    int plane_row0;  // first query row held by the Y workspace (rows are stored relative to it)
+    int qt_begin;    // this launch covers query tiles [qt_begin, qt_begin + gridDim.x)
+};
+
+template <int KD, bool PLANE>
+struct Smem {
+    static constexpr int Q_BYTES = BM * KD * 2;
+    static constexpr int K_BYTES = BN * KD * 2;
+    static constexpr int V_BYTES = BN * D * 2;
+    static constexpr int P_BYTES = BM * BN * 2;
+    static constexpr int Y_BYTES = PLANE ? BM * BN * 2 : 0;
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = OFF_Q + Q_BYTES;
+    static constexpr int OFF_V = OFF_K + 2 * K_BYTES;
+    static constexpr int OFF_P = OFF_V + 2 * V_BYTES;
+    static constexpr int OFF_Y = OFF_P + P_BYTES;
+    static constexpr int OFF_BAR = OFF_Y + 2 * Y_BYTES;
+    static constexpr int TOTAL = OFF_BAR + 256 + 1024;  // + alignment slack
+};
+
+template <int KD, bool PLANE>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ CUtensorMap tmQ,
+                const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                const __grid_constant__ CUtensorMap tmY) {
+    using L = Smem<KD, PLANE>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sQ = smem + L::OFF_Q;
+    uint8_t* sK = smem + L::OFF_K;
+    uint8_t* sV = smem + L::OFF_V;
+    uint8_t* sP = smem + L::OFF_P;
+    uint8_t* sY = smem + L::OFF_Y;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+    uint64_t* q_full = bars + 0;
+    uint64_t* kv_full = bars + 1;   // [2]
+    uint64_t* kv_empty = bars + 3;  // [2]
+    uint64_t* s_full = bars + 5;
+    uint64_t* s_free = bars + 6;
+    uint64_t* p_full = bars + 7;
+    uint64_t* pv_done = bars + 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 11);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int qt = p.qt_begin + (int)gridDim.x - 1 - (int)blockIdx.x;  // heavy tiles first
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int g = h / (p.Hq / p.Hkv);
+    const int nt = qt + 1;  // key tiles 0..qt
+    const int q0 = qt * BM;
+
+    if (tid == 0) {
+        mbar_init(q_full, 1);
+        mbar_init(kv_full + 0, 1); mbar_init(kv_full + 1, 1);
+        mbar_init(kv_empty + 0, 1); mbar_init(kv_empty + 1, 1);
+        mbar_init(s_full, 1);
+        mbar_init(s_free, 128);
+        mbar_init(p_full, 128);
+        mbar_init(pv_done, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 5) tmem_alloc(tmem_slot, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 128;
+
+    if (warp == 4) {
+        // ------------------------------ TMA producer ------------------------------
+        if (lane == 0) {
+            tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+            mbar_expect_tx(q_full, L::Q_BYTES);
+            for (int c = 0; c < KD / 64; ++c) tma_load_4d(sQ + c * (BM * 128), &tmQ, q_full, c * 64, h, q0, b);
+            for (int t = 0; t < nt; ++t) {
+                const int s = t & 1;
+                if (!mbar_wait(kv_empty + s, ((t >> 1) & 1) ^ 1, abort_flag)) break;
+                mbar_expect_tx(kv_full + s, L::K_BYTES + L::V_BYTES + L::Y_BYTES);
+                for (int c = 0; c < KD / 64; ++c) tma_load_4d(sK + s * L::K_BYTES + c * (BN * 128), &tmK, kv_full + s, c * 64, g, t * BN, b);
+                for (int c = 0; c < D / 64; ++c) tma_load_4d(sV + s * L::V_BYTES + c * (BN * 128), &tmV, kv_full + s, c * 64, g, t * BN, b);
+                if constexpr (PLANE)
+                    for (int c = 0; c < BN / 64; ++c)
+                        tma_load_3d(sY + s * L::Y_BYTES + c * (BM * 128), &tmY, kv_full + s, t * BN + c * 64, q0 - p.plane_row0,
+                                    b * p.Hq + h);
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            constexpr uint32_t IDESC_QK = umma_idesc_bf16(BM, BN, 0, 0);
+            constexpr uint32_t IDESC_PV = umma_idesc_bf16(BM, D, 0, 1);
+            auto issue_qk = [&](int t) {
+                const int s = t & 1;
+                const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + s * L::K_BYTES);
+#pragma unroll
+                for (int ks = 0; ks < KD / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * (BM * 128) + (ks & 3) * 32;
+                    umma_ss(tmem_S, umma_desc_sw128(qa + off, 16, 1024), umma_desc_sw128(ka + off, 16, 1024), IDESC_QK, ks > 0);
+                }
+                umma_commit(s_full);
+            };
+            bool ok = mbar_wait(q_full, 0, abort_flag) && mbar_wait(kv_full + 0, 0, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0);
+            }
+            for (int t = 0; ok && t < nt; ++t) {
+                const int s = t & 1;
+                if (t + 1 < nt) {
+                    ok = mbar_wait(kv_full + ((t + 1) & 1), ((t + 1) >> 1) & 1, abort_flag) && mbar_wait(s_free, t & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(t + 1);
+                }
+                if (!(ok = mbar_wait(p_full, t & 1, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t pa = smem_u32(sP), va = smem_u32(sV + s * L::V_BYTES);
+#pragma unroll
+                for (int ks = 0; ks < BN / 16; ++ks) {
+                    const uint32_t a_off = (ks >> 2) * (BM * 128) + (ks & 3) * 32;  // P: K-major, 64 keys per 128-byte row
+                    const uint32_t b_off = ks * 2048;                               // V: 16 keys = two 8-row groups
+                    umma_ss(tmem_O, umma_desc_sw128(pa + a_off, 16, 1024), umma_desc_sw128(va + b_off, BN * 128, 1024), IDESC_PV,
+                            (t > 0) || (ks > 0));
+                }
+                umma_commit(pv_done);
+                umma_commit(kv_empty + s);
+            }
+        }
+    } else {
+        // ------------------------------ softmax + epilogue (thread = query row) ------------------------------
+        const int row = tid;                       // 0..127, TMEM lane
+        const int qi = q0 + row;                   // global query index
+        const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+        float m_ref = -INFINITY, l_sum = 0.f;
+        bool ok = true;
+        for (int t = 0; t < nt; ++t) {
+            const int s = t & 1;
+            if (!(ok = mbar_wait(s_full, t & 1, abort_flag))) break;
+            tc_fence_after();
+            uint32_t sr[128];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(tmem_S + lane_sel + c * 32, sr + c * 32);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(s_free);
+            float* sf = reinterpret_cast<float*>(sr);
+            if constexpr (PLANE) {
+                // the stage's full barrier was already observed by the MMA warp; s_full implies it completed
+                const uint8_t* yb = sY + s * L::Y_BYTES;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const uint4 y = *reinterpret_cast<const uint4*>(yb + (c >> 3) * (BM * 128) + sw128_offset(row, c & 7));
+                    const uint32_t w[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        sf[c * 8 + 2 * e] = fmaf(sf[c * 8 + 2 * e], p.scale_log2, __uint_as_float(w[e] << 16) * 1.4426950408889634f);
+                        sf[c * 8 + 2 * e + 1] =
+                            fmaf(sf[c * 8 + 2 * e + 1], p.scale_log2, __uint_as_float(w[e] & 0xffff0000u) * 1.4426950408889634f);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 128; ++j) sf[j] *= p.scale_log2;
+            }
+            if (t == nt - 1) {
+#pragma unroll
+                for (int j = 0; j < 128; ++j)
+                    if (t * BN + j > qi) sf[j] = -INFINITY;
+            }
+            float m_t = sf[0];
+#pragma unroll
+            for (int j = 1; j < 128; ++j) m_t = fmaxf(m_t, sf[j]);
+            // lazy rescale: move the reference maximum only when some row of the warp outgrew it by 2^8
+            const bool grow = m_t > m_ref + 8.f;
+            const bool rescale = __any_sync(0xffffffffu, grow) || t == 0;
+            float factor = 1.f;
+            if (rescale) {
+                const float m_new = fmaxf(m_ref, m_t);
+                factor = fast_exp2(m_ref - m_new);
+                m_ref = m_new;
+            }
+            if (t > 0) {
+                if (!(ok = mbar_wait(pv_done, (t - 1) & 1, abort_flag))) break;
+                if (rescale) {
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t orr[32];
+                        tmem_ld32(tmem_O + lane_sel + c * 32, orr);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) orr[j] = __float_as_uint(__uint_as_float(orr[j]) * factor);
+                        tmem_st32(tmem_O + lane_sel + c * 32, orr);
+                    }
+                    tmem_wait_st();
+                }
+            }
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                float e[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    e[j] = fast_exp2(sf[c * 8 + j] - m_ref);
+                    sum += e[j];
+                }
+                uint4 v;
+                v.x = pack_bf16(e[0], e[1]); v.y = pack_bf16(e[2], e[3]); v.z = pack_bf16(e[4], e[5]); v.w = pack_bf16(e[6], e[7]);
+                *reinterpret_cast<uint4*>(sP + (c >> 3) * (BM * 128) + sw128_offset(row, c & 7)) = v;
+            }
+            l_sum = l_sum * factor + sum;
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive(p_full);
+        }
+        if (ok && mbar_wait(pv_done, (nt - 1) & 1, abort_flag)) {
+            tc_fence_after();
+            const float inv_l = 1.f / l_sum;
+            __nv_bfloat16* orow = p.o + b * p.o_sb + (int64_t)qi * p.o_sn + h * p.o_sh;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t orr[32];
+                tmem_ld32(tmem_O + lane_sel + c * 32, orr);
+                tmem_wait_ld();
+                if (qi < p.N) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint4 v;
+                        v.x = pack_bf16(__uint_as_float(orr[q * 8 + 0]) * inv_l, __uint_as_float(orr[q * 8 + 1]) * inv_l);
+                        v.y = pack_bf16(__uint_as_float(orr[q * 8 + 2]) * inv_l, __uint_as_float(orr[q * 8 + 3]) * inv_l);
+                        v.z = pack_bf16(__uint_as_float(orr[q * 8 + 4]) * inv_l, __uint_as_float(orr[q * 8 + 5]) * inv_l);
+                        v.w = pack_bf16(__uint_as_float(orr[q * 8 + 6]) * inv_l, __uint_as_float(orr[q * 8 + 7]) * inv_l);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + q * 8) = v;
+                    }
+                }
+            }
+        }
+    }
+    // ------------------------------ teardown ------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait ran out: give copies and MMAs still in flight time to land before the memory is released
+        if (tid == 0) atomicAdd(p.status + 1, 1);
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 5) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace
+
+
+bool make_tensor_map_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                          const uint32_t* box) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+            qres != cudaDriverEntryPointSuccess)
+            return false;
+        encode = reinterpret_cast<EncodeFn>(fn);
+    }
+    cuuint64_t gdims[5], gstr[4];
+    cuuint32_t gbox[5], estr[5];
+    for (int i = 0; i < rank; ++i) { gdims[i] = dims[i]; gbox[i] = box[i]; estr[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdims, gstr, gbox, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+bool tma_ok(const lisa_tensor& t) {
+    return t.dtype == LISA_BF16 && (reinterpret_cast<uintptr_t>(t.ptr) & 15u) == 0 && t.stride_b % 8 == 0 && t.stride_n % 8 == 0 &&
+           t.stride_h % 8 == 0 && t.stride_b > 0 && t.stride_n > 0 && t.stride_h > 0;
+}
+bool map_bnhx(CUtensorMap* m, const lisa_tensor& t, int B, int N, int H, int X) {
+    const uint64_t dims[4] = {(uint64_t)X, (uint64_t)H, (uint64_t)N, (uint64_t)B};
+    const uint64_t str[3] = {(uint64_t)t.stride_h * 2, (uint64_t)t.stride_n * 2, (uint64_t)t.stride_b * 2};
+    const uint32_t box[4] = {64, 1, 128, 1};
+    return make_tensor_map_bf16(m, t.ptr, 4, dims, str, box);
+}
+}  // namespace
+
+bool tc_flash_supported(const TcFlashArgs& a) {
+    return (a.kd == 128 || a.kd == 64) && tma_ok(a.qa) && tma_ok(a.ka) && tma_ok(a.v) && tma_ok(a.o) && a.Hq % a.Hkv == 0;
+}
+
+cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
+    CUtensorMap tmQ, tmK, tmV, tmY;
+    if (!map_bnhx(&tmQ, a.qa, a.B, a.N, a.Hq, a.kd) || !map_bnhx(&tmK, a.ka, a.B, a.N, a.Hkv, a.kd) ||
+        !map_bnhx(&tmV, a.v, a.B, a.N, a.Hkv, D))
+        return cudaErrorInvalidValue;
+    tmY = tmQ;
+    if (a.plane) {
+        const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * a.Hq};
+        const uint64_t str[2] = {(uint64_t)a.plane_cols * 2, (uint64_t)a.plane_cols * a.plane_rows * 2};
+        const uint32_t box[3] = {64, 128, 1};
+        if (!make_tensor_map_bf16(&tmY, a.plane, 3, dims, str, box)) return cudaErrorInvalidValue;
+    }
+    FlashParams p;
+    p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv;
+    p.scale_log2 = a.scale * 1.4426950408889634f;
+    p.o = reinterpret_cast<__nv_bfloat16*>(a.o.ptr);
+    p.o_sb = a.o.stride_b; p.o_sn = a.o.stride_n; p.o_sh = a.o.stride_h;
+    p.status = status_words();
+    if (!p.status) return cudaErrorUnknown;
+    p.plane_row0 = a.qt_begin * BM;
+    p.qt_begin = a.qt_begin;
+    dim3 grid(a.qt_count, a.Hq, a.B);
+    cudaError_t e;
+#define LISA_LAUNCH_FLASH(KD_, PL_)                                                                                        \
+    do {                                                                                                                   \
+        auto kern = tc_flash_kernel<KD_, PL_>;                                                                             \
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<KD_, PL_>::TOTAL)) != cudaSuccess) \
+            return e;                                                                                                      \
+        kern<<<grid, kThreads, Smem<KD_, PL_>::TOTAL, stream>>>(p, tmQ, tmK, tmV, tmY);                                    \
+    } while (0)
+    if (a.kd == 128 && !a.plane) LISA_LAUNCH_FLASH(128, false);
+    else if (a.kd == 64 && a.plane) LISA_LAUNCH_FLASH(64, true);
+    else if (a.kd == 64 && !a.plane) LISA_LAUNCH_FLASH(64, false);
+    else return cudaErrorInvalidValue;  // 128-wide scores plus a plane do not fit shared memory
+#undef LISA_LAUNCH_FLASH
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+}  // namespace lisa
