@@ -76,9 +76,33 @@ struct TcFlashArgs {
     const void* plane;
     int64_t plane_rows, plane_cols;
     int qt_begin, qt_count;
+    // emit_plane != nullptr: no attention; the scaled scores of the covered tiles are written there as bf16
+    // ([B*Hq][plane_rows][plane_cols], rows relative to qt_begin*128); v, o and plane are then ignored.
+    void* emit_plane = nullptr;
+    int ksteps = 0;  // 16-wide k-steps to issue (0 = kd/16); the columns beyond are zero padding
 };
 bool tc_flash_supported(const TcFlashArgs& a);
 cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t s);
+
+// Tensor-core aligner: applies the FFN chain of links[0..chain) to the score planes in place (see tc_align.cu).
+// planes[0] = A_0 in / Y out, planes[k] = D_k (already scaled) for k = 1..chain-1; all [B*32][plane_rows][plane_cols].
+struct TcAlignArgs {
+    int B, N, chain, qt_begin, qt_count;
+    int64_t plane_rows, plane_cols;
+    void* planes[4];
+    const lisa_link* links;
+    int ctas_per_tile = 0;
+};
+bool tc_align_supported(int Hq, const lisa_link* links, int chain);
+cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t s);
+
+// Packs Q' or K' ([B,N,H,r], any strides) into zero-padded bf16 [B][H][N][64] rows for the tensor-core kernels.
+cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int r, void* dst, cudaStream_t s);
+
+// Tensor-core prefill of a shared layer (tc_prefill.cu): emit planes -> align -> attention, wave by wave.
+bool tc_shared_prefill_supported(const lisa_shared_prefill_args& a);
+size_t tc_shared_prefill_workspace(const lisa_shared_prefill_args& a);
+cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws, cudaStream_t s);
 
 cudaError_t launch_kvcache_append(const lisa_kvcache_layer& c, const lisa_tensor& k, const lisa_tensor& v,
                                   const int32_t* lens_before, int n_new, cudaStream_t s);

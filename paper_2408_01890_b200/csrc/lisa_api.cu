@@ -173,6 +173,9 @@ lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes) 
         const lisa_shared_prefill_args* a = static_cast<const lisa_shared_prefill_args*>(args);
         if (a->struct_size != sizeof(lisa_shared_prefill_args)) return LISA_ERR_INVALID_ARG;
         *bytes = 0;
+        if (!g_force_general.load() && a->chain_len > 0 && a->links && a->Hq > 0 && a->Hkv > 0 && a->Hq % a->Hkv == 0 &&
+            tc_shared_prefill_supported(*a))
+            *bytes = tc_shared_prefill_workspace(*a);
         return LISA_OK;
     }
     if (op == LISA_OP_SHARED_DECODE) {
@@ -195,6 +198,12 @@ lisa_status_t lisa_attn_shared_prefill(const lisa_shared_prefill_args* a, lisa_s
             cudaError_t e = launch_tc_flash(f, s);
             return e == cudaSuccess ? LISA_OK : cuda_fail(e);
         }
+    }
+    if (!g_force_general.load() && a->chain_len > 0 && tc_shared_prefill_supported(*a)) {
+        const size_t need = tc_shared_prefill_workspace(*a);
+        if ((st = check_workspace(a->workspace, a->workspace_bytes, need)) != LISA_OK) return st;
+        cudaError_t e = launch_tc_shared_prefill(*a, a->workspace, s);
+        return e == cudaSuccess ? LISA_OK : cuda_fail(e);
     }
     cudaError_t e = launch_generic_prefill(*a, s);
     return e == cudaSuccess ? LISA_OK : cuda_fail(e);

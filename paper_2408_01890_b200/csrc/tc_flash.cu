@@ -38,14 +38,24 @@ struct FlashParams {
     int* status;
     int plane_row0;  // first query row held by the Y workspace (rows are stored relative to it)
     int qt_begin;    // this launch covers query tiles [qt_begin, qt_begin + gridDim.x)
+    int ksteps;      // 16-wide k-steps of the score MMA actually issued (<= KD/16; the rest is zero padding)
+    float scale;     // MODE_EMIT: scores are multiplied by this before rounding to bf16
+    __nv_bfloat16* plane_out;  // MODE_EMIT: [B*Hq][plane_rows][plane_cols]
+    int64_t plane_rows, plane_cols;
 };
 
-template <int KD, bool PLANE>
+// MODE_ATTN: softmax(QA.KA^T).V;  MODE_ATTN_PLANE: the same with the pre-computed tile Y added to the logits;
+// MODE_EMIT: no softmax, the scaled scores are written as bf16 to the plane workspace (for the aligner kernel).
+constexpr int MODE_ATTN = 0, MODE_ATTN_PLANE = 1, MODE_EMIT = 2;
+
+template <int KD, int MODE>
 struct Smem {
+    static constexpr bool PLANE = MODE == MODE_ATTN_PLANE;
+    static constexpr bool EMIT = MODE == MODE_EMIT;
     static constexpr int Q_BYTES = BM * KD * 2;
     static constexpr int K_BYTES = BN * KD * 2;
-    static constexpr int V_BYTES = BN * D * 2;
-    static constexpr int P_BYTES = BM * BN * 2;
+    static constexpr int V_BYTES = EMIT ? 0 : BN * D * 2;
+    static constexpr int P_BYTES = EMIT ? 0 : BM * BN * 2;
     static constexpr int Y_BYTES = PLANE ? BM * BN * 2 : 0;
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + Q_BYTES;
@@ -56,12 +66,13 @@ struct Smem {
     static constexpr int TOTAL = OFF_BAR + 256 + 1024;  // + alignment slack
 };
 
-template <int KD, bool PLANE>
+template <int KD, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ CUtensorMap tmQ,
                 const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmY) {
-    using L = Smem<KD, PLANE>;
+    using L = Smem<KD, MODE>;
+    constexpr bool PLANE = L::PLANE, EMIT = L::EMIT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem + L::OFF_Q;
@@ -116,7 +127,9 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 if (!mbar_wait(kv_empty + s, ((t >> 1) & 1) ^ 1, abort_flag)) break;
                 mbar_expect_tx(kv_full + s, L::K_BYTES + L::V_BYTES + L::Y_BYTES);
                 for (int c = 0; c < KD / 64; ++c) tma_load_4d(sK + s * L::K_BYTES + c * (BN * 128), &tmK, kv_full + s, c * 64, g, t * BN, b);
-                for (int c = 0; c < D / 64; ++c) tma_load_4d(sV + s * L::V_BYTES + c * (BN * 128), &tmV, kv_full + s, c * 64, g, t * BN, b);
+                if constexpr (!EMIT)
+                    for (int c = 0; c < D / 64; ++c)
+                        tma_load_4d(sV + s * L::V_BYTES + c * (BN * 128), &tmV, kv_full + s, c * 64, g, t * BN, b);
                 if constexpr (PLANE)
                     for (int c = 0; c < BN / 64; ++c)
                         tma_load_3d(sY + s * L::Y_BYTES + c * (BM * 128), &tmY, kv_full + s, t * BN + c * 64, q0 - p.plane_row0,
@@ -133,10 +146,14 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + s * L::K_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < KD / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * (BM * 128) + (ks & 3) * 32;
-                    umma_ss(tmem_S, umma_desc_sw128(qa + off, 16, 1024), umma_desc_sw128(ka + off, 16, 1024), IDESC_QK, ks > 0);
+                    if (ks < p.ksteps) {
+                        const uint32_t off = (ks >> 2) * (BM * 128) + (ks & 3) * 32;
+                        umma_ss(tmem_S, umma_desc_sw128(qa + off, 16, 1024), umma_desc_sw128(ka + off, 16, 1024), IDESC_QK, ks > 0);
+                    }
                 }
                 umma_commit(s_full);
+                if constexpr (EMIT)
+                    if (t + 2 < nt) umma_commit(kv_empty + s);  // nobody waits for the last two: do not arm them
             };
             bool ok = mbar_wait(q_full, 0, abort_flag) && mbar_wait(kv_full + 0, 0, abort_flag);
             if (ok) {
@@ -151,6 +168,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                     tc_fence_after();
                     issue_qk(t + 1);
                 }
+                if constexpr (EMIT) continue;
                 if (!(ok = mbar_wait(p_full, t & 1, abort_flag))) break;
                 tc_fence_after();
                 const uint32_t pa = smem_u32(sP), va = smem_u32(sV + s * L::V_BYTES);
@@ -162,7 +180,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                             (t > 0) || (ks > 0));
                 }
                 umma_commit(pv_done);
-                umma_commit(kv_empty + s);
+                if (t + 2 < nt) umma_commit(kv_empty + s);
             }
         }
     } else {
@@ -183,6 +201,21 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             tc_fence_before();
             mbar_arrive(s_free);
             float* sf = reinterpret_cast<float*>(sr);
+            if constexpr (EMIT) {
+                if (qi < p.N) {
+                    __nv_bfloat16* dst = p.plane_out + ((int64_t)(b * p.Hq + h) * p.plane_rows + (qi - p.plane_row0)) * p.plane_cols + t * BN;
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        uint4 v;
+                        v.x = pack_bf16(sf[c * 8 + 0] * p.scale, sf[c * 8 + 1] * p.scale);
+                        v.y = pack_bf16(sf[c * 8 + 2] * p.scale, sf[c * 8 + 3] * p.scale);
+                        v.z = pack_bf16(sf[c * 8 + 4] * p.scale, sf[c * 8 + 5] * p.scale);
+                        v.w = pack_bf16(sf[c * 8 + 6] * p.scale, sf[c * 8 + 7] * p.scale);
+                        *reinterpret_cast<uint4*>(dst + c * 8) = v;
+                    }
+                }
+                continue;
+            }
             if constexpr (PLANE) {
                 // the stage's full barrier was already observed by the MMA warp; s_full implies it completed
                 const uint8_t* yb = sY + s * L::Y_BYTES;
@@ -252,7 +285,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             tc_fence_before();
             mbar_arrive(p_full);
         }
-        if (ok && mbar_wait(pv_done, (nt - 1) & 1, abort_flag)) {
+        if (!EMIT && ok && mbar_wait(pv_done, (nt - 1) & 1, abort_flag)) {
             tc_fence_after();
             const float inv_l = 1.f / l_sum;
             __nv_bfloat16* orow = p.o + b * p.o_sb + (int64_t)qi * p.o_sn + h * p.o_sh;
@@ -332,14 +365,15 @@ bool map_bnhx(CUtensorMap* m, const lisa_tensor& t, int B, int N, int H, int X) 
 }  // namespace
 
 bool tc_flash_supported(const TcFlashArgs& a) {
-    return (a.kd == 128 || a.kd == 64) && tma_ok(a.qa) && tma_ok(a.ka) && tma_ok(a.v) && tma_ok(a.o) && a.Hq % a.Hkv == 0;
+    if (!((a.kd == 128 || a.kd == 64) && tma_ok(a.qa) && tma_ok(a.ka) && a.Hq % a.Hkv == 0)) return false;
+    return a.emit_plane ? true : (tma_ok(a.v) && tma_ok(a.o));
 }
 
 cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     CUtensorMap tmQ, tmK, tmV, tmY;
-    if (!map_bnhx(&tmQ, a.qa, a.B, a.N, a.Hq, a.kd) || !map_bnhx(&tmK, a.ka, a.B, a.N, a.Hkv, a.kd) ||
-        !map_bnhx(&tmV, a.v, a.B, a.N, a.Hkv, D))
-        return cudaErrorInvalidValue;
+    if (!map_bnhx(&tmQ, a.qa, a.B, a.N, a.Hq, a.kd) || !map_bnhx(&tmK, a.ka, a.B, a.N, a.Hkv, a.kd)) return cudaErrorInvalidValue;
+    tmV = tmQ;
+    if (!a.emit_plane && !map_bnhx(&tmV, a.v, a.B, a.N, a.Hkv, D)) return cudaErrorInvalidValue;
     tmY = tmQ;
     if (a.plane) {
         const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * a.Hq};
@@ -356,18 +390,25 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     if (!p.status) return cudaErrorUnknown;
     p.plane_row0 = a.qt_begin * BM;
     p.qt_begin = a.qt_begin;
+    p.ksteps = a.ksteps > 0 ? a.ksteps : a.kd / 16;
+    p.scale = a.scale;
+    p.plane_out = reinterpret_cast<__nv_bfloat16*>(a.emit_plane);
+    p.plane_rows = a.plane_rows; p.plane_cols = a.plane_cols;
     dim3 grid(a.qt_count, a.Hq, a.B);
     cudaError_t e;
-#define LISA_LAUNCH_FLASH(KD_, PL_)                                                                                        \
+#define LISA_LAUNCH_FLASH(KD_, PL_)                                                                                       \
     do {                                                                                                                   \
         auto kern = tc_flash_kernel<KD_, PL_>;                                                                             \
         if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<KD_, PL_>::TOTAL)) != cudaSuccess) \
             return e;                                                                                                      \
         kern<<<grid, kThreads, Smem<KD_, PL_>::TOTAL, stream>>>(p, tmQ, tmK, tmV, tmY);                                    \
     } while (0)
-    if (a.kd == 128 && !a.plane) LISA_LAUNCH_FLASH(128, false);
-    else if (a.kd == 64 && a.plane) LISA_LAUNCH_FLASH(64, true);
-    else if (a.kd == 64 && !a.plane) LISA_LAUNCH_FLASH(64, false);
+    if (a.emit_plane) {
+        if (a.kd == 128) LISA_LAUNCH_FLASH(128, MODE_EMIT);
+        else LISA_LAUNCH_FLASH(64, MODE_EMIT);
+    } else if (a.kd == 128 && !a.plane) LISA_LAUNCH_FLASH(128, MODE_ATTN);
+    else if (a.kd == 64 && a.plane) LISA_LAUNCH_FLASH(64, MODE_ATTN_PLANE);
+    else if (a.kd == 64 && !a.plane) LISA_LAUNCH_FLASH(64, MODE_ATTN);
     else return cudaErrorInvalidValue;  // 128-wide scores plus a plane do not fit shared memory
 #undef LISA_LAUNCH_FLASH
     count_launches(1);

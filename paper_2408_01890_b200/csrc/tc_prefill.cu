@@ -1,0 +1,163 @@
+// Tensor-core prefill of a shared layer (Sec. 5.1, Eq. 3-4, then Eq. 1): host-side orchestration.
+//
+// The aligner mixes all heads at one (query, key) position while softmax.V needs one running output per
+// head, so the layer runs as three tensor-core kernels that exchange bf16 score planes [head][row][col]
+// through a workspace sized to stay in L2, one wave of query tiles at a time:
+//   1. tc_flash (emit)   A_0 = Q0.K0^T/sqrt(d) per head, and D_k = Q'_k.K'_k^T/sqrt(r) for the links k < c
+//   2. tc_align          per position: the FFN chain over the head axis, Y written over A_0
+//   3. tc_flash (plane)  per head: logits = Y + Q'_c.K'_c^T/sqrt(r), causal softmax, .V
+// The N x N x Hq scores of the whole prompt are never stored; only the wave's strip of rows is.
+#include <algorithm>
+#include <cmath>
+
+#include "common.cuh"
+
+namespace lisa {
+namespace {
+
+constexpr int kTile = 128;
+constexpr int kPadRank = 64;
+constexpr size_t kWaveBytes = (size_t)64 << 20;  // score-plane bytes one wave may touch (L2 is 126 MB)
+
+__global__ void pack_lowrank_kernel(TView src, int B, int N, int H, int r, __nv_bfloat16* dst) {
+    const int64_t total = (int64_t)B * H * N * (kPadRank / 8);
+    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int chunk = (int)(e % (kPadRank / 8));
+        int64_t rest = e / (kPadRank / 8);
+        const int n = (int)(rest % N); rest /= N;
+        const int h = (int)(rest % H);
+        const int b = (int)(rest / H);
+        const __nv_bfloat16* sp = reinterpret_cast<const __nv_bfloat16*>(src.ptr) + b * src.sb + (int64_t)n * src.sn + h * src.sh;
+        __align__(16) __nv_bfloat16 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int x = chunk * 8 + j;
+            v[j] = x < r ? sp[x] : __float2bfloat16_rn(0.f);
+        }
+        *reinterpret_cast<uint4*>(dst + e * 8) = *reinterpret_cast<const uint4*>(v);
+    }
+}
+
+struct Wave { int begin, count; };
+
+// Consecutive query tiles are grouped while the causal part of their score planes stays within kWaveBytes.
+int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves) {
+    const int n_qt = (N + kTile - 1) / kTile;
+    const size_t per_col_tile = (size_t)B * Hq * kTile * kTile * 2 * c;
+    int n = 0, qt = 0;
+    while (qt < n_qt) {
+        size_t bytes = 0;
+        int cnt = 0;
+        while (qt + cnt < n_qt && (cnt == 0 || bytes + per_col_tile * (qt + cnt + 1) <= kWaveBytes)) {
+            bytes += per_col_tile * (qt + cnt + 1);
+            ++cnt;
+        }
+        if (waves && n < max_waves) waves[n] = Wave{qt, cnt};
+        ++n;
+        qt += cnt;
+    }
+    return n;
+}
+
+struct Layout {
+    size_t qp_off[kMaxChain], kp_off[kMaxChain], plane_off[kMaxChain];
+    int64_t plane_rows, plane_cols;
+    size_t total;
+};
+
+Layout plan_layout(const lisa_shared_prefill_args& a) {
+    Layout l{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 1023) & ~(size_t)1023; return o; };
+    for (int k = 0; k < a.chain_len; ++k) {
+        l.qp_off[k] = take((size_t)a.B * a.Hq * a.N * kPadRank * 2);
+        l.kp_off[k] = take((size_t)a.B * a.Hkv * a.N * kPadRank * 2);
+    }
+    const int n_qt = (a.N + kTile - 1) / kTile;
+    Wave waves[1024];
+    const int nw = plan_waves(a.B, a.N, a.Hq, a.chain_len, waves, 1024);
+    int max_cnt = 1;
+    for (int i = 0; i < std::min(nw, 1024); ++i) max_cnt = std::max(max_cnt, waves[i].count);
+    l.plane_rows = (int64_t)max_cnt * kTile;
+    l.plane_cols = (int64_t)n_qt * kTile;
+    for (int k = 0; k < a.chain_len; ++k) l.plane_off[k] = take((size_t)a.B * a.Hq * l.plane_rows * l.plane_cols * 2);
+    l.total = off;
+    return l;
+}
+
+lisa_tensor packed_view(void* ptr, int H, int N) {
+    return lisa_tensor{ptr, LISA_BF16, 0, (int64_t)H * N * kPadRank, (int64_t)kPadRank, (int64_t)N * kPadRank};
+}
+
+}  // namespace
+
+cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int r, void* dst, cudaStream_t s) {
+    const int64_t total = (int64_t)B * H * N * (kPadRank / 8);
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 32);
+    pack_lowrank_kernel<<<blocks, 256, 0, s>>>(make_view(src), B, N, H, r, reinterpret_cast<__nv_bfloat16*>(dst));
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+bool tc_shared_prefill_supported(const lisa_shared_prefill_args& a) {
+    if (a.d != 128 || a.chain_len < 1 || a.N > kTile * 1024) return false;
+    if (!tc_align_supported(a.Hq, a.links, a.chain_len)) return false;
+    for (int k = 0; k < a.chain_len; ++k)
+        if (a.links[k].qp.dtype != LISA_BF16 || a.links[k].kp.dtype != LISA_BF16 || a.links[k].r > 32) return false;
+    TcFlashArgs f{a.B, a.N, a.Hq, a.Hkv, 128, a.q0, a.k0, a.v, a.o, 1.f, nullptr, 0, 0, 0, 1};
+    return tc_flash_supported(f);
+}
+
+// + 1024: the launch aligns the caller's pointer up to the 1024 bytes the swizzled tiles need
+size_t tc_shared_prefill_workspace(const lisa_shared_prefill_args& a) { return plan_layout(a).total + 1024; }
+
+cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws, cudaStream_t s) {
+    const Layout l = plan_layout(a);
+    char* base = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(ws) + 1023) & ~(uintptr_t)1023);
+    const int c = a.chain_len;
+    cudaError_t e;
+    for (int k = 0; k < c; ++k) {
+        if ((e = launch_pack_lowrank(a.links[k].qp, a.B, a.N, a.Hq, a.links[k].r, base + l.qp_off[k], s)) != cudaSuccess) return e;
+        if ((e = launch_pack_lowrank(a.links[k].kp, a.B, a.N, a.Hkv, a.links[k].r, base + l.kp_off[k], s)) != cudaSuccess) return e;
+    }
+    Wave waves[1024];
+    const int nw = plan_waves(a.B, a.N, a.Hq, c, waves, 1024);
+    for (int w = 0; w < nw; ++w) {
+        const Wave wv = waves[w];
+        // 1. anchor scores and the differences of the links below the top one
+        TcFlashArgs f{a.B, a.N, a.Hq, a.Hkv, 128, a.q0, a.k0, a.v, a.o, 1.f / sqrtf((float)a.d), nullptr, l.plane_rows, l.plane_cols,
+                      wv.begin, wv.count};
+        f.emit_plane = base + l.plane_off[0];
+        if ((e = launch_tc_flash(f, s)) != cudaSuccess) return e;
+        for (int k = 0; k + 1 < c; ++k) {
+            TcFlashArgs fd = f;
+            fd.kd = kPadRank;
+            fd.qa = packed_view(base + l.qp_off[k], a.Hq, a.N);
+            fd.ka = packed_view(base + l.kp_off[k], a.Hkv, a.N);
+            fd.scale = 1.f / sqrtf((float)a.links[k].r);
+            fd.ksteps = (a.links[k].r + 15) / 16;
+            fd.emit_plane = base + l.plane_off[k + 1];
+            if ((e = launch_tc_flash(fd, s)) != cudaSuccess) return e;
+        }
+        // 2. the FFN chain over the head axis, in place
+        TcAlignArgs al{};
+        al.B = a.B; al.N = a.N; al.chain = c; al.qt_begin = wv.begin; al.qt_count = wv.count;
+        al.plane_rows = l.plane_rows; al.plane_cols = l.plane_cols;
+        for (int k = 0; k < c; ++k) al.planes[k] = base + l.plane_off[k];
+        al.links = a.links;
+        if ((e = launch_tc_align(al, s)) != cudaSuccess) return e;
+        // 3. this layer's own difference, softmax and .V
+        TcFlashArgs fv = f;
+        fv.emit_plane = nullptr;
+        fv.kd = kPadRank;
+        fv.qa = packed_view(base + l.qp_off[c - 1], a.Hq, a.N);
+        fv.ka = packed_view(base + l.kp_off[c - 1], a.Hkv, a.N);
+        fv.scale = 1.f / sqrtf((float)a.links[c - 1].r);
+        fv.ksteps = (a.links[c - 1].r + 15) / 16;
+        fv.plane = base + l.plane_off[0];
+        if ((e = launch_tc_flash(fv, s)) != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace lisa

@@ -28,3 +28,31 @@ def test_anchor_prefill_tensor_core(B, N, Hq, Hkv):
     finally:
         lb.lisa_force_general_kernels(False)
     assert_close(gen.float().cpu().numpy(), ref, "bf16", "general anchor prefill")
+
+
+def run_tc_shared(B, N, Hkv, chain, act, seed=0, bias=False, r=21):
+    w = synth.Workload("tc_shared", "bf16", B, N, 32, Hkv, 128, r, 64, act, chain)
+    t = synth.prefill_inputs(w, seed)
+    if bias:
+        for k in range(1, chain + 1):
+            t[f"b1_{k}"] = synth.as_dtype(synth.normal(f"b1_{k}", (64,), seed, std=0.5), "bf16")
+            t[f"b2_{k}"] = synth.as_dtype(synth.normal(f"b2_{k}", (32,), seed, std=0.5), "bf16")
+    dl, ol = make_links(t, chain, act, bias=bias)
+    n0 = lb.lisa_kernel_launches()
+    got = lb.lisa_attn_shared_prefill(dev(t["q0"]), dev(t["k0"]), dl, dev(t[f"v{chain}"]))
+    torch.cuda.synchronize()
+    assert lb.lisa_kernel_launches() - n0 >= 2 * chain + 3      # pack x2 per link, emit, align, attention
+    assert lb.lisa_check() == lb.OK
+    ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{chain}"]), ol)
+    return assert_close(got.float().cpu().numpy(), ref, "bf16", "tensor-core shared prefill N=%d c=%d" % (N, chain))
+
+
+@pytest.mark.parametrize("B,N,Hkv,chain,act", [(1, 128, 32, 1, "relu"), (1, 256, 32, 1, "silu"), (2, 300, 8, 1, "relu"),
+                                                 (1, 200, 32, 2, "relu"), (1, 513, 8, 3, "silu"), (1, 130, 32, 4, "none")])
+def test_shared_prefill_tensor_core(B, N, Hkv, chain, act):
+    run_tc_shared(B, N, Hkv, chain, act)
+
+
+def test_shared_prefill_tensor_core_bias_and_rank():
+    run_tc_shared(1, 260, 32, 2, "relu", seed=3, bias=True, r=32)
+    run_tc_shared(1, 140, 32, 1, "silu", seed=4, bias=True, r=8)
