@@ -197,8 +197,10 @@ def main():
     out = torch.empty_like(d["q0"])
     cache = lb.KVCacheLayer(lb.CACHE_SHARED, w.B, w.Hkv, w.N, w.d, w.r)
 
+    pws = lb._workspace(lb.OP_SHARED_PREFILL, lb._prefill_args(d["q0"], d["k0"], [link], d["v1"], out)[0])
+
     def prefill_step():
-        lb.lisa_attn_shared_prefill(d["q0"], d["k0"], [link], d["v1"], out=out)
+        lb.lisa_attn_shared_prefill(d["q0"], d["k0"], [link], d["v1"], out=out, workspace=pws)
         ev = torch.cuda.Event(enable_timing=True)
         ev.record()
         lb.lisa_kvcache_append(cache, d["kp1"], d["v1"])

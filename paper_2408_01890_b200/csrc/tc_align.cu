@@ -1,6 +1,7 @@
 // Head-axis aligner on tensor cores (Sec. 5.1): the FFN chain of a shared layer applied to score planes.
 //
-// Input: bf16 planes [B*Hq][rows][cols] holding A_0 = Q0.K0^T/sqrt(d) (Eq. 2) and, for chain depth c > 1, the
+// Input: fp16 planes [B*Hq][rows][cols] (fp16, not bf16: three more mantissa bits keep a chain of several links
+// inside the accuracy bar; scores are O(10), far from fp16's range limit, and conversions saturate) holding A_0 = Q0.K0^T/sqrt(d) (Eq. 2) and, for chain depth c > 1, the
 // already scaled differences D_k = Q'_k.K'_k^T/sqrt(r) (Eq. 3) of the links k < c.  Output, in place of the A_0
 // plane: Y = FFN_c(A_{c-1}) where A_k = FFN_k(A_{k-1}) + D_k (Eq. 4, ADD) -- the final link's D_c is added by the
 // attention kernel that consumes Y.  Hq = 32 heads, hidden width 64, two-layer FFNs.
@@ -9,7 +10,7 @@
 //   H  [128 x 64] = A [128 x 32] . W1 [32 x 64]     A read MN-major straight from the [head][position] planes
 //   Y  [128 x 32] = act(H + b1) [128 x 64] . W2 [64 x 32]  (+ D_k [128 x 32] . I [32 x 32] for k < c)
 // so the tensor core does the [head][position] -> [position][head] transposition.  One thread per position
-// applies bias and activation between the two MMAs and writes the result planes.
+// applies bias and activation between the two MMAs and writes the result planes.  Weights are converted to fp16.
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -31,7 +32,7 @@ struct AlignParams {
     int B, N, chain;         // chain = number of links applied here (c)
     int row0, qt_begin;      // planes hold query rows row0.. ; tiles [qt_begin, qt_begin + gridDim.y)
     int64_t plane_rows, plane_cols;
-    __nv_bfloat16* planes[kMaxTcChain];  // [0] = A_0 in / Y out; [k] = D_k for k = 1..c-1
+    __half* planes[kMaxTcChain];  // [0] = A_0 in / Y out; [k] = D_k for k = 1..c-1
     const void *w1[kMaxTcChain], *b1[kMaxTcChain], *w2[kMaxTcChain], *b2[kMaxTcChain];
     int w_dtype[kMaxTcChain], act[kMaxTcChain];
     int* status;
@@ -86,17 +87,15 @@ tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ T
     for (int e = tid; e < AT_BYTES / 16; e += kThreads) reinterpret_cast<uint4*>(sA)[e] = make_uint4(0, 0, 0, 0);
     __syncthreads();
     for (int e = tid; e < HQ; e += kThreads)  // identity: row g, k-slot g
-        *reinterpret_cast<__nv_bfloat16*>(sI + sw128_offset(e, e >> 3) + (e & 7) * 2) = __float2bfloat16_rn(1.f);
+        *reinterpret_cast<__half*>(sI + sw128_offset(e, e >> 3) + (e & 7) * 2) = __float2half_rn(1.f);
     for (int k = 0; k < c; ++k) {
         uint8_t* w1t = sW + k * (W1_BYTES + W2_BYTES);
         uint8_t* w2t = w1t + W1_BYTES;
         for (int e = tid; e < HQ * MH; e += kThreads) {
             const int hh = e / MH, u = e % MH;  // W1[hh][u] -> row u, k-slot hh
-            *reinterpret_cast<__nv_bfloat16*>(w1t + sw128_offset(u, hh >> 3) + (hh & 7) * 2) =
-                __float2bfloat16_rn(ld_elem(p.w1[k], e, p.w_dtype[k]));
+            *reinterpret_cast<__half*>(w1t + sw128_offset(u, hh >> 3) + (hh & 7) * 2) = __float2half_rn(ld_elem(p.w1[k], e, p.w_dtype[k]));
             const int u2 = e / HQ, gg = e % HQ;  // W2[u2][gg] -> row gg, k-slot u2
-            *reinterpret_cast<__nv_bfloat16*>(w2t + sw128_offset(gg, u2 >> 3) + (u2 & 7) * 2) =
-                __float2bfloat16_rn(ld_elem(p.w2[k], e, p.w_dtype[k]));
+            *reinterpret_cast<__half*>(w2t + sw128_offset(gg, u2 >> 3) + (u2 & 7) * 2) = __float2half_rn(ld_elem(p.w2[k], e, p.w_dtype[k]));
         }
         for (int e = tid; e < MH; e += kThreads) sBias[k * (MH + HQ) + e] = ldw(p.b1[k], e, p.w_dtype[k]);
         for (int e = tid; e < HQ; e += kThreads) sBias[k * (MH + HQ) + MH + e] = ldw(p.b2[k], e, p.w_dtype[k]);
@@ -109,10 +108,10 @@ tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ T
     const uint32_t tmem_D1 = tmem_base, tmem_D2 = tmem_base + 64;
     const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
 
-    constexpr uint32_t IDESC_1_MN = umma_idesc_bf16(UNIT, MH, 1, 0);
-    constexpr uint32_t IDESC_1_K = umma_idesc_bf16(UNIT, MH, 0, 0);
-    constexpr uint32_t IDESC_2 = umma_idesc_bf16(UNIT, HQ, 0, 0);
-    constexpr uint32_t IDESC_ID = umma_idesc_bf16(UNIT, HQ, 1, 0);
+    constexpr uint32_t IDESC_1_MN = umma_idesc_f16(UNIT, MH, 1, 0);
+    constexpr uint32_t IDESC_1_K = umma_idesc_f16(UNIT, MH, 0, 0);
+    constexpr uint32_t IDESC_2 = umma_idesc_f16(UNIT, HQ, 0, 0);
+    constexpr uint32_t IDESC_ID = umma_idesc_f16(UNIT, HQ, 1, 0);
 
     auto issue_loads = [&](int u, int stage) {  // thread 0 only
         const int row = qt * UNIT + u / nblk - p.row0, col = (u % nblk) * UNIT;
@@ -155,7 +154,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ T
             if (!(ok = mbar_wait(mma_bar, mma_phase, abort_flag))) break;
             mma_phase ^= 1;
             tc_fence_after();
-            // hidden layer: bias, activation, bf16, into the K-major H tile (row = this thread's position)
+            // hidden layer: bias, activation, fp16, into the K-major H tile (row = this thread's position)
 #pragma unroll
             for (int cc = 0; cc < 2; ++cc) {
                 uint32_t hr[32];
@@ -167,7 +166,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ T
 #pragma unroll
                     for (int j = 0; j < 8; ++j) e[j] = act_fast(__uint_as_float(hr[q * 8 + j]) + b1[cc * 32 + q * 8 + j], p.act[k]);
                     uint4 v;
-                    v.x = pack_bf16(e[0], e[1]); v.y = pack_bf16(e[2], e[3]); v.z = pack_bf16(e[4], e[5]); v.w = pack_bf16(e[6], e[7]);
+                    v.x = pack_f16(e[0], e[1]); v.y = pack_f16(e[2], e[3]); v.z = pack_f16(e[4], e[5]); v.w = pack_f16(e[6], e[7]);
                     *reinterpret_cast<uint4*>(sH + sw128_offset(tid, cc * 4 + q)) = v;
                 }
             }
@@ -200,20 +199,20 @@ tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ T
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     uint4 v;
-                    v.x = pack_bf16(__uint_as_float(yr[q * 8 + 0]) + b2[q * 8 + 0], __uint_as_float(yr[q * 8 + 1]) + b2[q * 8 + 1]);
-                    v.y = pack_bf16(__uint_as_float(yr[q * 8 + 2]) + b2[q * 8 + 2], __uint_as_float(yr[q * 8 + 3]) + b2[q * 8 + 3]);
-                    v.z = pack_bf16(__uint_as_float(yr[q * 8 + 4]) + b2[q * 8 + 4], __uint_as_float(yr[q * 8 + 5]) + b2[q * 8 + 5]);
-                    v.w = pack_bf16(__uint_as_float(yr[q * 8 + 6]) + b2[q * 8 + 6], __uint_as_float(yr[q * 8 + 7]) + b2[q * 8 + 7]);
+                    v.x = pack_f16(__uint_as_float(yr[q * 8 + 0]) + b2[q * 8 + 0], __uint_as_float(yr[q * 8 + 1]) + b2[q * 8 + 1]);
+                    v.y = pack_f16(__uint_as_float(yr[q * 8 + 2]) + b2[q * 8 + 2], __uint_as_float(yr[q * 8 + 3]) + b2[q * 8 + 3]);
+                    v.z = pack_f16(__uint_as_float(yr[q * 8 + 4]) + b2[q * 8 + 4], __uint_as_float(yr[q * 8 + 5]) + b2[q * 8 + 5]);
+                    v.w = pack_f16(__uint_as_float(yr[q * 8 + 6]) + b2[q * 8 + 6], __uint_as_float(yr[q * 8 + 7]) + b2[q * 8 + 7]);
                     *reinterpret_cast<uint4*>(sA + sw128_offset(tid, q)) = v;
                 }
                 fence_async_smem();
                 tc_fence_before();
                 __syncthreads();
             } else {
-                __nv_bfloat16* dst = p.planes[0] + ((int64_t)(b * HQ) * p.plane_rows + (row_g - p.row0)) * p.plane_cols + col0 + tid;
+                __half* dst = p.planes[0] + ((int64_t)(b * HQ) * p.plane_rows + (row_g - p.row0)) * p.plane_cols + col0 + tid;
                 const int64_t hstride = p.plane_rows * p.plane_cols;
 #pragma unroll
-                for (int g = 0; g < HQ; ++g) dst[g * hstride] = __float2bfloat16_rn(__uint_as_float(yr[g]) + b2[g]);
+                for (int g = 0; g < HQ; ++g) dst[g * hstride] = __float2half_rn(__uint_as_float(yr[g]) + b2[g]);
             }
         }
         // all reads of this stage's slabs (by the MMAs, now complete) and of D1/D2 are done before the
@@ -259,14 +258,14 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     p.row0 = a.qt_begin * UNIT; p.qt_begin = a.qt_begin;
     p.plane_rows = a.plane_rows; p.plane_cols = a.plane_cols;
     for (int k = 0; k < a.chain; ++k) {
-        p.planes[k] = reinterpret_cast<__nv_bfloat16*>(a.planes[k]);
+        p.planes[k] = reinterpret_cast<__half*>(a.planes[k]);
         const lisa_link& l = a.links[k];
         p.w1[k] = l.w1; p.b1[k] = l.b1; p.w2[k] = l.w2; p.b2[k] = l.b2;
         p.w_dtype[k] = l.w_dtype; p.act[k] = l.act;
         const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * HQ};
         const uint64_t str[2] = {(uint64_t)a.plane_cols * 2, (uint64_t)a.plane_cols * a.plane_rows * 2};
         const uint32_t box[3] = {64, 1, HQ};
-        if (!make_tensor_map_bf16(&maps.m[k], a.planes[k], 3, dims, str, box)) return cudaErrorInvalidValue;
+        if (!make_tensor_map_bf16(&maps.m[k], a.planes[k], 3, dims, str, box, true)) return cudaErrorInvalidValue;
     }
     for (int k = a.chain; k < kMaxTcChain; ++k) maps.m[k] = maps.m[0];
     p.status = status_words();

@@ -2,7 +2,7 @@
 //
 // One CTA per (batch b, query head h, 128-row query tile).  For every key tile j <= the query tile:
 //   scores  S = QA . KA^T            tcgen05.mma, fp32 accumulator in tensor memory
-//   logits  A = S * scale (+ Y)      Y: optional bf16 tile of pre-computed scores (the aligned part of a
+//   logits  A = S * scale (+ Y)      Y: optional fp16 tile of pre-computed scores (the aligned part of a
 //                                    shared layer, Eq. 4; then QA/KA are the layer's low-rank Q'/K', Eq. 3)
 //   causal mask (diagonal tile), online softmax in registers (one thread per query row), P as bf16
 //   O += P . V                       tcgen05.mma, V read MN-major straight from its [key][d] tile
@@ -40,12 +40,12 @@ struct FlashParams {
     int qt_begin;    // this launch covers query tiles [qt_begin, qt_begin + gridDim.x)
     int ksteps;      // 16-wide k-steps of the score MMA actually issued (<= KD/16; the rest is zero padding)
     float scale;     // MODE_EMIT: scores are multiplied by this before rounding to bf16
-    __nv_bfloat16* plane_out;  // MODE_EMIT: [B*Hq][plane_rows][plane_cols]
+    __half* plane_out;  // MODE_EMIT: fp16 [B*Hq][plane_rows][plane_cols]
     int64_t plane_rows, plane_cols;
 };
 
 // MODE_ATTN: softmax(QA.KA^T).V;  MODE_ATTN_PLANE: the same with the pre-computed tile Y added to the logits;
-// MODE_EMIT: no softmax, the scaled scores are written as bf16 to the plane workspace (for the aligner kernel).
+// MODE_EMIT: no softmax, the scaled scores are written as fp16 to the plane workspace (for the aligner kernel).
 constexpr int MODE_ATTN = 0, MODE_ATTN_PLANE = 1, MODE_EMIT = 2;
 
 template <int KD, int MODE>
@@ -203,14 +203,14 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             float* sf = reinterpret_cast<float*>(sr);
             if constexpr (EMIT) {
                 if (qi < p.N) {
-                    __nv_bfloat16* dst = p.plane_out + ((int64_t)(b * p.Hq + h) * p.plane_rows + (qi - p.plane_row0)) * p.plane_cols + t * BN;
+                    __half* dst = p.plane_out + ((int64_t)(b * p.Hq + h) * p.plane_rows + (qi - p.plane_row0)) * p.plane_cols + t * BN;
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
                         uint4 v;
-                        v.x = pack_bf16(sf[c * 8 + 0] * p.scale, sf[c * 8 + 1] * p.scale);
-                        v.y = pack_bf16(sf[c * 8 + 2] * p.scale, sf[c * 8 + 3] * p.scale);
-                        v.z = pack_bf16(sf[c * 8 + 4] * p.scale, sf[c * 8 + 5] * p.scale);
-                        v.w = pack_bf16(sf[c * 8 + 6] * p.scale, sf[c * 8 + 7] * p.scale);
+                        v.x = pack_f16(sf[c * 8 + 0] * p.scale, sf[c * 8 + 1] * p.scale);
+                        v.y = pack_f16(sf[c * 8 + 2] * p.scale, sf[c * 8 + 3] * p.scale);
+                        v.z = pack_f16(sf[c * 8 + 4] * p.scale, sf[c * 8 + 5] * p.scale);
+                        v.w = pack_f16(sf[c * 8 + 6] * p.scale, sf[c * 8 + 7] * p.scale);
                         *reinterpret_cast<uint4*>(dst + c * 8) = v;
                     }
                 }
@@ -225,9 +225,9 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                     const uint32_t w[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        sf[c * 8 + 2 * e] = fmaf(sf[c * 8 + 2 * e], p.scale_log2, __uint_as_float(w[e] << 16) * 1.4426950408889634f);
-                        sf[c * 8 + 2 * e + 1] =
-                            fmaf(sf[c * 8 + 2 * e + 1], p.scale_log2, __uint_as_float(w[e] & 0xffff0000u) * 1.4426950408889634f);
+                        const float2 yv = unpack_f16(w[e]);
+                        sf[c * 8 + 2 * e] = fmaf(sf[c * 8 + 2 * e], p.scale_log2, yv.x * 1.4426950408889634f);
+                        sf[c * 8 + 2 * e + 1] = fmaf(sf[c * 8 + 2 * e + 1], p.scale_log2, yv.y * 1.4426950408889634f);
                     }
                 }
             } else {
@@ -329,7 +329,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
 
 
 bool make_tensor_map_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                          const uint32_t* box) {
+                          const uint32_t* box, bool fp16) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -346,7 +346,7 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* base, int rank, const ui
     cuuint32_t gbox[5], estr[5];
     for (int i = 0; i < rank; ++i) { gdims[i] = dims[i]; gbox[i] = box[i]; estr[i] = 1; }
     for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
-    return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdims, gstr, gbox, estr,
+    return encode(map, fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdims, gstr, gbox, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -379,7 +379,7 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
         const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * a.Hq};
         const uint64_t str[2] = {(uint64_t)a.plane_cols * 2, (uint64_t)a.plane_cols * a.plane_rows * 2};
         const uint32_t box[3] = {64, 128, 1};
-        if (!make_tensor_map_bf16(&tmY, a.plane, 3, dims, str, box)) return cudaErrorInvalidValue;
+        if (!make_tensor_map_bf16(&tmY, a.plane, 3, dims, str, box, true)) return cudaErrorInvalidValue;
     }
     FlashParams p;
     p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv;
@@ -392,7 +392,7 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     p.qt_begin = a.qt_begin;
     p.ksteps = a.ksteps > 0 ? a.ksteps : a.kd / 16;
     p.scale = a.scale;
-    p.plane_out = reinterpret_cast<__nv_bfloat16*>(a.emit_plane);
+    p.plane_out = reinterpret_cast<__half*>(a.emit_plane);
     p.plane_rows = a.plane_rows; p.plane_cols = a.plane_cols;
     dim3 grid(a.qt_count, a.Hq, a.B);
     cudaError_t e;
