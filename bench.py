@@ -213,7 +213,6 @@ def main():
     l0 = lb.lisa_kernel_launches()
     total_ms, starts, marks = time_steps(prefill_step, args.steps, flush, barrier)
     launches = lb.lisa_kernel_launches() - l0
-    clocks = sampler.stop()
     kernel_ms = sum(s.elapsed_time(m) for s, m in zip(starts, marks)) / args.steps
     total_ms = max_over_ranks(total_ms)
     ms_per_step = total_ms / args.steps
@@ -301,6 +300,8 @@ def main():
                   "shared": res["shared"], "standard": res["standard"],
                   "shared_over_standard": res["shared"]["value"] / res["standard"]["value"]}
         del sh, st, prev, row, ws
+
+    clocks = sampler.stop()  # sampled across all timed regions above (prefill, end-to-end, decode)
 
     # ---------------- the CPU oracle on the host cores (rank 0, N = 1 only) ----------------
     cpu = None

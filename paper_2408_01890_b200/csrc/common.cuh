@@ -91,7 +91,7 @@ struct TcAlignArgs {
     int64_t plane_rows, plane_cols;
     void* planes[4];
     const lisa_link* links;
-    int ctas_per_tile = 0;
+    int ctas = 0;  // grid size (0 = three per SM)
 };
 bool tc_align_supported(int Hq, const lisa_link* links, int chain);
 cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t s);

@@ -11,6 +11,8 @@
 //   Y  [128 x 32] = act(H + b1) [128 x 64] . W2 [64 x 32]  (+ D_k [128 x 32] . I [32 x 32] for k < c)
 // so the tensor core does the [head][position] -> [position][head] transposition.  One thread per position
 // applies bias and activation between the two MMAs and writes the result planes.  Weights are converted to fp16.
+#include <algorithm>
+
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -30,7 +32,9 @@ constexpr int kMaxTcChain = 4;
 
 struct AlignParams {
     int B, N, chain;         // chain = number of links applied here (c)
-    int row0, qt_begin;      // planes hold query rows row0.. ; tiles [qt_begin, qt_begin + gridDim.y)
+    int row0, qt_begin, qt_count;  // planes hold query rows row0.. ; this launch covers tiles [qt_begin, qt_begin + qt_count)
+    int stages;              // depth of the slab ring (2..4)
+    int units_per_batch;     // sum over the covered tiles of valid rows x key blocks
     int64_t plane_rows, plane_cols;
     __half* planes[kMaxTcChain];  // [0] = A_0 in / Y out; [k] = D_k for k = 1..c-1
     const void *w1[kMaxTcChain], *b1[kMaxTcChain], *w2[kMaxTcChain], *b2[kMaxTcChain];
@@ -55,28 +59,39 @@ tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ T
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int c = p.chain;
-    // layout: [stage 0 slabs (c)] [stage 1 slabs (c)] [H tile] [A tile] [identity] [W1,W2 per link] [biases] [barriers]
+    const int S = p.stages;
+    // layout: [S stages of c slabs] [H tile] [A tile] [identity] [W1,W2 per link] [biases] [barriers]
     uint8_t* sSlab = smem;
-    uint8_t* sH = sSlab + 2 * c * SLAB_BYTES;
+    uint8_t* sH = sSlab + S * c * SLAB_BYTES;
     uint8_t* sA = sH + AT_BYTES;
     uint8_t* sI = sA + AT_BYTES;
     uint8_t* sW = sI + W2_BYTES;
     float* sBias = reinterpret_cast<float*>(sW + c * (W1_BYTES + W2_BYTES));  // per link: b1[64], b2[32]
     uint64_t* bars = reinterpret_cast<uint64_t*>(sBias + c * (MH + HQ));
-    uint64_t* full = bars;      // [2]
-    uint64_t* mma_bar = bars + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 4);
+    uint64_t* full = bars;      // [4]
+    uint64_t* mma_bar = bars + 4;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 6);
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int qt = p.qt_begin + blockIdx.y, b = blockIdx.z;
-    const int nblk = qt + 1;
-    const int rows_valid = min(UNIT, p.N - qt * UNIT);
-    const int n_units = rows_valid * nblk;
+    const int n_units = p.units_per_batch * p.B;
+    // unit index -> (batch, query row, first key column): units are numbered tile by tile, row by row
+    auto decode = [&](int u, int& b, int& row_g, int& col0) {
+        b = u / p.units_per_batch;
+        int rem = u - b * p.units_per_batch;
+        int t = p.qt_begin;
+        for (;; ++t) {
+            const int n_t = min(UNIT, p.N - t * UNIT) * (t + 1);
+            if (rem < n_t || t + 1 >= p.qt_begin + p.qt_count) break;
+            rem -= n_t;
+        }
+        row_g = t * UNIT + rem / (t + 1);
+        col0 = (rem % (t + 1)) * UNIT;
+    };
 
     // ---- one-time set-up: barriers, TMEM, weights as swizzled MMA operands ----
     if (tid == 0) {
-        mbar_init(full + 0, 1); mbar_init(full + 1, 1);
+        for (int i = 0; i < 4; ++i) mbar_init(full + i, 1);
         mbar_init(mma_bar, 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -114,26 +129,30 @@ tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ T
     constexpr uint32_t IDESC_ID = umma_idesc_f16(UNIT, HQ, 1, 0);
 
     auto issue_loads = [&](int u, int stage) {  // thread 0 only
-        const int row = qt * UNIT + u / nblk - p.row0, col = (u % nblk) * UNIT;
+        int b, row_g, col0;
+        decode(u, b, row_g, col0);
         mbar_expect_tx(full + stage, c * SLAB_BYTES);
         for (int k = 0; k < c; ++k)
             for (int half = 0; half < 2; ++half)
-                tma_load_3d(sSlab + (stage * c + k) * SLAB_BYTES + half * (HQ * 128), &maps.m[k], full + stage, col + half * 64, row,
-                            b * HQ);
+                tma_load_3d(sSlab + (stage * c + k) * SLAB_BYTES + half * (HQ * 128), &maps.m[k], full + stage, col0 + half * 64,
+                            row_g - p.row0, b * HQ);
     };
 
     uint32_t mma_phase = 0;
     bool ok = true;
     int it = 0;
-    if (tid == 0 && (int)blockIdx.x < n_units) issue_loads(blockIdx.x, 0);
+    if (tid == 0)
+        for (int i = 0; i < S - 1; ++i)
+            if ((int)blockIdx.x + i * (int)gridDim.x < n_units) issue_loads(blockIdx.x + i * gridDim.x, i);
     for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x, ++it) {
-        const int stage = it & 1;
-        const int un = u + gridDim.x;
-        // every thread finished reading the other stage's slabs and D2 of the previous unit before this point
-        if (tid == 0 && un < n_units) issue_loads(un, stage ^ 1);
-        if (!(ok = mbar_wait(full + stage, (it >> 1) & 1, abort_flag))) break;
+        const int stage = it % S;
+        const int un = u + (S - 1) * gridDim.x;
+        // the stage refilled here held unit it-1, whose slabs and results every thread is done with (loop-end barrier)
+        if (tid == 0 && un < n_units) issue_loads(un, (it + S - 1) % S);
+        if (!(ok = mbar_wait(full + stage, (it / S) & 1, abort_flag))) break;
+        int b, row_g, col0;
+        decode(u, b, row_g, col0);
         const uint8_t* slabs = sSlab + stage * c * SLAB_BYTES;
-        const int row_g = qt * UNIT + u / nblk, col0 = (u % nblk) * UNIT;
         for (int k = 0; k < c; ++k) {
             const uint8_t* w1t = sW + k * (W1_BYTES + W2_BYTES);
             const uint8_t* w2t = w1t + W1_BYTES;
@@ -235,8 +254,8 @@ tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ T
     }
 }
 
-size_t align_smem_bytes(int c) {
-    return (size_t)2 * c * SLAB_BYTES + 2 * AT_BYTES + W2_BYTES + (size_t)c * (W1_BYTES + W2_BYTES) + (size_t)c * (MH + HQ) * 4 + 64 + 1024;
+size_t align_smem_bytes(int c, int stages) {
+    return (size_t)stages * c * SLAB_BYTES + 2 * AT_BYTES + W2_BYTES + (size_t)c * (W1_BYTES + W2_BYTES) + (size_t)c * (MH + HQ) * 4 + 64 + 1024;
 }
 
 }  // namespace
@@ -255,7 +274,10 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     AlignParams p{};
     TensorMaps maps;
     p.B = a.B; p.N = a.N; p.chain = a.chain;
-    p.row0 = a.qt_begin * UNIT; p.qt_begin = a.qt_begin;
+    p.row0 = a.qt_begin * UNIT; p.qt_begin = a.qt_begin; p.qt_count = a.qt_count;
+    p.stages = a.chain == 1 ? 3 : 2;
+    p.units_per_batch = 0;
+    for (int t = a.qt_begin; t < a.qt_begin + a.qt_count; ++t) p.units_per_batch += std::min(UNIT, a.N - t * UNIT) * (t + 1);
     p.plane_rows = a.plane_rows; p.plane_cols = a.plane_cols;
     for (int k = 0; k < a.chain; ++k) {
         p.planes[k] = reinterpret_cast<__half*>(a.planes[k]);
@@ -270,10 +292,13 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     for (int k = a.chain; k < kMaxTcChain; ++k) maps.m[k] = maps.m[0];
     p.status = status_words();
     if (!p.status) return cudaErrorUnknown;
-    const size_t smem = align_smem_bytes(a.chain);
+    const size_t smem = align_smem_bytes(a.chain, p.stages);
     cudaError_t e = cudaFuncSetAttribute(tc_align_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    dim3 grid(a.ctas_per_tile > 0 ? a.ctas_per_tile : 16, a.qt_count, a.B);
+    const int64_t total_units = (int64_t)p.units_per_batch * a.B;
+    if (total_units <= 0 || total_units > 0x7fffffff) return cudaErrorInvalidValue;
+    const int max_ctas = a.ctas > 0 ? a.ctas : 148 * 3;
+    dim3 grid((unsigned)std::min<int64_t>(total_units, max_ctas));
     tc_align_kernel<<<grid, kThreads, smem, stream>>>(p, maps);
     count_launches(1);
     return cudaGetLastError();
