@@ -30,6 +30,7 @@ namespace {
 
 lisa_status_t cuda_fail(cudaError_t e) {
     t_last_cuda_error = (int)e;
+    (void)cudaGetLastError();  // do not let a non-sticky error leak into the next call's launch check
     return LISA_ERR_CUDA;
 }
 
