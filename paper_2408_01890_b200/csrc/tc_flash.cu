@@ -118,23 +118,33 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
 
     if (warp == 4) {
         // ------------------------------ TMA producer ------------------------------
-        if (lane == 0) {
-            tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
-            mbar_expect_tx(q_full, L::Q_BYTES);
-            for (int c = 0; c < KD / 64; ++c) tma_load_4d(sQ + c * (BM * 128), &tmQ, q_full, c * 64, h, q0, b);
-            for (int t = 0; t < nt; ++t) {
-                const int s = t & 1;
-                if (!mbar_wait(kv_empty + s, ((t >> 1) & 1) ^ 1, abort_flag)) break;
-                mbar_expect_tx(kv_full + s, L::K_BYTES + L::V_BYTES + L::Y_BYTES);
-                for (int c = 0; c < KD / 64; ++c) tma_load_4d(sK + s * L::K_BYTES + c * (BN * 128), &tmK, kv_full + s, c * 64, g, t * BN, b);
-                if constexpr (!EMIT)
-                    for (int c = 0; c < D / 64; ++c)
-                        tma_load_4d(sV + s * L::V_BYTES + c * (BN * 128), &tmV, kv_full + s, c * 64, g, t * BN, b);
-                if constexpr (PLANE)
-                    for (int c = 0; c < BN / 64; ++c)
-                        tma_load_3d(sY + s * L::Y_BYTES + c * (BM * 128), &tmY, kv_full + s, t * BN + c * 64, q0 - p.plane_row0,
-                                    b * p.Hq + h);
+        // Lane 0 waits for the stage and arms its barrier; then the copies of the stage are issued by different
+        // lanes of the warp at once (one 64-column box each): a single thread issuing them back to back is
+        // several hundred cycles slower per copy.
+        if (lane == 0) { tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); }
+        if (lane == 0) mbar_expect_tx(q_full, L::Q_BYTES);
+        __syncwarp();
+        if (lane < KD / 64) tma_load_4d(sQ + lane * (BM * 128), &tmQ, q_full, lane * 64, h, q0, b);
+        bool okp = true;
+        for (int t = 0; t < nt; ++t) {
+            const int s = t & 1;
+            if (lane == 0) {
+                okp = mbar_wait(kv_empty + s, ((t >> 1) & 1) ^ 1, abort_flag);
+                if (okp) mbar_expect_tx(kv_full + s, L::K_BYTES + L::V_BYTES + L::Y_BYTES);
             }
+            okp = __shfl_sync(0xffffffffu, okp, 0);
+            if (!okp) break;
+            constexpr int NK = KD / 64, NV = EMIT ? 0 : D / 64, NY = PLANE ? BN / 64 : 0;
+            if (lane < NK) {
+                tma_load_4d(sK + s * L::K_BYTES + lane * (BN * 128), &tmK, kv_full + s, lane * 64, g, t * BN, b);
+            } else if (lane < NK + NV) {
+                const int c = lane - NK;
+                tma_load_4d(sV + s * L::V_BYTES + c * (BN * 128), &tmV, kv_full + s, c * 64, g, t * BN, b);
+            } else if (lane < NK + NV + NY) {
+                const int c = lane - NK - NV;
+                tma_load_3d(sY + s * L::Y_BYTES + c * (BM * 128), &tmY, kv_full + s, t * BN + c * 64, q0 - p.plane_row0, b * p.Hq + h);
+            }
+            __syncwarp();
         }
     } else if (warp == 5) {
         // ------------------------------ MMA issuer ------------------------------

@@ -17,7 +17,12 @@ namespace {
 
 constexpr int kTile = 128;
 constexpr int kPadRank = 64;
-constexpr size_t kWaveBytes = (size_t)64 << 20;  // score-plane bytes one wave may touch (L2 is 126 MB)
+// A wave takes query tiles until its head-partitioned kernels have at least kWaveMinCtas CTAs (four per SM: with
+// fewer, the grids do not fill the GPU and launch and tail costs dominate) and then further tiles while the causal
+// part of its score planes stays within kWaveBytes.  Measured on B200: grid fill matters far more than keeping
+// the planes inside the 126 MB L2.
+constexpr size_t kWaveBytes = (size_t)256 << 20;
+constexpr int kWaveMinCtas = 4 * 148;
 
 __global__ void pack_lowrank_kernel(TView src, int B, int N, int H, int r, __nv_bfloat16* dst) {
     const int64_t total = (int64_t)B * H * N * (kPadRank / 8);
@@ -40,7 +45,6 @@ __global__ void pack_lowrank_kernel(TView src, int B, int N, int H, int r, __nv_
 
 struct Wave { int begin, count; };
 
-// Consecutive query tiles are grouped while the causal part of their score planes stays within kWaveBytes.
 int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves) {
     const int n_qt = (N + kTile - 1) / kTile;
     const size_t per_col_tile = (size_t)B * Hq * kTile * kTile * 2 * c;
@@ -48,7 +52,7 @@ int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves) {
     while (qt < n_qt) {
         size_t bytes = 0;
         int cnt = 0;
-        while (qt + cnt < n_qt && (cnt == 0 || bytes + per_col_tile * (qt + cnt + 1) <= kWaveBytes)) {
+        while (qt + cnt < n_qt && (B * Hq * cnt < kWaveMinCtas || bytes + per_col_tile * (qt + cnt + 1) <= kWaveBytes)) {
             bytes += per_col_tile * (qt + cnt + 1);
             ++cnt;
         }
