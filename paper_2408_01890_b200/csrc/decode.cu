@@ -58,6 +58,72 @@ __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float* f) {
 
 __device__ __forceinline__ float ldw(const void* p, int idx, int dtype) { return p ? ld_elem(p, idx, dtype) : 0.f; }
 
+// Partial P.V of a FULL chunk (all kChunk rows valid), bf16 cache, LPR = d/8 lanes per V row.  A warp streams the
+// V rows of its heads as one software-pipelined sequence: two register sets of eight 16-byte loads per lane
+// alternate, and the last batch of a head already prefetches the first batch of the warp's next head, so loads
+// stay in flight across batches and across heads.  All offsets are compile-time constants off one pointer.
+template <int LPR>
+__device__ __forceinline__ void pv_full_chunk(const DecodeParams& p, const float* s_s, int b, size_t part, int j0) {
+    constexpr int RSTEP = 32 / LPR;            // rows fetched by one warp-wide load
+    constexpr int NB = kChunk / RSTEP / 8;     // batches of 8 loads per head (even)
+    constexpr int D = LPR * 8;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane % LPR, rsel = lane / LPR;
+    const int Hq = p.Hq, G = p.Hq / p.Hkv;
+    auto head_ptr = [&](int h) {
+        return reinterpret_cast<const uint4*>(p.vcache) + (((size_t)b * p.Hkv + h / G) * p.L_cap + j0 + rsel) * LPR + sub;
+    };
+    if (warp >= Hq) return;
+    const uint4* hp = head_ptr(warp);
+    uint4 ra[8], rb[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) ra[u] = ld_stream16(hp + u * RSTEP * LPR);
+    for (int h = warp; h < Hq; h += kWarps) {
+        const bool has_next = h + kWarps < Hq;
+        const uint4* np = has_next ? head_ptr(h + kWarps) : hp;
+        const float* ps = s_s + h * kChunk + rsel;
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int bi = 0; bi < NB; bi += 2) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) rb[u] = ld_stream16(hp + ((bi + 1) * 8 + u) * RSTEP * LPR);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                float f[8];
+                bf16x8_to_f32(ra[u], f);
+                const float pj = ps[(bi * 8 + u) * RSTEP];
+#pragma unroll
+                for (int t = 0; t < 8; ++t) acc[t] = fmaf(pj, f[t], acc[t]);
+            }
+            if (bi + 2 < NB) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) ra[u] = ld_stream16(hp + ((bi + 2) * 8 + u) * RSTEP * LPR);
+            } else if (has_next) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) ra[u] = ld_stream16(np + u * RSTEP * LPR);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                float f[8];
+                bf16x8_to_f32(rb[u], f);
+                const float pj = ps[((bi + 1) * 8 + u) * RSTEP];
+#pragma unroll
+                for (int t = 0; t < 8; ++t) acc[t] = fmaf(pj, f[t], acc[t]);
+            }
+        }
+#pragma unroll
+        for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+            for (int t = 0; t < 8; ++t) acc[t] += __shfl_xor_sync(0xffffffffu, acc[t], off);
+        if (rsel == 0) {
+            float4* dst = reinterpret_cast<float4*>(p.ws_o + (part + h) * D + sub * 8);
+            dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+        }
+        hp = np;
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Phase B: s_s[h][kChunk] holds the chunk's scores (-inf beyond the sequence end). Produces the
 // chunk's (max, sum, unnormalised P.V) per head into the workspace.
@@ -93,42 +159,33 @@ __device__ __forceinline__ void softmax_pv_chunk(const DecodeParams& p, float* s
     __syncthreads();
     const int j0 = chunk * kChunk;
     if (p.cache_dtype == LISA_BF16) {
-        const int lpr = d / 8;          // lanes per V row (16 bytes each)
-        const int rstep = 32 / lpr;     // rows fetched by one warp-wide load
-        const int sub = lane % lpr, rsel = lane / lpr;
-        for (int h = warp; h < Hq; h += kWarps) {
-            const uint4* vbase = reinterpret_cast<const uint4*>(p.vcache) +
-                                 (((size_t)b * p.Hkv + h / G) * p.L_cap + j0) * lpr + sub;
-            const float* ps = s_s + h * kChunk;
-            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            int jj = rsel;
-            for (; jj + 7 * rstep < nrows; jj += 8 * rstep) {
-                uint4 raw[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) raw[u] = ld_stream16(vbase + (size_t)(jj + u * rstep) * lpr);
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
+        if (nrows == kChunk) {
+            if (d == 128) pv_full_chunk<16>(p, s_s, b, part, j0);
+            else if (d == 64) pv_full_chunk<8>(p, s_s, b, part, j0);
+            else pv_full_chunk<4>(p, s_s, b, part, j0);
+        } else {
+            // ragged last chunk of a sequence: plain loop
+            const int lpr = d / 8, rstep = 32 / lpr, sub = lane % lpr, rsel = lane / lpr;
+            for (int h = warp; h < Hq; h += kWarps) {
+                const uint4* vbase = reinterpret_cast<const uint4*>(p.vcache) +
+                                     (((size_t)b * p.Hkv + h / G) * p.L_cap + j0) * lpr + sub;
+                const float* ps = s_s + h * kChunk;
+                float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                for (int jj = rsel; jj < nrows; jj += rstep) {
                     float f[8];
-                    bf16x8_to_f32(raw[u], f);
-                    const float pj = ps[jj + u * rstep];
+                    bf16x8_to_f32(ld_stream16(vbase + (size_t)jj * lpr), f);
+                    const float pj = ps[jj];
 #pragma unroll
                     for (int t = 0; t < 8; ++t) acc[t] = fmaf(pj, f[t], acc[t]);
                 }
-            }
-            for (; jj < nrows; jj += rstep) {
-                float f[8];
-                bf16x8_to_f32(ld_stream16(vbase + (size_t)jj * lpr), f);
-                const float pj = ps[jj];
+                for (int off = lpr; off < 32; off <<= 1)
 #pragma unroll
-                for (int t = 0; t < 8; ++t) acc[t] = fmaf(pj, f[t], acc[t]);
-            }
-            for (int off = lpr; off < 32; off <<= 1)
-#pragma unroll
-                for (int t = 0; t < 8; ++t) acc[t] += __shfl_xor_sync(0xffffffffu, acc[t], off);
-            if (rsel == 0) {
-                float4* dst = reinterpret_cast<float4*>(p.ws_o + (part + h) * d + sub * 8);
-                dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-                dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+                    for (int t = 0; t < 8; ++t) acc[t] += __shfl_xor_sync(0xffffffffu, acc[t], off);
+                if (rsel == 0) {
+                    float4* dst = reinterpret_cast<float4*>(p.ws_o + (part + h) * d + sub * 8);
+                    dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+                    dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+                }
             }
         }
     } else {
@@ -191,12 +248,19 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
             if (j0 + j8 * 8 < p.L_cap) {
                 const __nv_bfloat16* base = reinterpret_cast<const __nv_bfloat16*>(p.kpT) +
                                             ((size_t)b * p.Hkv + h / G) * r * p.L_cap + j0 + j8 * 8;
-                for (int x = 0; x < r; ++x) {
-                    float f[8];
-                    bf16x8_to_f32(ld_stream16(base + (size_t)x * p.L_cap), f);
-                    const float qx = qp_s[h * kMaxRank + x];
+                for (int x0 = 0; x0 < r; x0 += 8) {   // eight independent 16-byte loads in flight per lane
+                    uint4 raw[8];
 #pragma unroll
-                    for (int t = 0; t < 8; ++t) acc[t] = fmaf(qx, f[t], acc[t]);
+                    for (int e = 0; e < 8; ++e)
+                        raw[e] = x0 + e < r ? ld_stream16(base + (size_t)(x0 + e) * p.L_cap) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        float f[8];
+                        bf16x8_to_f32(raw[e], f);
+                        const float qx = x0 + e < r ? qp_s[h * kMaxRank + x0 + e] : 0.f;
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) acc[t] = fmaf(qx, f[t], acc[t]);
+                    }
                 }
             }
             float4* dst = reinterpret_cast<float4*>(s_s + h * kChunk + j8 * 8);
