@@ -206,10 +206,10 @@ def main():
         lb.lisa_kvcache_append(cache, d["kp1"], d["v1"])
         return ev
 
+    sampler = ClockSampler(local)   # runs from the warm-up to the end of the last timed region
+    sampler.start()
     for _ in range(args.warmup):
         flush(); prefill_step()
-    sampler = ClockSampler(local)
-    sampler.start()
     l0 = lb.lisa_kernel_launches()
     total_ms, starts, marks = time_steps(prefill_step, args.steps, flush, barrier)
     launches = lb.lisa_kernel_launches() - l0
