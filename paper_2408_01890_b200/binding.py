@@ -191,12 +191,27 @@ def lisa_kvcache_append(cache: KVCacheLayer, k_or_kp: torch.Tensor, v: torch.Ten
                                       int(v.shape[1]), _stream()), "lisa_kvcache_append")
 
 
-def _workspace(op: int, args) -> Optional[torch.Tensor]:
+def _workspace_bytes(op: int, args) -> int:
     n = C.c_size_t()
     _check(load().lisa_workspace_bytes(op, C.byref(args), C.byref(n)), "lisa_workspace_bytes")
-    if n.value == 0:
+    return int(n.value)
+
+
+def _workspace(op: int, args) -> Optional[torch.Tensor]:
+    n = _workspace_bytes(op, args)
+    if n == 0:
         return None
-    return torch.empty(n.value, dtype=torch.uint8, device="cuda")
+    return torch.empty(n, dtype=torch.uint8, device="cuda")
+
+
+def decode_workspace_bytes(B: int, Hq: int, d: int, L: int) -> int:
+    """Scratch bytes of one decode call (shared or standard layer) for up to B sequences of up to L positions."""
+    cache = CCacheLayer(CACHE_SHARED, BF16, B, Hq, (L + 7) // 8 * 8, d, 1, 0, None, None)
+    a = SharedDecodeArgs()
+    a.struct_size = C.sizeof(SharedDecodeArgs)
+    a.B, a.Hq, a.L = B, Hq, L
+    a.cache = C.pointer(cache)
+    return _workspace_bytes(OP_SHARED_DECODE, a)
 
 
 def lisa_attn_anchor(q: torch.Tensor, k: Optional[torch.Tensor] = None, v: Optional[torch.Tensor] = None, *,

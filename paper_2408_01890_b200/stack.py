@@ -1,0 +1,153 @@
+"""A stack of attention layers driven through the library: prefill of a prompt, then token-by-token decode.
+
+Only orchestration lives here: which layer is standard and which is shared (Sec. 5.1 "Selecting layers": LiSA
+applied at intervals, each shared layer taking the scores of the layer before it), the per-layer caches
+(Sec. 5.2: a shared layer stores K_LR instead of K), the ping-pong score rows handed from layer to layer in
+decode, and timing.  Every layer's inputs are seeded synthetic tensors (the projections that would produce them
+lie outside the library).  All arithmetic runs in the library's kernels.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+from . import binding as lb
+from . import synth
+
+
+def default_standard_layers(n_layers: int = 32) -> List[int]:
+    """Layers 0-3 and every 4th layer thereafter are standard; the rest are shared, in chains of three."""
+    return sorted(set(range(4)) | set(range(3, n_layers, 4)))
+
+
+@dataclass
+class Probe:
+    """What to keep for checking against the oracle: layers, prefill rows (b, i), decode steps and sequences."""
+    layers: Sequence[int] = ()
+    rows_b: Sequence[int] = ()
+    rows_i: Sequence[int] = ()
+    steps: Sequence[int] = ()
+    seqs: Sequence[int] = ()
+    prefill: Dict[int, dict] = field(default_factory=dict)
+    decode: Dict[tuple, dict] = field(default_factory=dict)
+
+
+class AttentionStack:
+    def __init__(self, n_layers=32, standard_layers: Optional[Sequence[int]] = None, B=32, N=2048, T=256, Hq=32, Hkv=32,
+                 d=128, r=21, m=64, act="relu", seed=0):
+        self.n_layers, self.B, self.N, self.T = n_layers, B, N, T
+        self.Hq, self.Hkv, self.d, self.r, self.m, self.act, self.seed = Hq, Hkv, d, r, m, act, seed
+        std = set(default_standard_layers(n_layers) if standard_layers is None else standard_layers)
+        assert 0 in std, "layer 0 has no previous scores to share"
+        self.is_standard = [l in std for l in range(n_layers)]
+        self.L_cap = (N + T + 7) // 8 * 8
+        self.caches = [lb.KVCacheLayer(lb.CACHE_STANDARD if s else lb.CACHE_SHARED, B, Hkv, self.L_cap, d, 0 if s else r)
+                       for s in self.is_standard]
+        self.weights = {}
+        for l in range(n_layers):
+            if not self.is_standard[l]:
+                w1 = synth.as_dtype(synth.normal(f"w1/{l}", (Hq, m), seed, std=Hq ** -0.5), "bf16").cuda()
+                w2 = synth.as_dtype(synth.normal(f"w2/{l}", (m, Hq), seed, std=m ** -0.5), "bf16").cuda()
+                self.weights[l] = (w1, w2)
+        self.rows = [torch.empty((B, Hq, self.L_cap), dtype=torch.float32, device="cuda") for _ in range(2)]
+
+    def draw(self, name: str, layer: int, shape):
+        return synth.device_normal(f"{name}/{layer}", shape, self.seed)
+
+    def next_is_shared(self, l: int) -> bool:
+        return l + 1 < self.n_layers and not self.is_standard[l + 1]
+
+    # ------------------------------------------------------------------ prefill
+    def prefill(self, probe: Optional[Probe] = None) -> float:
+        """Runs every layer over the prompt and fills the caches. Returns the device time in milliseconds."""
+        B, N, Hq, Hkv, d, r = self.B, self.N, self.Hq, self.Hkv, self.d, self.r
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        out = torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device="cuda")
+        # every layer's inputs are drawn before the clock starts
+        drawn = []
+        for l in range(self.n_layers):
+            if self.is_standard[l]:
+                drawn.append((self.draw("q", l, (B, N, Hq, d)), self.draw("k", l, (B, N, Hkv, d)), self.draw("v", l, (B, N, Hkv, d))))
+            else:
+                drawn.append((self.draw("qp", l, (B, N, Hq, r)), self.draw("kp", l, (B, N, Hkv, r)),
+                              self.draw("v", l, (B, N, Hkv, d))))
+        ws = None
+        torch.cuda.synchronize()
+        t0.record()
+        q0 = k0 = None
+        links: List[lb.Link] = []
+        for l in range(self.n_layers):
+            a, b_, v = drawn[l]
+            if self.is_standard[l]:
+                lb.lisa_attn_anchor(a, b_, v, out=out)
+                lb.lisa_kvcache_append(self.caches[l], b_, v)
+                q0, k0, links = a, b_, []
+            else:
+                w1, w2 = self.weights[l]
+                links = links + [lb.Link(a, b_, w1, w2, act=lb.ACTS[self.act])]
+                args = lb._prefill_args(q0, k0, links, v, out)[0]
+                need = lb._workspace_bytes(lb.OP_SHARED_PREFILL, args)
+                if ws is None or ws.numel() < need:
+                    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+                lb.lisa_attn_shared_prefill(q0, k0, links, v, out=out, workspace=ws)
+                lb.lisa_kvcache_append(self.caches[l], b_, v)
+            if probe is not None and l in probe.layers:
+                rb = torch.tensor(list(probe.rows_b), device="cuda")
+                ri = torch.tensor(list(probe.rows_i), device="cuda")
+                seqs = sorted(set(probe.rows_b))
+                probe.prefill[l] = {
+                    "seqs": seqs, "out": out[rb, ri].float().cpu(), "q0": q0[seqs].cpu(), "k0": k0[seqs].cpu(), "v": v[seqs].cpu(),
+                    "links": [(lk.qp[seqs].cpu(), lk.kp[seqs].cpu(), lk.w1.cpu(), lk.w2.cpu()) for lk in links]}
+        t1.record()
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1)
+
+    # ------------------------------------------------------------------ decode
+    def decode(self, probe: Optional[Probe] = None) -> float:
+        """T decode steps through all layers (one new token per sequence and step). Returns milliseconds."""
+        B, N, T, Hq, Hkv, d, r = self.B, self.N, self.T, self.Hq, self.Hkv, self.d, self.r
+        new = []
+        for l in range(self.n_layers):
+            if self.is_standard[l]:
+                new.append((self.draw("dq", l, (B, 1, Hq, d)), self.draw("dk", l, (B, 1, Hkv, d)), self.draw("dv", l, (B, 1, Hkv, d))))
+            else:
+                new.append((self.draw("dqp", l, (B, 1, Hq, r)), self.draw("dkp", l, (B, 1, Hkv, r)), self.draw("dv", l, (B, 1, Hkv, d))))
+        out = torch.empty((B, 1, Hq, d), dtype=torch.bfloat16, device="cuda")
+        ws = torch.empty(lb.decode_workspace_bytes(B, Hq, d, self.L_cap), dtype=torch.uint8, device="cuda")
+        before = torch.empty((B,), dtype=torch.int32, device="cuda")
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0.record()
+        for t in range(T):
+            L = N + t + 1
+            before.fill_(L - 1)
+            cur = 0
+            for l in range(self.n_layers):
+                a, kn, vn = new[l]
+                cache = self.caches[l]
+                lb.lisa_kvcache_append(cache, kn, vn, before)
+                row_out = self.rows[cur ^ 1] if self.next_is_shared(l) else None
+                if self.is_standard[l]:
+                    lb.lisa_attn_anchor(a, cache=cache, L=L, out=out, out_scores=row_out, workspace=ws)
+                else:
+                    w1, w2 = self.weights[l]
+                    lb.lisa_attn_shared_decode(self.rows[cur], lb.Link(a, None, w1, w2, act=lb.ACTS[self.act]), cache, L=L, out=out,
+                                               out_scores=row_out, workspace=ws)
+                if probe is not None and t in probe.steps and l in probe.layers:
+                    s = list(probe.seqs)
+                    rec = {"L": L, "out": out[s, 0].float().cpu(), "a": a[s, 0].cpu(), "v": cache.v[s, :, :L].cpu(),
+                           "k": cache.k[s][..., :L].cpu() if not self.is_standard[l] else cache.k[s, :, :L].cpu(),
+                           "row": None if row_out is None else row_out[s, :, :L].cpu(),
+                           "prev": None if self.is_standard[l] else self.rows[cur][s, :, :L].cpu()}
+                    probe.decode[(t, l)] = rec
+                if row_out is not None:
+                    cur ^= 1
+        t1.record()
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1)
+
+    def tokens_per_s(self, prefill_ms: float, decode_ms: float) -> float:
+        """(prompt tokens + generated tokens) / (prompt time + decoding time), the paper's throughput definition."""
+        return self.B * (self.N + self.T) / ((prefill_ms + decode_ms) * 1e-3)
