@@ -154,6 +154,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-decode", action="store_true", help="skip the decode section")
+    ap.add_argument("--no-stack", action="store_true", help="skip the 32-layer stack section")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
@@ -301,7 +302,29 @@ def main():
                   "shared_over_standard": res["shared"]["value"] / res["standard"]["value"]}
         del sh, st, prev, row, ws
 
-    clocks = sampler.stop()  # sampled across all timed regions above (prefill, end-to-end, decode)
+    # ---------------- 32-layer stack: prefill 2048 + 256 decode steps, LiSA pattern vs all standard (N = 1 only) ----------------
+    stack = None
+    if not args.no_stack and world == 1:
+        from paper_2408_01890_b200 import stack as lstack
+        ws5 = synth.WORKLOADS["cfg5_llama2_7b_stack"]
+        res5 = {}
+        for name, std_layers in (("lisa", None), ("standard", list(range(32)))):
+            torch.cuda.empty_cache()
+            stk = lstack.AttentionStack(n_layers=32, standard_layers=std_layers, B=ws5.B, N=ws5.N, T=256, Hq=ws5.Hq, Hkv=ws5.Hkv,
+                                        d=ws5.d, r=ws5.r, m=ws5.m, act=ws5.act, seed=rank)
+            l1 = lb.lisa_kernel_launches()
+            pre_ms = stk.prefill()
+            dec_ms = stk.decode()
+            launches += lb.lisa_kernel_launches() - l1
+            res5[name] = {"value": stk.tokens_per_s(pre_ms, dec_ms), "unit": "tokens/s", "prefill_ms": pre_ms, "decode_ms": dec_ms,
+                          "shared_layers": 32 - sum(stk.is_standard)}
+            del stk
+        torch.cuda.empty_cache()
+        stack = {"workload": "cfg5_llama2_7b_stack", "B": ws5.B, "prompt": ws5.N, "decode_steps": 256, "layers": 32,
+                 "lisa": res5["lisa"], "standard": res5["standard"], "lisa_over_standard": res5["lisa"]["value"] / res5["standard"]["value"],
+                 "note": "one run each, calls made from Python through the C ABI"}
+
+    clocks = sampler.stop()  # sampled across all timed regions above (prefill, end-to-end, decode, stack)
 
     # ---------------- the CPU oracle on the host cores (rank 0, N = 1 only) ----------------
     cpu = None
@@ -327,7 +350,7 @@ def main():
                        "act": w.act, "chain_len": 1, "l2": "256 MiB buffer written between timed iterations",
                        "step": "lisa_attn_shared_prefill + lisa_kvcache_append"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
-            "decode": decode}))
+            "decode": decode, "stack": stack}))
     if dist is not None:
         dist.destroy_process_group()
 
