@@ -155,8 +155,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-decode", action="store_true", help="skip the decode section")
     ap.add_argument("--no-stack", action="store_true", help="skip the 32-layer stack section")
+    ap.add_argument("--only", choices=["prefill", "decode"], default=None,
+                    help="profiling aid: run just that section (prefill: no end-to-end, decode, stack or CPU legs)")
+    ap.add_argument("--decode-batch", type=int, default=0, help="profiling aid: decode batch size (default: the workload's 64)")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.only is None:
+        args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.only == "prefill":
+        args.no_decode = args.no_stack = True
+    if args.only == "decode":
+        args.no_stack = True
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -227,28 +235,31 @@ def main():
 
 
     # ---------------- end to end through the host-memory entry point ----------------
-    hp = {k: t[k].pin_memory() for k in ("q0", "k0", "v1", "qp1", "kp1", "w1_1", "w2_1")}
-    hlink = lb.Link(hp["qp1"], hp["kp1"], hp["w1_1"], hp["w2_1"], act=lb.ACTS[w.act])
-    hout = torch.empty_like(t["q0"]).pin_memory()
-    arena = torch.empty(lb.lisa_host_arena_bytes(hp["q0"], hp["k0"], [hlink], hp["v1"], hout), dtype=torch.uint8, device="cuda")
-    h2d = sum(x.numel() * x.element_size() for x in hp.values())
-    d2h = hout.numel() * hout.element_size()
+    def measure_e2e():
+        hp = {k: t[k].pin_memory() for k in ("q0", "k0", "v1", "qp1", "kp1", "w1_1", "w2_1")}
+        hlink = lb.Link(hp["qp1"], hp["kp1"], hp["w1_1"], hp["w2_1"], act=lb.ACTS[w.act])
+        hout = torch.empty_like(t["q0"]).pin_memory()
+        arena = torch.empty(lb.lisa_host_arena_bytes(hp["q0"], hp["k0"], [hlink], hp["v1"], hout), dtype=torch.uint8, device="cuda")
+        h2d = sum(x.numel() * x.element_size() for x in hp.values())
+        d2h = hout.numel() * hout.element_size()
 
-    def e2e_step():
-        lb.lisa_attn_shared_prefill_host(hp["q0"], hp["k0"], [hlink], hp["v1"], hout, arena)
+        def e2e_step():
+            lb.lisa_attn_shared_prefill_host(hp["q0"], hp["k0"], [hlink], hp["v1"], hout, arena)
 
-    for _ in range(3):
-        e2e_step()
-    e2e_total, _, _ = time_steps(e2e_step, args.steps, flush, barrier)
-    e2e_ms = max_over_ranks(e2e_total) / args.steps
-    e2e = {"value": world * tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
-           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        for _ in range(3):
+            e2e_step()
+        e2e_total, _, _ = time_steps(e2e_step, args.steps, flush, barrier)
+        e2e_ms = max_over_ranks(e2e_total) / args.steps
+        return {"value": world * tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    e2e = measure_e2e() if args.only is None else None
 
     # ---------------- decode step and the library's own standard-attention decode ----------------
     decode = None
     if not args.no_decode:
         wd = synth.WORKLOADS[DECODE]
-        B, L = wd.B, wd.N
+        B, L = (args.decode_batch or wd.B), wd.N
         sh = lb.KVCacheLayer(lb.CACHE_SHARED, B, wd.Hkv, L, wd.d, wd.r)
         st = lb.KVCacheLayer(lb.CACHE_STANDARD, B, wd.Hkv, L, wd.d)
         sh.k.copy_(synth.device_normal("kpT", sh.k.shape, rank)); sh.v.copy_(synth.device_normal("v", sh.v.shape, rank))
@@ -328,7 +339,7 @@ def main():
 
     # ---------------- the CPU oracle on the host cores (rank 0, N = 1 only) ----------------
     cpu = None
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and args.only is None:
         import oracle
         ol = [oracle.Link(synth.to_f64(t["qp1"]), synth.to_f64(t["kp1"]), synth.to_f64(t["w1_1"]), synth.to_f64(t["w2_1"]),
                           r=w.r, act={"relu": oracle.ACT_RELU, "silu": oracle.ACT_SILU, "none": oracle.ACT_NONE}[w.act])]
