@@ -46,13 +46,13 @@ def prefill_flops(w, c):
     return positions * per_pos
 
 
-def decode_bytes(w, shared=True):
+def decode_bytes(w, shared=True, B=None):
     """Algorithmic HBM bytes of one decode step: score row in and out (fp32), K' (or K) and V caches (bf16)."""
     if shared:
         per_seq = 2 * w.Hq * w.N * 4 + w.Hkv * w.N * w.r * 2 + w.Hkv * w.N * w.d * 2
     else:
         per_seq = w.Hq * w.N * 4 + 2 * w.Hkv * w.N * w.d * 2
-    return w.B * per_seq
+    return (B or w.B) * per_seq
 
 
 class ClockSampler:
@@ -302,12 +302,12 @@ def main():
             ends_ms = max_over_ranks(tot) / args.steps
             append_ms = sum(s.elapsed_time(m) for s, m in zip(sts, mks)) / args.steps
             k_ms = ends_ms - append_ms
-            gbs = decode_bytes(wd, shared) / (k_ms * 1e-3) / 1e9
+            gbs = decode_bytes(wd, shared, B) / (k_ms * 1e-3) / 1e9
             res[name] = {"value": world * B / (ends_ms * 1e-3), "unit": "tokens/s", "ms_per_step": ends_ms,
                          "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                       "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0,
                                       "peak_source": peaks["source"], "kernel_ms": k_ms,
-                                      "bytes_per_launch": decode_bytes(wd, shared), "traffic": None}}
+                                      "bytes_per_launch": decode_bytes(wd, shared, B), "traffic": None}}
         decode = {"workload": DECODE, "B": B, "L": L, "Hq": wd.Hq, "d": wd.d, "r": wd.r, "m": wd.m,
                   "shared": res["shared"], "standard": res["standard"],
                   "shared_over_standard": res["shared"]["value"] / res["standard"]["value"]}

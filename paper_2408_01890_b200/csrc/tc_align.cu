@@ -3,7 +3,7 @@
 // Input: fp16 planes [B*Hq][rows][cols] (fp16, not bf16: three more mantissa bits keep a chain of several links
 // inside the accuracy bar; scores are O(10), far from fp16's range limit, and conversions saturate) holding A_0 = Q0.K0^T/sqrt(d) (Eq. 2) and, for chain depth c > 1, the
 // already scaled differences D_k = Q'_k.K'_k^T/sqrt(r) (Eq. 3) of the links k < c.  Output, in place of the A_0
-// plane: Y = FFN_c(A_{c-1}) where A_k = FFN_k(A_{k-1}) + D_k (Eq. 4, ADD) -- the final link's D_c is added by the
+// plane: Y = log2(e) * FFN_c(A_{c-1}) where A_k = FFN_k(A_{k-1}) + D_k (Eq. 4, ADD) -- the final link's D_c is added by the
 // attention kernel that consumes Y.  Hq = 32 heads, hidden width 64, two-layer FFNs.
 //
 // A work unit is 128 consecutive key positions of one query row; positions are the M dimension of the MMAs:
@@ -28,6 +28,8 @@ constexpr int W1_BYTES = MH * 128;         // B operand, K-major: row = hidden u
 constexpr int W2_BYTES = HQ * 128;         // row = output head, k = 64 hidden units
 constexpr int AT_BYTES = UNIT * 128;       // A operand, K-major: row = position, 64 k-slots
 constexpr uint32_t TMEM_COLS = 256;        // D1[2]: [0,128), D2[2]: [128,192)
+constexpr float kLog2e = 1.4426950408889634f;  // the last link's output leaves multiplied by log2(e): the attention
+                                               // kernel that adds it to its logits works in the exp2 domain
 constexpr int kMaxTcChain = 3;  // shared memory holds the slabs and weights of at most three links
 
 struct AlignParams {
@@ -173,10 +175,12 @@ tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ T
             const int hh = e / MH, u = e % MH;  // W1[hh][u] -> row u, k-slot hh
             *reinterpret_cast<__half*>(w1t + sw128_offset(u, hh >> 3) + (hh & 7) * 2) = __float2half_rn(ld_elem(p.w1[k], e, p.w_dtype[k]));
             const int u2 = e / HQ, gg = e % HQ;  // W2[u2][gg] -> row gg, k-slot u2
-            *reinterpret_cast<__half*>(w2t + sw128_offset(gg, u2 >> 3) + (u2 & 7) * 2) = __float2half_rn(ld_elem(p.w2[k], e, p.w_dtype[k]));
+            *reinterpret_cast<__half*>(w2t + sw128_offset(gg, u2 >> 3) + (u2 & 7) * 2) =
+                __float2half_rn(ld_elem(p.w2[k], e, p.w_dtype[k]) * (k == c - 1 ? kLog2e : 1.f));
         }
         for (int e = tid; e < MH; e += blockDim.x) sBias[k * (MH + HQ) + e] = ldw(p.b1[k], e, p.w_dtype[k]);
-        for (int e = tid; e < HQ; e += blockDim.x) sBias[k * (MH + HQ) + MH + e] = ldw(p.b2[k], e, p.w_dtype[k]);
+        for (int e = tid; e < HQ; e += blockDim.x)
+            sBias[k * (MH + HQ) + MH + e] = ldw(p.b2[k], e, p.w_dtype[k]) * (k == c - 1 ? kLog2e : 1.f);
     }
     fence_async_smem();
     tc_fence_before();

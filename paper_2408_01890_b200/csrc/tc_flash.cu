@@ -1,15 +1,18 @@
 // Tensor-core flash kernel (tcgen05 + TMEM + TMA) for head width 128, bf16.
 //
 // One CTA per (batch b, query head h, 128-row query tile).  For every key tile j <= the query tile:
-//   scores  S = QA . KA^T            tcgen05.mma, fp32 accumulator in tensor memory
+//   scores  S = QA . KA^T            tcgen05.mma, fp32 accumulator in tensor memory (two buffers, so S(t+1) is
+//                                    computed while the softmax of tile t runs)
 //   logits  A = S * scale (+ Y)      Y: optional fp16 tile of pre-computed scores (the aligned part of a
 //                                    shared layer, Eq. 4; then QA/KA are the layer's low-rank Q'/K', Eq. 3)
 //   causal mask (diagonal tile), online softmax in registers (one thread per query row), P as bf16
 //   O += P . V                       tcgen05.mma, V read MN-major straight from its [key][d] tile
-// With QA/KA = Q/K and no Y this is standard attention (Eq. 1-2).
+// With QA/KA = Q/K and no Y this is standard attention (Eq. 1-2).  In MODE_EMIT there is no softmax: the scaled
+// scores leave as fp16 tiles (staged in shared memory, stored with TMA) for the aligner kernel.
 //
 // Warp roles: warps 0-3 softmax/epilogue (thread = query row = TMEM lane), warp 4 TMA producer,
-// warp 5 MMA issuer and TMEM owner.  Two-stage K/V(/Y) ring; S(t+1) is issued before P.V(t).
+// warp 5 MMA issuer and TMEM owner.  K and V(/Y) have their own two-stage rings: a K stage is free again as
+// soon as its score MMA has run, a V stage after its P.V MMA.
 // Every wait is bounded; on expiry the CTA records it in the status word, drains and exits.
 #include "common.cuh"
 #include "tc_common.cuh"
@@ -28,7 +31,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
 }
 
 constexpr int kThreads = 192;
-constexpr uint32_t TMEM_COLS = 256;  // S: [0,128), O: [128,256)
+constexpr uint32_t TMEM_COLS = 512;  // S[2]: [0,256), O: [256,384)
 
 struct FlashParams {
     int B, N, Hq, Hkv;
@@ -36,16 +39,14 @@ struct FlashParams {
     __nv_bfloat16* o;
     int64_t o_sb, o_sn, o_sh;
     int* status;
-    int plane_row0;  // first query row held by the Y workspace (rows are stored relative to it)
+    int plane_row0;  // first query row held by the plane workspace (rows are stored relative to it)
     int qt_begin;    // this launch covers query tiles [qt_begin, qt_begin + gridDim.x)
     int ksteps;      // 16-wide k-steps of the score MMA actually issued (<= KD/16; the rest is zero padding)
-    float scale;     // MODE_EMIT: scores are multiplied by this before rounding to bf16
-    __half* plane_out;  // MODE_EMIT: fp16 [B*Hq][plane_rows][plane_cols]
-    int64_t plane_rows, plane_cols;
+    float scale;     // MODE_EMIT: scores are multiplied by this before rounding to fp16
 };
 
-// MODE_ATTN: softmax(QA.KA^T).V;  MODE_ATTN_PLANE: the same with the pre-computed tile Y added to the logits;
-// MODE_EMIT: no softmax, the scaled scores are written as fp16 to the plane workspace (for the aligner kernel).
+// MODE_ATTN: softmax(QA.KA^T).V;  MODE_ATTN_PLANE: the same with the pre-computed tile Y added to the logits
+// (Y arrives already multiplied by log2(e));  MODE_EMIT: no softmax, the scaled scores go to the plane workspace.
 constexpr int MODE_ATTN = 0, MODE_ATTN_PLANE = 1, MODE_EMIT = 2;
 
 template <int KD, int MODE>
@@ -57,12 +58,14 @@ struct Smem {
     static constexpr int V_BYTES = EMIT ? 0 : BN * D * 2;
     static constexpr int P_BYTES = EMIT ? 0 : BM * BN * 2;
     static constexpr int Y_BYTES = PLANE ? BM * BN * 2 : 0;
+    static constexpr int STG_BYTES = EMIT ? 4 * 2 * 8192 : 0;  // per epilogue warp: two buffers of [2 halves][32 rows][128 B]
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + Q_BYTES;
     static constexpr int OFF_V = OFF_K + 2 * K_BYTES;
     static constexpr int OFF_P = OFF_V + 2 * V_BYTES;
     static constexpr int OFF_Y = OFF_P + P_BYTES;
-    static constexpr int OFF_BAR = OFF_Y + 2 * Y_BYTES;
+    static constexpr int OFF_STG = OFF_Y + 2 * Y_BYTES;
+    static constexpr int OFF_BAR = OFF_STG + STG_BYTES;
     static constexpr int TOTAL = OFF_BAR + 256 + 1024;  // + alignment slack
 };
 
@@ -80,16 +83,19 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     uint8_t* sV = smem + L::OFF_V;
     uint8_t* sP = smem + L::OFF_P;
     uint8_t* sY = smem + L::OFF_Y;
+    uint8_t* sStg = smem + L::OFF_STG;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
     uint64_t* q_full = bars + 0;
-    uint64_t* kv_full = bars + 1;   // [2]
-    uint64_t* kv_empty = bars + 3;  // [2]
-    uint64_t* s_full = bars + 5;
-    uint64_t* s_free = bars + 6;
-    uint64_t* p_full = bars + 7;
-    uint64_t* pv_done = bars + 8;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 11);
+    uint64_t* k_full = bars + 1;    // [2]
+    uint64_t* k_empty = bars + 3;   // [2]
+    uint64_t* v_full = bars + 5;    // [2] V and Y of a stage
+    uint64_t* v_empty = bars + 7;   // [2]
+    uint64_t* s_full = bars + 9;    // [2] score buffer written by the MMA
+    uint64_t* s_free = bars + 11;   // [2] score buffer copied to registers by all 128 rows
+    uint64_t* p_full = bars + 13;
+    uint64_t* pv_done = bars + 14;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 17);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int qt = p.qt_begin + (int)gridDim.x - 1 - (int)blockIdx.x;  // heavy tiles first
@@ -100,10 +106,11 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
 
     if (tid == 0) {
         mbar_init(q_full, 1);
-        mbar_init(kv_full + 0, 1); mbar_init(kv_full + 1, 1);
-        mbar_init(kv_empty + 0, 1); mbar_init(kv_empty + 1, 1);
-        mbar_init(s_full, 1);
-        mbar_init(s_free, 128);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1);
+            mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
+            mbar_init(s_full + i, 1); mbar_init(s_free + i, 128);
+        }
         mbar_init(p_full, 128);
         mbar_init(pv_done, 1);
         *abort_flag = 0;
@@ -114,72 +121,78 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 128;
+    const uint32_t tmem_O = tmem_base + 256;
 
     if (warp == 4) {
         // ------------------------------ TMA producer ------------------------------
-        // Lane 0 waits for the stage and arms its barrier; then the copies of the stage are issued by different
-        // lanes of the warp at once (one 64-column box each): a single thread issuing them back to back is
-        // several hundred cycles slower per copy.
-        if (lane == 0) { tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); }
-        if (lane == 0) mbar_expect_tx(q_full, L::Q_BYTES);
+        // Lane 0 waits for a stage and arms its barrier; then the copies are issued by different lanes at once
+        // (one 64-column box each): one thread issuing them back to back is several hundred cycles slower per copy.
+        if (lane == 0) {
+            tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
+            if (!EMIT) tma_prefetch_desc(&tmV);
+            mbar_expect_tx(q_full, L::Q_BYTES);
+        }
         __syncwarp();
         if (lane < KD / 64) tma_load_4d(sQ + lane * (BM * 128), &tmQ, q_full, lane * 64, h, q0, b);
+        constexpr int NK = KD / 64, NV = EMIT ? 0 : D / 64, NY = PLANE ? BN / 64 : 0;
         bool okp = true;
         for (int t = 0; t < nt; ++t) {
             const int s = t & 1;
+            const uint32_t par = ((t >> 1) & 1) ^ 1;
             if (lane == 0) {
-                okp = mbar_wait(kv_empty + s, ((t >> 1) & 1) ^ 1, abort_flag);
-                if (okp) mbar_expect_tx(kv_full + s, L::K_BYTES + L::V_BYTES + L::Y_BYTES);
+                okp = mbar_wait(k_empty + s, par, abort_flag);
+                if (okp) mbar_expect_tx(k_full + s, L::K_BYTES);
             }
             okp = __shfl_sync(0xffffffffu, okp, 0);
             if (!okp) break;
-            constexpr int NK = KD / 64, NV = EMIT ? 0 : D / 64, NY = PLANE ? BN / 64 : 0;
-            if (lane < NK) {
-                tma_load_4d(sK + s * L::K_BYTES + lane * (BN * 128), &tmK, kv_full + s, lane * 64, g, t * BN, b);
-            } else if (lane < NK + NV) {
-                const int c = lane - NK;
-                tma_load_4d(sV + s * L::V_BYTES + c * (BN * 128), &tmV, kv_full + s, c * 64, g, t * BN, b);
-            } else if (lane < NK + NV + NY) {
-                const int c = lane - NK - NV;
-                tma_load_3d(sY + s * L::Y_BYTES + c * (BM * 128), &tmY, kv_full + s, t * BN + c * 64, q0 - p.plane_row0, b * p.Hq + h);
-            }
+            if (lane < NK) tma_load_4d(sK + s * L::K_BYTES + lane * (BN * 128), &tmK, k_full + s, lane * 64, g, t * BN, b);
             __syncwarp();
+            if constexpr (!EMIT) {
+                if (lane == 0) {
+                    okp = mbar_wait(v_empty + s, par, abort_flag);
+                    if (okp) mbar_expect_tx(v_full + s, L::V_BYTES + L::Y_BYTES);
+                }
+                okp = __shfl_sync(0xffffffffu, okp, 0);
+                if (!okp) break;
+                if (lane < NV) {
+                    tma_load_4d(sV + s * L::V_BYTES + lane * (BN * 128), &tmV, v_full + s, lane * 64, g, t * BN, b);
+                } else if (lane < NV + NY) {
+                    const int c = lane - NV;
+                    tma_load_3d(sY + s * L::Y_BYTES + c * (BM * 128), &tmY, v_full + s, t * BN + c * 64, q0 - p.plane_row0, b * p.Hq + h);
+                }
+                __syncwarp();
+            }
         }
     } else if (warp == 5) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             constexpr uint32_t IDESC_QK = umma_idesc_bf16(BM, BN, 0, 0);
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(BM, D, 0, 1);
-            auto issue_qk = [&](int t) {
+            const int ksteps = p.ksteps;
+            // scores of tile t into buffer t&1; needs K(t) loaded and (t >= 2) the buffer read by the softmax of t-2
+            auto issue_qk = [&](int t) -> bool {
                 const int s = t & 1;
+                if (!mbar_wait(k_full + s, (t >> 1) & 1, abort_flag)) return false;
+                if (!mbar_wait(s_free + s, ((t >> 1) & 1) ^ 1, abort_flag)) return false;
+                tc_fence_after();
                 const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + s * L::K_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < KD / 16; ++ks) {
-                    if (ks < p.ksteps) {
+                    if (ks < ksteps) {
                         const uint32_t off = (ks >> 2) * (BM * 128) + (ks & 3) * 32;
-                        umma_ss(tmem_S, umma_desc_sw128(qa + off, 16, 1024), umma_desc_sw128(ka + off, 16, 1024), IDESC_QK, ks > 0);
+                        umma_ss(tmem_base + s * 128, umma_desc_sw128(qa + off, 16, 1024), umma_desc_sw128(ka + off, 16, 1024), IDESC_QK, ks > 0);
                     }
                 }
-                umma_commit(s_full);
-                if constexpr (EMIT)
-                    if (t + 2 < nt) umma_commit(kv_empty + s);  // nobody waits for the last two: do not arm them
+                umma_commit(s_full + s);
+                if (t + 2 < nt) umma_commit(k_empty + s);  // nobody waits for the last two: do not arm them
+                return true;
             };
-            bool ok = mbar_wait(q_full, 0, abort_flag) && mbar_wait(kv_full + 0, 0, abort_flag);
-            if (ok) {
-                tc_fence_after();
-                issue_qk(0);
-            }
+            bool ok = mbar_wait(q_full, 0, abort_flag) && issue_qk(0);
             for (int t = 0; ok && t < nt; ++t) {
                 const int s = t & 1;
-                if (t + 1 < nt) {
-                    ok = mbar_wait(kv_full + ((t + 1) & 1), ((t + 1) >> 1) & 1, abort_flag) && mbar_wait(s_free, t & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_qk(t + 1);
-                }
+                if (t + 1 < nt && !(ok = issue_qk(t + 1))) break;
                 if constexpr (EMIT) continue;
-                if (!(ok = mbar_wait(p_full, t & 1, abort_flag))) break;
+                if (!(ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag) && mbar_wait(p_full, t & 1, abort_flag))) break;
                 tc_fence_after();
                 const uint32_t pa = smem_u32(sP), va = smem_u32(sV + s * L::V_BYTES);
 #pragma unroll
@@ -190,44 +203,53 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                             (t > 0) || (ks > 0));
                 }
                 umma_commit(pv_done);
-                if (t + 2 < nt) umma_commit(kv_empty + s);
+                if (t + 2 < nt) umma_commit(v_empty + s);
             }
         }
     } else {
-        // ------------------------------ softmax + epilogue (thread = query row) ------------------------------
+        // ------------------------------ softmax / epilogue (thread = query row) ------------------------------
         const int row = tid;                       // 0..127, TMEM lane
         const int qi = q0 + row;                   // global query index
         const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+        const float scale_log2 = p.scale_log2, emit_scale = p.scale;
         float m_ref = -INFINITY, l_sum = 0.f;
         bool ok = true;
         for (int t = 0; t < nt; ++t) {
             const int s = t & 1;
-            if (!(ok = mbar_wait(s_full, t & 1, abort_flag))) break;
+            if (!(ok = mbar_wait(s_full + s, (t >> 1) & 1, abort_flag))) break;
             tc_fence_after();
             uint32_t sr[128];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tmem_S + lane_sel + c * 32, sr + c * 32);
+            for (int c = 0; c < 4; ++c) tmem_ld32(tmem_base + s * 128 + lane_sel + c * 32, sr + c * 32);
             tmem_wait_ld();
             tc_fence_before();
-            mbar_arrive(s_free);
+            mbar_arrive(s_free + s);
             float* sf = reinterpret_cast<float*>(sr);
             if constexpr (EMIT) {
-                if (qi < p.N) {
-                    __half* dst = p.plane_out + ((int64_t)(b * p.Hq + h) * p.plane_rows + (qi - p.plane_row0)) * p.plane_cols + t * BN;
+                // this warp's 32 rows x 128 columns as fp16 into its staging buffer (two 64-column halves, swizzled
+                // like any other tile), then lanes 0 and 1 store one half each with TMA
+                uint8_t* stg = sStg + (warp * 2 + s) * 8192;
+                if (t >= 2 && lane < 2) tma_store_wait_read<1>();  // the store of tile t-2 has read this buffer
+                __syncwarp();
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        uint4 v;
-                        v.x = pack_f16(sf[c * 8 + 0] * p.scale, sf[c * 8 + 1] * p.scale);
-                        v.y = pack_f16(sf[c * 8 + 2] * p.scale, sf[c * 8 + 3] * p.scale);
-                        v.z = pack_f16(sf[c * 8 + 4] * p.scale, sf[c * 8 + 5] * p.scale);
-                        v.w = pack_f16(sf[c * 8 + 6] * p.scale, sf[c * 8 + 7] * p.scale);
-                        *reinterpret_cast<uint4*>(dst + c * 8) = v;
-                    }
+                for (int c = 0; c < 16; ++c) {
+                    uint4 v;
+                    v.x = pack_f16(sf[c * 8 + 0] * emit_scale, sf[c * 8 + 1] * emit_scale);
+                    v.y = pack_f16(sf[c * 8 + 2] * emit_scale, sf[c * 8 + 3] * emit_scale);
+                    v.z = pack_f16(sf[c * 8 + 4] * emit_scale, sf[c * 8 + 5] * emit_scale);
+                    v.w = pack_f16(sf[c * 8 + 6] * emit_scale, sf[c * 8 + 7] * emit_scale);
+                    *reinterpret_cast<uint4*>(stg + (c >> 3) * 4096 + sw128_offset(lane, c & 7)) = v;
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane < 2) {
+                    tma_store_3d(&tmY, stg + lane * 4096, t * BN + lane * 64, q0 - p.plane_row0 + warp * 32, b * p.Hq + h);
+                    tma_store_commit();
                 }
                 continue;
             }
             if constexpr (PLANE) {
-                // the stage's full barrier was already observed by the MMA warp; s_full implies it completed
+                if (!(ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag))) break;  // Y of this stage has landed
                 const uint8_t* yb = sY + s * L::Y_BYTES;
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
@@ -236,14 +258,12 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const float2 yv = unpack_f16(w[e]);
-                        sf[c * 8 + 2 * e] = fmaf(sf[c * 8 + 2 * e], p.scale_log2, yv.x * 1.4426950408889634f);
-                        sf[c * 8 + 2 * e + 1] = fmaf(sf[c * 8 + 2 * e + 1], p.scale_log2, yv.y * 1.4426950408889634f);
+                        sf[c * 8 + 2 * e] = fmaf(sf[c * 8 + 2 * e], scale_log2, yv.x);
+                        sf[c * 8 + 2 * e + 1] = fmaf(sf[c * 8 + 2 * e + 1], scale_log2, yv.y);
                     }
                 }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 128; ++j) sf[j] *= p.scale_log2;
             }
+            // from here on: PLANE -> sf holds log2-domain logits; otherwise raw scores, scaled inside the exp
             if (t == nt - 1) {
 #pragma unroll
                 for (int j = 0; j < 128; ++j)
@@ -252,6 +272,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             float m_t = sf[0];
 #pragma unroll
             for (int j = 1; j < 128; ++j) m_t = fmaxf(m_t, sf[j]);
+            if constexpr (!PLANE) m_t *= scale_log2;
             // lazy rescale: move the reference maximum only when some row of the warp outgrew it by 2^8
             const bool grow = m_t > m_ref + 8.f;
             const bool rescale = __any_sync(0xffffffffu, grow) || t == 0;
@@ -278,12 +299,13 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 }
             }
             float sum = 0.f;
+            const float neg_m = -m_ref;
 #pragma unroll
             for (int c = 0; c < 16; ++c) {
                 float e[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    e[j] = fast_exp2(sf[c * 8 + j] - m_ref);
+                    e[j] = PLANE ? fast_exp2(sf[c * 8 + j] + neg_m) : fast_exp2(fmaf(sf[c * 8 + j], scale_log2, neg_m));
                     sum += e[j];
                 }
                 uint4 v;
@@ -295,7 +317,9 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             tc_fence_before();
             mbar_arrive(p_full);
         }
-        if (!EMIT && ok && mbar_wait(pv_done, (nt - 1) & 1, abort_flag)) {
+        if constexpr (EMIT) {
+            if (lane < 2) tma_store_wait_all<0>();
+        } else if (ok && mbar_wait(pv_done, (nt - 1) & 1, abort_flag)) {
             tc_fence_after();
             const float inv_l = 1.f / l_sum;
             __nv_bfloat16* orow = p.o + b * p.o_sb + (int64_t)qi * p.o_sn + h * p.o_sh;
@@ -324,8 +348,8 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     if (*abort_flag) {
         // a wait ran out: give copies and MMAs still in flight time to land before the memory is released
         if (tid == 0) atomicAdd(p.status + 1, 1);
-        const uint64_t t0 = global_timer_ns();
-        while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
+        const long long t0 = clock64();
+        while (clock64() - t0 < 4000000ll) __nanosleep(1000);
         __syncthreads();
     }
     if (warp == 5) {
@@ -336,7 +360,6 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
 }
 
 }  // namespace
-
 
 bool make_tensor_map_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                           const uint32_t* box, bool fp16) {
@@ -385,6 +408,12 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     tmV = tmQ;
     if (!a.emit_plane && !map_bnhx(&tmV, a.v, a.B, a.N, a.Hkv, D)) return cudaErrorInvalidValue;
     tmY = tmQ;
+    if (a.emit_plane) {  // store map: one epilogue warp's 32 rows x 64 columns per copy
+        const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * a.Hq};
+        const uint64_t str[2] = {(uint64_t)a.plane_cols * 2, (uint64_t)a.plane_cols * a.plane_rows * 2};
+        const uint32_t box[3] = {64, 32, 1};
+        if (!make_tensor_map_bf16(&tmY, a.emit_plane, 3, dims, str, box, true)) return cudaErrorInvalidValue;
+    }
     if (a.plane) {
         const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * a.Hq};
         const uint64_t str[2] = {(uint64_t)a.plane_cols * 2, (uint64_t)a.plane_cols * a.plane_rows * 2};
@@ -402,8 +431,7 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     p.qt_begin = a.qt_begin;
     p.ksteps = a.ksteps > 0 ? a.ksteps : a.kd / 16;
     p.scale = a.scale;
-    p.plane_out = reinterpret_cast<__half*>(a.emit_plane);
-    p.plane_rows = a.plane_rows; p.plane_cols = a.plane_cols;
+
     dim3 grid(a.qt_count, a.Hq, a.B);
     cudaError_t e;
 #define LISA_LAUNCH_FLASH(KD_, PL_)                                                                                       \
