@@ -29,6 +29,10 @@ from paper_2408_01890_b200 import synth  # noqa: E402
 PREFILL = "cfg2_llama2_7b_prefill"
 DECODE = "cfg4_llama2_13b_decode"
 METRIC = "lisa_attention_tokens_per_s"
+# dram bytes (read + write) per launch from the ncu captures summarised under profiles/ (cold cache, same workload);
+# None for a kernel that has changed since its counters were taken
+PREFILL_TRAFFIC = {"align": 142717952 + 83444480, "emit_scores": 33583360 + 85699840, "attention": 176216320 + 10768896}
+DECODE_TRAFFIC_PER_SEQ = (395937024 + 4827392) / 8  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
 
 
 def measured_peaks():
@@ -228,10 +232,27 @@ def main():
     tokens = w.B * w.N
     value = world * tokens / (ms_per_step * 1e-3)
     flops = prefill_flops(w, 1)
-    achieved = flops / (kernel_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "lisa_attn_shared_prefill", "achieved": achieved, "peak": peaks["bf16_tflops"],
+    # per-kernel device times of the same step (events recorded inside the library around each of its kernels)
+    lb.lisa_prefill_phase_timing(True)
+    for _ in range(args.steps):
+        flush(); prefill_step()
+    phase_ms = [x / args.steps for x in lb.lisa_prefill_phase_times()]
+    lb.lisa_prefill_phase_timing(False)
+    positions = w.B * w.N * (w.N + 1) // 2
+    phase_flops = {"pack": 0, "emit_scores": positions * 2 * w.Hq * w.d, "align": positions * 4 * w.Hq * w.m,
+                   "attention": positions * (2 * w.Hq * w.r + 2 * w.Hq * w.d)}
+    names = ["pack", "emit_scores", "align", "attention"]
+    kernels = {n: {"ms": phase_ms[i], "flops": phase_flops[n],
+                   "tflops": (phase_flops[n] / (phase_ms[i] * 1e-3) / 1e12) if phase_ms[i] > 0 else None,
+                   "share": phase_ms[i] / max(sum(phase_ms), 1e-9)} for i, n in enumerate(names)}
+    dom = max(names, key=lambda n: kernels[n]["ms"])
+    achieved = kernels[dom]["tflops"] or 0.0
+    call_tflops = flops / (kernel_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "lisa_attn_shared_prefill/" + dom, "achieved": achieved, "peak": peaks["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",
-                "traffic": None, "kernel_ms": kernel_ms, "flops_per_launch": flops}
+                "traffic": PREFILL_TRAFFIC.get(dom), "kernel_ms": kernels[dom]["ms"], "flops_per_launch": kernels[dom]["flops"],
+                "kernels": kernels,
+                "whole_call": {"ms": kernel_ms, "flops": flops, "achieved": call_tflops, "frac": call_tflops / peaks["bf16_tflops"]}}
 
 
     # ---------------- end to end through the host-memory entry point ----------------
@@ -307,7 +328,8 @@ def main():
                          "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                       "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0,
                                       "peak_source": peaks["source"], "kernel_ms": k_ms,
-                                      "bytes_per_launch": decode_bytes(wd, shared, B), "traffic": None}}
+                                      "bytes_per_launch": decode_bytes(wd, shared, B),
+                                      "traffic": DECODE_TRAFFIC_PER_SEQ * B if shared else None}}
         decode = {"workload": DECODE, "B": B, "L": L, "Hq": wd.Hq, "d": wd.d, "r": wd.r, "m": wd.m,
                   "shared": res["shared"], "standard": res["standard"],
                   "shared_over_standard": res["shared"]["value"] / res["standard"]["value"]}

@@ -26,7 +26,7 @@ OP_ANCHOR, OP_SHARED_PREFILL, OP_SHARED_DECODE = 0, 1, 2
 ACTS = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
 
 EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_host", "lisa_host_arena_bytes",
-           "lisa_attn_shared_decode", "lisa_attn_shared_decode_static", "lisa_kvcache_append", "lisa_kvcache_bytes", "lisa_workspace_bytes", "lisa_check",
+           "lisa_attn_shared_decode", "lisa_attn_shared_decode_static", "lisa_kvcache_append", "lisa_kvcache_bytes", "lisa_prefill_phase_times", "lisa_prefill_phase_timing", "lisa_workspace_bytes", "lisa_check",
            "lisa_force_general_kernels", "lisa_kernel_launches", "lisa_last_cuda_error", "lisa_status_string", "lisa_version"]
 
 
@@ -344,3 +344,15 @@ def lisa_kernel_launches() -> int:
 def lisa_force_general_kernels(on: bool) -> None:
     """Route every later call through the general SIMT kernels (True) or restore the default choice (False)."""
     load().lisa_force_general_kernels(1 if on else 0)
+
+
+def lisa_prefill_phase_timing(enable: bool) -> None:
+    """Turns the per-kernel event timing of the tensor-core prefill on or off."""
+    _check(load().lisa_prefill_phase_timing(1 if enable else 0), "lisa_prefill_phase_timing")
+
+
+def lisa_prefill_phase_times():
+    """Milliseconds per phase (pack, emit, align, attention) summed since the last read."""
+    ms = (C.c_float * 4)()
+    _check(load().lisa_prefill_phase_times(ms), "lisa_prefill_phase_times")
+    return [float(x) for x in ms]

@@ -103,6 +103,8 @@ cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int
 bool tc_shared_prefill_supported(const lisa_shared_prefill_args& a);
 size_t tc_shared_prefill_workspace(const lisa_shared_prefill_args& a);
 cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws, cudaStream_t s);
+cudaError_t prefill_phase_timing(bool enable);
+cudaError_t prefill_phase_times(float* ms4);
 
 cudaError_t launch_kvcache_append(const lisa_kvcache_layer& c, const lisa_tensor& k, const lisa_tensor& v,
                                   const int32_t* lens_before, int n_new, cudaStream_t s);

@@ -286,6 +286,17 @@ lisa_status_t lisa_kvcache_append(const lisa_kvcache_layer* layer, const lisa_te
     return e == cudaSuccess ? LISA_OK : cuda_fail(e);
 }
 
+lisa_status_t lisa_prefill_phase_timing(int enable) {
+    cudaError_t e = prefill_phase_timing(enable != 0);
+    return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+}
+
+lisa_status_t lisa_prefill_phase_times(float* ms4) {
+    if (!ms4) return LISA_ERR_INVALID_ARG;
+    cudaError_t e = prefill_phase_times(ms4);
+    return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+}
+
 lisa_status_t lisa_check(lisa_stream_t stream) {
     cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e);

@@ -43,6 +43,32 @@ __global__ void pack_lowrank_kernel(TView src, int B, int N, int H, int r, __nv_
     }
 }
 
+// Optional per-phase timing of the tensor-core prefill (lisa_prefill_phase_timing): CUDA events recorded on the
+// caller's stream around each internal kernel, summed per phase when read.  Off by default.
+constexpr int kPhases = 4;       // 0 pack, 1 emit score planes, 2 aligner, 3 attention
+constexpr int kMaxMarks = 2048;
+struct PhaseTimer {
+    bool on = false;
+    int n = 0;
+    cudaEvent_t ev[2 * kMaxMarks];
+    int phase[kMaxMarks];
+} g_pt;
+
+struct PhaseMark {
+    cudaStream_t s;
+    int idx;
+    PhaseMark(int phase, cudaStream_t stream) : s(stream), idx(-1) {
+        if (g_pt.on && g_pt.n < kMaxMarks) {
+            idx = g_pt.n++;
+            g_pt.phase[idx] = phase;
+            cudaEventRecord(g_pt.ev[2 * idx], s);
+        }
+    }
+    ~PhaseMark() {
+        if (idx >= 0) cudaEventRecord(g_pt.ev[2 * idx + 1], s);
+    }
+};
+
 struct Wave { int begin, count; };
 
 int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves) {
@@ -121,6 +147,7 @@ cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws
     const int c = a.chain_len;
     cudaError_t e;
     for (int k = 0; k < c; ++k) {
+        PhaseMark mark(0, s);
         if ((e = launch_pack_lowrank(a.links[k].qp, a.B, a.N, a.Hq, a.links[k].r, base + l.qp_off[k], s)) != cudaSuccess) return e;
         if ((e = launch_pack_lowrank(a.links[k].kp, a.B, a.N, a.Hkv, a.links[k].r, base + l.kp_off[k], s)) != cudaSuccess) return e;
     }
@@ -132,8 +159,12 @@ cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws
         TcFlashArgs f{a.B, a.N, a.Hq, a.Hkv, 128, a.q0, a.k0, a.v, a.o, 1.f / sqrtf((float)a.d), nullptr, l.plane_rows, l.plane_cols,
                       wv.begin, wv.count};
         f.emit_plane = base + l.plane_off[0];
-        if ((e = launch_tc_flash(f, s)) != cudaSuccess) return e;
+        {
+            PhaseMark mark(1, s);
+            if ((e = launch_tc_flash(f, s)) != cudaSuccess) return e;
+        }
         for (int k = 0; k + 1 < c; ++k) {
+            PhaseMark mark(1, s);
             TcFlashArgs fd = f;
             fd.kd = kPadRank;
             fd.qa = packed_view(base + l.qp_off[k], a.Hq, a.N);
@@ -149,7 +180,10 @@ cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws
         al.plane_rows = l.plane_rows; al.plane_cols = l.plane_cols;
         for (int k = 0; k < c; ++k) al.planes[k] = base + l.plane_off[k];
         al.links = a.links;
-        if ((e = launch_tc_align(al, s)) != cudaSuccess) return e;
+        {
+            PhaseMark mark(2, s);
+            if ((e = launch_tc_align(al, s)) != cudaSuccess) return e;
+        }
         // 3. this layer's own difference, softmax and .V
         TcFlashArgs fv = f;
         fv.emit_plane = nullptr;
@@ -159,8 +193,38 @@ cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws
         fv.scale = 1.f / sqrtf((float)a.links[c - 1].r);
         fv.ksteps = (a.links[c - 1].r + 15) / 16;
         fv.plane = base + l.plane_off[0];
+        PhaseMark mark(3, s);
         if ((e = launch_tc_flash(fv, s)) != cudaSuccess) return e;
     }
+    return cudaSuccess;
+}
+
+cudaError_t prefill_phase_timing(bool enable) {
+    if (enable == g_pt.on) { g_pt.n = 0; return cudaSuccess; }
+    if (enable) {
+        for (int i = 0; i < 2 * kMaxMarks; ++i) {
+            cudaError_t e = cudaEventCreate(&g_pt.ev[i]);
+            if (e != cudaSuccess) return e;
+        }
+    } else {
+        for (int i = 0; i < 2 * kMaxMarks; ++i) cudaEventDestroy(g_pt.ev[i]);
+    }
+    g_pt.on = enable;
+    g_pt.n = 0;
+    return cudaSuccess;
+}
+
+cudaError_t prefill_phase_times(float* ms) {
+    for (int i = 0; i < kPhases; ++i) ms[i] = 0.f;
+    if (!g_pt.on) return cudaSuccess;
+    for (int i = 0; i < g_pt.n; ++i) {
+        cudaError_t e = cudaEventSynchronize(g_pt.ev[2 * i + 1]);
+        if (e != cudaSuccess) return e;
+        float t = 0.f;
+        if ((e = cudaEventElapsedTime(&t, g_pt.ev[2 * i], g_pt.ev[2 * i + 1])) != cudaSuccess) return e;
+        ms[g_pt.phase[i]] += t;
+    }
+    g_pt.n = 0;
     return cudaSuccess;
 }
 
