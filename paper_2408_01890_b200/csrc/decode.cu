@@ -370,6 +370,80 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
     softmax_pv_chunk(p, s_s, b, chunk, nrows);
 }
 
+// Scores of a FULL chunk for a standard layer, d = 128, bf16 cache: s_s[h][j] = q_h . K_j / sqrt(d).  Same streaming
+// scheme as pv_full_chunk (two register sets of eight 16-byte loads per lane, prefetch across heads).  A lane holds
+// the partial dot products of eight rows over its 8 of the 128 dimensions; the sum over the 16 lanes of a row is a
+// butterfly that halves the number of live values at every step (8 shuffles per batch instead of 32).
+__device__ __forceinline__ void anchor_qk_full_chunk(const DecodeParams& p, float* s_s, const float* q_s, int b, int j0,
+                                                     float inv_sqrt_d) {
+    constexpr int LPR = 16, RSTEP = 2, NB = kChunk / RSTEP / 8;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane & 15, rsel = lane >> 4;
+    const int Hq = p.Hq, G = p.Hq / p.Hkv;
+    auto head_ptr = [&](int h) {
+        return reinterpret_cast<const uint4*>(p.kcache) + (((size_t)b * p.Hkv + h / G) * p.L_cap + j0 + rsel) * LPR + sub;
+    };
+    if (warp >= Hq) return;
+    const uint4* hp = head_ptr(warp);
+    uint4 ra[8], rb[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) ra[u] = ld_stream16(hp + u * RSTEP * LPR);
+    const int urow = ((sub & 8) ? 4 : 0) + ((sub & 4) ? 2 : 0) + ((sub & 2) ? 1 : 0);  // row of the batch this lane ends up with
+    auto reduce_store = [&](const uint4* regs, const float* qv, float* srow, int bi) {
+        float dot[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            float f[8];
+            bf16x8_to_f32(regs[u], f);
+            float acc = 0.f;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) acc = fmaf(qv[t], f[t], acc);
+            dot[u] = acc;
+        }
+        float v4[4], v2[2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float send = (sub & 8) ? dot[i] : dot[i + 4];
+            const float keep = (sub & 8) ? dot[i + 4] : dot[i];
+            v4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const float send = (sub & 4) ? v4[i] : v4[i + 2];
+            const float keep = (sub & 4) ? v4[i + 2] : v4[i];
+            v2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+        }
+        const float send = (sub & 2) ? v2[0] : v2[1];
+        const float keep = (sub & 2) ? v2[1] : v2[0];
+        float v1 = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+        v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+        if ((sub & 1) == 0) srow[(bi * 8 + urow) * RSTEP + rsel] = v1 * inv_sqrt_d;
+    };
+    for (int h = warp; h < Hq; h += kWarps) {
+        const bool has_next = h + kWarps < Hq;
+        const uint4* np = has_next ? head_ptr(h + kWarps) : hp;
+        float qv[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) qv[t] = q_s[h * 128 + sub * 8 + t];
+        float* srow = s_s + h * kChunk;
+#pragma unroll
+        for (int bi = 0; bi < NB; bi += 2) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) rb[u] = ld_stream16(hp + ((bi + 1) * 8 + u) * RSTEP * LPR);
+            reduce_store(ra, qv, srow, bi);
+            if (bi + 2 < NB) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) ra[u] = ld_stream16(hp + ((bi + 2) * 8 + u) * RSTEP * LPR);
+            } else if (has_next) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) ra[u] = ld_stream16(np + u * RSTEP * LPR);
+            }
+            reduce_store(rb, qv, srow, bi + 1);
+        }
+        hp = np;
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Standard layer: scores from the K cache.
 // ---------------------------------------------------------------------------------------------
@@ -389,7 +463,9 @@ __global__ void __launch_bounds__(kThreads, 2) anchor_decode_chunk_kernel(const 
     }
     __syncthreads();
     const float inv_sqrt_d = rsqrtf((float)d);
-    if (p.cache_dtype == LISA_BF16) {
+    if (p.cache_dtype == LISA_BF16 && d == 128 && nrows == kChunk) {
+        anchor_qk_full_chunk(p, s_s, q_s, b, j0, inv_sqrt_d);
+    } else if (p.cache_dtype == LISA_BF16) {
         const int lpr = d / 8, rstep = 32 / lpr, sub = lane % lpr, rsel = lane / lpr;
         for (int h = warp; h < Hq; h += kWarps) {
             float qv[8];
