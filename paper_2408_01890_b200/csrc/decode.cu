@@ -58,6 +58,18 @@ __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float* f) {
 
 __device__ __forceinline__ float ldw(const void* p, int idx, int dtype) { return p ? ld_elem(p, idx, dtype) : 0.f; }
 
+__device__ __forceinline__ uint32_t f32_to_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+// d += a (16x8, row) . b (8x8, col), tf32 in, fp32 accumulate
+__device__ __forceinline__ void mma_tf32(float* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
 // Partial P.V of a FULL chunk (all kChunk rows valid), bf16 cache, LPR = d/8 lanes per V row.  A warp streams the
 // V rows of its heads as one software-pipelined sequence: two register sets of eight 16-byte loads per lane
 // alternate, and the last batch of a head already prefetches the first batch of the warp's next head, so loads
@@ -201,8 +213,8 @@ __device__ __forceinline__ void softmax_pv_chunk(const DecodeParams& p, float* s
 }
 
 // ---------------------------------------------------------------------------------------------
-// Shared layer.  HQ_C/M_C > 0: compile-time sizes, aligner in registers (ADD, two layers, bf16 cache,
-// M_C % 8 == 0, HQ_C % 4 == 0).  HQ_C == 0: any supported mode and size, per-thread scratch arrays.
+// Shared layer.  HQ_C/M_C > 0: compile-time sizes, aligner on the tensor cores (ADD, two layers, bf16 cache,
+// M_C % 8 == 0, HQ_C % 8 == 0).  HQ_C == 0: any supported mode and size, per-thread scratch arrays.
 // ---------------------------------------------------------------------------------------------
 template <int HQ_C, int M_C>
 __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_kernel(const __grid_constant__ DecodeParams p) {
@@ -220,9 +232,12 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
     float* s_s = smem;                      // [Hq][kChunk]  delta, then scores, then exp
     float* part_s = s_s + Hq * kChunk;      // [Hq][kChunk]  partial FFN output of the upper half
     float* qp_s = part_s + Hq * kChunk;     // [Hq][kMaxRank]
-    float* w1_s = qp_s + Hq * kMaxRank;     // [h_in][m]
-    float* w2_s = w1_s + h_in * m;          // [m][Hq]
-    float* b1_s = w2_s + m * Hq;            // [m]
+    // weight rows are padded in the tensor-core path (strides m + 8 and Hq + 4) so that the fragment loads of a
+    // warp spread over all shared-memory banks
+    const int w1_ld = HQ_C ? m + 8 : m, w2_ld = HQ_C ? Hq + 4 : Hq;
+    float* w1_s = qp_s + Hq * kMaxRank;     // [h_in][w1_ld]
+    float* w2_s = w1_s + h_in * w1_ld;      // [m][w2_ld]
+    float* b1_s = w2_s + m * w2_ld;         // [m]
     float* b2_s = b1_s + m;                 // [Hq]
 
     for (int e = tid; e < Hq * r; e += kThreads) {
@@ -230,10 +245,10 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
         qp_s[h * kMaxRank + x] = ld_elem(p.qp.ptr, b * p.qp.sb + h * p.qp.sh + x, p.qp.dtype);
     }
     if (p.integrate != LISA_INTEGRATE_PLUS) {
-        for (int e = tid; e < h_in * m; e += kThreads) w1_s[e] = ld_elem(p.w1, e, p.w_dtype);
+        for (int e = tid; e < h_in * m; e += kThreads) w1_s[(e / m) * w1_ld + e % m] = ld_elem(p.w1, e, p.w_dtype);
         for (int e = tid; e < m; e += kThreads) b1_s[e] = ldw(p.b1, e, p.w_dtype);
         if (p.ffn_layers == 2) {
-            for (int e = tid; e < m * Hq; e += kThreads) w2_s[e] = ld_elem(p.w2, e, p.w_dtype);
+            for (int e = tid; e < m * Hq; e += kThreads) w2_s[(e / Hq) * w2_ld + e % Hq] = ld_elem(p.w2, e, p.w_dtype);
             for (int e = tid; e < Hq; e += kThreads) b2_s[e] = ldw(p.b2, e, p.w_dtype);
         }
     }
@@ -286,48 +301,69 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
     float* outrow = p.out_scores ? p.out_scores + b * p.sc_sb + j0 + pos : nullptr;
 
     if constexpr (HQ_C > 0) {
-        // ADD, two-layer FFN; the two halves of the CTA split the hidden units of each position
-        constexpr int MH = M_C / 2;
-        float a[HQ_C], y[HQ_C];
+        // ADD, two-layer FFN on the tensor cores (mma.sync m16n8k8, tf32 operands, fp32 accumulation): a warp owns
+        // 16 positions of the chunk as the M dimension.  Layer 1: [16 x HQ] . [HQ x M]; its accumulator fragments,
+        // after bias and activation, ARE the A fragments of layer 2 when hidden unit 8j + 2t / 8j + 2t + 1 is taken
+        // as k-index t / t + 4 of k-step j (the order of the hidden units inside the sum is free), so nothing moves
+        // between lanes.  bf16 weights are exact in tf32; the fp32 score row is rounded to tf32 (2^-11 relative).
+        constexpr int KS1 = HQ_C / 8, NT1 = M_C / 8, KS2 = M_C / 8, NT2 = HQ_C / 8;
+        const int lane = tid & 31, warp = tid >> 5;
+        const int g = lane >> 2, t = lane & 3;
+        const int p0 = warp * 16 + g, p1 = p0 + 8;              // this lane's two position rows
+        const bool ok0 = p0 < nrows, ok1 = p1 < nrows;
+        const float* prow = p.prev + b * p.prev_sb + j0;
+        uint32_t afr[KS1][4];
 #pragma unroll
-        for (int h = 0; h < HQ_C; ++h) {
-            a[h] = valid ? prev[h * p.prev_sh] : 0.f;
-            y[h] = 0.f;
+        for (int ks = 0; ks < KS1; ++ks) {
+            const float* r0 = prow + (int64_t)(ks * 8 + t) * p.prev_sh;
+            const float* r1 = prow + (int64_t)(ks * 8 + t + 4) * p.prev_sh;
+            afr[ks][0] = f32_to_tf32(ok0 ? r0[p0] : 0.f);
+            afr[ks][1] = f32_to_tf32(ok1 ? r0[p1] : 0.f);
+            afr[ks][2] = f32_to_tf32(ok0 ? r1[p0] : 0.f);
+            afr[ks][3] = f32_to_tf32(ok1 ? r1[p1] : 0.f);
         }
-        const int u0 = half * MH;
-#pragma unroll 1
-        for (int ub = 0; ub < MH; ub += 4) {
-            float4 hacc = *reinterpret_cast<const float4*>(b1_s + u0 + ub);
+        float yacc[NT2][4];
 #pragma unroll
-            for (int h = 0; h < HQ_C; ++h) {
-                const float4 w = *reinterpret_cast<const float4*>(w1_s + h * M_C + u0 + ub);
-                hacc.x = fmaf(a[h], w.x, hacc.x); hacc.y = fmaf(a[h], w.y, hacc.y);
-                hacc.z = fmaf(a[h], w.z, hacc.z); hacc.w = fmaf(a[h], w.w, hacc.w);
+        for (int j2 = 0; j2 < NT2; ++j2) {
+            const float bb0 = b2_s[j2 * 8 + 2 * t], bb1 = b2_s[j2 * 8 + 2 * t + 1];
+            yacc[j2][0] = bb0; yacc[j2][1] = bb1; yacc[j2][2] = bb0; yacc[j2][3] = bb1;
+        }
+#pragma unroll
+        for (int j = 0; j < NT1; ++j) {
+            // one 8-wide slice of hidden units: layer 1, activation, then straight into layer 2 as k-step j
+            float hacc[4];
+            hacc[0] = hacc[2] = b1_s[j * 8 + 2 * t];
+            hacc[1] = hacc[3] = b1_s[j * 8 + 2 * t + 1];
+#pragma unroll
+            for (int ks = 0; ks < KS1; ++ks) {
+                const uint32_t w0 = __float_as_uint(w1_s[(ks * 8 + t) * w1_ld + j * 8 + g]);
+                const uint32_t w1v = __float_as_uint(w1_s[(ks * 8 + t + 4) * w1_ld + j * 8 + g]);
+                mma_tf32(hacc, afr[ks], w0, w1v);
             }
-            const float hv[4] = {act_apply(hacc.x, p.act), act_apply(hacc.y, p.act), act_apply(hacc.z, p.act),
-                                 act_apply(hacc.w, p.act)};
+            uint32_t hfr[4];
+            hfr[0] = f32_to_tf32(act_apply(hacc[0], p.act));   // (row g,   k = t)     <- column 2t
+            hfr[1] = f32_to_tf32(act_apply(hacc[2], p.act));   // (row g+8, k = t)
+            hfr[2] = f32_to_tf32(act_apply(hacc[1], p.act));   // (row g,   k = t + 4) <- column 2t + 1
+            hfr[3] = f32_to_tf32(act_apply(hacc[3], p.act));   // (row g+8, k = t + 4)
 #pragma unroll
-            for (int uu = 0; uu < 4; ++uu) {
-                const float* wrow = w2_s + (u0 + ub + uu) * HQ_C;
-#pragma unroll
-                for (int g4 = 0; g4 < HQ_C / 4; ++g4) {
-                    const float4 w = *reinterpret_cast<const float4*>(wrow + g4 * 4);
-                    y[g4 * 4 + 0] = fmaf(hv[uu], w.x, y[g4 * 4 + 0]); y[g4 * 4 + 1] = fmaf(hv[uu], w.y, y[g4 * 4 + 1]);
-                    y[g4 * 4 + 2] = fmaf(hv[uu], w.z, y[g4 * 4 + 2]); y[g4 * 4 + 3] = fmaf(hv[uu], w.w, y[g4 * 4 + 3]);
-                }
+            for (int j2 = 0; j2 < NT2; ++j2) {
+                const uint32_t w0 = __float_as_uint(w2_s[(j * 8 + 2 * t) * w2_ld + j2 * 8 + g]);
+                const uint32_t w1v = __float_as_uint(w2_s[(j * 8 + 2 * t + 1) * w2_ld + j2 * 8 + g]);
+                mma_tf32(yacc[j2], hfr, w0, w1v);
             }
         }
-        if (half == 1) {
+        // scores = FFN + A_Delta; yacc[j2]: [0] (p0, head 8 j2 + 2t), [1] (p0, +1), [2] (p1, 2t), [3] (p1, +1)
+        float* out0 = p.out_scores ? p.out_scores + b * p.sc_sb + j0 : nullptr;
 #pragma unroll
-            for (int g = 0; g < HQ_C; ++g) part_s[g * kChunk + pos] = y[g];
-        }
-        __syncthreads();
-        if (half == 0) {
+        for (int j2 = 0; j2 < NT2; ++j2) {
 #pragma unroll
-            for (int g = 0; g < HQ_C; ++g) {
-                const float sc = y[g] + part_s[g * kChunk + pos] + b2_s[g] + s_s[g * kChunk + pos];
-                s_s[g * kChunk + pos] = valid ? sc : -INFINITY;
-                if (valid && outrow) outrow[g * p.sc_sh] = sc;
+            for (int e = 0; e < 4; ++e) {
+                const int hh = j2 * 8 + 2 * t + (e & 1);
+                const int pp = (e & 2) ? p1 : p0;
+                const bool okp = (e & 2) ? ok1 : ok0;
+                const float sc = yacc[j2][e] + s_s[hh * kChunk + pp];
+                s_s[hh * kChunk + pp] = okp ? sc : -INFINITY;
+                if (okp && out0) out0[(int64_t)hh * p.sc_sh + pp] = sc;
             }
         }
     } else {
@@ -579,7 +615,7 @@ cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cud
     const int h_in = p.integrate == LISA_INTEGRATE_CONCAT ? 2 * p.Hq : p.Hq;
     const int m = p.integrate == LISA_INTEGRATE_PLUS ? 0 : p.m;
     const size_t smem = sizeof(float) * ((size_t)2 * p.Hq * kChunk + (size_t)p.Hq * kMaxRank + (size_t)h_in * m +
-                                         (size_t)m * p.Hq + m + p.Hq + 8);
+                                         (size_t)m * p.Hq + m + p.Hq + 8 + (size_t)h_in * 8 + (size_t)m * 4);
     dim3 grid(p.n_chunks, p.B);
     const bool fast = p.integrate == LISA_INTEGRATE_ADD && p.ffn_layers == 2 && c.dtype == LISA_BF16;
     cudaError_t e;
