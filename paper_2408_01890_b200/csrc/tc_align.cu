@@ -69,55 +69,67 @@ __device__ __forceinline__ void mma_f16(float* d, const uint32_t* a, uint32_t b0
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// Activation of two hidden units, packed to fp16 (the A-fragment format of the next MMA).
 template <int ACT>
-__device__ __forceinline__ float act1(float x) {
-    if constexpr (ACT == LISA_ACT_RELU) return fmaxf(x, 0.f);
+__device__ __forceinline__ uint32_t act_pack(float x0, float x1) {
+    if constexpr (ACT == LISA_ACT_RELU) return pack_f16(fmaxf(x0, 0.f), fmaxf(x1, 0.f));
     if constexpr (ACT == LISA_ACT_SILU) {
-        // x * sigmoid(x): one ex2 and one rcp (full-rate MUFU ops; the packed tanh is a quarter-rate op on this part)
-        float e, r;
-        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * -1.4426950408889634f));
-        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.f + e));
-        return x * r;
+        // x * sigmoid(x) = x / (1 + 2^(-x log2 e)).  The transcendental pipe is the scarce unit here (64 hidden units
+        // per position), so the pair shares its MUFU work: one packed-fp16 ex2 for both exponentials and ONE
+        // reciprocal, of the product of the two denominators (1/d0 = d1 * r, 1/d1 = d0 * r).  Denominators are
+        // clamped so that their product stays finite; sigmoid is then below 2^-60 anyway.
+        const __half2 xh = __floats2half2_rn(x0 * -1.4426950408889634f, x1 * -1.4426950408889634f);
+        uint32_t eh;
+        asm("ex2.approx.ftz.f16x2 %0, %1;" : "=r"(eh) : "r"(*reinterpret_cast<const uint32_t*>(&xh)));
+        const float2 e = unpack_f16(eh);
+        const float d0 = fminf(1.f + e.x, 1e18f), d1 = fminf(1.f + e.y, 1e18f);
+        float r;
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(d0 * d1));
+        return pack_f16(x0 * (d1 * r), x1 * (d0 * r));
     }
-    return x;
+    return pack_f16(x0, x1);
 }
 
 // One link on a warp's 16 positions: afr = A fragments (2 k-steps of 16 heads) -> y = W2^T act(W1^T a + b1) + b2
-// as four accumulator tiles of 8 heads.
+// as four accumulator tiles of 8 heads.  All eight hidden tiles are accumulated before the activation, so that
+// sixteen independent MMAs are in flight, then the sixteen of the second layer.
 template <int ACT>
 __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* w1f, const uint2* w2f, const float* b1, const float* b2,
                                          int lane, float (*y)[4]) {
     const int t = lane & 3;
+    float h[8][4];
 #pragma unroll
-    for (int j2 = 0; j2 < 4; ++j2) {
-        const float c0 = b2[j2 * 8 + 2 * t], c1 = b2[j2 * 8 + 2 * t + 1];
-        y[j2][0] = c0; y[j2][1] = c1; y[j2][2] = c0; y[j2][3] = c1;
+    for (int j = 0; j < 8; ++j) {
+        const float2 bb = *reinterpret_cast<const float2*>(b1 + j * 8 + 2 * t);
+        h[j][0] = bb.x; h[j][1] = bb.y; h[j][2] = bb.x; h[j][3] = bb.y;
     }
 #pragma unroll
-    for (int s = 0; s < 4; ++s) {   // 16 hidden units at a time: layer 1, activation, then k-step s of layer 2
-        float h[2][4];
+    for (int ks = 0; ks < 2; ++ks)
 #pragma unroll
-        for (int jj = 0; jj < 2; ++jj) {
-            const int j = 2 * s + jj;
-            const float c0 = b1[j * 8 + 2 * t], c1 = b1[j * 8 + 2 * t + 1];
-            h[jj][0] = c0; h[jj][1] = c1; h[jj][2] = c0; h[jj][3] = c1;
-#pragma unroll
-            for (int ks = 0; ks < 2; ++ks) {
-                const uint2 w = w1f[(ks * 8 + j) * 32 + lane];
-                mma_f16(h[jj], afr[ks], w.x, w.y);
-            }
+        for (int j = 0; j < 8; ++j) {
+            const uint2 w = w1f[(ks * 8 + j) * 32 + lane];
+            mma_f16(h[j], afr[ks], w.x, w.y);
         }
-        uint32_t hfr[4];
-        hfr[0] = pack_f16(act1<ACT>(h[0][0]), act1<ACT>(h[0][1]));
-        hfr[1] = pack_f16(act1<ACT>(h[0][2]), act1<ACT>(h[0][3]));
-        hfr[2] = pack_f16(act1<ACT>(h[1][0]), act1<ACT>(h[1][1]));
-        hfr[3] = pack_f16(act1<ACT>(h[1][2]), act1<ACT>(h[1][3]));
+    uint32_t hfr[4][4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        hfr[s][0] = act_pack<ACT>(h[2 * s][0], h[2 * s][1]);
+        hfr[s][1] = act_pack<ACT>(h[2 * s][2], h[2 * s][3]);
+        hfr[s][2] = act_pack<ACT>(h[2 * s + 1][0], h[2 * s + 1][1]);
+        hfr[s][3] = act_pack<ACT>(h[2 * s + 1][2], h[2 * s + 1][3]);
+    }
+#pragma unroll
+    for (int j2 = 0; j2 < 4; ++j2) {
+        const float2 bb = *reinterpret_cast<const float2*>(b2 + j2 * 8 + 2 * t);
+        y[j2][0] = bb.x; y[j2][1] = bb.y; y[j2][2] = bb.x; y[j2][3] = bb.y;
+    }
+#pragma unroll
+    for (int s = 0; s < 4; ++s)
 #pragma unroll
         for (int j2 = 0; j2 < 4; ++j2) {
             const uint2 w = w2f[(s * 4 + j2) * 32 + lane];
-            mma_f16(y[j2], hfr, w.x, w.y);
+            mma_f16(y[j2], hfr[s], w.x, w.y);
         }
-    }
 }
 
 struct TensorMaps {
