@@ -80,7 +80,7 @@ __device__ __forceinline__ uint32_t act_pack(float x0, float x1) {
         // clamped so that their product stays finite; sigmoid is then below 2^-60 anyway.
         const __half2 xh = __floats2half2_rn(x0 * -1.4426950408889634f, x1 * -1.4426950408889634f);
         uint32_t eh;
-        asm("ex2.approx.ftz.f16x2 %0, %1;" : "=r"(eh) : "r"(*reinterpret_cast<const uint32_t*>(&xh)));
+        asm("ex2.approx.f16x2 %0, %1;" : "=r"(eh) : "r"(*reinterpret_cast<const uint32_t*>(&xh)));
         const float2 e = unpack_f16(eh);
         const float d0 = fminf(1.f + e.x, 1e18f), d1 = fminf(1.f + e.y, 1e18f);
         float r;
