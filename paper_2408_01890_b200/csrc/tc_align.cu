@@ -7,21 +7,22 @@
 // Y = log2(e) * FFN_c(A_{c-1}) where A_k = FFN_k(A_{k-1}) + D_k (Eq. 4, ADD) -- the final link's D_c is added by
 // the attention kernel that consumes Y.  Hq = 32 heads, hidden width 64, two-layer FFNs.
 //
-// A work unit is 128 consecutive key positions of one query row: one [head][position] slab of 8 KB per plane,
-// brought in by one TMA copy.  A warp owns 16 positions as the M dimension of warp-level MMAs (mma.sync m16n8k16,
-// fp16 in, fp32 accumulate) and keeps the whole chain in registers:
-//   H = A [16 x 32] . W1 [32 x 64]      A fragments come straight from the slab with ldmatrix.trans, so the
+// A warp owns strips of 16 key positions of one query row as the M dimension of warp-level MMAs (mma.sync
+// m16n8k16, fp16 in, fp32 accumulate) and keeps the whole chain in registers:
+//   H = A [16 x 32] . W1 [32 x 64]      A fragments: lane h loads [head h][16 positions] (32 B), parks it in the warp's
+//                                        scratch and ldmatrix.trans hands out the fragments, so the
 //                                        [head][position] -> [position][head] transposition costs nothing
 //   Y = act(H + b1) [16 x 64] . W2      the accumulator fragments of H, packed to fp16, ARE the A fragments of this MMA
 //   A_k = Y + b2 + D_k                  D_k read with the same ldmatrix.trans; packed again it feeds the next link
-// and the last Y goes back to a slab-shaped staging buffer with stmatrix.trans and out with one TMA store.
+// and the last Y goes back through the scratch with stmatrix.trans, 32 bytes per head and lane.
 // Why not tcgen05 here: the contractions are tiny (K = 32/64, N = 64/32) and an elementwise step sits between any
 // two of them, so with tensor-memory accumulators every step pays a round trip through TMEM, shared memory and an
 // mbarrier hand-off between the issuing thread and the threads that apply the activation; measured on B200 that
 // version spent ~13 clocks per position and link (tensor pipe 5% busy).  mma.sync runs at a quarter of the tcgen05
 // rate (measured 555 TFLOP/s) but needs 4 clocks per position and link with nothing leaving the registers.
-// Warp roles: eight MMA warps, one producer warp (TMA loads ahead through a ring of slab slots, TMA stores).
-// Every wait is bounded; on expiry the CTA records it in the status word and exits.
+// A TMA-fed variant of this kernel (producer warp, slab ring) was slower: one copy per 128 positions gathers 64
+// rows of 128 bytes from 32 planes and took the issuing thread ~2000 cycles.  Here every warp is independent: no
+// block-wide barrier after set-up, no mbarrier, no wait that could hang.
 #include <algorithm>
 
 #include "common.cuh"
@@ -47,6 +48,8 @@ struct AlignParams {
     int B, N, chain;               // chain = number of links applied here (c)
     int row0, qt_begin, qt_count;  // planes hold query rows row0.. ; this launch covers tiles [qt_begin, qt_begin + qt_count)
     int units_per_batch;           // sum over the covered tiles of valid rows x key blocks
+    int64_t plane_rows, plane_cols;
+    __half* planes[kMaxTcChain];   // [0] = A_0 in / Y out; [k] = D_k for k = 1..c-1; each [B*32][plane_rows][plane_cols]
     const void *w1[kMaxTcChain], *b1[kMaxTcChain], *w2[kMaxTcChain], *b2[kMaxTcChain];
     int w_dtype[kMaxTcChain], act[kMaxTcChain];
     int* status;
@@ -132,39 +135,63 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
         }
 }
 
-struct TensorMaps {
-    CUtensorMap m[kMaxTcChain];
-};
-
-__global__ void __launch_bounds__(kThreads, 2)
-tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ TensorMaps maps) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+// Each warp works alone on strips of 16 key positions of one query row: no block-wide barrier, no producer warp.
+//   global -> registers  lane h loads the 32 bytes [head h][16 positions] of every input plane (prefetched one
+//                        strip ahead, so the loads overlap the previous strip's MMAs)
+//   registers -> shared  into the warp's private scratch, then ldmatrix.trans yields the A / D fragments
+//   chain in registers   (ffn_link)
+//   result               stmatrix.trans into the scratch, lane h reads its 32 bytes back and stores them
+__global__ void __launch_bounds__(kWorkers, 2)
+tc_align_kernel(const __grid_constant__ AlignParams p) {
+    extern __shared__ __align__(16) uint8_t smem[];
     const int c = p.chain;
-    // layout: [kStages slots][c slabs] | out staging [2] | per link: W1 fragments, W2 fragments, b1[64], b2[32] | barriers
-    uint8_t* sSlab = smem;
-    uint8_t* sOut = sSlab + kStages * c * SLAB_BYTES;
-    uint8_t* sW = sOut + 2 * SLAB_BYTES;
     constexpr int LINK_BYTES = W1F_BYTES + W2F_BYTES + (MH + HQ) * 4;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sW + c * LINK_BYTES);
-    uint64_t* full = bars;                     // [kStages] slot filled by TMA
-    uint64_t* slot_free = bars + kStages;      // [kStages] all eight MMA warps are done with the slot
-    uint64_t* out_ready = bars + 2 * kStages;  // [2] staging buffer written by all eight warps
-    uint64_t* out_free = out_ready + 2;        // [2] its TMA store has read it
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(out_free + 2);
-
+    uint8_t* sW = smem;                               // per link: W1 fragments, W2 fragments, b1[64], b2[32]
+    uint8_t* sScr = sW + c * LINK_BYTES;              // per warp: c planes x [32 heads][32 B]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n_units = p.units_per_batch * p.B;
-    // Every CTA owns a contiguous range of units; units are numbered batch by batch, tile by tile, row by row,
-    // key block by key block, so a cursor steps through them without any division.
-    const int per_cta = (n_units + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int u_begin = min(n_units, (int)blockIdx.x * per_cta), u_end = min(n_units, u_begin + per_cta);
-    const int n_mine = u_end - u_begin;
-    struct Cursor { int b, t, row, jb; };   // batch, query tile, row inside the tile, key block
-    auto cursor_at = [&](int u) {
-        Cursor cu;
-        cu.b = u / p.units_per_batch;
-        int rem = u - cu.b * p.units_per_batch;
+
+    // ---- one-time set-up: weights as ready-made B fragments (fp16, the last link's W2/b2 times log2 e) ----
+    for (int k = 0; k < c; ++k) {
+        uint2* w1f = reinterpret_cast<uint2*>(sW + k * LINK_BYTES);
+        uint2* w2f = reinterpret_cast<uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
+        float* bias = reinterpret_cast<float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
+        const float out_scale = k == c - 1 ? kLog2e : 1.f;
+        const int wd = p.w_dtype[k];
+        for (int e = tid; e < 2 * 8 * 32; e += kWorkers) {   // W1 [32 heads][64 hidden]: k = head, n = hidden
+            const int ln = e & 31, j = (e >> 5) & 7, ks = e >> 8, g = ln >> 2, t = ln & 3;
+            const int k0 = ks * 16 + 2 * t, n = j * 8 + g;
+            uint2 w;
+            w.x = pack_f16(ld_elem(p.w1[k], k0 * MH + n, wd), ld_elem(p.w1[k], (k0 + 1) * MH + n, wd));
+            w.y = pack_f16(ld_elem(p.w1[k], (k0 + 8) * MH + n, wd), ld_elem(p.w1[k], (k0 + 9) * MH + n, wd));
+            w1f[e] = w;
+        }
+        for (int e = tid; e < 4 * 4 * 32; e += kWorkers) {   // W2 [64 hidden][32 heads]: k = hidden, n = head
+            const int ln = e & 31, j2 = (e >> 5) & 3, s2 = e >> 7, g = ln >> 2, t = ln & 3;
+            const int k0 = s2 * 16 + 2 * t, n = j2 * 8 + g;
+            uint2 w;
+            w.x = pack_f16(ld_elem(p.w2[k], k0 * HQ + n, wd) * out_scale, ld_elem(p.w2[k], (k0 + 1) * HQ + n, wd) * out_scale);
+            w.y = pack_f16(ld_elem(p.w2[k], (k0 + 8) * HQ + n, wd) * out_scale, ld_elem(p.w2[k], (k0 + 9) * HQ + n, wd) * out_scale);
+            w2f[e] = w;
+        }
+        for (int e = tid; e < MH; e += kWorkers) bias[e] = ldw(p.b1[k], e, wd);
+        for (int e = tid; e < HQ; e += kWorkers) bias[MH + e] = ldw(p.b2[k], e, wd) * out_scale;
+    }
+    __syncthreads();
+
+    // ---- this warp's contiguous range of strips; strips are numbered unit by unit (8 per 128-position unit) ----
+    const long long n_strips = (long long)p.units_per_batch * p.B * 8;
+    const long long n_warps = (long long)gridDim.x * (kWorkers / 32);
+    const long long per_warp = (n_strips + n_warps - 1) / n_warps;
+    const long long s_begin = min(n_strips, ((long long)blockIdx.x * (kWorkers / 32) + warp) * per_warp);
+    const long long s_end = min(n_strips, s_begin + per_warp);
+    if (s_begin >= s_end) return;
+    struct Cursor { int b, t, row, jb, sub; };   // batch, query tile, row in the tile, key block, 16-position strip in the block
+    Cursor cu;
+    {
+        const long long u = s_begin >> 3;
+        cu.sub = (int)(s_begin & 7);
+        cu.b = (int)(u / p.units_per_batch);
+        int rem = (int)(u - (long long)cu.b * p.units_per_batch);
         cu.t = p.qt_begin;
         for (;; ++cu.t) {
             const int n_t = min(UNIT, p.N - cu.t * UNIT) * (cu.t + 1);
@@ -173,165 +200,116 @@ tc_align_kernel(const __grid_constant__ AlignParams p, const __grid_constant__ T
         }
         cu.row = rem / (cu.t + 1);
         cu.jb = rem - cu.row * (cu.t + 1);
-        return cu;
+    }
+    auto advance = [&](Cursor& x) {
+        if (++x.sub < 8) return;
+        x.sub = 0;
+        if (++x.jb <= x.t) return;
+        x.jb = 0;
+        if (++x.row < min(UNIT, p.N - x.t * UNIT)) return;
+        x.row = 0;
+        if (++x.t < p.qt_begin + p.qt_count) return;
+        x.t = p.qt_begin;
+        ++x.b;
     };
-    auto advance = [&](Cursor& cu) {
-        if (++cu.jb <= cu.t) return;
-        cu.jb = 0;
-        if (++cu.row < min(UNIT, p.N - cu.t * UNIT)) return;
-        cu.row = 0;
-        if (++cu.t < p.qt_begin + p.qt_count) return;
-        cu.t = p.qt_begin;
-        ++cu.b;
+    // element offset of [head = lane][this strip] inside a plane set
+    auto strip_off = [&](const Cursor& x) {
+        return ((int64_t)(x.b * HQ + lane) * p.plane_rows + (x.t * UNIT + x.row - p.row0)) * p.plane_cols + x.jb * UNIT + x.sub * 16;
     };
 
-    // ---- one-time set-up: barriers; weights as ready-made B fragments (fp16, the last link's W2/b2 times log2 e) ----
-    if (tid == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(full + i, 1); mbar_init(slot_free + i, 8); }
-        for (int i = 0; i < 2; ++i) { mbar_init(out_ready + i, 8); mbar_init(out_free + i, 1); }
-        *abort_flag = 0;
-        fence_barrier_init();
-    }
-    for (int k = 0; k < c; ++k) {
-        uint2* w1f = reinterpret_cast<uint2*>(sW + k * LINK_BYTES);
-        uint2* w2f = reinterpret_cast<uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
-        float* bias = reinterpret_cast<float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
-        const float out_scale = k == c - 1 ? kLog2e : 1.f;
-        const int wd = p.w_dtype[k];
-        for (int e = tid; e < 2 * 8 * 32; e += kThreads) {   // W1 [32 heads][64 hidden]: k = head, n = hidden
-            const int ln = e & 31, j = (e >> 5) & 7, ks = e >> 8, g = ln >> 2, t = ln & 3;
-            const int k0 = ks * 16 + 2 * t, n = j * 8 + g;
-            uint2 w;
-            w.x = pack_f16(ld_elem(p.w1[k], k0 * MH + n, wd), ld_elem(p.w1[k], (k0 + 1) * MH + n, wd));
-            w.y = pack_f16(ld_elem(p.w1[k], (k0 + 8) * MH + n, wd), ld_elem(p.w1[k], (k0 + 9) * MH + n, wd));
-            w1f[e] = w;
-        }
-        for (int e = tid; e < 4 * 4 * 32; e += kThreads) {   // W2 [64 hidden][32 heads]: k = hidden, n = head
-            const int ln = e & 31, j2 = (e >> 5) & 3, s2 = e >> 7, g = ln >> 2, t = ln & 3;
-            const int k0 = s2 * 16 + 2 * t, n = j2 * 8 + g;
-            uint2 w;
-            w.x = pack_f16(ld_elem(p.w2[k], k0 * HQ + n, wd) * out_scale, ld_elem(p.w2[k], (k0 + 1) * HQ + n, wd) * out_scale);
-            w.y = pack_f16(ld_elem(p.w2[k], (k0 + 8) * HQ + n, wd) * out_scale, ld_elem(p.w2[k], (k0 + 9) * HQ + n, wd) * out_scale);
-            w2f[e] = w;
-        }
-        for (int e = tid; e < MH; e += kThreads) bias[e] = ldw(p.b1[k], e, wd);
-        for (int e = tid; e < HQ; e += kThreads) bias[MH + e] = ldw(p.b2[k], e, wd) * out_scale;
-    }
-    __syncthreads();
+    uint8_t* scr = sScr + warp * c * 1024;
+    // scratch layout per plane: row = head (32 B), its two 16-byte halves swapped for heads 4..7 of every 8 so that
+    // the eight rows of an 8x8 matrix fall into distinct banks
+    const int my_sw = (lane >> 2) & 1;
+    const uint32_t st_off0 = lane * 32 + ((0 ^ my_sw) << 4), st_off1 = lane * 32 + ((1 ^ my_sw) << 4);
+    const int mi = lane >> 3, lr = lane & 7;               // ldmatrix/stmatrix: matrix index and row supplied by this lane
+    auto frag_off = [&](int x) {                           // 16-head block x, head block half (mi >> 1), position half (mi & 1)
+        const int head = x * 16 + 8 * (mi >> 1) + lr;
+        return (uint32_t)(head * 32 + (((mi & 1) ^ ((head >> 2) & 1)) << 4));
+    };
+    const uint32_t off0 = frag_off(0), off1 = frag_off(1);
+    const uint32_t scr_a = smem_u32(scr);
 
-    if (warp == 8) {
-        // =========================== producer: TMA loads ahead, TMA stores behind ===========================
-        Cursor cl = cursor_at(u_begin), cs = cl;
-        if (lane == 0) for (int k = 0; k < c; ++k) tma_prefetch_desc(&maps.m[k]);
-        bool ok = true;
-        int n_loaded = 0;
-        auto load_next = [&]() {   // whole warp; lanes 0..c-1 issue one slab copy each
-            const int slot = n_loaded % kStages;
-            if (lane == 0) {
-                ok = n_loaded < kStages || mbar_wait(slot_free + slot, (n_loaded / kStages - 1) & 1, abort_flag);
-                if (ok) mbar_expect_tx(full + slot, c * SLAB_BYTES);
+    uint4 cur[kMaxTcChain][2], nxt[kMaxTcChain][2];
+    {
+        const int64_t o = strip_off(cu);
+#pragma unroll
+        for (int k = 0; k < kMaxTcChain; ++k)
+            if (k < c) {
+                const uint4* src = reinterpret_cast<const uint4*>(p.planes[k] + o);
+                cur[k][0] = src[0]; cur[k][1] = src[1];
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (ok && lane < c)
-                tma_load_4d(sSlab + (slot * c + lane) * SLAB_BYTES, &maps.m[lane], full + slot, 0, cl.b * HQ, cl.jb * 2,
-                            cl.t * UNIT + cl.row - p.row0);
-            __syncwarp();
-            advance(cl);
-            ++n_loaded;
-        };
-        for (int i = 0; i < kStages - 1 && n_loaded < n_mine && ok; ++i) load_next();
-        for (int u = 0; ok && u < n_mine; ++u) {
-            if (n_loaded < n_mine) load_next();
-            if (!ok) break;
-            const int buf = u & 1;
-            if (lane == 0) {
-                ok = mbar_wait(out_ready + buf, (u >> 1) & 1, abort_flag);
-                if (ok) {
-                    tma_store_4d(&maps.m[0], sOut + buf * SLAB_BYTES, 0, cs.b * HQ, cs.jb * 2, cs.t * UNIT + cs.row - p.row0);
-                    tma_store_commit();
-                    tma_store_wait_read<0>();
-                    mbar_arrive(out_free + buf);
+    }
+    for (long long sidx = s_begin; sidx < s_end; ++sidx) {
+        const int64_t o_cur = strip_off(cu);
+        advance(cu);
+#pragma unroll
+        for (int k = 0; k < kMaxTcChain; ++k)
+            if (k < c) {
+                *reinterpret_cast<uint4*>(scr + k * 1024 + st_off0) = cur[k][0];
+                *reinterpret_cast<uint4*>(scr + k * 1024 + st_off1) = cur[k][1];
+            }
+        __syncwarp();
+        if (sidx + 1 < s_end) {
+            const int64_t o = strip_off(cu);
+#pragma unroll
+            for (int k = 0; k < kMaxTcChain; ++k)
+                if (k < c) {
+                    const uint4* src = reinterpret_cast<const uint4*>(p.planes[k] + o);
+                    nxt[k][0] = src[0]; nxt[k][1] = src[1];
                 }
-            }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            advance(cs);
         }
-        if (lane == 0) tma_store_wait_all<0>();
-    } else {
-        // =========================== MMA warps: 16 positions each ===========================
-        const int half = warp >> 2, c0 = (warp & 3) * 2;       // 64-position half and first 8-position chunk of this warp
-        const int mi = lane >> 3, lr = lane & 7;               // ldmatrix/stmatrix: matrix index and row supplied by this lane
-        const int chunk = c0 + (mi & 1);
-        // byte offset inside a slab of the 16-byte row this lane addresses, for the head block (mi >> 1) of k-step/tile pair x
-        auto frag_off = [&](int x) {
-            const int head = x * 16 + 8 * (mi >> 1) + lr;
-            return half * (HQ * 128) + head * 128 + ((chunk ^ (head & 7)) << 4);
-        };
-        const int off0 = frag_off(0), off1 = frag_off(1);
-        bool ok = true;
-        for (int u = 0; ok && u < n_mine; ++u) {
-            const int slot = u % kStages;
-            if (!(ok = mbar_wait(full + slot, (u / kStages) & 1, abort_flag))) break;
-            const uint32_t slabs = smem_u32(sSlab + slot * c * SLAB_BYTES);
-            uint32_t afr[2][4];
-            ldmatrix_x4_trans(afr[0], slabs + off0);
-            ldmatrix_x4_trans(afr[1], slabs + off1);
-            float y[4][4];
-            for (int k = 0; k < c; ++k) {
-                const uint2* w1f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES);
-                const uint2* w2f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
-                const float* b1 = reinterpret_cast<const float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
-                const int act = p.act[k];
-                if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU>(afr, w1f, w2f, b1, b1 + MH, lane, y);
-                else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU>(afr, w1f, w2f, b1, b1 + MH, lane, y);
-                else ffn_link<LISA_ACT_NONE>(afr, w1f, w2f, b1, b1 + MH, lane, y);
-                if (k + 1 < c) {
-                    // A_{k+1} = y + D_{k+1}; the difference comes in the same fragment arrangement as A did
+        uint32_t afr[2][4];
+        ldmatrix_x4_trans(afr[0], scr_a + off0);
+        ldmatrix_x4_trans(afr[1], scr_a + off1);
+        float y[4][4];
+        for (int k = 0; k < c; ++k) {
+            const uint2* w1f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES);
+            const uint2* w2f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
+            const float* b1 = reinterpret_cast<const float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
+            const int act = p.act[k];
+            if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU>(afr, w1f, w2f, b1, b1 + MH, lane, y);
+            else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU>(afr, w1f, w2f, b1, b1 + MH, lane, y);
+            else ffn_link<LISA_ACT_NONE>(afr, w1f, w2f, b1, b1 + MH, lane, y);
+            if (k + 1 < c) {
+                // A_{k+1} = y + D_{k+1}; the difference comes in the same fragment arrangement as A did
 #pragma unroll
-                    for (int x = 0; x < 2; ++x) {
-                        uint32_t dfr[4];
-                        ldmatrix_x4_trans(dfr, slabs + (k + 1) * SLAB_BYTES + (x ? off1 : off0));
+                for (int x = 0; x < 2; ++x) {
+                    uint32_t dfr[4];
+                    ldmatrix_x4_trans(dfr, scr_a + (k + 1) * 1024 + (x ? off1 : off0));
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float2 dv = unpack_f16(dfr[q]);
-                            float* yy = y[2 * x + (q >> 1)] + 2 * (q & 1);
-                            afr[x][q] = pack_f16(yy[0] + dv.x, yy[1] + dv.y);
-                        }
+                    for (int q = 0; q < 4; ++q) {
+                        const float2 dv = unpack_f16(dfr[q]);
+                        float* yy = y[2 * x + (q >> 1)] + 2 * (q & 1);
+                        afr[x][q] = pack_f16(yy[0] + dv.x, yy[1] + dv.y);
                     }
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(slot_free + slot);   // this warp has read everything it needs from the slot
-            // result -> slab-shaped staging buffer ([head][position], swizzled), transposed by stmatrix
-            const int buf = u & 1;
-            if (u >= 2 && !(ok = mbar_wait(out_free + buf, ((u >> 1) - 1) & 1, abort_flag))) break;
-            const uint32_t stg = smem_u32(sOut + buf * SLAB_BYTES);
-#pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                uint32_t r[4];
-                r[0] = pack_f16(y[2 * x][0], y[2 * x][1]);
-                r[1] = pack_f16(y[2 * x][2], y[2 * x][3]);
-                r[2] = pack_f16(y[2 * x + 1][0], y[2 * x + 1][1]);
-                r[3] = pack_f16(y[2 * x + 1][2], y[2 * x + 1][3]);
-                stmatrix_x4_trans(stg + (x ? off1 : off0), r);
-            }
-            fence_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(out_ready + buf);
         }
-    }
-    __syncthreads();
-    if (*abort_flag) {
-        // a wait ran out: record it and give copies still in flight time to land before the CTA's memory is released
-        if (tid == 0) atomicAdd(p.status + 1, 1);
-        const long long t0 = clock64();
-        while (clock64() - t0 < 4000000ll) __nanosleep(1000);
-        __syncthreads();
+        // result -> scratch plane 0 ([head][position]), transposed by stmatrix; then lane h stores head h's 32 bytes
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            uint32_t r[4];
+            r[0] = pack_f16(y[2 * x][0], y[2 * x][1]);
+            r[1] = pack_f16(y[2 * x][2], y[2 * x][3]);
+            r[2] = pack_f16(y[2 * x + 1][0], y[2 * x + 1][1]);
+            r[3] = pack_f16(y[2 * x + 1][2], y[2 * x + 1][3]);
+            stmatrix_x4_trans(scr_a + (x ? off1 : off0), r);
+        }
+        __syncwarp();
+        {
+            uint4* dst = reinterpret_cast<uint4*>(p.planes[0] + o_cur);
+            dst[0] = *reinterpret_cast<const uint4*>(scr + st_off0);
+            dst[1] = *reinterpret_cast<const uint4*>(scr + st_off1);
+        }
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < kMaxTcChain; ++k) { cur[k][0] = nxt[k][0]; cur[k][1] = nxt[k][1]; }
     }
 }
 
 size_t align_smem_bytes(int c) {
-    return (size_t)kStages * c * SLAB_BYTES + 2 * SLAB_BYTES + (size_t)c * (W1F_BYTES + W2F_BYTES + (MH + HQ) * 4) + 256 + 1024;
+    return (size_t)c * (W1F_BYTES + W2F_BYTES + (MH + HQ) * 4) + (size_t)(kWorkers / 32) * c * 1024 + 16;
 }
 
 }  // namespace
@@ -347,33 +325,28 @@ bool tc_align_supported(int Hq, const lisa_link* links, int chain) {
 
 cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     AlignParams p{};
-    TensorMaps maps;
     p.B = a.B; p.N = a.N; p.chain = a.chain;
     p.row0 = a.qt_begin * UNIT; p.qt_begin = a.qt_begin; p.qt_count = a.qt_count;
+    p.plane_rows = a.plane_rows; p.plane_cols = a.plane_cols;
     p.units_per_batch = 0;
     for (int t = a.qt_begin; t < a.qt_begin + a.qt_count; ++t) p.units_per_batch += std::min(UNIT, a.N - t * UNIT) * (t + 1);
     for (int k = 0; k < a.chain; ++k) {
+        p.planes[k] = reinterpret_cast<__half*>(a.planes[k]);
         const lisa_link& l = a.links[k];
         p.w1[k] = l.w1; p.b1[k] = l.b1; p.w2[k] = l.w2; p.b2[k] = l.b2;
         p.w_dtype[k] = l.w_dtype; p.act[k] = l.act;
-        // 4-D view of the [B*Hq][rows][cols] planes: (column inside a 64-block, plane, 64-block, row).  A box of
-        // 64 x 32 x 2 x 1 lands in shared memory as [half][head][64 positions]: one unit's slab in one copy.
-        const uint64_t dims[4] = {64, (uint64_t)a.B * HQ, (uint64_t)a.plane_cols / 64, (uint64_t)a.plane_rows};
-        const uint64_t str[3] = {(uint64_t)a.plane_cols * a.plane_rows * 2, 128, (uint64_t)a.plane_cols * 2};
-        const uint32_t box[4] = {64, HQ, 2, 1};
-        if (!make_tensor_map_bf16(&maps.m[k], a.planes[k], 4, dims, str, box, true)) return cudaErrorInvalidValue;
     }
-    for (int k = a.chain; k < kMaxTcChain; ++k) maps.m[k] = maps.m[0];
     p.status = status_words();
     if (!p.status) return cudaErrorUnknown;
+    if (a.plane_cols % 16 != 0) return cudaErrorInvalidValue;   // strips are loaded as aligned 32-byte pieces
     const size_t smem = align_smem_bytes(a.chain);
     cudaError_t e = cudaFuncSetAttribute(tc_align_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const int64_t total_units = (int64_t)p.units_per_batch * a.B;
     if (total_units <= 0 || total_units > 0x7fffffff) return cudaErrorInvalidValue;
     const int max_ctas = a.ctas > 0 ? a.ctas : 148 * 2;
-    dim3 grid((unsigned)std::min<int64_t>((total_units + 7) / 8, max_ctas));  // at least eight units per CTA
-    tc_align_kernel<<<grid, kThreads, smem, stream>>>(p, maps);
+    dim3 grid((unsigned)std::min<int64_t>((total_units + 3) / 4, max_ctas));  // at least four strips per warp
+    tc_align_kernel<<<grid, kWorkers, smem, stream>>>(p);
     count_launches(1);
     return cudaGetLastError();
 }
