@@ -135,19 +135,18 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
         }
 }
 
-// Each warp works alone on strips of 16 key positions of one query row: no block-wide barrier, no producer warp.
-//   global -> registers  lane h loads the 32 bytes [head h][16 positions] of every input plane (prefetched one
-//                        strip ahead, so the loads overlap the previous strip's MMAs)
-//   registers -> shared  into the warp's private scratch, then ldmatrix.trans yields the A / D fragments
+// Each warp works alone on pieces of 32 key positions of one query row: no block-wide barrier, no producer warp.
+//   global -> scratch    cp.async, 16 bytes per lane, four lanes per head (64 contiguous bytes), one piece ahead
+//   scratch -> fragments ldmatrix.trans per 16-position strip
 //   chain in registers   (ffn_link)
-//   result               stmatrix.trans into the scratch, lane h reads its 32 bytes back and stores them
+//   result               stmatrix.trans back into the scratch, then 16 bytes per lane to the plane
 __global__ void __launch_bounds__(kWorkers, 2)
 tc_align_kernel(const __grid_constant__ AlignParams p) {
     extern __shared__ __align__(16) uint8_t smem[];
     const int c = p.chain;
     constexpr int LINK_BYTES = W1F_BYTES + W2F_BYTES + (MH + HQ) * 4;
     uint8_t* sW = smem;                               // per link: W1 fragments, W2 fragments, b1[64], b2[32]
-    uint8_t* sScr = sW + c * LINK_BYTES;              // per warp: c planes x [32 heads][32 B]
+    uint8_t* sScr = sW + c * LINK_BYTES;              // per warp: two buffers of c planes x [32 heads][64 B]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // ---- one-time set-up: weights as ready-made B fragments (fp16, the last link's W2/b2 times log2 e) ----
@@ -178,18 +177,18 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
     }
     __syncthreads();
 
-    // ---- this warp's contiguous range of strips; strips are numbered unit by unit (8 per 128-position unit) ----
-    const long long n_strips = (long long)p.units_per_batch * p.B * 8;
+    // ---- this warp's contiguous range of pieces; a piece is 32 positions (4 per 128-position unit) ----
+    const long long n_pieces = (long long)p.units_per_batch * p.B * 4;
     const long long n_warps = (long long)gridDim.x * (kWorkers / 32);
-    const long long per_warp = (n_strips + n_warps - 1) / n_warps;
-    const long long s_begin = min(n_strips, ((long long)blockIdx.x * (kWorkers / 32) + warp) * per_warp);
-    const long long s_end = min(n_strips, s_begin + per_warp);
+    const long long per_warp = (n_pieces + n_warps - 1) / n_warps;
+    const long long s_begin = min(n_pieces, ((long long)blockIdx.x * (kWorkers / 32) + warp) * per_warp);
+    const long long s_end = min(n_pieces, s_begin + per_warp);
     if (s_begin >= s_end) return;
-    struct Cursor { int b, t, row, jb, sub; };   // batch, query tile, row in the tile, key block, 16-position strip in the block
+    struct Cursor { int b, t, row, jb, sub; };   // batch, query tile, row in the tile, key block, 32-position piece in the block
     Cursor cu;
     {
-        const long long u = s_begin >> 3;
-        cu.sub = (int)(s_begin & 7);
+        const long long u = s_begin >> 2;
+        cu.sub = (int)(s_begin & 3);
         cu.b = (int)(u / p.units_per_batch);
         int rem = (int)(u - (long long)cu.b * p.units_per_batch);
         cu.t = p.qt_begin;
@@ -202,7 +201,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         cu.jb = rem - cu.row * (cu.t + 1);
     }
     auto advance = [&](Cursor& x) {
-        if (++x.sub < 8) return;
+        if (++x.sub < 4) return;
         x.sub = 0;
         if (++x.jb <= x.t) return;
         x.jb = 0;
@@ -212,104 +211,101 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         x.t = p.qt_begin;
         ++x.b;
     };
-    // element offset of [head = lane][this strip] inside a plane set
-    auto strip_off = [&](const Cursor& x) {
-        return ((int64_t)(x.b * HQ + lane) * p.plane_rows + (x.t * UNIT + x.row - p.row0)) * p.plane_cols + x.jb * UNIT + x.sub * 16;
+    // Global <-> scratch: four lanes cover the 64 bytes [head][32 positions] of one head, so one warp-wide access
+    // touches 8 heads (8 lines); four accesses move a piece.  Scratch rows are 64 bytes (one head); the 16-byte chunk
+    // index is XOR-ed with (head / 2) % 4 so that the 8 rows of an 8x8 matrix fall into distinct banks.
+    const int l_head = lane >> 2, l_chunk = lane & 3;
+    auto piece_off = [&](const Cursor& x, int head) {   // element offset of [head][this piece] + this lane's chunk
+        return ((int64_t)(x.b * HQ + head) * p.plane_rows + (x.t * UNIT + x.row - p.row0)) * p.plane_cols + x.jb * UNIT + x.sub * 32 +
+               l_chunk * 8;
     };
-
-    uint8_t* scr = sScr + warp * c * 1024;
-    // scratch layout per plane: row = head (32 B), its two 16-byte halves swapped for heads 4..7 of every 8 so that
-    // the eight rows of an 8x8 matrix fall into distinct banks
-    const int my_sw = (lane >> 2) & 1;
-    const uint32_t st_off0 = lane * 32 + ((0 ^ my_sw) << 4), st_off1 = lane * 32 + ((1 ^ my_sw) << 4);
-    const int mi = lane >> 3, lr = lane & 7;               // ldmatrix/stmatrix: matrix index and row supplied by this lane
-    auto frag_off = [&](int x) {                           // 16-head block x, head block half (mi >> 1), position half (mi & 1)
-        const int head = x * 16 + 8 * (mi >> 1) + lr;
-        return (uint32_t)(head * 32 + (((mi & 1) ^ ((head >> 2) & 1)) << 4));
-    };
-    const uint32_t off0 = frag_off(0), off1 = frag_off(1);
-    const uint32_t scr_a = smem_u32(scr);
-
-    uint4 cur[kMaxTcChain][2], nxt[kMaxTcChain][2];
-    {
-        const int64_t o = strip_off(cu);
+    auto scr_off = [&](int head, int chunk) { return (uint32_t)(head * 64 + ((chunk ^ ((head >> 1) & 3)) << 4)); };
+    uint8_t* scr = sScr + warp * (2 * c * 2048);          // [2 buffers][c planes][32 heads][64 B]
+    auto fetch = [&](const Cursor& x, int buf) {          // asynchronous global -> scratch copy of a piece, all planes
 #pragma unroll
         for (int k = 0; k < kMaxTcChain; ++k)
             if (k < c) {
-                const uint4* src = reinterpret_cast<const uint4*>(p.planes[k] + o);
-                cur[k][0] = src[0]; cur[k][1] = src[1];
-            }
-    }
-    for (long long sidx = s_begin; sidx < s_end; ++sidx) {
-        const int64_t o_cur = strip_off(cu);
-        advance(cu);
 #pragma unroll
-        for (int k = 0; k < kMaxTcChain; ++k)
-            if (k < c) {
-                *reinterpret_cast<uint4*>(scr + k * 1024 + st_off0) = cur[k][0];
-                *reinterpret_cast<uint4*>(scr + k * 1024 + st_off1) = cur[k][1];
-            }
-        __syncwarp();
-        if (sidx + 1 < s_end) {
-            const int64_t o = strip_off(cu);
-#pragma unroll
-            for (int k = 0; k < kMaxTcChain; ++k)
-                if (k < c) {
-                    const uint4* src = reinterpret_cast<const uint4*>(p.planes[k] + o);
-                    nxt[k][0] = src[0]; nxt[k][1] = src[1];
+                for (int i = 0; i < 4; ++i) {
+                    const int head = l_head + 8 * i;
+                    const uint32_t dst = smem_u32(scr + (buf * c + k) * 2048) + scr_off(head, l_chunk);
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(p.planes[k] + piece_off(x, head)) : "memory");
                 }
+            }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    const int mi = lane >> 3, lr = lane & 7;               // ldmatrix/stmatrix: matrix index and row supplied by this lane
+    // strip s2 (16 positions) of the piece, 16-head block x: head block half (mi >> 1), position half (mi & 1)
+    auto frag_off = [&](int s2, int x) { return scr_off(x * 16 + 8 * (mi >> 1) + lr, 2 * s2 + (mi & 1)); };
+
+    fetch(cu, 0);
+    int buf = 0;
+    for (long long sidx = s_begin; sidx < s_end; ++sidx, buf ^= 1) {
+        const Cursor here = cu;
+        advance(cu);
+        if (sidx + 1 < s_end) {
+            fetch(cu, buf ^ 1);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
-        uint32_t afr[2][4];
-        ldmatrix_x4_trans(afr[0], scr_a + off0);
-        ldmatrix_x4_trans(afr[1], scr_a + off1);
-        float y[4][4];
-        for (int k = 0; k < c; ++k) {
-            const uint2* w1f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES);
-            const uint2* w2f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
-            const float* b1 = reinterpret_cast<const float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
-            const int act = p.act[k];
-            if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU>(afr, w1f, w2f, b1, b1 + MH, lane, y);
-            else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU>(afr, w1f, w2f, b1, b1 + MH, lane, y);
-            else ffn_link<LISA_ACT_NONE>(afr, w1f, w2f, b1, b1 + MH, lane, y);
-            if (k + 1 < c) {
-                // A_{k+1} = y + D_{k+1}; the difference comes in the same fragment arrangement as A did
+        __syncwarp();
+        const uint32_t base = smem_u32(scr + buf * c * 2048);
+#pragma unroll 1
+        for (int s2 = 0; s2 < 2; ++s2) {
+            const uint32_t off0 = frag_off(s2, 0), off1 = frag_off(s2, 1);
+            uint32_t afr[2][4];
+            ldmatrix_x4_trans(afr[0], base + off0);
+            ldmatrix_x4_trans(afr[1], base + off1);
+            float y[4][4];
+            for (int k = 0; k < c; ++k) {
+                const uint2* w1f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES);
+                const uint2* w2f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
+                const float* b1 = reinterpret_cast<const float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
+                const int act = p.act[k];
+                if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU>(afr, w1f, w2f, b1, b1 + MH, lane, y);
+                else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU>(afr, w1f, w2f, b1, b1 + MH, lane, y);
+                else ffn_link<LISA_ACT_NONE>(afr, w1f, w2f, b1, b1 + MH, lane, y);
+                if (k + 1 < c) {
+                    // A_{k+1} = y + D_{k+1}; the difference comes in the same fragment arrangement as A did
 #pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    uint32_t dfr[4];
-                    ldmatrix_x4_trans(dfr, scr_a + (k + 1) * 1024 + (x ? off1 : off0));
+                    for (int x = 0; x < 2; ++x) {
+                        uint32_t dfr[4];
+                        ldmatrix_x4_trans(dfr, base + (k + 1) * 2048 + (x ? off1 : off0));
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float2 dv = unpack_f16(dfr[q]);
-                        float* yy = y[2 * x + (q >> 1)] + 2 * (q & 1);
-                        afr[x][q] = pack_f16(yy[0] + dv.x, yy[1] + dv.y);
+                        for (int q = 0; q < 4; ++q) {
+                            const float2 dv = unpack_f16(dfr[q]);
+                            float* yy = y[2 * x + (q >> 1)] + 2 * (q & 1);
+                            afr[x][q] = pack_f16(yy[0] + dv.x, yy[1] + dv.y);
+                        }
                     }
                 }
             }
-        }
-        // result -> scratch plane 0 ([head][position]), transposed by stmatrix; then lane h stores head h's 32 bytes
+            // result over this strip's place in scratch plane 0 (every lane's ldmatrix of it is done), transposed back
+            __syncwarp();
 #pragma unroll
-        for (int x = 0; x < 2; ++x) {
-            uint32_t r[4];
-            r[0] = pack_f16(y[2 * x][0], y[2 * x][1]);
-            r[1] = pack_f16(y[2 * x][2], y[2 * x][3]);
-            r[2] = pack_f16(y[2 * x + 1][0], y[2 * x + 1][1]);
-            r[3] = pack_f16(y[2 * x + 1][2], y[2 * x + 1][3]);
-            stmatrix_x4_trans(scr_a + (x ? off1 : off0), r);
-        }
-        __syncwarp();
-        {
-            uint4* dst = reinterpret_cast<uint4*>(p.planes[0] + o_cur);
-            dst[0] = *reinterpret_cast<const uint4*>(scr + st_off0);
-            dst[1] = *reinterpret_cast<const uint4*>(scr + st_off1);
+            for (int x = 0; x < 2; ++x) {
+                uint32_t r[4];
+                r[0] = pack_f16(y[2 * x][0], y[2 * x][1]);
+                r[1] = pack_f16(y[2 * x][2], y[2 * x][3]);
+                r[2] = pack_f16(y[2 * x + 1][0], y[2 * x + 1][1]);
+                r[3] = pack_f16(y[2 * x + 1][2], y[2 * x + 1][3]);
+                stmatrix_x4_trans(base + (x ? off1 : off0), r);
+            }
         }
         __syncwarp();
 #pragma unroll
-        for (int k = 0; k < kMaxTcChain; ++k) { cur[k][0] = nxt[k][0]; cur[k][1] = nxt[k][1]; }
+        for (int i = 0; i < 4; ++i) {
+            const int head = l_head + 8 * i;
+            *reinterpret_cast<uint4*>(p.planes[0] + piece_off(here, head)) =
+                *reinterpret_cast<const uint4*>(scr + buf * c * 2048 + scr_off(head, l_chunk));
+        }
+        __syncwarp();   // the next iteration's fetch overwrites the other buffer only; this one is refilled one iteration later
     }
 }
 
 size_t align_smem_bytes(int c) {
-    return (size_t)c * (W1F_BYTES + W2F_BYTES + (MH + HQ) * 4) + (size_t)(kWorkers / 32) * c * 1024 + 16;
+    return (size_t)c * (W1F_BYTES + W2F_BYTES + (MH + HQ) * 4) + (size_t)(kWorkers / 32) * 2 * c * 2048 + 16;
 }
 
 }  // namespace
@@ -338,7 +334,7 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     }
     p.status = status_words();
     if (!p.status) return cudaErrorUnknown;
-    if (a.plane_cols % 16 != 0) return cudaErrorInvalidValue;   // strips are loaded as aligned 32-byte pieces
+    if (a.plane_cols % 32 != 0) return cudaErrorInvalidValue;   // pieces are moved as aligned 16-byte chunks
     const size_t smem = align_smem_bytes(a.chain);
     cudaError_t e = cudaFuncSetAttribute(tc_align_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
