@@ -34,8 +34,8 @@ namespace {
 using namespace tc;
 
 constexpr int HQ = 32, MH = 64, UNIT = 128;
-constexpr int kWorkers = 256;                 // eight warps x 16 positions
-constexpr int kThreads = kWorkers + 32;       // + producer warp
+constexpr int kWorkers = 256;                 // threads per CTA, weights read from shared memory (two CTAs per SM)
+constexpr int kRegwThreads = 128;             // threads per CTA, weights held in registers (three CTAs per SM)
 constexpr int SLAB_BYTES = 2 * HQ * 128;      // [2 halves of 64 positions][32 heads][128 B], 128-byte swizzle
 constexpr int kStages = 3;                    // ring of slab slots (each holds the c slabs of one unit)
 constexpr int W1F_BYTES = 2 * 8 * 32 * 8;     // B fragments of W1: [k-step][n-tile][lane] x (b0, b1)
@@ -96,9 +96,12 @@ __device__ __forceinline__ uint32_t act_pack(float x0, float x1) {
 // One link on a warp's 16 positions: afr = A fragments (2 k-steps of 16 heads) -> y = W2^T act(W1^T a + b1) + b2
 // as four accumulator tiles of 8 heads.  All eight hidden tiles are accumulated before the activation, so that
 // sixteen independent MMAs are in flight, then the sixteen of the second layer.
-template <int ACT>
-__device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* w1f, const uint2* w2f, const float* b1, const float* b2,
-                                         int lane, float (*y)[4]) {
+// The fragments of W1 and W2 come either from shared memory (w1f/w2f, one 8-byte load per MMA) or, when REGW, from
+// the register copies w1r/w2r that a warp keeps for its whole life (single-link calls: shared-memory bandwidth, not
+// the tensor pipe, is what the per-MMA loads run into).
+template <int ACT, bool REGW>
+__device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* w1f, const uint2* w2f, const uint2* w1r, const uint2* w2r,
+                                         const float* b1, const float* b2, int lane, float (*y)[4]) {
     const int t = lane & 3;
     float h[8][4];
 #pragma unroll
@@ -110,7 +113,7 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
     for (int ks = 0; ks < 2; ++ks)
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const uint2 w = w1f[(ks * 8 + j) * 32 + lane];
+            const uint2 w = REGW ? w1r[ks * 8 + j] : w1f[(ks * 8 + j) * 32 + lane];
             mma_f16(h[j], afr[ks], w.x, w.y);
         }
     uint32_t hfr[4][4];
@@ -130,7 +133,7 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
     for (int s = 0; s < 4; ++s)
 #pragma unroll
         for (int j2 = 0; j2 < 4; ++j2) {
-            const uint2 w = w2f[(s * 4 + j2) * 32 + lane];
+            const uint2 w = REGW ? w2r[s * 4 + j2] : w2f[(s * 4 + j2) * 32 + lane];
             mma_f16(y[j2], hfr[s], w.x, w.y);
         }
 }
@@ -140,8 +143,10 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
 //   scratch -> fragments ldmatrix.trans per 16-position strip
 //   chain in registers   (ffn_link)
 //   result               stmatrix.trans back into the scratch, then 16 bytes per lane to the plane
-__global__ void __launch_bounds__(kWorkers, 2)
+template <bool REGW>
+__global__ void __launch_bounds__(REGW ? kRegwThreads : kWorkers, REGW ? 3 : 2)
 tc_align_kernel(const __grid_constant__ AlignParams p) {
+    constexpr int NT = REGW ? kRegwThreads : kWorkers;
     extern __shared__ __align__(16) uint8_t smem[];
     const int c = p.chain;
     constexpr int LINK_BYTES = W1F_BYTES + W2F_BYTES + (MH + HQ) * 4;
@@ -156,7 +161,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         float* bias = reinterpret_cast<float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
         const float out_scale = k == c - 1 ? kLog2e : 1.f;
         const int wd = p.w_dtype[k];
-        for (int e = tid; e < 2 * 8 * 32; e += kWorkers) {   // W1 [32 heads][64 hidden]: k = head, n = hidden
+        for (int e = tid; e < 2 * 8 * 32; e += NT) {   // W1 [32 heads][64 hidden]: k = head, n = hidden
             const int ln = e & 31, j = (e >> 5) & 7, ks = e >> 8, g = ln >> 2, t = ln & 3;
             const int k0 = ks * 16 + 2 * t, n = j * 8 + g;
             uint2 w;
@@ -164,7 +169,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             w.y = pack_f16(ld_elem(p.w1[k], (k0 + 8) * MH + n, wd), ld_elem(p.w1[k], (k0 + 9) * MH + n, wd));
             w1f[e] = w;
         }
-        for (int e = tid; e < 4 * 4 * 32; e += kWorkers) {   // W2 [64 hidden][32 heads]: k = hidden, n = head
+        for (int e = tid; e < 4 * 4 * 32; e += NT) {   // W2 [64 hidden][32 heads]: k = hidden, n = head
             const int ln = e & 31, j2 = (e >> 5) & 3, s2 = e >> 7, g = ln >> 2, t = ln & 3;
             const int k0 = s2 * 16 + 2 * t, n = j2 * 8 + g;
             uint2 w;
@@ -172,16 +177,16 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             w.y = pack_f16(ld_elem(p.w2[k], (k0 + 8) * HQ + n, wd) * out_scale, ld_elem(p.w2[k], (k0 + 9) * HQ + n, wd) * out_scale);
             w2f[e] = w;
         }
-        for (int e = tid; e < MH; e += kWorkers) bias[e] = ldw(p.b1[k], e, wd);
-        for (int e = tid; e < HQ; e += kWorkers) bias[MH + e] = ldw(p.b2[k], e, wd) * out_scale;
+        for (int e = tid; e < MH; e += NT) bias[e] = ldw(p.b1[k], e, wd);
+        for (int e = tid; e < HQ; e += NT) bias[MH + e] = ldw(p.b2[k], e, wd) * out_scale;
     }
     __syncthreads();
 
     // ---- this warp's contiguous range of pieces; a piece is 32 positions (4 per 128-position unit) ----
     const long long n_pieces = (long long)p.units_per_batch * p.B * 4;
-    const long long n_warps = (long long)gridDim.x * (kWorkers / 32);
+    const long long n_warps = (long long)gridDim.x * (NT / 32);
     const long long per_warp = (n_pieces + n_warps - 1) / n_warps;
-    const long long s_begin = min(n_pieces, ((long long)blockIdx.x * (kWorkers / 32) + warp) * per_warp);
+    const long long s_begin = min(n_pieces, ((long long)blockIdx.x * (NT / 32) + warp) * per_warp);
     const long long s_end = min(n_pieces, s_begin + per_warp);
     if (s_begin >= s_end) return;
     struct Cursor { int b, t, row, jb, sub; };   // batch, query tile, row in the tile, key block, 32-position piece in the block
@@ -238,6 +243,14 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
     // strip s2 (16 positions) of the piece, 16-head block x: head block half (mi >> 1), position half (mi & 1)
     auto frag_off = [&](int s2, int x) { return scr_off(x * 16 + 8 * (mi >> 1) + lr, 2 * s2 + (mi & 1)); };
 
+    uint2 w1r[16], w2r[16];
+    if constexpr (REGW) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            w1r[i] = reinterpret_cast<const uint2*>(sW)[i * 32 + lane];
+            w2r[i] = reinterpret_cast<const uint2*>(sW + W1F_BYTES)[i * 32 + lane];
+        }
+    }
     fetch(cu, 0);
     int buf = 0;
     for (long long sidx = s_begin; sidx < s_end; ++sidx, buf ^= 1) {
@@ -263,9 +276,9 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                 const uint2* w2f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
                 const float* b1 = reinterpret_cast<const float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
                 const int act = p.act[k];
-                if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU>(afr, w1f, w2f, b1, b1 + MH, lane, y);
-                else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU>(afr, w1f, w2f, b1, b1 + MH, lane, y);
-                else ffn_link<LISA_ACT_NONE>(afr, w1f, w2f, b1, b1 + MH, lane, y);
+                if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, REGW>(afr, w1f, w2f, w1r, w2r, b1, b1 + MH, lane, y);
+                else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, REGW>(afr, w1f, w2f, w1r, w2r, b1, b1 + MH, lane, y);
+                else ffn_link<LISA_ACT_NONE, REGW>(afr, w1f, w2f, w1r, w2r, b1, b1 + MH, lane, y);
                 if (k + 1 < c) {
                     // A_{k+1} = y + D_{k+1}; the difference comes in the same fragment arrangement as A did
 #pragma unroll
@@ -304,8 +317,8 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
     }
 }
 
-size_t align_smem_bytes(int c) {
-    return (size_t)c * (W1F_BYTES + W2F_BYTES + (MH + HQ) * 4) + (size_t)(kWorkers / 32) * 2 * c * 2048 + 16;
+size_t align_smem_bytes(int c, int threads) {
+    return (size_t)c * (W1F_BYTES + W2F_BYTES + (MH + HQ) * 4) + (size_t)(threads / 32) * 2 * c * 2048 + 16;
 }
 
 }  // namespace
@@ -335,14 +348,18 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     p.status = status_words();
     if (!p.status) return cudaErrorUnknown;
     if (a.plane_cols % 32 != 0) return cudaErrorInvalidValue;   // pieces are moved as aligned 16-byte chunks
-    const size_t smem = align_smem_bytes(a.chain);
-    cudaError_t e = cudaFuncSetAttribute(tc_align_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const bool regw = a.chain == 1;   // a single link's weight fragments fit in registers
+    const int threads = regw ? kRegwThreads : kWorkers;
+    const size_t smem = align_smem_bytes(a.chain, threads);
+    cudaError_t e = regw ? cudaFuncSetAttribute(tc_align_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                         : cudaFuncSetAttribute(tc_align_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const int64_t total_units = (int64_t)p.units_per_batch * a.B;
     if (total_units <= 0 || total_units > 0x7fffffff) return cudaErrorInvalidValue;
-    const int max_ctas = a.ctas > 0 ? a.ctas : 148 * 2;
-    dim3 grid((unsigned)std::min<int64_t>((total_units + 3) / 4, max_ctas));  // at least four strips per warp
-    tc_align_kernel<<<grid, kWorkers, smem, stream>>>(p);
+    const int max_ctas = a.ctas > 0 ? a.ctas : 148 * (regw ? 3 : 2);
+    dim3 grid((unsigned)std::min<int64_t>((total_units + 3) / 4, max_ctas));  // at least a unit per warp
+    if (regw) tc_align_kernel<true><<<grid, threads, smem, stream>>>(p);
+    else tc_align_kernel<false><<<grid, threads, smem, stream>>>(p);
     count_launches(1);
     return cudaGetLastError();
 }
