@@ -72,65 +72,79 @@ __device__ __forceinline__ void mma_f16(float* d, const uint32_t* a, uint32_t b0
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// Activation of two hidden units, packed to fp16 (the A-fragment format of the next MMA).
+// d = a (16x16, row) . b (16x8, col) + c with fp16 accumulators: the two result registers hold rows g and g+8 as
+// packed pairs of columns (2t, 2t+1), which is exactly the A-fragment arrangement of a following MMA.
+__device__ __forceinline__ void mma_f16acc(uint32_t* d, const uint32_t* a, uint32_t b0, uint32_t b1, uint32_t c0, uint32_t c1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f16.f16.f16.f16 {%0,%1}, {%2,%3,%4,%5}, {%6,%7}, {%8,%9};"
+                 : "=r"(d[0]), "=r"(d[1])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(c0), "r"(c1));
+}
+// d = a . b + c, fp32 accumulators, c given separately (a bias pair repeated for both rows)
+__device__ __forceinline__ void mma_f16_bias(float* d, const uint32_t* a, uint32_t b0, uint32_t b1, float c0, float c1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%10,%11};"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(c0), "f"(c1));
+}
+
+// Activation of two hidden units held as a packed fp16 pair; the result is again a packed pair (an A-fragment
+// register of the second layer's MMA).
 template <int ACT>
-__device__ __forceinline__ uint32_t act_pack(float x0, float x1) {
-    if constexpr (ACT == LISA_ACT_RELU) return pack_f16(fmaxf(x0, 0.f), fmaxf(x1, 0.f));
-    if constexpr (ACT == LISA_ACT_SILU) {
-        // x * sigmoid(x) = x / (1 + 2^(-x log2 e)).  The transcendental pipe is the scarce unit here (64 hidden units
-        // per position), so the pair shares its MUFU work: one packed-fp16 ex2 for both exponentials and ONE
-        // reciprocal, of the product of the two denominators (1/d0 = d1 * r, 1/d1 = d0 * r).  Denominators are
-        // clamped so that their product stays finite; sigmoid is then below 2^-60 anyway.
-        const __half2 xh = __floats2half2_rn(x0 * -1.4426950408889634f, x1 * -1.4426950408889634f);
-        uint32_t eh;
-        asm("ex2.approx.f16x2 %0, %1;" : "=r"(eh) : "r"(*reinterpret_cast<const uint32_t*>(&xh)));
-        const float2 e = unpack_f16(eh);
-        const float d0 = fminf(1.f + e.x, 1e18f), d1 = fminf(1.f + e.y, 1e18f);
-        float r;
-        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(d0 * d1));
-        return pack_f16(x0 * (d1 * r), x1 * (d0 * r));
+__device__ __forceinline__ uint32_t act_h2(uint32_t x) {
+    if constexpr (ACT == LISA_ACT_RELU) {
+        uint32_t r;
+        asm("max.f16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(0u));
+        return r;
     }
-    return pack_f16(x0, x1);
+    if constexpr (ACT == LISA_ACT_SILU) {
+        // x * sigmoid(x) = (x/2) tanh(x/2) + x/2: one packed multiply, one packed tanh, one packed fused multiply-add
+        uint32_t hx, th, r;
+        asm("mul.f16x2 %0, %1, %2;" : "=r"(hx) : "r"(x), "r"(0x38003800u));   // 0.5, 0.5
+        asm("tanh.approx.f16x2 %0, %1;" : "=r"(th) : "r"(hx));
+        asm("fma.rn.f16x2 %0, %1, %2, %1;" : "=r"(r) : "r"(hx), "r"(th));
+        return r;
+    }
+    return x;
 }
 
 // One link on a warp's 16 positions: afr = A fragments (2 k-steps of 16 heads) -> y = W2^T act(W1^T a + b1) + b2
-// as four accumulator tiles of 8 heads.  All eight hidden tiles are accumulated before the activation, so that
-// sixteen independent MMAs are in flight, then the sixteen of the second layer.
+// as four accumulator tiles of 8 heads.  The first layer accumulates in fp16 (32 products per hidden unit, the
+// result is rounded to fp16 for the second layer's operand in any case): its accumulator registers ARE the second
+// layer's A fragments, so the activation is one to three packed instructions per register and nothing is converted
+// or repacked.  The second layer accumulates in fp32.  b1h holds b1 as packed fp16 pairs, b2 is fp32.
 // The fragments of W1 and W2 come either from shared memory (w1f/w2f, one 8-byte load per MMA) or, when REGW, from
-// the register copies w1r/w2r that a warp keeps for its whole life (single-link calls: shared-memory bandwidth, not
-// the tensor pipe, is what the per-MMA loads run into).
+// the register copies w1r/w2r that a warp keeps for its whole life (single-link calls).
 template <int ACT, bool REGW>
 __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* w1f, const uint2* w2f, const uint2* w1r, const uint2* w2r,
-                                         const float* b1, const float* b2, int lane, float (*y)[4]) {
+                                         const uint32_t* b1h, const float* b2, int lane, float (*y)[4]) {
     const int t = lane & 3;
-    float h[8][4];
+    uint32_t h[8][2];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const float2 bb = *reinterpret_cast<const float2*>(b1 + j * 8 + 2 * t);
-        h[j][0] = bb.x; h[j][1] = bb.y; h[j][2] = bb.x; h[j][3] = bb.y;
+        const uint32_t bb = b1h[j * 4 + t];
+        const uint2 w = REGW ? w1r[j] : w1f[j * 32 + lane];
+        mma_f16acc(h[j], afr[0], w.x, w.y, bb, bb);
     }
 #pragma unroll
-    for (int ks = 0; ks < 2; ++ks)
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const uint2 w = REGW ? w1r[ks * 8 + j] : w1f[(ks * 8 + j) * 32 + lane];
-            mma_f16(h[j], afr[ks], w.x, w.y);
-        }
+    for (int j = 0; j < 8; ++j) {
+        const uint2 w = REGW ? w1r[8 + j] : w1f[(8 + j) * 32 + lane];
+        mma_f16acc(h[j], afr[1], w.x, w.y, h[j][0], h[j][1]);
+    }
     uint32_t hfr[4][4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-        hfr[s][0] = act_pack<ACT>(h[2 * s][0], h[2 * s][1]);
-        hfr[s][1] = act_pack<ACT>(h[2 * s][2], h[2 * s][3]);
-        hfr[s][2] = act_pack<ACT>(h[2 * s + 1][0], h[2 * s + 1][1]);
-        hfr[s][3] = act_pack<ACT>(h[2 * s + 1][2], h[2 * s + 1][3]);
+        hfr[s][0] = act_h2<ACT>(h[2 * s][0]);
+        hfr[s][1] = act_h2<ACT>(h[2 * s][1]);
+        hfr[s][2] = act_h2<ACT>(h[2 * s + 1][0]);
+        hfr[s][3] = act_h2<ACT>(h[2 * s + 1][1]);
     }
 #pragma unroll
     for (int j2 = 0; j2 < 4; ++j2) {
         const float2 bb = *reinterpret_cast<const float2*>(b2 + j2 * 8 + 2 * t);
-        y[j2][0] = bb.x; y[j2][1] = bb.y; y[j2][2] = bb.x; y[j2][3] = bb.y;
+        const uint2 w = REGW ? w2r[j2] : w2f[j2 * 32 + lane];
+        mma_f16_bias(y[j2], hfr[0], w.x, w.y, bb.x, bb.y);
     }
 #pragma unroll
-    for (int s = 0; s < 4; ++s)
+    for (int s = 1; s < 4; ++s)
 #pragma unroll
         for (int j2 = 0; j2 < 4; ++j2) {
             const uint2 w = REGW ? w2r[s * 4 + j2] : w2f[(s * 4 + j2) * 32 + lane];
@@ -177,7 +191,8 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             w.y = pack_f16(ld_elem(p.w2[k], (k0 + 8) * HQ + n, wd) * out_scale, ld_elem(p.w2[k], (k0 + 9) * HQ + n, wd) * out_scale);
             w2f[e] = w;
         }
-        for (int e = tid; e < MH; e += NT) bias[e] = ldw(p.b1[k], e, wd);
+        for (int e = tid; e < MH / 2; e += NT)   // b1 as packed fp16 pairs (the first layer's accumulator format)
+            reinterpret_cast<uint32_t*>(bias)[e] = pack_f16(ldw(p.b1[k], 2 * e, wd), ldw(p.b1[k], 2 * e + 1, wd));
         for (int e = tid; e < HQ; e += NT) bias[MH + e] = ldw(p.b2[k], e, wd) * out_scale;
     }
     __syncthreads();
@@ -275,10 +290,11 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                 const uint2* w1f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES);
                 const uint2* w2f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
                 const float* b1 = reinterpret_cast<const float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
+                const uint32_t* b1h = reinterpret_cast<const uint32_t*>(b1);
                 const int act = p.act[k];
-                if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, REGW>(afr, w1f, w2f, w1r, w2r, b1, b1 + MH, lane, y);
-                else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, REGW>(afr, w1f, w2f, w1r, w2r, b1, b1 + MH, lane, y);
-                else ffn_link<LISA_ACT_NONE, REGW>(afr, w1f, w2f, w1r, w2r, b1, b1 + MH, lane, y);
+                if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
+                else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
+                else ffn_link<LISA_ACT_NONE, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
                 if (k + 1 < c) {
                     // A_{k+1} = y + D_{k+1}; the difference comes in the same fragment arrangement as A did
 #pragma unroll
