@@ -236,7 +236,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
     // index is XOR-ed with (head / 2) % 4 so that the 8 rows of an 8x8 matrix fall into distinct banks.
     const int l_head = lane >> 2, l_chunk = lane & 3;
     auto piece_off = [&](const Cursor& x, int head) {   // element offset of [head][this piece] + this lane's chunk
-        return ((int64_t)(x.b * HQ + head) * p.plane_rows + (x.t * UNIT + x.row - p.row0)) * p.plane_cols + x.jb * UNIT + x.sub * 32 +
+        return ((int64_t)(x.t * UNIT + x.row - p.row0) * (p.B * HQ) + (x.b * HQ + head)) * p.plane_cols + x.jb * UNIT + x.sub * 32 +
                l_chunk * 8;
     };
     auto scr_off = [&](int head, int chunk) { return (uint32_t)(head * 64 + ((chunk ^ ((head >> 1) & 3)) << 4)); };

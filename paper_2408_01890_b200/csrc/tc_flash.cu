@@ -410,13 +410,13 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     tmY = tmQ;
     if (a.emit_plane) {  // store map: one epilogue warp's 32 rows x 64 columns per copy
         const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * a.Hq};
-        const uint64_t str[2] = {(uint64_t)a.plane_cols * 2, (uint64_t)a.plane_cols * a.plane_rows * 2};
+        const uint64_t str[2] = {(uint64_t)a.B * a.Hq * a.plane_cols * 2, (uint64_t)a.plane_cols * 2};   // [row][b*Hq+h][col]
         const uint32_t box[3] = {64, 32, 1};
         if (!make_tensor_map_bf16(&tmY, a.emit_plane, 3, dims, str, box, true)) return cudaErrorInvalidValue;
     }
     if (a.plane) {
         const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * a.Hq};
-        const uint64_t str[2] = {(uint64_t)a.plane_cols * 2, (uint64_t)a.plane_cols * a.plane_rows * 2};
+        const uint64_t str[2] = {(uint64_t)a.B * a.Hq * a.plane_cols * 2, (uint64_t)a.plane_cols * 2};   // [row][b*Hq+h][col]
         const uint32_t box[3] = {64, 128, 1};
         if (!make_tensor_map_bf16(&tmY, a.plane, 3, dims, str, box, true)) return cudaErrorInvalidValue;
     }
