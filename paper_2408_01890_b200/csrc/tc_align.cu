@@ -34,10 +34,8 @@ namespace {
 using namespace tc;
 
 constexpr int HQ = 32, MH = 64, UNIT = 128;
-constexpr int kWorkers = 256;                 // threads per CTA, weights read from shared memory (two CTAs per SM)
-constexpr int kRegwThreads = 128;             // threads per CTA, weights held in registers (three CTAs per SM)
-constexpr int SLAB_BYTES = 2 * HQ * 128;      // [2 halves of 64 positions][32 heads][128 B], 128-byte swizzle
-constexpr int kStages = 3;                    // ring of slab slots (each holds the c slabs of one unit)
+constexpr int kWorkers = 384, kStages = 2;                        // weights read from shared memory: one CTA per SM
+constexpr int kRegwThreads = 128, kRegwCtas = 3, kRegwStages = 4; // weights held in registers (single link)
 constexpr int W1F_BYTES = 2 * 8 * 32 * 8;     // B fragments of W1: [k-step][n-tile][lane] x (b0, b1)
 constexpr int W2F_BYTES = 4 * 4 * 32 * 8;     // B fragments of W2
 constexpr float kLog2e = 1.4426950408889634f; // the last link's output leaves multiplied by log2(e): the attention
@@ -157,15 +155,14 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
 //   scratch -> fragments ldmatrix.trans per 16-position strip
 //   chain in registers   (ffn_link)
 //   result               stmatrix.trans back into the scratch, then 16 bytes per lane to the plane
-template <bool REGW>
-__global__ void __launch_bounds__(REGW ? kRegwThreads : kWorkers, REGW ? 3 : 2)
+template <bool REGW, int NT, int MIN_CTAS, int STAGES>
+__global__ void __launch_bounds__(NT, MIN_CTAS)
 tc_align_kernel(const __grid_constant__ AlignParams p) {
-    constexpr int NT = REGW ? kRegwThreads : kWorkers;
     extern __shared__ __align__(16) uint8_t smem[];
     const int c = p.chain;
     constexpr int LINK_BYTES = W1F_BYTES + W2F_BYTES + (MH + HQ) * 4;
     uint8_t* sW = smem;                               // per link: W1 fragments, W2 fragments, b1[64], b2[32]
-    uint8_t* sScr = sW + c * LINK_BYTES;              // per warp: two buffers of c planes x [32 heads][64 B]
+    uint8_t* sScr = sW + c * LINK_BYTES;              // per warp: STAGES buffers of c planes x [32 heads][64 B]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // ---- one-time set-up: weights as ready-made B fragments (fp16, the last link's W2/b2 times log2 e) ----
@@ -240,7 +237,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                l_chunk * 8;
     };
     auto scr_off = [&](int head, int chunk) { return (uint32_t)(head * 64 + ((chunk ^ ((head >> 1) & 3)) << 4)); };
-    uint8_t* scr = sScr + warp * (2 * c * 2048);          // [2 buffers][c planes][32 heads][64 B]
+    uint8_t* scr = sScr + warp * (STAGES * c * 2048);     // [STAGES buffers][c planes][32 heads][64 B]
     auto fetch = [&](const Cursor& x, int buf) {          // asynchronous global -> scratch copy of a piece, all planes
 #pragma unroll
         for (int k = 0; k < kMaxTcChain; ++k)
@@ -266,17 +263,23 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             w2r[i] = reinterpret_cast<const uint2*>(sW + W1F_BYTES)[i * 32 + lane];
         }
     }
-    fetch(cu, 0);
-    int buf = 0;
-    for (long long sidx = s_begin; sidx < s_end; ++sidx, buf ^= 1) {
+    // STAGES - 1 pieces are in flight ahead of the one being worked on; one commit group per piece (an empty group
+    // past the end keeps the count uniform), so waiting for all but the newest STAGES - 1 groups completes this one.
+    Cursor ahead = cu;
+    long long fidx = s_begin;
+#pragma unroll
+    for (int i = 0; i < STAGES - 1; ++i, ++fidx) {
+        if (fidx < s_end) { fetch(ahead, i); advance(ahead); }
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    int buf = 0, fbuf = STAGES - 1;
+    for (long long sidx = s_begin; sidx < s_end; ++sidx, ++fidx) {
         const Cursor here = cu;
         advance(cu);
-        if (sidx + 1 < s_end) {
-            fetch(cu, buf ^ 1);
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
-        } else {
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-        }
+        if (fidx < s_end) { fetch(ahead, fbuf); advance(ahead); }
+        else asm volatile("cp.async.commit_group;" ::: "memory");
+        fbuf = fbuf + 1 == STAGES ? 0 : fbuf + 1;
+        asm volatile("cp.async.wait_group %0;" ::"n"(STAGES - 1) : "memory");
         __syncwarp();
         const uint32_t base = smem_u32(scr + buf * c * 2048);
 #pragma unroll 1
@@ -329,12 +332,13 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             *reinterpret_cast<uint4*>(p.planes[0] + piece_off(here, head)) =
                 *reinterpret_cast<const uint4*>(scr + buf * c * 2048 + scr_off(head, l_chunk));
         }
-        __syncwarp();   // the next iteration's fetch overwrites the other buffer only; this one is refilled one iteration later
+        __syncwarp();   // the next iteration's fetch refills the buffer that was stored one iteration ago, not this one
+        buf = buf + 1 == STAGES ? 0 : buf + 1;
     }
 }
 
-size_t align_smem_bytes(int c, int threads) {
-    return (size_t)c * (W1F_BYTES + W2F_BYTES + (MH + HQ) * 4) + (size_t)(threads / 32) * 2 * c * 2048 + 16;
+size_t align_smem_bytes(int c, int threads, int stages) {
+    return (size_t)c * (W1F_BYTES + W2F_BYTES + (MH + HQ) * 4) + (size_t)(threads / 32) * stages * c * 2048 + 16;
 }
 
 }  // namespace
@@ -364,18 +368,20 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     p.status = status_words();
     if (!p.status) return cudaErrorUnknown;
     if (a.plane_cols % 32 != 0) return cudaErrorInvalidValue;   // pieces are moved as aligned 16-byte chunks
-    const bool regw = a.chain == 1;   // a single link's weight fragments fit in registers
+    // One link: its weight fragments live in registers, 4-warp CTAs, three per SM, three pieces in flight per warp.
+    // Longer chains: weights in shared memory, one 12-warp CTA per SM, one piece in flight per warp.
+    const bool regw = a.chain == 1;
     const int threads = regw ? kRegwThreads : kWorkers;
-    const size_t smem = align_smem_bytes(a.chain, threads);
-    cudaError_t e = regw ? cudaFuncSetAttribute(tc_align_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                         : cudaFuncSetAttribute(tc_align_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const int ctas_per_sm = regw ? kRegwCtas : 1;
+    const size_t smem = align_smem_bytes(a.chain, threads, regw ? kRegwStages : kStages);
+    auto kernel = regw ? tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages> : tc_align_kernel<false, kWorkers, 1, kStages>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const int64_t total_units = (int64_t)p.units_per_batch * a.B;
     if (total_units <= 0 || total_units > 0x7fffffff) return cudaErrorInvalidValue;
-    const int max_ctas = a.ctas > 0 ? a.ctas : 148 * (regw ? 3 : 2);
+    const int max_ctas = a.ctas > 0 ? a.ctas : 148 * ctas_per_sm;
     dim3 grid((unsigned)std::min<int64_t>((total_units + 3) / 4, max_ctas));  // at least a unit per warp
-    if (regw) tc_align_kernel<true><<<grid, threads, smem, stream>>>(p);
-    else tc_align_kernel<false><<<grid, threads, smem, stream>>>(p);
+    kernel<<<grid, threads, smem, stream>>>(p);
     count_launches(1);
     return cudaGetLastError();
 }
