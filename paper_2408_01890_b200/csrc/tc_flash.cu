@@ -40,7 +40,7 @@ struct FlashParams {
     int64_t o_sb, o_sn, o_sh;
     int* status;
     int plane_row0;  // first query row held by the plane workspace (rows are stored relative to it)
-    int qt_begin;    // this launch covers query tiles [qt_begin, qt_begin + gridDim.x)
+    int qt_begin;    // this launch covers query tiles [qt_begin, qt_begin + gridDim.y)
     int ksteps;      // 16-wide k-steps of the score MMA actually issued (<= KD/16; the rest is zero padding)
     float scale;     // MODE_EMIT: scores are multiplied by this before rounding to fp16
 };
@@ -98,8 +98,10 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 17);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int qt = p.qt_begin + (int)gridDim.x - 1 - (int)blockIdx.x;  // heavy tiles first
-    const int h = blockIdx.y, b = blockIdx.z;
+    // blockIdx.x (the fastest-dispatched index) runs over (batch, head), blockIdx.y over query tiles from the last one
+    // down: every CTA of the heaviest tile is handed out before any lighter one, so the SMs finish close together
+    const int qt = p.qt_begin + (int)gridDim.y - 1 - (int)blockIdx.y;
+    const int h = (int)blockIdx.x % p.Hq, b = (int)blockIdx.x / p.Hq;
     const int g = h / (p.Hq / p.Hkv);
     const int nt = qt + 1;  // key tiles 0..qt
     const int q0 = qt * BM;
@@ -432,7 +434,8 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     p.ksteps = a.ksteps > 0 ? a.ksteps : a.kd / 16;
     p.scale = a.scale;
 
-    dim3 grid(a.qt_count, a.Hq, a.B);
+    if (a.qt_count < 1 || a.qt_count > 65535) return cudaErrorInvalidValue;
+    dim3 grid(a.Hq * a.B, a.qt_count);
     cudaError_t e;
 #define LISA_LAUNCH_FLASH(KD_, PL_)                                                                                       \
     do {                                                                                                                   \
