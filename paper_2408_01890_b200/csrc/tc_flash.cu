@@ -1,18 +1,22 @@
 // Tensor-core flash kernel (tcgen05 + TMEM + TMA) for head width 128, bf16.
 //
-// One CTA per (batch b, query head h, 128-row query tile).  For every key tile j <= the query tile:
-//   scores  S = QA . KA^T            tcgen05.mma, fp32 accumulator in tensor memory (two buffers, so S(t+1) is
-//                                    computed while the softmax of tile t runs)
+// One CTA per (batch b, query head h, 128-row query tile).  For every 64-key tile j up to the diagonal:
+//   scores  S = QA . KA^T            tcgen05.mma (M 128, N 64), fp32 accumulator in tensor memory (two buffers, so
+//                                    S(t+1) is computed while the softmax of tile t runs)
 //   logits  A = S * scale (+ Y)      Y: optional fp16 tile of pre-computed scores (the aligned part of a
 //                                    shared layer, Eq. 4; then QA/KA are the layer's low-rank Q'/K', Eq. 3)
-//   causal mask (diagonal tile), online softmax in registers (one thread per query row), P as bf16
-//   O += P . V                       tcgen05.mma, V read MN-major straight from its [key][d] tile
+//   causal mask (tiles that reach past the first query row), online softmax in registers (one thread per query
+//   row), P as bf16
+//   O += P . V                       tcgen05.mma (M 128, N 128, K 64), V read MN-major straight from its [key][d] tile
 // With QA/KA = Q/K and no Y this is standard attention (Eq. 1-2).  In MODE_EMIT there is no softmax: the scaled
 // scores leave as fp16 tiles (staged in shared memory, stored with TMA) for the aligner kernel.
 //
 // Warp roles: warps 0-3 softmax/epilogue (thread = query row = TMEM lane), warp 4 TMA producer,
-// warp 5 MMA issuer and TMEM owner.  K and V(/Y) have their own two-stage rings: a K stage is free again as
-// soon as its score MMA has run, a V stage after its P.V MMA.
+// warp 5 MMA issuer and TMEM owner.  K and V(/Y) have their own rings: a K stage is free again as soon as its
+// score MMA has run, a V stage after its P.V MMA.
+// Sizing: the softmax warps are the slow stage (one exp2 per score on the 16-lane transcendental unit) and every
+// hand-off between the roles costs a few hundred cycles of latency, so TWO CTAs share an SM and fill each other's
+// gaps, prologues and epilogues: 64-key tiles keep a CTA at 112 KB of shared memory and 256 tensor-memory columns.
 // Every wait is bounded; on expiry the CTA records it in the status word, drains and exits.
 #include "common.cuh"
 #include "tc_common.cuh"
@@ -22,7 +26,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int BM = 128, BN = 128, D = 128;
+constexpr int BM = 128, BN = 64, D = 128;
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -31,7 +35,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
 }
 
 constexpr int kThreads = 192;
-constexpr uint32_t TMEM_COLS = 512;  // S[2]: [0,256), O: [256,384)
 
 struct FlashParams {
     int B, N, Hq, Hkv;
@@ -53,31 +56,40 @@ template <int KD, int MODE>
 struct Smem {
     static constexpr bool PLANE = MODE == MODE_ATTN_PLANE;
     static constexpr bool EMIT = MODE == MODE_EMIT;
+    static constexpr int KST = EMIT ? 3 : 2;             // K ring depth (V/Y: two stages)
     static constexpr int Q_BYTES = BM * KD * 2;
     static constexpr int K_BYTES = BN * KD * 2;
     static constexpr int V_BYTES = EMIT ? 0 : BN * D * 2;
     static constexpr int P_BYTES = EMIT ? 0 : BM * BN * 2;
     static constexpr int Y_BYTES = PLANE ? BM * BN * 2 : 0;
-    static constexpr int STG_BYTES = EMIT ? 4 * 2 * 8192 : 0;  // per epilogue warp: two buffers of [2 halves][32 rows][128 B]
+    static constexpr int STG_BYTES = EMIT ? 4 * 2 * 4096 : 0;  // per epilogue warp: two buffers of [32 rows][128 B]
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + Q_BYTES;
-    static constexpr int OFF_V = OFF_K + 2 * K_BYTES;
+    static constexpr int OFF_V = OFF_K + KST * K_BYTES;
     static constexpr int OFF_P = OFF_V + 2 * V_BYTES;
     static constexpr int OFF_Y = OFF_P + P_BYTES;
     static constexpr int OFF_STG = OFF_Y + 2 * Y_BYTES;
     static constexpr int OFF_BAR = OFF_STG + STG_BYTES;
-    static constexpr int TOTAL = OFF_BAR + 256 + 1024;  // + alignment slack
+    static constexpr int TOTAL = OFF_BAR + 256;
+    static constexpr uint32_t TMEM_COLS = EMIT ? 128 : 256;   // S[2]: [0,128), O: [128,256)
+    static_assert(TOTAL <= 115712, "two CTAs must fit one SM's shared memory");
 };
 
 template <int KD, int MODE>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ CUtensorMap tmQ,
                 const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmY) {
     using L = Smem<KD, MODE>;
     constexpr bool PLANE = L::PLANE, EMIT = L::EMIT;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr int KST = L::KST;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    // 128-byte-swizzled tiles need 1024-byte aligned bases; the dynamic window starts on such a boundary (there is no
+    // static shared memory in this kernel).  Should that ever not hold, refuse loudly instead of computing garbage.
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (threadIdx.x == 0) atomicAdd(p.status + 1, 1);
+        return;
+    }
     uint8_t* sQ = smem + L::OFF_Q;
     uint8_t* sK = smem + L::OFF_K;
     uint8_t* sV = smem + L::OFF_V;
@@ -86,16 +98,16 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     uint8_t* sStg = smem + L::OFF_STG;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
     uint64_t* q_full = bars + 0;
-    uint64_t* k_full = bars + 1;    // [2]
-    uint64_t* k_empty = bars + 3;   // [2]
-    uint64_t* v_full = bars + 5;    // [2] V and Y of a stage
-    uint64_t* v_empty = bars + 7;   // [2]
-    uint64_t* s_full = bars + 9;    // [2] score buffer written by the MMA
-    uint64_t* s_free = bars + 11;   // [2] score buffer copied to registers by all 128 rows
-    uint64_t* p_full = bars + 13;
-    uint64_t* pv_done = bars + 14;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 17);
+    uint64_t* k_full = bars + 1;    // [KST <= 3]
+    uint64_t* k_empty = bars + 4;   // [KST <= 3]
+    uint64_t* v_full = bars + 7;    // [2] V and Y of a stage
+    uint64_t* v_empty = bars + 9;   // [2]
+    uint64_t* s_full = bars + 11;   // [2] score buffer written by the MMA
+    uint64_t* s_free = bars + 13;   // [2] score buffer copied to registers by all 128 rows
+    uint64_t* p_full = bars + 15;
+    uint64_t* pv_done = bars + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 19);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // blockIdx.x (the fastest-dispatched index) runs over (batch, head), blockIdx.y over query tiles from the last one
@@ -103,13 +115,13 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     const int qt = p.qt_begin + (int)gridDim.y - 1 - (int)blockIdx.y;
     const int h = (int)blockIdx.x % p.Hq, b = (int)blockIdx.x / p.Hq;
     const int g = h / (p.Hq / p.Hkv);
-    const int nt = qt + 1;  // key tiles 0..qt
     const int q0 = qt * BM;
+    const int nt = min((q0 + BM) / BN, (p.N + BN - 1) / BN);  // key tiles 0..nt-1 reach the last query row / the last key
 
     if (tid == 0) {
         mbar_init(q_full, 1);
+        for (int i = 0; i < KST; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1);
             mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
             mbar_init(s_full + i, 1); mbar_init(s_free + i, 128);
         }
@@ -118,12 +130,12 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         *abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == 5) tmem_alloc(tmem_slot, TMEM_COLS);
+    if (warp == 5) tmem_alloc(tmem_slot, L::TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_O = tmem_base + 256;
+    const uint32_t tmem_O = tmem_base + 128;
 
     if (warp == 4) {
         // ------------------------------ TMA producer ------------------------------
@@ -132,35 +144,34 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         if (lane == 0) {
             tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
             if (!EMIT) tma_prefetch_desc(&tmV);
+            if (PLANE) tma_prefetch_desc(&tmY);
             mbar_expect_tx(q_full, L::Q_BYTES);
         }
         __syncwarp();
         if (lane < KD / 64) tma_load_4d(sQ + lane * (BM * 128), &tmQ, q_full, lane * 64, h, q0, b);
-        constexpr int NK = KD / 64, NV = EMIT ? 0 : D / 64, NY = PLANE ? BN / 64 : 0;
+        constexpr int NK = KD / 64, NV = EMIT ? 0 : D / 64, NY = PLANE ? 1 : 0;
         bool okp = true;
         for (int t = 0; t < nt; ++t) {
-            const int s = t & 1;
-            const uint32_t par = ((t >> 1) & 1) ^ 1;
+            const int sk = t % KST, sv = t & 1;
             if (lane == 0) {
-                okp = mbar_wait(k_empty + s, par, abort_flag);
-                if (okp) mbar_expect_tx(k_full + s, L::K_BYTES);
+                okp = mbar_wait(k_empty + sk, ((t / KST) & 1) ^ 1, abort_flag);
+                if (okp) mbar_expect_tx(k_full + sk, L::K_BYTES);
             }
             okp = __shfl_sync(0xffffffffu, okp, 0);
             if (!okp) break;
-            if (lane < NK) tma_load_4d(sK + s * L::K_BYTES + lane * (BN * 128), &tmK, k_full + s, lane * 64, g, t * BN, b);
+            if (lane < NK) tma_load_4d(sK + sk * L::K_BYTES + lane * (BN * 128), &tmK, k_full + sk, lane * 64, g, t * BN, b);
             __syncwarp();
             if constexpr (!EMIT) {
                 if (lane == 0) {
-                    okp = mbar_wait(v_empty + s, par, abort_flag);
-                    if (okp) mbar_expect_tx(v_full + s, L::V_BYTES + L::Y_BYTES);
+                    okp = mbar_wait(v_empty + sv, ((t >> 1) & 1) ^ 1, abort_flag);
+                    if (okp) mbar_expect_tx(v_full + sv, L::V_BYTES + L::Y_BYTES);
                 }
                 okp = __shfl_sync(0xffffffffu, okp, 0);
                 if (!okp) break;
                 if (lane < NV) {
-                    tma_load_4d(sV + s * L::V_BYTES + lane * (BN * 128), &tmV, v_full + s, lane * 64, g, t * BN, b);
+                    tma_load_4d(sV + sv * L::V_BYTES + lane * (BN * 128), &tmV, v_full + sv, lane * 64, g, t * BN, b);
                 } else if (lane < NV + NY) {
-                    const int c = lane - NV;
-                    tma_load_3d(sY + s * L::Y_BYTES + c * (BM * 128), &tmY, v_full + s, t * BN + c * 64, q0 - p.plane_row0, b * p.Hq + h);
+                    tma_load_3d(sY + sv * L::Y_BYTES, &tmY, v_full + sv, t * BN, q0 - p.plane_row0, b * p.Hq + h);
                 }
                 __syncwarp();
             }
@@ -173,20 +184,21 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             const int ksteps = p.ksteps;
             // scores of tile t into buffer t&1; needs K(t) loaded and (t >= 2) the buffer read by the softmax of t-2
             auto issue_qk = [&](int t) -> bool {
-                const int s = t & 1;
-                if (!mbar_wait(k_full + s, (t >> 1) & 1, abort_flag)) return false;
+                const int s = t & 1, sk = t % KST;
+                if (!mbar_wait(k_full + sk, (t / KST) & 1, abort_flag)) return false;
                 if (!mbar_wait(s_free + s, ((t >> 1) & 1) ^ 1, abort_flag)) return false;
                 tc_fence_after();
-                const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + s * L::K_BYTES);
+                const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + sk * L::K_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < KD / 16; ++ks) {
                     if (ks < ksteps) {
-                        const uint32_t off = (ks >> 2) * (BM * 128) + (ks & 3) * 32;
-                        umma_ss(tmem_base + s * 128, umma_desc_sw128(qa + off, 16, 1024), umma_desc_sw128(ka + off, 16, 1024), IDESC_QK, ks > 0);
+                        const uint32_t q_off = (ks >> 2) * (BM * 128) + (ks & 3) * 32;
+                        const uint32_t k_off = (ks >> 2) * (BN * 128) + (ks & 3) * 32;
+                        umma_ss(tmem_base + s * BN, umma_desc_sw128(qa + q_off, 16, 1024), umma_desc_sw128(ka + k_off, 16, 1024), IDESC_QK, ks > 0);
                     }
                 }
                 umma_commit(s_full + s);
-                if (t + 2 < nt) umma_commit(k_empty + s);  // nobody waits for the last two: do not arm them
+                if (t + KST < nt) umma_commit(k_empty + sk);  // nobody waits for the last ones: do not arm them
                 return true;
             };
             bool ok = mbar_wait(q_full, 0, abort_flag) && issue_qk(0);
@@ -199,9 +211,9 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 const uint32_t pa = smem_u32(sP), va = smem_u32(sV + s * L::V_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < BN / 16; ++ks) {
-                    const uint32_t a_off = (ks >> 2) * (BM * 128) + (ks & 3) * 32;  // P: K-major, 64 keys per 128-byte row
-                    const uint32_t b_off = ks * 2048;                               // V: 16 keys = two 8-row groups
-                    umma_ss(tmem_O, umma_desc_sw128(pa + a_off, 16, 1024), umma_desc_sw128(va + b_off, BN * 128, 1024), IDESC_PV,
+                    // P: K-major, 64 keys per 128-byte row; V: 16 keys = two 8-row groups, the next 64 d-columns
+                    // BN * 128 bytes further on
+                    umma_ss(tmem_O, umma_desc_sw128(pa + ks * 32, 16, 1024), umma_desc_sw128(va + ks * 2048, BN * 128, 1024), IDESC_PV,
                             (t > 0) || (ks > 0));
                 }
                 umma_commit(pv_done);
@@ -220,32 +232,32 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             const int s = t & 1;
             if (!(ok = mbar_wait(s_full + s, (t >> 1) & 1, abort_flag))) break;
             tc_fence_after();
-            uint32_t sr[128];
+            uint32_t sr[BN];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tmem_base + s * 128 + lane_sel + c * 32, sr + c * 32);
+            for (int c = 0; c < BN / 32; ++c) tmem_ld32(tmem_base + s * BN + lane_sel + c * 32, sr + c * 32);
             tmem_wait_ld();
             tc_fence_before();
             mbar_arrive(s_free + s);
             float* sf = reinterpret_cast<float*>(sr);
             if constexpr (EMIT) {
-                // this warp's 32 rows x 128 columns as fp16 into its staging buffer (two 64-column halves, swizzled
-                // like any other tile), then lanes 0 and 1 store one half each with TMA
-                uint8_t* stg = sStg + (warp * 2 + s) * 8192;
-                if (t >= 2 && lane < 2) tma_store_wait_read<1>();  // the store of tile t-2 has read this buffer
+                // this warp's 32 rows x 64 columns as fp16 into its staging buffer (swizzled like any other tile),
+                // then lane 0 stores it with TMA
+                uint8_t* stg = sStg + (warp * 2 + s) * 4096;
+                if (t >= 2 && lane == 0) tma_store_wait_read<1>();  // the store of tile t-2 has read this buffer
                 __syncwarp();
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
+                for (int c = 0; c < BN / 8; ++c) {
                     uint4 v;
                     v.x = pack_f16(sf[c * 8 + 0] * emit_scale, sf[c * 8 + 1] * emit_scale);
                     v.y = pack_f16(sf[c * 8 + 2] * emit_scale, sf[c * 8 + 3] * emit_scale);
                     v.z = pack_f16(sf[c * 8 + 4] * emit_scale, sf[c * 8 + 5] * emit_scale);
                     v.w = pack_f16(sf[c * 8 + 6] * emit_scale, sf[c * 8 + 7] * emit_scale);
-                    *reinterpret_cast<uint4*>(stg + (c >> 3) * 4096 + sw128_offset(lane, c & 7)) = v;
+                    *reinterpret_cast<uint4*>(stg + sw128_offset(lane, c)) = v;
                 }
                 fence_async_smem();
                 __syncwarp();
-                if (lane < 2) {
-                    tma_store_3d(&tmY, stg + lane * 4096, t * BN + lane * 64, q0 - p.plane_row0 + warp * 32, b * p.Hq + h);
+                if (lane == 0) {
+                    tma_store_3d(&tmY, stg, t * BN, q0 - p.plane_row0 + warp * 32, b * p.Hq + h);
                     tma_store_commit();
                 }
                 continue;
@@ -254,8 +266,8 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 if (!(ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag))) break;  // Y of this stage has landed
                 const uint8_t* yb = sY + s * L::Y_BYTES;
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const uint4 y = *reinterpret_cast<const uint4*>(yb + (c >> 3) * (BM * 128) + sw128_offset(row, c & 7));
+                for (int c = 0; c < BN / 8; ++c) {
+                    const uint4 y = *reinterpret_cast<const uint4*>(yb + sw128_offset(row, c));
                     const uint32_t w[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -266,16 +278,17 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 }
             }
             // from here on: PLANE -> sf holds log2-domain logits; otherwise raw scores, scaled inside the exp
-            if (t == nt - 1) {
+            if (t * BN + BN - 1 > q0) {   // the tile reaches past the CTA's first query row: mask keys after each row
 #pragma unroll
-                for (int j = 0; j < 128; ++j)
+                for (int j = 0; j < BN; ++j)
                     if (t * BN + j > qi) sf[j] = -INFINITY;
             }
             float m_t = sf[0];
 #pragma unroll
-            for (int j = 1; j < 128; ++j) m_t = fmaxf(m_t, sf[j]);
+            for (int j = 1; j < BN; ++j) m_t = fmaxf(m_t, sf[j]);
             if constexpr (!PLANE) m_t *= scale_log2;
             // lazy rescale: move the reference maximum only when some row of the warp outgrew it by 2^8
+            // (a row with every key of this tile masked has m_t = -inf and never asks for it)
             const bool grow = m_t > m_ref + 8.f;
             const bool rescale = __any_sync(0xffffffffu, grow) || t == 0;
             float factor = 1.f;
@@ -303,7 +316,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             float sum = 0.f;
             const float neg_m = -m_ref;
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
+            for (int c = 0; c < BN / 8; ++c) {
                 float e[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -312,7 +325,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 }
                 uint4 v;
                 v.x = pack_bf16(e[0], e[1]); v.y = pack_bf16(e[2], e[3]); v.z = pack_bf16(e[4], e[5]); v.w = pack_bf16(e[6], e[7]);
-                *reinterpret_cast<uint4*>(sP + (c >> 3) * (BM * 128) + sw128_offset(row, c & 7)) = v;
+                *reinterpret_cast<uint4*>(sP + sw128_offset(row, c)) = v;
             }
             l_sum = l_sum * factor + sum;
             fence_async_smem();
@@ -320,7 +333,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             mbar_arrive(p_full);
         }
         if constexpr (EMIT) {
-            if (lane < 2) tma_store_wait_all<0>();
+            if (lane == 0) tma_store_wait_all<0>();
         } else if (ok && mbar_wait(pv_done, (nt - 1) & 1, abort_flag)) {
             tc_fence_after();
             const float inv_l = 1.f / l_sum;
@@ -357,7 +370,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     if (warp == 5) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        tmem_dealloc(tmem_base, L::TMEM_COLS);
     }
 }
 
@@ -391,10 +404,10 @@ bool tma_ok(const lisa_tensor& t) {
     return t.dtype == LISA_BF16 && (reinterpret_cast<uintptr_t>(t.ptr) & 15u) == 0 && t.stride_b % 8 == 0 && t.stride_n % 8 == 0 &&
            t.stride_h % 8 == 0 && t.stride_b > 0 && t.stride_n > 0 && t.stride_h > 0;
 }
-bool map_bnhx(CUtensorMap* m, const lisa_tensor& t, int B, int N, int H, int X) {
+bool map_bnhx(CUtensorMap* m, const lisa_tensor& t, int B, int N, int H, int X, int rows) {
     const uint64_t dims[4] = {(uint64_t)X, (uint64_t)H, (uint64_t)N, (uint64_t)B};
     const uint64_t str[3] = {(uint64_t)t.stride_h * 2, (uint64_t)t.stride_n * 2, (uint64_t)t.stride_b * 2};
-    const uint32_t box[4] = {64, 1, 128, 1};
+    const uint32_t box[4] = {64, 1, (uint32_t)rows, 1};
     return make_tensor_map_bf16(m, t.ptr, 4, dims, str, box);
 }
 }  // namespace
@@ -406,9 +419,9 @@ bool tc_flash_supported(const TcFlashArgs& a) {
 
 cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     CUtensorMap tmQ, tmK, tmV, tmY;
-    if (!map_bnhx(&tmQ, a.qa, a.B, a.N, a.Hq, a.kd) || !map_bnhx(&tmK, a.ka, a.B, a.N, a.Hkv, a.kd)) return cudaErrorInvalidValue;
+    if (!map_bnhx(&tmQ, a.qa, a.B, a.N, a.Hq, a.kd, BM) || !map_bnhx(&tmK, a.ka, a.B, a.N, a.Hkv, a.kd, BN)) return cudaErrorInvalidValue;
     tmV = tmQ;
-    if (!a.emit_plane && !map_bnhx(&tmV, a.v, a.B, a.N, a.Hkv, D)) return cudaErrorInvalidValue;
+    if (!a.emit_plane && !map_bnhx(&tmV, a.v, a.B, a.N, a.Hkv, D, BN)) return cudaErrorInvalidValue;
     tmY = tmQ;
     if (a.emit_plane) {  // store map: one epilogue warp's 32 rows x 64 columns per copy
         const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * a.Hq};
@@ -441,6 +454,8 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     do {                                                                                                                   \
         auto kern = tc_flash_kernel<KD_, PL_>;                                                                             \
         if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<KD_, PL_>::TOTAL)) != cudaSuccess) \
+            return e;                                                                                                      \
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) \
             return e;                                                                                                      \
         kern<<<grid, kThreads, Smem<KD_, PL_>::TOTAL, stream>>>(p, tmQ, tmK, tmV, tmY);                                    \
     } while (0)
