@@ -56,23 +56,34 @@ template <int KD, int MODE>
 struct Smem {
     static constexpr bool PLANE = MODE == MODE_ATTN_PLANE;
     static constexpr bool EMIT = MODE == MODE_EMIT;
-    static constexpr int KST = EMIT ? 3 : 2;             // K ring depth (V/Y: two stages)
+    // P (the bf16 probabilities, A operand of P.V) is double-buffered so that the softmax of tile t+1 never waits
+    // for the P.V of tile t.  To stay inside half an SM's shared memory it borrows a buffer whose content is dead
+    // by then: with a plane, the Y tile of the same stage (each thread has read its own row of Y and overwrites just
+    // that row); with 128-wide keys, the K tile of the same stage (its score MMA has completed before the softmax
+    // starts), which is then released by the P.V MMA instead of the score MMA -- hence three K stages.  64-wide
+    // keys without a plane leave room for two buffers of their own.
+    static constexpr bool P_IN_Y = PLANE;
+    static constexpr bool P_IN_K = !EMIT && !PLANE && KD == 128;
+    static constexpr bool P_OWN = !EMIT && !P_IN_Y && !P_IN_K;
+    static constexpr int KST = (EMIT || P_IN_K) ? 3 : 2;  // K ring depth (V/Y: two stages)
     static constexpr int Q_BYTES = BM * KD * 2;
     static constexpr int K_BYTES = BN * KD * 2;
     static constexpr int V_BYTES = EMIT ? 0 : BN * D * 2;
-    static constexpr int P_BYTES = EMIT ? 0 : BM * BN * 2;
+    static constexpr int P_BYTES = BM * BN * 2;
+    static constexpr int P_OWN_BYTES = P_OWN ? 2 * P_BYTES : 0;
     static constexpr int Y_BYTES = PLANE ? BM * BN * 2 : 0;
     static constexpr int STG_BYTES = EMIT ? 4 * 2 * 4096 : 0;  // per epilogue warp: two buffers of [32 rows][128 B]
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + Q_BYTES;
     static constexpr int OFF_V = OFF_K + KST * K_BYTES;
     static constexpr int OFF_P = OFF_V + 2 * V_BYTES;
-    static constexpr int OFF_Y = OFF_P + P_BYTES;
+    static constexpr int OFF_Y = OFF_P + P_OWN_BYTES;
     static constexpr int OFF_STG = OFF_Y + 2 * Y_BYTES;
     static constexpr int OFF_BAR = OFF_STG + STG_BYTES;
     static constexpr int TOTAL = OFF_BAR + 256;
     static constexpr uint32_t TMEM_COLS = EMIT ? 128 : 256;   // S[2]: [0,128), O: [128,256)
     static_assert(TOTAL <= 115712, "two CTAs must fit one SM's shared memory");
+    static_assert(!P_IN_K || K_BYTES >= P_BYTES, "P must fit the K stage it borrows");
 };
 
 template <int KD, int MODE>
@@ -104,10 +115,16 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     uint64_t* v_empty = bars + 9;   // [2]
     uint64_t* s_full = bars + 11;   // [2] score buffer written by the MMA
     uint64_t* s_free = bars + 13;   // [2] score buffer copied to registers by all 128 rows
-    uint64_t* p_full = bars + 15;
-    uint64_t* pv_done = bars + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 19);
+    uint64_t* p_full = bars + 15;   // [2]
+    uint64_t* pv_done = bars + 17;  // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 19);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 20);
+    // P of tile t
+    auto p_buf = [&](int t) -> uint8_t* {
+        if constexpr (L::P_IN_Y) return sY + (t & 1) * L::Y_BYTES;
+        else if constexpr (L::P_IN_K) return sK + (t % KST) * L::K_BYTES;
+        else return sP + (t & 1) * L::P_BYTES;
+    };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // blockIdx.x (the fastest-dispatched index) runs over (batch, head), blockIdx.y over query tiles from the last one
@@ -124,9 +141,8 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         for (int i = 0; i < 2; ++i) {
             mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1);
             mbar_init(s_full + i, 1); mbar_init(s_free + i, 128);
+            mbar_init(p_full + i, 128); mbar_init(pv_done + i, 1);
         }
-        mbar_init(p_full, 128);
-        mbar_init(pv_done, 1);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -198,7 +214,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                     }
                 }
                 umma_commit(s_full + s);
-                if (t + KST < nt) umma_commit(k_empty + sk);  // nobody waits for the last ones: do not arm them
+                if (!L::P_IN_K && t + KST < nt) umma_commit(k_empty + sk);  // nobody waits for the last ones: do not arm them
                 return true;
             };
             bool ok = mbar_wait(q_full, 0, abort_flag) && issue_qk(0);
@@ -206,9 +222,9 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 const int s = t & 1;
                 if (t + 1 < nt && !(ok = issue_qk(t + 1))) break;
                 if constexpr (EMIT) continue;
-                if (!(ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag) && mbar_wait(p_full, t & 1, abort_flag))) break;
+                if (!(ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag) && mbar_wait(p_full + s, (t >> 1) & 1, abort_flag))) break;
                 tc_fence_after();
-                const uint32_t pa = smem_u32(sP), va = smem_u32(sV + s * L::V_BYTES);
+                const uint32_t pa = smem_u32(p_buf(t)), va = smem_u32(sV + s * L::V_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < BN / 16; ++ks) {
                     // P: K-major, 64 keys per 128-byte row; V: 16 keys = two 8-row groups, the next 64 d-columns
@@ -216,8 +232,9 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                     umma_ss(tmem_O, umma_desc_sw128(pa + ks * 32, 16, 1024), umma_desc_sw128(va + ks * 2048, BN * 128, 1024), IDESC_PV,
                             (t > 0) || (ks > 0));
                 }
-                umma_commit(pv_done);
+                umma_commit(pv_done + s);
                 if (t + 2 < nt) umma_commit(v_empty + s);
+                if (L::P_IN_K && t + KST < nt) umma_commit(k_empty + t % KST);
             }
         }
     } else {
@@ -283,9 +300,13 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 for (int j = 0; j < BN; ++j)
                     if (t * BN + j > qi) sf[j] = -INFINITY;
             }
-            float m_t = sf[0];
+            float mx[4] = {sf[0], sf[1], sf[2], sf[3]};   // four independent chains instead of one of 64 dependent steps
 #pragma unroll
-            for (int j = 1; j < BN; ++j) m_t = fmaxf(m_t, sf[j]);
+            for (int j = 4; j < BN; j += 4) {
+                mx[0] = fmaxf(mx[0], sf[j]); mx[1] = fmaxf(mx[1], sf[j + 1]);
+                mx[2] = fmaxf(mx[2], sf[j + 2]); mx[3] = fmaxf(mx[3], sf[j + 3]);
+            }
+            float m_t = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             if constexpr (!PLANE) m_t *= scale_log2;
             // lazy rescale: move the reference maximum only when some row of the warp outgrew it by 2^8
             // (a row with every key of this tile masked has m_t = -inf and never asks for it)
@@ -297,9 +318,9 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 factor = fast_exp2(m_ref - m_new);
                 m_ref = m_new;
             }
-            if (t > 0) {
-                if (!(ok = mbar_wait(pv_done, (t - 1) & 1, abort_flag))) break;
-                if (rescale) {
+            if (t > 0 && rescale) {   // the accumulator is touched only after every P.V issued so far has landed in it
+                if (!(ok = mbar_wait(pv_done + ((t - 1) & 1), ((t - 1) >> 1) & 1, abort_flag))) break;
+                {
                     tc_fence_after();
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -313,6 +334,10 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                     tmem_wait_st();
                 }
             }
+            if constexpr (L::P_OWN) {   // this buffer was the A operand of the P.V two tiles back
+                if (t >= 2 && !(ok = mbar_wait(pv_done + s, ((t - 2) >> 1) & 1, abort_flag))) break;
+            }
+            uint8_t* pb = p_buf(t);
             float sum = 0.f;
             const float neg_m = -m_ref;
 #pragma unroll
@@ -325,16 +350,16 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 }
                 uint4 v;
                 v.x = pack_bf16(e[0], e[1]); v.y = pack_bf16(e[2], e[3]); v.z = pack_bf16(e[4], e[5]); v.w = pack_bf16(e[6], e[7]);
-                *reinterpret_cast<uint4*>(sP + sw128_offset(row, c)) = v;
+                *reinterpret_cast<uint4*>(pb + sw128_offset(row, c)) = v;
             }
             l_sum = l_sum * factor + sum;
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(p_full);
+            mbar_arrive(p_full + s);
         }
         if constexpr (EMIT) {
             if (lane == 0) tma_store_wait_all<0>();
-        } else if (ok && mbar_wait(pv_done, (nt - 1) & 1, abort_flag)) {
+        } else if (ok && mbar_wait(pv_done + ((nt - 1) & 1), ((nt - 1) >> 1) & 1, abort_flag)) {
             tc_fence_after();
             const float inv_l = 1.f / l_sum;
             __nv_bfloat16* orow = p.o + b * p.o_sb + (int64_t)qi * p.o_sn + h * p.o_sh;
