@@ -155,42 +155,51 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
 
     if (warp == 4) {
         // ------------------------------ TMA producer ------------------------------
-        // Lane 0 waits for a stage and arms its barrier; then the copies are issued by different lanes at once
-        // (one 64-column box each): one thread issuing them back to back is several hundred cycles slower per copy.
+        // The two single-thread roles (this one and the MMA issuer) share their scheduler with busy softmax warps and
+        // get an instruction slot every several cycles, so their loops are kept to a few dozen instructions per tile:
+        // running stage counters instead of divisions, one wait/arm section by lane 0 per tile, then every copy of
+        // the tile issued at once by different lanes (one 64-column box each).
+        // V(t) (with Y(t)) travels together with K(t+1): both wait for the P.V of tile t-2 at the latest.
+        constexpr int NQ = KD / 64, NK = KD / 64, NV = EMIT ? 0 : D / 64, NY = PLANE ? 1 : 0;
         if (lane == 0) {
             tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
             if (!EMIT) tma_prefetch_desc(&tmV);
             if (PLANE) tma_prefetch_desc(&tmY);
             mbar_expect_tx(q_full, L::Q_BYTES);
+            mbar_expect_tx(k_full, L::K_BYTES);
         }
         __syncwarp();
-        if (lane < KD / 64) tma_load_4d(sQ + lane * (BM * 128), &tmQ, q_full, lane * 64, h, q0, b);
-        constexpr int NK = KD / 64, NV = EMIT ? 0 : D / 64, NY = PLANE ? 1 : 0;
-        bool okp = true;
+        if (lane < NQ) tma_load_4d(sQ + lane * (BM * 128), &tmQ, q_full, lane * 64, h, q0, b);
+        else if (lane < NQ + NK) tma_load_4d(sK + (lane - NQ) * (BN * 128), &tmK, k_full, (lane - NQ) * 64, g, 0, b);
+        __syncwarp();
+        int ks_next = 1 % KST;              // K stage of tile t+1
+        uint32_t kpar_next = 1;             // parity to wait for on its "empty" barrier (first pass: passes at once)
         for (int t = 0; t < nt; ++t) {
-            const int sk = t % KST, sv = t & 1;
+            const int sv = t & 1;
+            const bool more_k = t + 1 < nt;
+            bool okp = true;
             if (lane == 0) {
-                okp = mbar_wait(k_empty + sk, ((t / KST) & 1) ^ 1, abort_flag);
-                if (okp) mbar_expect_tx(k_full + sk, L::K_BYTES);
-            }
-            okp = __shfl_sync(0xffffffffu, okp, 0);
-            if (!okp) break;
-            if (lane < NK) tma_load_4d(sK + sk * L::K_BYTES + lane * (BN * 128), &tmK, k_full + sk, lane * 64, g, t * BN, b);
-            __syncwarp();
-            if constexpr (!EMIT) {
-                if (lane == 0) {
+                if constexpr (!EMIT) {
                     okp = mbar_wait(v_empty + sv, ((t >> 1) & 1) ^ 1, abort_flag);
                     if (okp) mbar_expect_tx(v_full + sv, L::V_BYTES + L::Y_BYTES);
                 }
-                okp = __shfl_sync(0xffffffffu, okp, 0);
-                if (!okp) break;
-                if (lane < NV) {
-                    tma_load_4d(sV + sv * L::V_BYTES + lane * (BN * 128), &tmV, v_full + sv, lane * 64, g, t * BN, b);
-                } else if (lane < NV + NY) {
-                    tma_load_3d(sY + sv * L::Y_BYTES, &tmY, v_full + sv, t * BN, q0 - p.plane_row0, b * p.Hq + h);
+                if (okp && more_k) {
+                    okp = mbar_wait(k_empty + ks_next, kpar_next, abort_flag);
+                    if (okp) mbar_expect_tx(k_full + ks_next, L::K_BYTES);
                 }
-                __syncwarp();
             }
+            okp = __shfl_sync(0xffffffffu, okp, 0);
+            if (!okp) break;
+            if (lane < NV) {
+                tma_load_4d(sV + sv * L::V_BYTES + lane * (BN * 128), &tmV, v_full + sv, lane * 64, g, t * BN, b);
+            } else if (lane < NV + NY) {
+                tma_load_3d(sY + sv * L::Y_BYTES, &tmY, v_full + sv, t * BN, q0 - p.plane_row0, b * p.Hq + h);
+            } else if (lane < NV + NY + NK && more_k) {
+                const int c = lane - NV - NY;
+                tma_load_4d(sK + ks_next * L::K_BYTES + c * (BN * 128), &tmK, k_full + ks_next, c * 64, g, (t + 1) * BN, b);
+            }
+            __syncwarp();
+            if (++ks_next == KST) { ks_next = 0; kpar_next ^= 1; }
         }
     } else if (warp == 5) {
         // ------------------------------ MMA issuer ------------------------------
@@ -198,43 +207,59 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             constexpr uint32_t IDESC_QK = umma_idesc_bf16(BM, BN, 0, 0);
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(BM, D, 0, 1);
             const int ksteps = p.ksteps;
-            // scores of tile t into buffer t&1; needs K(t) loaded and (t >= 2) the buffer read by the softmax of t-2
-            auto issue_qk = [&](int t) -> bool {
-                const int s = t & 1, sk = t % KST;
-                if (!mbar_wait(k_full + sk, (t / KST) & 1, abort_flag)) return false;
+            // Descriptors are built once; per MMA only the start-address field (bits 0-13 of the low word, in
+            // 16-byte units) moves, by a compile-time constant or a stage offset: no carry can leave the field.
+            auto desc_off = [](uint64_t d, uint32_t bytes) -> uint64_t {
+                return (d & 0xffffffff00000000ull) | (uint32_t)((uint32_t)d + (bytes >> 4));
+            };
+            const uint64_t dq0 = umma_desc_sw128(smem_u32(sQ), 16, 1024);
+            const uint64_t dk0 = umma_desc_sw128(smem_u32(sK), 16, 1024);
+            const uint64_t dv0 = umma_desc_sw128(smem_u32(sV), BN * 128, 1024);
+            const uint64_t dp0 = umma_desc_sw128(smem_u32(p_buf(0)), 16, 1024);
+            constexpr uint32_t P_STRIDE = L::P_IN_Y ? L::Y_BYTES : (L::P_IN_K ? L::K_BYTES : L::P_BYTES);
+            // scores of the next tile into buffer t&1; needs K(t) loaded and (t >= 2) the buffer read by the softmax of t-2
+            int qk_t = 0, qk_sk = 0;
+            uint32_t qk_kpar = 0;
+            auto issue_qk = [&]() -> bool {
+                const int t = qk_t, s = t & 1;
+                if (!mbar_wait(k_full + qk_sk, qk_kpar, abort_flag)) return false;
                 if (!mbar_wait(s_free + s, ((t >> 1) & 1) ^ 1, abort_flag)) return false;
                 tc_fence_after();
-                const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + sk * L::K_BYTES);
+                const uint64_t dk = desc_off(dk0, qk_sk * L::K_BYTES);
+                const uint32_t dst = tmem_base + s * BN;
 #pragma unroll
                 for (int ks = 0; ks < KD / 16; ++ks) {
                     if (ks < ksteps) {
-                        const uint32_t q_off = (ks >> 2) * (BM * 128) + (ks & 3) * 32;
-                        const uint32_t k_off = (ks >> 2) * (BN * 128) + (ks & 3) * 32;
-                        umma_ss(tmem_base + s * BN, umma_desc_sw128(qa + q_off, 16, 1024), umma_desc_sw128(ka + k_off, 16, 1024), IDESC_QK, ks > 0);
+                        umma_ss(dst, desc_off(dq0, (ks >> 2) * (BM * 128) + (ks & 3) * 32), desc_off(dk, (ks >> 2) * (BN * 128) + (ks & 3) * 32),
+                                IDESC_QK, ks > 0);
                     }
                 }
                 umma_commit(s_full + s);
-                if (!L::P_IN_K && t + KST < nt) umma_commit(k_empty + sk);  // nobody waits for the last ones: do not arm them
+                if (!L::P_IN_K && t + KST < nt) umma_commit(k_empty + qk_sk);  // nobody waits for the last ones: do not arm them
+                ++qk_t;
+                if (++qk_sk == KST) { qk_sk = 0; qk_kpar ^= 1; }
                 return true;
             };
-            bool ok = mbar_wait(q_full, 0, abort_flag) && issue_qk(0);
+            bool ok = mbar_wait(q_full, 0, abort_flag) && issue_qk();
+            int pk = 0;   // P_IN_K: K stage that holds P(t)
             for (int t = 0; ok && t < nt; ++t) {
                 const int s = t & 1;
-                if (t + 1 < nt && !(ok = issue_qk(t + 1))) break;
+                if (t + 1 < nt && !(ok = issue_qk())) break;
                 if constexpr (EMIT) continue;
                 if (!(ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag) && mbar_wait(p_full + s, (t >> 1) & 1, abort_flag))) break;
                 tc_fence_after();
-                const uint32_t pa = smem_u32(p_buf(t)), va = smem_u32(sV + s * L::V_BYTES);
+                const uint64_t dp = desc_off(dp0, (L::P_IN_K ? pk : s) * P_STRIDE);
+                const uint64_t dv = desc_off(dv0, s * L::V_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < BN / 16; ++ks) {
                     // P: K-major, 64 keys per 128-byte row; V: 16 keys = two 8-row groups, the next 64 d-columns
                     // BN * 128 bytes further on
-                    umma_ss(tmem_O, umma_desc_sw128(pa + ks * 32, 16, 1024), umma_desc_sw128(va + ks * 2048, BN * 128, 1024), IDESC_PV,
-                            (t > 0) || (ks > 0));
+                    umma_ss(tmem_O, desc_off(dp, ks * 32), desc_off(dv, ks * 2048), IDESC_PV, (t > 0) || (ks > 0));
                 }
                 umma_commit(pv_done + s);
                 if (t + 2 < nt) umma_commit(v_empty + s);
-                if (L::P_IN_K && t + KST < nt) umma_commit(k_empty + t % KST);
+                if (L::P_IN_K && t + KST < nt) umma_commit(k_empty + pk);
+                if (++pk == KST) pk = 0;
             }
         }
     } else {
