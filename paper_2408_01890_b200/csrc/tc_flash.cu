@@ -194,7 +194,10 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         }
     } else if (warp == 5) {
         // ------------------------------ MMA issuer ------------------------------
-        if (lane == 0) {
+        // Every lane of the warp runs the loop (waits, stage counters, descriptor arithmetic: all warp-uniform);
+        // only the MMA and commit instructions themselves are predicated on lane 0.
+        {
+            const uint32_t issue = lane == 0;
             constexpr uint32_t IDESC_QK = umma_idesc_bf16(BM, BN, 0, 0);
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(BM, D, 0, 1);
             const int ksteps = p.ksteps;
@@ -213,31 +216,32 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             uint32_t qk_kpar = 0;
             auto issue_qk = [&]() -> bool {
                 const int t = qk_t, s = t & 1;
-                if (!mbar_wait(k_full + qk_sk, qk_kpar, abort_flag)) return false;
-                if (!mbar_wait(s_free + s, ((t >> 1) & 1) ^ 1, abort_flag)) return false;
+                const bool ready = mbar_wait(k_full + qk_sk, qk_kpar, abort_flag) && mbar_wait(s_free + s, ((t >> 1) & 1) ^ 1, abort_flag);
+                if (!__all_sync(0xffffffffu, ready)) return false;   // one verdict for the whole warp
                 tc_fence_after();
                 const uint64_t dk = desc_off(dk0, qk_sk * L::K_BYTES);
                 const uint32_t dst = tmem_base + s * BN;
 #pragma unroll
                 for (int ks = 0; ks < KD / 16; ++ks) {
                     if (ks < ksteps) {
-                        umma_ss(dst, desc_off(dq0, (ks >> 2) * (BM * 128) + (ks & 3) * 32), desc_off(dk, (ks >> 2) * (BN * 128) + (ks & 3) * 32),
+                        umma_ss_if(issue, dst, desc_off(dq0, (ks >> 2) * (BM * 128) + (ks & 3) * 32), desc_off(dk, (ks >> 2) * (BN * 128) + (ks & 3) * 32),
                                 IDESC_QK, ks > 0);
                     }
                 }
-                umma_commit(s_full + s);
-                if (!L::P_IN_K && t + KST < nt) umma_commit(k_empty + qk_sk);  // nobody waits for the last ones: do not arm them
+                umma_commit_if(issue, s_full + s);
+                if (!L::P_IN_K && t + KST < nt) umma_commit_if(issue, k_empty + qk_sk);  // nobody waits for the last ones: do not arm them
                 ++qk_t;
                 if (++qk_sk == KST) { qk_sk = 0; qk_kpar ^= 1; }
                 return true;
             };
-            bool ok = mbar_wait(q_full, 0, abort_flag) && issue_qk();
+            bool ok = __all_sync(0xffffffffu, mbar_wait(q_full, 0, abort_flag)) && issue_qk();
             int pk = 0;   // P_IN_K: K stage that holds P(t)
             for (int t = 0; ok && t < nt; ++t) {
                 const int s = t & 1;
                 if (t + 1 < nt && !(ok = issue_qk())) break;
                 if constexpr (EMIT) continue;
-                if (!(ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag) && mbar_wait(p_full + s, (t >> 1) & 1, abort_flag))) break;
+                ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag) && mbar_wait(p_full + s, (t >> 1) & 1, abort_flag);
+                if (!(ok = __all_sync(0xffffffffu, ok))) break;
                 tc_fence_after();
                 const uint64_t dp = desc_off(dp0, (L::P_IN_K ? pk : s) * P_STRIDE);
                 const uint64_t dv = desc_off(dv0, s * L::V_BYTES);
@@ -245,11 +249,11 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 for (int ks = 0; ks < BN / 16; ++ks) {
                     // P: K-major, 64 keys per 128-byte row; V: 16 keys = two 8-row groups, the next 64 d-columns
                     // BN * 128 bytes further on
-                    umma_ss(tmem_O, desc_off(dp, ks * 32), desc_off(dv, ks * 2048), IDESC_PV, (t > 0) || (ks > 0));
+                    umma_ss_if(issue, tmem_O, desc_off(dp, ks * 32), desc_off(dv, ks * 2048), IDESC_PV, (t > 0) || (ks > 0));
                 }
-                umma_commit(pv_done + s);
-                if (t + 2 < nt) umma_commit(v_empty + s);
-                if (L::P_IN_K && t + KST < nt) umma_commit(k_empty + pk);
+                umma_commit_if(issue, pv_done + s);
+                if (t + 2 < nt) umma_commit_if(issue, v_empty + s);
+                if (L::P_IN_K && t + KST < nt) umma_commit_if(issue, k_empty + pk);
                 if (++pk == KST) pk = 0;
             }
         }
