@@ -155,42 +155,57 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
 
     if (warp == 4) {
         // ------------------------------ TMA producer ------------------------------
-        // Lane 0 waits for a stage and arms its barrier; then the copies are issued by different lanes at once
-        // (one 64-column box each): one thread issuing them back to back is several hundred cycles slower per copy.
+        // The two single-thread roles (this one and the MMA issuer) share their scheduler with busy softmax warps and
+        // get an instruction slot every several cycles, so their loops are kept to a few dozen instructions per tile:
+        // running stage counters instead of divisions, one wait/arm section by lane 0 per tile, then every copy of
+        // the tile issued by different lanes (one 64-column box each).
+        // V(t) (with Y(t)) travels together with K(t+1): both wait for the P.V of tile t-2 at the latest.
+        constexpr int NQ = KD / 64, NK = KD / 64, NV = EMIT ? 0 : D / 64;
         if (lane == 0) {
             tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
             if (!EMIT) tma_prefetch_desc(&tmV);
             if (PLANE) tma_prefetch_desc(&tmY);
             mbar_expect_tx(q_full, L::Q_BYTES);
+            mbar_expect_tx(k_full, L::K_BYTES);
         }
         __syncwarp();
-        if (lane < KD / 64) tma_load_4d(sQ + lane * (BM * 128), &tmQ, q_full, lane * 64, h, q0, b);
-        constexpr int NK = KD / 64, NV = EMIT ? 0 : D / 64, NY = PLANE ? 1 : 0;
-        bool okp = true;
+        // One call site per tensor map, each reached with the map and the barrier uniform over the warp and only the
+        // lane-dependent box differing, and a reconvergence point between sites.
+        if (lane < NQ) tma_load_4d(sQ + lane * (BM * 128), &tmQ, q_full, lane * 64, h, q0, b);
+        __syncwarp();
+        if (lane < NK) tma_load_4d(sK + lane * (BN * 128), &tmK, k_full, lane * 64, g, 0, b);
+        __syncwarp();
+        int ks_next = 1 % KST;              // K stage of tile t+1
+        uint32_t kpar_next = 1;             // parity to wait for on its "empty" barrier (first pass: passes at once)
         for (int t = 0; t < nt; ++t) {
-            const int sk = t % KST, sv = t & 1;
+            const int sv = t & 1;
+            const bool more_k = t + 1 < nt;
+            bool okp = true;
             if (lane == 0) {
-                okp = mbar_wait(k_empty + sk, ((t / KST) & 1) ^ 1, abort_flag);
-                if (okp) mbar_expect_tx(k_full + sk, L::K_BYTES);
-            }
-            okp = __shfl_sync(0xffffffffu, okp, 0);
-            if (!okp) break;
-            if (lane < NK) tma_load_4d(sK + sk * L::K_BYTES + lane * (BN * 128), &tmK, k_full + sk, lane * 64, g, t * BN, b);
-            __syncwarp();
-            if constexpr (!EMIT) {
-                if (lane == 0) {
+                if constexpr (!EMIT) {
                     okp = mbar_wait(v_empty + sv, ((t >> 1) & 1) ^ 1, abort_flag);
                     if (okp) mbar_expect_tx(v_full + sv, L::V_BYTES + L::Y_BYTES);
                 }
-                okp = __shfl_sync(0xffffffffu, okp, 0);
-                if (!okp) break;
-                if (lane < NV) {
-                    tma_load_4d(sV + sv * L::V_BYTES + lane * (BN * 128), &tmV, v_full + sv, lane * 64, g, t * BN, b);
-                } else if (lane < NV + NY) {
-                    tma_load_3d(sY + sv * L::Y_BYTES, &tmY, v_full + sv, t * BN, q0 - p.plane_row0, b * p.Hq + h);
+                if (okp && more_k) {
+                    okp = mbar_wait(k_empty + ks_next, kpar_next, abort_flag);
+                    if (okp) mbar_expect_tx(k_full + ks_next, L::K_BYTES);
                 }
+            }
+            okp = __shfl_sync(0xffffffffu, okp, 0);
+            if (!okp) break;
+            if constexpr (!EMIT) {
+                if (lane < NV) tma_load_4d(sV + sv * L::V_BYTES + lane * (BN * 128), &tmV, v_full + sv, lane * 64, g, t * BN, b);
                 __syncwarp();
             }
+            if constexpr (PLANE) {
+                if (lane == 0) tma_load_3d(sY + sv * L::Y_BYTES, &tmY, v_full + sv, t * BN, q0 - p.plane_row0, b * p.Hq + h);
+                __syncwarp();
+            }
+            if (more_k) {
+                if (lane < NK) tma_load_4d(sK + ks_next * L::K_BYTES + lane * (BN * 128), &tmK, k_full + ks_next, lane * 64, g, (t + 1) * BN, b);
+                __syncwarp();
+            }
+            if (++ks_next == KST) { ks_next = 0; kpar_next ^= 1; }
         }
     } else if (warp == 5) {
         // ------------------------------ MMA issuer ------------------------------
