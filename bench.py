@@ -31,8 +31,8 @@ DECODE = "cfg4_llama2_13b_decode"
 METRIC = "lisa_attention_tokens_per_s"
 # dram bytes (read + write) per launch from the ncu captures summarised under profiles/ (cold cache, same workload);
 # None for a kernel that has changed since its counters were taken
-PREFILL_TRAFFIC = {"align": 142717952 + 83444480, "emit_scores": 33583360 + 85699840, "attention": 176216320 + 10768896}
-DECODE_TRAFFIC_PER_SEQ = (395937024 + 4827392) / 8  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
+PREFILL_TRAFFIC = {"align": None, "emit_scores": None, "attention": None}
+DECODE_TRAFFIC_PER_SEQ = None  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
 
 
 def measured_peaks():
@@ -241,18 +241,36 @@ def main():
     positions = w.B * w.N * (w.N + 1) // 2
     phase_flops = {"pack": 0, "emit_scores": positions * 2 * w.Hq * w.d, "align": positions * 4 * w.Hq * w.m,
                    "attention": positions * (2 * w.Hq * w.r + 2 * w.Hq * w.d)}
+    # Algorithmic HBM bytes of each kernel.  The three kernels hand the scores of every causal position to one
+    # another as fp16 planes (2 bytes per position and head); those planes, not the flops, set each kernel's floor:
+    # at 60 flop per plane byte every one of them sits far left of the ridge (about 250 flop/byte).
+    plane = positions * w.Hq * 2
+    qk_lr = w.B * w.N * (w.Hq + w.Hkv) * 2
+    phase_bytes = {"pack": qk_lr * (w.r + 64), "emit_scores": qk_lr * w.d + plane, "align": 2 * plane,
+                   "attention": plane + qk_lr * 64 + w.B * w.N * (w.Hkv + w.Hq) * w.d * 2}
     names = ["pack", "emit_scores", "align", "attention"]
-    kernels = {n: {"ms": phase_ms[i], "flops": phase_flops[n],
-                   "tflops": (phase_flops[n] / (phase_ms[i] * 1e-3) / 1e12) if phase_ms[i] > 0 else None,
-                   "share": phase_ms[i] / max(sum(phase_ms), 1e-9)} for i, n in enumerate(names)}
+    kernels = {}
+    for i, n in enumerate(names):
+        sec = phase_ms[i] * 1e-3
+        t_tensor, t_hbm = phase_flops[n] / (peaks["bf16_tflops"] * 1e12), phase_bytes[n] / (peaks["hbm_gbs"] * 1e9)
+        kernels[n] = {"ms": phase_ms[i], "share": phase_ms[i] / max(sum(phase_ms), 1e-9), "flops": phase_flops[n],
+                      "bytes": phase_bytes[n], "tflops": phase_flops[n] / sec / 1e12 if sec > 0 else None,
+                      "gbs": phase_bytes[n] / sec / 1e9 if sec > 0 else None, "bound": "hbm" if t_hbm >= t_tensor else "tensor",
+                      "frac": max(t_tensor, t_hbm) / sec if sec > 0 else None, "traffic": PREFILL_TRAFFIC.get(n)}
     dom = max(names, key=lambda n: kernels[n]["ms"])
-    achieved = kernels[dom]["tflops"] or 0.0
+    kd = kernels[dom]
     call_tflops = flops / (kernel_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "lisa_attn_shared_prefill/" + dom, "achieved": achieved, "peak": peaks["bf16_tflops"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",
-                "traffic": PREFILL_TRAFFIC.get(dom), "kernel_ms": kernels[dom]["ms"], "flops_per_launch": kernels[dom]["flops"],
-                "kernels": kernels,
-                "whole_call": {"ms": kernel_ms, "flops": flops, "achieved": call_tflops, "frac": call_tflops / peaks["bf16_tflops"]}}
+    if kd["bound"] == "hbm":
+        roofline = {"bound": "hbm", "kernel": "lisa_attn_shared_prefill/" + dom, "achieved": kd["gbs"], "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": kd["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                    "bytes_per_launch": kd["bytes"]}
+    else:
+        roofline = {"bound": "tensor", "kernel": "lisa_attn_shared_prefill/" + dom, "achieved": kd["tflops"], "peak": peaks["bf16_tflops"],
+                    "unit": "TFLOP/s", "frac": kd["tflops"] / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",
+                    "flops_per_launch": kd["flops"]}
+    roofline.update({"traffic": kd["traffic"], "kernel_ms": kd["ms"], "kernels": kernels,
+                     "whole_call": {"bound": "tensor", "ms": kernel_ms, "flops": flops, "achieved": call_tflops, "unit": "TFLOP/s",
+                                    "frac": call_tflops / peaks["bf16_tflops"]}})
 
 
     # ---------------- end to end through the host-memory entry point ----------------
@@ -329,7 +347,7 @@ def main():
                                       "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0,
                                       "peak_source": peaks["source"], "kernel_ms": k_ms,
                                       "bytes_per_launch": decode_bytes(wd, shared, B),
-                                      "traffic": DECODE_TRAFFIC_PER_SEQ * B if shared else None}}
+                                      "traffic": DECODE_TRAFFIC_PER_SEQ * B if shared and DECODE_TRAFFIC_PER_SEQ else None}}
         decode = {"workload": DECODE, "B": B, "L": L, "Hq": wd.Hq, "d": wd.d, "r": wd.r, "m": wd.m,
                   "shared": res["shared"], "standard": res["standard"],
                   "shared_over_standard": res["shared"]["value"] / res["standard"]["value"]}
