@@ -31,8 +31,8 @@ DECODE = "cfg4_llama2_13b_decode"
 METRIC = "lisa_attention_tokens_per_s"
 # dram bytes (read + write) per launch from the ncu captures summarised under profiles/ (cold cache, same workload);
 # None for a kernel that has changed since its counters were taken
-PREFILL_TRAFFIC = {"align": None, "emit_scores": None, "attention": None}
-DECODE_TRAFFIC_PER_SEQ = None  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
+PREFILL_TRAFFIC = {"align": 142647296 + 88310784, "emit_scores": 39532544 + 86390528, "attention": 186269184 + 5880064}
+DECODE_TRAFFIC_PER_SEQ = (395953152 + 5092608) / 8  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
 
 
 def measured_peaks():
