@@ -1,28 +1,28 @@
 // Head-axis aligner on tensor cores (Sec. 5.1): the FFN chain of a shared layer applied to score planes.
 //
-// Input: fp16 planes [B*Hq][rows][cols] (fp16, not bf16: three more mantissa bits keep a chain of several links
+// Input: fp16 planes [rows][B*Hq][cols] (fp16, not bf16: three more mantissa bits keep a chain of several links
 // inside the accuracy bar; scores are O(10), far from fp16's range limit, and conversions saturate) holding
 // A_0 = Q0.K0^T/sqrt(d) (Eq. 2) and, for chain depth c > 1, the already scaled differences
 // D_k = Q'_k.K'_k^T/sqrt(r) (Eq. 3) of the links k < c.  Output, in place of the A_0 plane:
 // Y = log2(e) * FFN_c(A_{c-1}) where A_k = FFN_k(A_{k-1}) + D_k (Eq. 4, ADD) -- the final link's D_c is added by
 // the attention kernel that consumes Y.  Hq = 32 heads, hidden width 64, two-layer FFNs.
 //
-// A warp owns strips of 16 key positions of one query row as the M dimension of warp-level MMAs (mma.sync
-// m16n8k16, fp16 in, fp32 accumulate) and keeps the whole chain in registers:
-//   H = A [16 x 32] . W1 [32 x 64]      A fragments: lane h loads [head h][16 positions] (32 B), parks it in the warp's
-//                                        scratch and ldmatrix.trans hands out the fragments, so the
-//                                        [head][position] -> [position][head] transposition costs nothing
-//   Y = act(H + b1) [16 x 64] . W2      the accumulator fragments of H, packed to fp16, ARE the A fragments of this MMA
-//   A_k = Y + b2 + D_k                  D_k read with the same ldmatrix.trans; packed again it feeds the next link
-// and the last Y goes back through the scratch with stmatrix.trans, 32 bytes per head and lane.
+// A warp owns pieces of 32 key positions of one query row and, within a piece, strips of 16 positions as the M
+// dimension of warp-level MMAs (mma.sync m16n8k16), keeping the whole chain in registers:
+//   global -> scratch      cp.async, 16 bytes per lane, four lanes per head, several pieces ahead
+//   H = A [16 x 32] . W1   A fragments by ldmatrix.trans from the warp's [head][position] scratch, so the
+//                          [head][position] -> [position][head] transposition costs nothing; fp16 accumulators
+//   Y = act(H + b1) . W2   the accumulator registers of H ARE the A fragments of this MMA (packed activation, no
+//                          conversion); fp32 accumulators
+//   A_k = Y + b2 + D_k     D_k read with the same ldmatrix.trans; packed again it feeds the next link
+// and the last Y goes back through the scratch with stmatrix.trans and out with 16-byte stores.
 // Why not tcgen05 here: the contractions are tiny (K = 32/64, N = 64/32) and an elementwise step sits between any
 // two of them, so with tensor-memory accumulators every step pays a round trip through TMEM, shared memory and an
 // mbarrier hand-off between the issuing thread and the threads that apply the activation; measured on B200 that
 // version spent ~13 clocks per position and link (tensor pipe 5% busy).  mma.sync runs at a quarter of the tcgen05
-// rate (measured 555 TFLOP/s) but needs 4 clocks per position and link with nothing leaving the registers.
-// A TMA-fed variant of this kernel (producer warp, slab ring) was slower: one copy per 128 positions gathers 64
-// rows of 128 bytes from 32 planes and took the issuing thread ~2000 cycles.  Here every warp is independent: no
-// block-wide barrier after set-up, no mbarrier, no wait that could hang.
+// rate (measured 555 TFLOP/s) but nothing leaves the registers.  Every warp is independent: no block-wide barrier
+// after set-up, no mbarrier, no wait that could hang.  The kernel is bound by the planes it moves (4 bytes per
+// position and head for one link), not by its arithmetic.
 #include <algorithm>
 
 #include "common.cuh"
@@ -47,7 +47,7 @@ struct AlignParams {
     int row0, qt_begin, qt_count;  // planes hold query rows row0.. ; this launch covers tiles [qt_begin, qt_begin + qt_count)
     int units_per_batch;           // sum over the covered tiles of valid rows x key blocks
     int64_t plane_rows, plane_cols;
-    __half* planes[kMaxTcChain];   // [0] = A_0 in / Y out; [k] = D_k for k = 1..c-1; each [B*32][plane_rows][plane_cols]
+    __half* planes[kMaxTcChain];   // [0] = A_0 in / Y out; [k] = D_k for k = 1..c-1; each [plane_rows][B*32][plane_cols]
     const void *w1[kMaxTcChain], *b1[kMaxTcChain], *w2[kMaxTcChain], *b2[kMaxTcChain];
     int w_dtype[kMaxTcChain], act[kMaxTcChain];
     int* status;

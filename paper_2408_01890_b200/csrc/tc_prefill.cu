@@ -1,7 +1,7 @@
 // Tensor-core prefill of a shared layer (Sec. 5.1, Eq. 3-4, then Eq. 1): host-side orchestration.
 //
 // The aligner mixes all heads at one (query, key) position while softmax.V needs one running output per
-// head, so the layer runs as three tensor-core kernels that exchange fp16 score planes [head][row][col]
+// head, so the layer runs as three tensor-core kernels that exchange fp16 score planes [row][head][col]
 // through a workspace sized to stay in L2, one wave of query tiles at a time:
 //   1. tc_flash (emit)   A_0 = Q0.K0^T/sqrt(d) per head, and D_k = Q'_k.K'_k^T/sqrt(r) for the links k < c
 //   2. tc_align          per position: the FFN chain over the head axis, Y written over A_0
