@@ -68,7 +68,7 @@ size_t decode_workspace(int B, int Hq, int d, int L);
 
 // Tensor-core flash kernel (head width 128, bf16): O = softmax_causal(QA.KA^T * scale [+ plane]) . V for query tiles
 // [qt_begin, qt_begin + qt_count).  qa [B,N,Hq,kd], ka [B,N,Hkv,kd] with kd in {64,128}; plane (optional) holds
-// bf16 [plane_rows][B*Hq][plane_cols] pre-computed scores for query rows qt_begin*128 onwards.
+// bf16 blocked [rows/128][cols/64][128][B*Hq][64] pre-computed scores for query rows qt_begin*128 onwards.
 struct TcFlashArgs {
     int B, N, Hq, Hkv, kd;
     lisa_tensor qa, ka, v, o;
@@ -77,7 +77,7 @@ struct TcFlashArgs {
     int64_t plane_rows, plane_cols;
     int qt_begin, qt_count;
     // emit_plane != nullptr: no attention; the scaled scores of the covered tiles are written there as bf16
-    // ([plane_rows][B*Hq][plane_cols], rows relative to qt_begin*128); v, o and plane are then ignored.
+    // (blocked [rows/128][cols/64][128][B*Hq][64], rows relative to qt_begin*128); v, o and plane are then ignored.
     void* emit_plane = nullptr;
     int ksteps = 0;  // 16-wide k-steps to issue (0 = kd/16); the columns beyond are zero padding
 };
@@ -85,7 +85,7 @@ bool tc_flash_supported(const TcFlashArgs& a);
 cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t s);
 
 // Tensor-core aligner: applies the FFN chain of links[0..chain) to the score planes in place (see tc_align.cu).
-// planes[0] = A_0 in / Y out, planes[k] = D_k (already scaled) for k = 1..chain-1; all [plane_rows][B*32][plane_cols].
+// planes[0] = A_0 in / Y out, planes[k] = D_k (already scaled) for k = 1..chain-1; all blocked [rows/128][cols/64][128][B*32][64].
 struct TcAlignArgs {
     int B, N, chain, qt_begin, qt_count;
     int64_t plane_rows, plane_cols;

@@ -1,6 +1,6 @@
 // Head-axis aligner on tensor cores (Sec. 5.1): the FFN chain of a shared layer applied to score planes.
 //
-// Input: fp16 planes [rows][B*Hq][cols] (fp16, not bf16: three more mantissa bits keep a chain of several links
+// Input: fp16 planes, blocked [row block of 128][column block of 64][row][B*Hq][64 columns], (fp16, not bf16: three more mantissa bits keep a chain of several links
 // inside the accuracy bar; scores are O(10), far from fp16's range limit, and conversions saturate) holding
 // A_0 = Q0.K0^T/sqrt(d) (Eq. 2) and, for chain depth c > 1, the already scaled differences
 // D_k = Q'_k.K'_k^T/sqrt(r) (Eq. 3) of the links k < c.  Output, in place of the A_0 plane:
@@ -47,7 +47,7 @@ struct AlignParams {
     int row0, qt_begin, qt_count;  // planes hold query rows row0.. ; this launch covers tiles [qt_begin, qt_begin + qt_count)
     int units_per_batch;           // sum over the covered tiles of valid rows x key blocks
     int64_t plane_rows, plane_cols;
-    __half* planes[kMaxTcChain];   // [0] = A_0 in / Y out; [k] = D_k for k = 1..c-1; each [plane_rows][B*32][plane_cols]
+    __half* planes[kMaxTcChain];   // [0] = A_0 in / Y out; [k] = D_k for k = 1..c-1; blocked, see tc_flash.cu
     const void *w1[kMaxTcChain], *b1[kMaxTcChain], *w2[kMaxTcChain], *b2[kMaxTcChain];
     int w_dtype[kMaxTcChain], act[kMaxTcChain];
     int* status;
@@ -233,8 +233,10 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
     // index is XOR-ed with (head / 2) % 4 so that the 8 rows of an 8x8 matrix fall into distinct banks.
     const int l_head = lane >> 2, l_chunk = lane & 3;
     auto piece_off = [&](const Cursor& x, int head) {   // element offset of [head][this piece] + this lane's chunk
-        return ((int64_t)(x.t * UNIT + x.row - p.row0) * (p.B * HQ) + (x.b * HQ + head)) * p.plane_cols + x.jb * UNIT + x.sub * 32 +
-               l_chunk * 8;
+        // blocked plane: [row block of 128][column block of 64][row in block][b*HQ + head][64 columns]
+        const int r = x.t * UNIT + x.row - p.row0;
+        const int64_t blk = (int64_t)(r >> 7) * (p.plane_cols >> 6) + (x.jb * 2 + (x.sub >> 1));
+        return ((blk * 128 + (r & 127)) * (p.B * HQ) + (x.b * HQ + head)) * 64 + (x.sub & 1) * 32 + l_chunk * 8;
     };
     auto scr_off = [&](int head, int chunk) { return (uint32_t)(head * 64 + ((chunk ^ ((head >> 1) & 3)) << 4)); };
     uint8_t* scr = sScr + warp * (STAGES * c * 2048);     // [STAGES buffers][c planes][32 heads][64 B]
@@ -367,7 +369,7 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     }
     p.status = status_words();
     if (!p.status) return cudaErrorUnknown;
-    if (a.plane_cols % 32 != 0) return cudaErrorInvalidValue;   // pieces are moved as aligned 16-byte chunks
+    if (a.plane_cols % 64 != 0 || a.plane_rows % 128 != 0) return cudaErrorInvalidValue;   // whole blocks
     // One link: its weight fragments live in registers, 4-warp CTAs, three per SM, three pieces in flight per warp.
     // Longer chains: weights in shared memory, one 12-warp CTA per SM, one piece in flight per warp.
     const bool regw = a.chain == 1;

@@ -198,7 +198,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 __syncwarp();
             }
             if constexpr (PLANE) {
-                if (lane == 0) tma_load_3d(sY + sv * L::Y_BYTES, &tmY, v_full + sv, t * BN, q0 - p.plane_row0, b * p.Hq + h);
+                if (lane == 0) tma_load_5d(sY + sv * L::Y_BYTES, &tmY, v_full + sv, 0, b * p.Hq + h, 0, t, (q0 - p.plane_row0) / BM);
                 __syncwarp();
             }
             if (more_k) {
@@ -309,7 +309,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_3d(&tmY, stg, t * BN, q0 - p.plane_row0 + warp * 32, b * p.Hq + h);
+                    tma_store_5d(&tmY, stg, 0, b * p.Hq + h, warp * 32, t, (q0 - p.plane_row0) / BM);
                     tma_store_commit();
                 }
                 continue;
@@ -483,17 +483,17 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     tmV = tmQ;
     if (!a.emit_plane && !map_bnhx(&tmV, a.v, a.B, a.N, a.Hkv, D, BN)) return cudaErrorInvalidValue;
     tmY = tmQ;
-    if (a.emit_plane) {  // store map: one epilogue warp's 32 rows x 64 columns per copy
-        const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * a.Hq};
-        const uint64_t str[2] = {(uint64_t)a.B * a.Hq * a.plane_cols * 2, (uint64_t)a.plane_cols * 2};   // [row][b*Hq+h][col]
-        const uint32_t box[3] = {64, 32, 1};
-        if (!make_tensor_map_bf16(&tmY, a.emit_plane, 3, dims, str, box, true)) return cudaErrorInvalidValue;
-    }
-    if (a.plane) {
-        const uint64_t dims[3] = {(uint64_t)a.plane_cols, (uint64_t)a.plane_rows, (uint64_t)a.B * a.Hq};
-        const uint64_t str[2] = {(uint64_t)a.B * a.Hq * a.plane_cols * 2, (uint64_t)a.plane_cols * 2};   // [row][b*Hq+h][col]
-        const uint32_t box[3] = {64, 128, 1};
-        if (!make_tensor_map_bf16(&tmY, a.plane, 3, dims, str, box, true)) return cudaErrorInvalidValue;
+    // Score planes are blocked [row block of 128][column block of 64][row in block][b*Hq + h][64 columns]: the 32
+    // heads of a position lie 128 bytes apart (the aligner gathers them), and a head's 128 x 64 tile is 128 rows of 128
+    // bytes spread over one 128 * B*Hq * 128-byte block, which the CTAs of all heads fill or drain at about the same time.
+    if (a.emit_plane || a.plane) {
+        if (a.plane_rows % BM != 0 || a.plane_cols % BN != 0) return cudaErrorInvalidValue;
+        const uint64_t bh = (uint64_t)a.B * a.Hq, ncb = (uint64_t)a.plane_cols / BN, nrb = (uint64_t)a.plane_rows / BM;
+        const uint64_t dims[5] = {(uint64_t)BN, bh, (uint64_t)BM, ncb, nrb};
+        const uint64_t str[4] = {(uint64_t)BN * 2, bh * BN * 2, (uint64_t)BM * bh * BN * 2, ncb * BM * bh * BN * 2};
+        // emit: one epilogue warp's 32 rows x 64 columns per copy; attention: the CTA's 128 rows x 64 columns
+        const uint32_t box[5] = {(uint32_t)BN, 1, a.emit_plane ? 32u : (uint32_t)BM, 1, 1};
+        if (!make_tensor_map_bf16(&tmY, a.emit_plane ? a.emit_plane : a.plane, 5, dims, str, box, true)) return cudaErrorInvalidValue;
     }
     FlashParams p;
     p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv;
