@@ -11,10 +11,9 @@
 // With QA/KA = Q/K and no Y this is standard attention (Eq. 1-2).  In MODE_EMIT there is no softmax: the scaled
 // scores leave as fp16 tiles (staged in shared memory, stored with TMA) for the aligner kernel.
 //
-// Warp roles: warps 0-3 softmax/epilogue (thread = query row = TMEM lane), then one TMA producer warp and one MMA
-// issuer warp that also owns the tensor memory.  MODE_EMIT carries no state from tile to tile and has a second
-// epilogue warpgroup (warps 4-7); the two take alternate tiles.  K and V(/Y) have their own rings: a K stage is
-// free again as soon as its score MMA has run, a V stage after its P.V MMA.
+// Warp roles: warps 0-3 softmax/epilogue (thread = query row = TMEM lane), warp 4 TMA producer,
+// warp 5 MMA issuer and TMEM owner.  K and V(/Y) have their own rings: a K stage is free again as soon as its
+// score MMA has run, a V stage after its P.V MMA.
 // Sizing: the softmax warps are the slow stage (one exp2 per score on the 16-lane transcendental unit) and every
 // hand-off between the roles costs a few hundred cycles of latency, so TWO CTAs share an SM and fill each other's
 // gaps, prologues and epilogues: 64-key tiles keep a CTA at 112 KB of shared memory and 256 tensor-memory columns.
@@ -35,9 +34,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-// Epilogue warpgroups: one (the softmax carries a running state from tile to tile); the emit mode has no such state
-// and runs two that take alternate tiles (group g always reads score buffer g).
-constexpr int flash_threads(int mode) { return mode == 2 ? 320 : 192; }
+constexpr int kThreads = 192;
 
 struct FlashParams {
     int B, N, Hq, Hkv;
@@ -75,7 +72,7 @@ struct Smem {
     static constexpr int P_BYTES = BM * BN * 2;
     static constexpr int P_OWN_BYTES = P_OWN ? 2 * P_BYTES : 0;
     static constexpr int Y_BYTES = PLANE ? BM * BN * 2 : 0;
-    static constexpr int STG_BYTES = EMIT ? 8 * 4096 : 0;      // per epilogue warp (two warpgroups): [32 rows][128 B]
+    static constexpr int STG_BYTES = EMIT ? 4 * 2 * 4096 : 0;  // per epilogue warp: two buffers of [32 rows][128 B]
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + Q_BYTES;
     static constexpr int OFF_V = OFF_K + KST * K_BYTES;
@@ -90,14 +87,13 @@ struct Smem {
 };
 
 template <int KD, int MODE>
-__global__ void __launch_bounds__(flash_threads(MODE), 2)
+__global__ void __launch_bounds__(kThreads, 2)
 tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ CUtensorMap tmQ,
                 const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                 const __grid_constant__ CUtensorMap tmY) {
     using L = Smem<KD, MODE>;
     constexpr bool PLANE = L::PLANE, EMIT = L::EMIT;
     constexpr int KST = L::KST;
-    constexpr int NWG = EMIT ? 2 : 1, PW = 4 * NWG, MW = PW + 1;   // epilogue warpgroups; producer and MMA warp
     extern __shared__ __align__(1024) uint8_t smem[];
     // 128-byte-swizzled tiles need 1024-byte aligned bases; the dynamic window starts on such a boundary (there is no
     // static shared memory in this kernel).  Should that ever not hold, refuse loudly instead of computing garbage.
@@ -150,14 +146,14 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         *abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == MW) tmem_alloc(tmem_slot, L::TMEM_COLS);
+    if (warp == 5) tmem_alloc(tmem_slot, L::TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_O = tmem_base + 128;
 
-    if (warp == PW) {
+    if (warp == 4) {
         // ------------------------------ TMA producer ------------------------------
         // The two single-thread roles (this one and the MMA issuer) share their scheduler with busy softmax warps and
         // get an instruction slot every several cycles, so their loops are kept to a few dozen instructions per tile:
@@ -211,7 +207,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             }
             if (++ks_next == KST) { ks_next = 0; kpar_next ^= 1; }
         }
-    } else if (warp == MW) {
+    } else if (warp == 5) {
         // ------------------------------ MMA issuer ------------------------------
         // Every lane of the warp runs the loop (waits, stage counters, descriptor arithmetic: all warp-uniform);
         // only the MMA and commit instructions themselves are predicated on lane 0.
@@ -278,14 +274,13 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         }
     } else {
         // ------------------------------ softmax / epilogue (thread = query row) ------------------------------
-        const int row = tid & 127;                 // 0..127, TMEM lane
-        const int wg = warp >> 2, wq = warp & 3;   // warpgroup; warp within it = TMEM lane quarter
+        const int row = tid;                       // 0..127, TMEM lane
         const int qi = q0 + row;                   // global query index
-        const uint32_t lane_sel = (uint32_t)(wq * 32) << 16;
+        const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
         const float scale_log2 = p.scale_log2, emit_scale = p.scale;
         float m_ref = -INFINITY, l_sum = 0.f;
         bool ok = true;
-        for (int t = EMIT ? wg : 0; t < nt; t += NWG) {
+        for (int t = 0; t < nt; ++t) {
             const int s = t & 1;
             if (!(ok = mbar_wait(s_full + s, (t >> 1) & 1, abort_flag))) break;
             tc_fence_after();
@@ -299,8 +294,8 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             if constexpr (EMIT) {
                 // this warp's 32 rows x 64 columns as fp16 into its staging buffer (swizzled like any other tile),
                 // then lane 0 stores it with TMA
-                uint8_t* stg = sStg + warp * 4096;
-                if (lane == 0) tma_store_wait_read<0>();  // this warp's previous store (two tiles back) has read the buffer
+                uint8_t* stg = sStg + (warp * 2 + s) * 4096;
+                if (t >= 2 && lane == 0) tma_store_wait_read<1>();  // the store of tile t-2 has read this buffer
                 __syncwarp();
 #pragma unroll
                 for (int c = 0; c < BN / 8; ++c) {
@@ -314,7 +309,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    tma_store_5d(&tmY, stg, 0, b * p.Hq + h, wq * 32, t, (q0 - p.plane_row0) / BM);
+                    tma_store_5d(&tmY, stg, 0, b * p.Hq + h, warp * 32, t, (q0 - p.plane_row0) / BM);
                     tma_store_commit();
                 }
                 continue;
@@ -432,7 +427,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         while (clock64() - t0 < 4000000ll) __nanosleep(1000);
         __syncthreads();
     }
-    if (warp == MW) {
+    if (warp == 5) {
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, L::TMEM_COLS);
@@ -522,7 +517,7 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
             return e;                                                                                                      \
         if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) \
             return e;                                                                                                      \
-        kern<<<grid, flash_threads(PL_), Smem<KD_, PL_>::TOTAL, stream>>>(p, tmQ, tmK, tmV, tmY);                                    \
+        kern<<<grid, kThreads, Smem<KD_, PL_>::TOTAL, stream>>>(p, tmQ, tmK, tmV, tmY);                                    \
     } while (0)
     if (a.emit_plane) {
         if (a.kd == 128) LISA_LAUNCH_FLASH(128, MODE_EMIT);
