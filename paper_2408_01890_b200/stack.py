@@ -60,8 +60,13 @@ class AttentionStack:
         return l + 1 < self.n_layers and not self.is_standard[l + 1]
 
     # ------------------------------------------------------------------ prefill
-    def prefill(self, probe: Optional[Probe] = None) -> float:
-        """Runs every layer over the prompt and fills the caches. Returns the device time in milliseconds."""
+    def prefill(self, probe: Optional[Probe] = None, nf: bool = False) -> float:
+        """Runs every layer over the prompt and fills the caches. Returns the device time in milliseconds.
+
+        nf=True is the paper's lossless-prefill recipe (Sec. 5.2, "NF"): a shared layer attends over the prompt with
+        standard attention on its own full Q and K, and only what it caches differs (K_LR instead of K); sharing
+        starts with the first decoded token.  Prefill then costs what a standard stack costs.
+        """
         B, N, Hq, Hkv, d, r = self.B, self.N, self.Hq, self.Hkv, self.d, self.r
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         out = torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device="cuda")
@@ -70,6 +75,9 @@ class AttentionStack:
         for l in range(self.n_layers):
             if self.is_standard[l]:
                 drawn.append((self.draw("q", l, (B, N, Hq, d)), self.draw("k", l, (B, N, Hkv, d)), self.draw("v", l, (B, N, Hkv, d))))
+            elif nf:
+                drawn.append((self.draw("q", l, (B, N, Hq, d)), self.draw("k", l, (B, N, Hkv, d)), self.draw("v", l, (B, N, Hkv, d)),
+                              self.draw("kp", l, (B, N, Hkv, r))))
             else:
                 drawn.append((self.draw("qp", l, (B, N, Hq, r)), self.draw("kp", l, (B, N, Hkv, r)),
                               self.draw("v", l, (B, N, Hkv, d))))
@@ -79,8 +87,12 @@ class AttentionStack:
         q0 = k0 = None
         links: List[lb.Link] = []
         for l in range(self.n_layers):
-            a, b_, v = drawn[l]
-            if self.is_standard[l]:
+            a, b_, v = drawn[l][:3]
+            if nf and not self.is_standard[l]:
+                lb.lisa_attn_anchor(a, b_, v, out=out)
+                lb.lisa_kvcache_append(self.caches[l], drawn[l][3], v)
+                q0, k0, links = a, b_, []
+            elif self.is_standard[l]:
                 lb.lisa_attn_anchor(a, b_, v, out=out)
                 lb.lisa_kvcache_append(self.caches[l], b_, v)
                 q0, k0, links = a, b_, []

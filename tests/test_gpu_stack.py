@@ -49,6 +49,22 @@ def test_small_stack_every_layer():
     check_probe(st, probe)
 
 
+def test_small_stack_lossless_prefill():
+    """Sec. 5.2 "NF": shared layers attend over the prompt with standard attention on their own Q and K and cache
+    K_LR; sharing starts with the first decoded token."""
+    st = lstack.AttentionStack(n_layers=8, B=2, N=200, T=4, seed=5)
+    probe = lstack.Probe(layers=range(8), rows_b=[0, 1, 1, 0], rows_i=[0, 199, 64, 129], steps=[0, 3], seqs=[0, 1])
+    st.prefill(probe, nf=True)
+    for l in range(8):
+        if not st.is_standard[l]:
+            assert probe.prefill[l]["links"] == []                       # plain attention in prefill ...
+            kp = st.draw("kp", l, (2, 200, st.Hkv, st.r))                 # ... and K_LR (transposed) in the cache
+            assert torch.equal(st.caches[l].k[:, :, :, :200], kp.permute(0, 2, 3, 1))
+    st.decode(probe)
+    assert lb.lisa_check() == lb.OK
+    check_probe(st, probe)
+
+
 def test_cfg5_llama2_7b_stack_sampled():
     w = synth.WORKLOADS["cfg5_llama2_7b_stack"]
     st = lstack.AttentionStack(n_layers=32, B=w.B, N=w.N, T=256, Hq=w.Hq, Hkv=w.Hkv, d=w.d, r=w.r, m=w.m, act=w.act, seed=0)
