@@ -153,9 +153,9 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         // ------------------------------ TMA producer ------------------------------
         // The two single-thread roles (this one and the MMA issuer) share their scheduler with busy softmax warps and
         // get an instruction slot every several cycles, so their loops are kept to a few dozen instructions per tile:
-        // running stage counters instead of divisions, one wait/arm section by lane 0 per tile, then the copies of
-        // the tile issued by different lanes (one 64-column box each), one call site per tensor map with the map and
-        // the barrier uniform over the warp and a reconvergence point between sites.
+        // running stage counters instead of divisions, the copies issued by different lanes (one 64-column box each),
+        // one call site per tensor map with the map and the barrier uniform over the warp and a reconvergence point
+        // between sites.
         // K runs two tiles ahead of V (the score MMA of tile t+2 is issued before the P.V of tile t): per tile,
         // K(t+2) (its stage was freed by the score MMA of tile t) and V(t+1) (freed by the P.V of tile t-1).
         constexpr int NQ = KD / 64, NK = KD / 64, NV = EMIT ? 0 : D / 64;
@@ -190,31 +190,31 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         for (int t = 0; t < nt; ++t) {
             const int sv1 = (t + 1) & 1;
             const bool more_k = t + 2 < nt, more_v = !EMIT && t + 1 < nt;
+            // K first, in a section of its own: its stage is free long before the V stage is, and the score MMA two
+            // tiles ahead must not wait for a P.V to complete
             bool okp = true;
-            if (lane == 0) {
-                if (more_k) {
+            if (more_k) {
+                if (lane == 0) {
                     okp = mbar_wait(k_empty + ks2, kpar2, abort_flag);
                     if (okp) mbar_expect_tx(k_full + ks2, L::K_BYTES);
                 }
-                if (okp && more_v) {
-                    okp = mbar_wait(v_empty + sv1, (((t + 1) >> 1) & 1) ^ 1, abort_flag);
-                    if (okp) mbar_expect_tx(v_full + sv1, L::V_BYTES + L::Y_BYTES);
-                }
-            }
-            okp = __shfl_sync(0xffffffffu, okp, 0);
-            if (!okp) break;
-            if (more_k) {
+                okp = __shfl_sync(0xffffffffu, okp, 0);
+                if (!okp) break;
                 if (lane < NK) tma_load_4d(sK + ks2 * L::K_BYTES + lane * (BN * 128), &tmK, k_full + ks2, lane * 64, g, (t + 2) * BN, b);
                 __syncwarp();
             }
-            if constexpr (!EMIT) {
-                if (more_v) {
+            if (more_v) {
+                if (lane == 0) {
+                    okp = mbar_wait(v_empty + sv1, (((t + 1) >> 1) & 1) ^ 1, abort_flag);
+                    if (okp) mbar_expect_tx(v_full + sv1, L::V_BYTES + L::Y_BYTES);
+                }
+                okp = __shfl_sync(0xffffffffu, okp, 0);
+                if (!okp) break;
+                if constexpr (!EMIT) {
                     if (lane < NV) tma_load_4d(sV + sv1 * L::V_BYTES + lane * (BN * 128), &tmV, v_full + sv1, lane * 64, g, (t + 1) * BN, b);
                     __syncwarp();
                 }
-            }
-            if constexpr (PLANE) {
-                if (more_v) {
+                if constexpr (PLANE) {
                     if (lane == 0) tma_load_5d(sY + sv1 * L::Y_BYTES, &tmY, v_full + sv1, 0, b * p.Hq + h, 0, t + 1, (q0 - p.plane_row0) / BM);
                     __syncwarp();
                 }
