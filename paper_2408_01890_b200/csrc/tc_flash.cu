@@ -56,19 +56,21 @@ template <int KD, int MODE>
 struct Smem {
     static constexpr bool PLANE = MODE == MODE_ATTN_PLANE;
     static constexpr bool EMIT = MODE == MODE_EMIT;
-    // P (the bf16 probabilities, A operand of P.V).  With a plane it is written over the Y tile of the same stage
-    // (each thread has read its own row of Y and overwrites just that row), which makes it double-buffered for
-    // free.  Otherwise it has buffers of its own: two where 64-wide keys leave room, one with 128-wide keys (the
-    // softmax then waits for the previous P.V before it writes, a wait that is usually over by then).
+    // P (the bf16 probabilities, A operand of P.V) is double-buffered so that the softmax of tile t+1 never waits
+    // for the P.V of tile t.  To stay inside half an SM's shared memory it borrows a buffer whose content is dead
+    // by then: with a plane, the Y tile of the same stage (each thread has read its own row of Y and overwrites just
+    // that row); with 128-wide keys, the K tile of the same stage (its score MMA has completed before the softmax
+    // starts), which is then released by the P.V MMA instead of the score MMA -- hence three K stages.  64-wide
+    // keys without a plane leave room for two buffers of their own.
     static constexpr bool P_IN_Y = PLANE;
-    static constexpr bool P_OWN = !EMIT && !P_IN_Y;
-    static constexpr int NPB = !P_OWN ? 0 : (KD == 128 ? 1 : 2);   // own P buffers
-    static constexpr int KST = EMIT ? 3 : 2;               // K ring depth (V/Y: two stages)
+    static constexpr bool P_IN_K = !EMIT && !PLANE && KD == 128;
+    static constexpr bool P_OWN = !EMIT && !P_IN_Y && !P_IN_K;
+    static constexpr int KST = (EMIT || P_IN_K) ? 3 : 2;  // K ring depth (V/Y: two stages)
     static constexpr int Q_BYTES = BM * KD * 2;
     static constexpr int K_BYTES = BN * KD * 2;
     static constexpr int V_BYTES = EMIT ? 0 : BN * D * 2;
     static constexpr int P_BYTES = BM * BN * 2;
-    static constexpr int P_OWN_BYTES = NPB * P_BYTES;
+    static constexpr int P_OWN_BYTES = P_OWN ? 2 * P_BYTES : 0;
     static constexpr int Y_BYTES = PLANE ? BM * BN * 2 : 0;
     static constexpr int STG_BYTES = EMIT ? 4 * 2 * 4096 : 0;  // per epilogue warp: two buffers of [32 rows][128 B]
     static constexpr int OFF_Q = 0;
@@ -81,6 +83,7 @@ struct Smem {
     static constexpr int TOTAL = OFF_BAR + 256;
     static constexpr uint32_t TMEM_COLS = EMIT ? 128 : 256;   // S[2]: [0,128), O: [128,256)
     static_assert(TOTAL <= 115712, "two CTAs must fit one SM's shared memory");
+    static_assert(!P_IN_K || K_BYTES >= P_BYTES, "P must fit the K stage it borrows");
 };
 
 template <int KD, int MODE>
@@ -119,7 +122,8 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     // P of tile t
     auto p_buf = [&](int t) -> uint8_t* {
         if constexpr (L::P_IN_Y) return sY + (t & 1) * L::Y_BYTES;
-        else return sP + (L::NPB == 2 ? (t & 1) : 0) * L::P_BYTES;
+        else if constexpr (L::P_IN_K) return sK + (t % KST) * L::K_BYTES;
+        else return sP + (t & 1) * L::P_BYTES;
     };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -153,11 +157,9 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         // ------------------------------ TMA producer ------------------------------
         // The two single-thread roles (this one and the MMA issuer) share their scheduler with busy softmax warps and
         // get an instruction slot every several cycles, so their loops are kept to a few dozen instructions per tile:
-        // running stage counters instead of divisions, the copies issued by different lanes (one 64-column box each),
-        // one call site per tensor map with the map and the barrier uniform over the warp and a reconvergence point
-        // between sites.
-        // K runs two tiles ahead of V (the score MMA of tile t+2 is issued before the P.V of tile t): per tile,
-        // K(t+2) (its stage was freed by the score MMA of tile t) and V(t+1) (freed by the P.V of tile t-1).
+        // running stage counters instead of divisions, one wait/arm section by lane 0 per tile, then every copy of
+        // the tile issued by different lanes (one 64-column box each).
+        // V(t) (with Y(t)) travels together with K(t+1): both wait for the P.V of tile t-2 at the latest.
         constexpr int NQ = KD / 64, NK = KD / 64, NV = EMIT ? 0 : D / 64;
         if (lane == 0) {
             tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
@@ -165,61 +167,45 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             if (PLANE) tma_prefetch_desc(&tmY);
             mbar_expect_tx(q_full, L::Q_BYTES);
             mbar_expect_tx(k_full, L::K_BYTES);
-            if (nt > 1) mbar_expect_tx(k_full + 1, L::K_BYTES);
-            if (!EMIT) mbar_expect_tx(v_full, L::V_BYTES + L::Y_BYTES);
         }
         __syncwarp();
+        // One call site per tensor map, each reached with the map and the barrier uniform over the warp and only the
+        // lane-dependent box differing, and a reconvergence point between sites.
         if (lane < NQ) tma_load_4d(sQ + lane * (BM * 128), &tmQ, q_full, lane * 64, h, q0, b);
         __syncwarp();
         if (lane < NK) tma_load_4d(sK + lane * (BN * 128), &tmK, k_full, lane * 64, g, 0, b);
         __syncwarp();
-        if constexpr (!EMIT) {
-            if (lane < NV) tma_load_4d(sV + lane * (BN * 128), &tmV, v_full, lane * 64, g, 0, b);
-            __syncwarp();
-        }
-        if constexpr (PLANE) {
-            if (lane == 0) tma_load_5d(sY, &tmY, v_full, 0, b * p.Hq + h, 0, 0, (q0 - p.plane_row0) / BM);
-            __syncwarp();
-        }
-        if (nt > 1) {
-            if (lane < NK) tma_load_4d(sK + L::K_BYTES + lane * (BN * 128), &tmK, k_full + 1, lane * 64, g, BN, b);
-            __syncwarp();
-        }
-        int ks2 = 2 % KST;                        // K stage of tile t+2
-        uint32_t kpar2 = (2 / KST) & 1 ? 0u : 1u; // parity to wait for on its "empty" barrier: ((tile / KST) & 1) ^ 1
+        int ks_next = 1 % KST;              // K stage of tile t+1
+        uint32_t kpar_next = 1;             // parity to wait for on its "empty" barrier (first pass: passes at once)
         for (int t = 0; t < nt; ++t) {
-            const int sv1 = (t + 1) & 1;
-            const bool more_k = t + 2 < nt, more_v = !EMIT && t + 1 < nt;
-            // K first, in a section of its own: its stage is free long before the V stage is, and the score MMA two
-            // tiles ahead must not wait for a P.V to complete
+            const int sv = t & 1;
+            const bool more_k = t + 1 < nt;
             bool okp = true;
-            if (more_k) {
-                if (lane == 0) {
-                    okp = mbar_wait(k_empty + ks2, kpar2, abort_flag);
-                    if (okp) mbar_expect_tx(k_full + ks2, L::K_BYTES);
+            if (lane == 0) {
+                if constexpr (!EMIT) {
+                    okp = mbar_wait(v_empty + sv, ((t >> 1) & 1) ^ 1, abort_flag);
+                    if (okp) mbar_expect_tx(v_full + sv, L::V_BYTES + L::Y_BYTES);
                 }
-                okp = __shfl_sync(0xffffffffu, okp, 0);
-                if (!okp) break;
-                if (lane < NK) tma_load_4d(sK + ks2 * L::K_BYTES + lane * (BN * 128), &tmK, k_full + ks2, lane * 64, g, (t + 2) * BN, b);
+                if (okp && more_k) {
+                    okp = mbar_wait(k_empty + ks_next, kpar_next, abort_flag);
+                    if (okp) mbar_expect_tx(k_full + ks_next, L::K_BYTES);
+                }
+            }
+            okp = __shfl_sync(0xffffffffu, okp, 0);
+            if (!okp) break;
+            if constexpr (!EMIT) {
+                if (lane < NV) tma_load_4d(sV + sv * L::V_BYTES + lane * (BN * 128), &tmV, v_full + sv, lane * 64, g, t * BN, b);
                 __syncwarp();
             }
-            if (more_v) {
-                if (lane == 0) {
-                    okp = mbar_wait(v_empty + sv1, (((t + 1) >> 1) & 1) ^ 1, abort_flag);
-                    if (okp) mbar_expect_tx(v_full + sv1, L::V_BYTES + L::Y_BYTES);
-                }
-                okp = __shfl_sync(0xffffffffu, okp, 0);
-                if (!okp) break;
-                if constexpr (!EMIT) {
-                    if (lane < NV) tma_load_4d(sV + sv1 * L::V_BYTES + lane * (BN * 128), &tmV, v_full + sv1, lane * 64, g, (t + 1) * BN, b);
-                    __syncwarp();
-                }
-                if constexpr (PLANE) {
-                    if (lane == 0) tma_load_5d(sY + sv1 * L::Y_BYTES, &tmY, v_full + sv1, 0, b * p.Hq + h, 0, t + 1, (q0 - p.plane_row0) / BM);
-                    __syncwarp();
-                }
+            if constexpr (PLANE) {
+                if (lane == 0) tma_load_5d(sY + sv * L::Y_BYTES, &tmY, v_full + sv, 0, b * p.Hq + h, 0, t, (q0 - p.plane_row0) / BM);
+                __syncwarp();
             }
-            if (++ks2 == KST) { ks2 = 0; kpar2 ^= 1; }
+            if (more_k) {
+                if (lane < NK) tma_load_4d(sK + ks_next * L::K_BYTES + lane * (BN * 128), &tmK, k_full + ks_next, lane * 64, g, (t + 1) * BN, b);
+                __syncwarp();
+            }
+            if (++ks_next == KST) { ks_next = 0; kpar_next ^= 1; }
         }
     } else if (warp == 5) {
         // ------------------------------ MMA issuer ------------------------------
@@ -239,11 +225,8 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             const uint64_t dk0 = umma_desc_sw128(smem_u32(sK), 16, 1024);
             const uint64_t dv0 = umma_desc_sw128(smem_u32(sV), BN * 128, 1024);
             const uint64_t dp0 = umma_desc_sw128(smem_u32(p_buf(0)), 16, 1024);
-            constexpr uint32_t P_STRIDE = L::P_IN_Y ? L::Y_BYTES : (L::NPB == 2 ? L::P_BYTES : 0);
-            // scores of the next tile into buffer t&1; needs K(t) loaded and (t >= 2) the buffer read by the softmax of t-2.
-            // They run two tiles ahead of the P.V products: S(t+2) is issued as soon as the softmax of tile t has
-            // copied S(t) out of tensor memory, i.e. while that softmax is still computing, and is complete long
-            // before the softmax of tile t+1 ends; P.V(t) follows when P(t) arrives.
+            constexpr uint32_t P_STRIDE = L::P_IN_Y ? L::Y_BYTES : (L::P_IN_K ? L::K_BYTES : L::P_BYTES);
+            // scores of the next tile into buffer t&1; needs K(t) loaded and (t >= 2) the buffer read by the softmax of t-2
             int qk_t = 0, qk_sk = 0;
             uint32_t qk_kpar = 0;
             auto issue_qk = [&]() -> bool {
@@ -261,21 +244,21 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                     }
                 }
                 umma_commit_if(issue, s_full + s);
-                if (t + KST < nt) umma_commit_if(issue, k_empty + qk_sk);  // nobody waits for the last ones: do not arm them
+                if (!L::P_IN_K && t + KST < nt) umma_commit_if(issue, k_empty + qk_sk);  // nobody waits for the last ones: do not arm them
                 ++qk_t;
                 if (++qk_sk == KST) { qk_sk = 0; qk_kpar ^= 1; }
                 return true;
             };
             bool ok = __all_sync(0xffffffffu, mbar_wait(q_full, 0, abort_flag)) && issue_qk();
-            if (ok && nt > 1) ok = issue_qk();
+            int pk = 0;   // P_IN_K: K stage that holds P(t)
             for (int t = 0; ok && t < nt; ++t) {
                 const int s = t & 1;
-                if (t + 2 < nt && !(ok = issue_qk())) break;
+                if (t + 1 < nt && !(ok = issue_qk())) break;
                 if constexpr (EMIT) continue;
                 ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag) && mbar_wait(p_full + s, (t >> 1) & 1, abort_flag);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;
                 tc_fence_after();
-                const uint64_t dp = desc_off(dp0, s * P_STRIDE);
+                const uint64_t dp = desc_off(dp0, (L::P_IN_K ? pk : s) * P_STRIDE);
                 const uint64_t dv = desc_off(dv0, s * L::V_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < BN / 16; ++ks) {
@@ -285,6 +268,8 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 }
                 umma_commit_if(issue, pv_done + s);
                 if (t + 2 < nt) umma_commit_if(issue, v_empty + s);
+                if (L::P_IN_K && t + KST < nt) umma_commit_if(issue, k_empty + pk);
+                if (++pk == KST) pk = 0;
             }
         }
     } else {
@@ -384,9 +369,8 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                     tmem_wait_st();
                 }
             }
-            if constexpr (L::P_OWN) {   // this buffer was the A operand of the P.V one or two tiles back
-                constexpr int NPB = L::NPB;
-                if (t >= NPB && !(ok = mbar_wait(pv_done + ((t - NPB) & 1), ((t - NPB) >> 1) & 1, abort_flag))) break;
+            if constexpr (L::P_OWN) {   // this buffer was the A operand of the P.V two tiles back
+                if (t >= 2 && !(ok = mbar_wait(pv_done + s, ((t - 2) >> 1) & 1, abort_flag))) break;
             }
             uint8_t* pb = p_buf(t);
             float sum = 0.f;
