@@ -55,7 +55,7 @@ typedef enum lisa_act_t { LISA_ACT_NONE = 0, LISA_ACT_RELU = 1, LISA_ACT_SILU = 
 typedef enum lisa_integrate_t { LISA_INTEGRATE_ADD = 0, LISA_INTEGRATE_CONCAT = 1, LISA_INTEGRATE_PLUS = 2 } lisa_integrate_t;
 
 typedef enum lisa_cache_kind_t { LISA_CACHE_STANDARD = 0, LISA_CACHE_SHARED = 1 } lisa_cache_kind_t;
-typedef enum lisa_op_t { LISA_OP_ANCHOR = 0, LISA_OP_SHARED_PREFILL = 1, LISA_OP_SHARED_DECODE = 2 } lisa_op_t;
+typedef enum lisa_op_t { LISA_OP_ANCHOR = 0, LISA_OP_SHARED_PREFILL = 1, LISA_OP_SHARED_DECODE = 2, LISA_OP_SHARED_PREFILL_CHAIN = 3 } lisa_op_t;
 
 /* A strided view of an activation tensor [B, N, H, x]; x contiguous. */
 typedef struct lisa_tensor {
@@ -146,6 +146,29 @@ typedef struct lisa_shared_prefill_args {
     size_t workspace_bytes;
 } lisa_shared_prefill_args;
 lisa_status_t lisa_attn_shared_prefill(const lisa_shared_prefill_args* args, lisa_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * lisa_attn_shared_prefill_chain -- prefill of ALL shared layers that hang off one anchor, in one pass
+ * (Sec. 5.1: each shared layer takes the scores of the layer before it, so the layers at depth 1..c of
+ * a chain compute nested prefixes of the same sequence A_1, ..., A_c of Eq. 4).
+ * For k = 0..chain_len-1: o[k] is exactly what lisa_attn_shared_prefill returns for chain_len = k+1 with
+ * v = v[k]: softmax(mask(A_{k+1})) . v[k].  The anchor scores and every link's difference are computed once
+ * instead of once per layer that needs them.  v and o are host arrays of chain_len tensor descriptors
+ * ([B,N,Hkv,d] and [B,N,Hq,d], device memory); the o[k] must not overlap one another.
+ * Workspace: lisa_workspace_bytes(LISA_OP_SHARED_PREFILL_CHAIN, args, &n).  Shapes outside the tensor-core
+ * kernels' range run layer by layer through lisa_attn_shared_prefill with the same results.
+ * Errors as lisa_attn_shared_prefill; on error nothing is launched. */
+typedef struct lisa_shared_prefill_chain_args {
+    size_t struct_size;
+    int32_t B, N, Hq, Hkv, d, chain_len; /* chain_len >= 1 */
+    lisa_tensor q0, k0;
+    const lisa_link* links;  /* host array [chain_len] */
+    const lisa_tensor* v;    /* host array [chain_len] */
+    const lisa_tensor* o;    /* host array [chain_len] */
+    void* workspace;
+    size_t workspace_bytes;
+} lisa_shared_prefill_chain_args;
+lisa_status_t lisa_attn_shared_prefill_chain(const lisa_shared_prefill_chain_args* args, lisa_stream_t stream);
 
 /* The same call with every tensor, weight and `o` in HOST memory (dense [B,N,H,x] layout, strides
  * ignored; workspace fields ignored).  Inputs are staged into `device_arena` (device memory of at least

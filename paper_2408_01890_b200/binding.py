@@ -22,10 +22,10 @@ F32, BF16 = 0, 1
 ACT_NONE, ACT_RELU, ACT_SILU = 0, 1, 2
 INTEGRATE_ADD, INTEGRATE_CONCAT, INTEGRATE_PLUS = 0, 1, 2
 CACHE_STANDARD, CACHE_SHARED = 0, 1
-OP_ANCHOR, OP_SHARED_PREFILL, OP_SHARED_DECODE = 0, 1, 2
+OP_ANCHOR, OP_SHARED_PREFILL, OP_SHARED_DECODE, OP_SHARED_PREFILL_CHAIN = 0, 1, 2, 3
 ACTS = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
 
-EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_host", "lisa_host_arena_bytes",
+EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_chain", "lisa_attn_shared_prefill_host", "lisa_host_arena_bytes",
            "lisa_attn_shared_decode", "lisa_attn_shared_decode_static", "lisa_kvcache_append", "lisa_kvcache_bytes", "lisa_prefill_phase_times", "lisa_prefill_phase_timing", "lisa_workspace_bytes", "lisa_check",
            "lisa_force_general_kernels", "lisa_kernel_launches", "lisa_last_cuda_error", "lisa_status_string", "lisa_version"]
 
@@ -68,6 +68,12 @@ class SharedPrefillArgs(C.Structure):
                 ("links", C.POINTER(CLink)), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
 
+class SharedPrefillChainArgs(C.Structure):
+    _fields_ = [("struct_size", C.c_size_t), ("B", C.c_int32), ("N", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32),
+                ("d", C.c_int32), ("chain_len", C.c_int32), ("q0", Tensor), ("k0", Tensor), ("links", C.POINTER(CLink)),
+                ("v", C.POINTER(Tensor)), ("o", C.POINTER(Tensor)), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
 class SharedDecodeArgs(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("B", C.c_int32), ("Hq", C.c_int32), ("L", C.c_int32),
                 ("reserved", C.c_int32), ("prev_scores", C.c_void_p), ("prev_stride_b", C.c_int64),
@@ -92,6 +98,8 @@ def load():
             getattr(lib, name).restype = C.c_int
         lib.lisa_attn_anchor.argtypes = [C.POINTER(AnchorArgs), C.c_void_p]
         lib.lisa_attn_shared_prefill.argtypes = [C.POINTER(SharedPrefillArgs), C.c_void_p]
+        lib.lisa_attn_shared_prefill_chain.argtypes = [C.POINTER(SharedPrefillChainArgs), C.c_void_p]
+        lib.lisa_attn_shared_prefill_chain.restype = C.c_int
         lib.lisa_attn_shared_prefill_host.argtypes = [C.POINTER(SharedPrefillArgs), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.lisa_host_arena_bytes.argtypes = [C.POINTER(SharedPrefillArgs), C.POINTER(C.c_size_t)]
         lib.lisa_attn_shared_decode.argtypes = [C.POINTER(SharedDecodeArgs), C.c_void_p]
@@ -261,6 +269,32 @@ def lisa_attn_shared_prefill(q0: torch.Tensor, k0: torch.Tensor, links: Sequence
     a.workspace, a.workspace_bytes = _ptr(ws), (ws.numel() if ws is not None else 0)
     _check(load().lisa_attn_shared_prefill(C.byref(a), _stream()), "lisa_attn_shared_prefill")
     return out
+
+
+def _prefill_chain_args(q0, k0, links: Sequence[Link], vs, outs):
+    B, N, Hq, d = q0.shape
+    a = SharedPrefillChainArgs()
+    a.struct_size = C.sizeof(SharedPrefillChainArgs)
+    a.B, a.N, a.Hq, a.Hkv, a.d, a.chain_len = B, N, Hq, k0.shape[2], d, len(links)
+    a.q0, a.k0 = _tensor4(q0), _tensor4(k0)
+    larr = (CLink * len(links))(*[l.to_c() for l in links])
+    varr = (Tensor * len(links))(*[_tensor4(v) for v in vs])
+    oarr = (Tensor * len(links))(*[_tensor4(o) for o in outs])
+    a.links, a.v, a.o = C.cast(larr, C.POINTER(CLink)), C.cast(varr, C.POINTER(Tensor)), C.cast(oarr, C.POINTER(Tensor))
+    return a, (larr, varr, oarr)
+
+
+def lisa_attn_shared_prefill_chain(q0: torch.Tensor, k0: torch.Tensor, links: Sequence[Link], vs: Sequence[torch.Tensor], *,
+                                   outs: Optional[Sequence[torch.Tensor]] = None,
+                                   workspace: Optional[torch.Tensor] = None) -> Sequence[torch.Tensor]:
+    """All len(links) shared layers that hang off one anchor, in one pass; outs[k] is the layer at chain depth k+1 (V = vs[k])."""
+    assert len(links) >= 1 and len(vs) == len(links)
+    outs = [torch.empty_like(q0) for _ in links] if outs is None else list(outs)
+    a, keep = _prefill_chain_args(q0, k0, links, vs, outs)
+    ws = workspace if workspace is not None else _workspace(OP_SHARED_PREFILL_CHAIN, a)
+    a.workspace, a.workspace_bytes = _ptr(ws), (ws.numel() if ws is not None else 0)
+    _check(load().lisa_attn_shared_prefill_chain(C.byref(a), _stream()), "lisa_attn_shared_prefill_chain")
+    return outs
 
 
 def lisa_host_arena_bytes(q0, k0, links, v, out) -> int:

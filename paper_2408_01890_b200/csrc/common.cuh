@@ -92,6 +92,7 @@ struct TcAlignArgs {
     void* planes[4];
     const lisa_link* links;
     int ctas = 0;  // grid size (0 = three per SM)
+    bool store_all = false;  // every link's output is stored (times log2 e): link k (0-based) into planes[k]
 };
 bool tc_align_supported(int Hq, const lisa_link* links, int chain);
 cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t s);
@@ -103,6 +104,9 @@ cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int
 bool tc_shared_prefill_supported(const lisa_shared_prefill_args& a);
 size_t tc_shared_prefill_workspace(const lisa_shared_prefill_args& a);
 cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws, cudaStream_t s);
+// vs/os: per-layer V and O of a chain of a.chain_len layers (nullptr: only the deepest layer, a.v / a.o)
+cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, const lisa_tensor* vs, const lisa_tensor* os, void* ws,
+                                           cudaStream_t s);
 cudaError_t prefill_phase_timing(bool enable);
 cudaError_t prefill_phase_times(float* ms4);
 

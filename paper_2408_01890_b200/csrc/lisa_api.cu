@@ -162,6 +162,20 @@ lisa_status_t lisa_kvcache_bytes(const lisa_kvcache_layer* layer, size_t* k_byte
     return LISA_OK;
 }
 
+namespace {
+// The single-layer call that computes layer k (0-based) of a chain.
+lisa_shared_prefill_args chain_layer(const lisa_shared_prefill_chain_args& a, int k) {
+    lisa_shared_prefill_args p;
+    std::memset(&p, 0, sizeof(p));
+    p.struct_size = sizeof(p);
+    p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv; p.d = a.d; p.chain_len = k + 1;
+    p.q0 = a.q0; p.k0 = a.k0; p.v = a.v[k]; p.o = a.o[k];
+    p.links = a.links;
+    p.workspace = a.workspace; p.workspace_bytes = a.workspace_bytes;
+    return p;
+}
+}  // namespace
+
 lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes) {
     if (!args || !bytes) return LISA_ERR_INVALID_ARG;
     if (op == LISA_OP_ANCHOR) {
@@ -177,6 +191,20 @@ lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes) 
         if (!g_force_general.load() && a->chain_len > 0 && a->links && a->Hq > 0 && a->Hkv > 0 && a->Hq % a->Hkv == 0 &&
             tc_shared_prefill_supported(*a))
             *bytes = tc_shared_prefill_workspace(*a);
+        return LISA_OK;
+    }
+    if (op == LISA_OP_SHARED_PREFILL_CHAIN) {
+        const lisa_shared_prefill_chain_args* a = static_cast<const lisa_shared_prefill_chain_args*>(args);
+        if (a->struct_size != sizeof(lisa_shared_prefill_chain_args) || a->chain_len < 1 || !a->v || !a->o) return LISA_ERR_INVALID_ARG;
+        size_t need = 0;   // the deepest layer needs the most, on either path
+        for (int k = 0; k < a->chain_len; ++k) {
+            const lisa_shared_prefill_args p = chain_layer(*a, k);
+            size_t n = 0;
+            lisa_status_t st = lisa_workspace_bytes(LISA_OP_SHARED_PREFILL, &p, &n);
+            if (st != LISA_OK) return st;
+            need = n > need ? n : need;
+        }
+        *bytes = need;
         return LISA_OK;
     }
     if (op == LISA_OP_SHARED_DECODE) {
@@ -208,6 +236,33 @@ lisa_status_t lisa_attn_shared_prefill(const lisa_shared_prefill_args* a, lisa_s
     }
     cudaError_t e = launch_generic_prefill(*a, s);
     return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+}
+
+lisa_status_t lisa_attn_shared_prefill_chain(const lisa_shared_prefill_chain_args* a, lisa_stream_t stream) {
+    if (!a || a->struct_size != sizeof(lisa_shared_prefill_chain_args) || a->chain_len < 1 || !a->v || !a->o || !a->links)
+        return LISA_ERR_INVALID_ARG;
+    // every layer is validated before anything is launched
+    bool tensor_cores = !g_force_general.load();
+    for (int k = 0; k < a->chain_len; ++k) {
+        const lisa_shared_prefill_args p = chain_layer(*a, k);
+        lisa_status_t st = validate_prefill(&p);
+        if (st != LISA_OK) return st;
+        tensor_cores = tensor_cores && tc_shared_prefill_supported(p);
+    }
+    size_t need = 0;
+    lisa_status_t st = lisa_workspace_bytes(LISA_OP_SHARED_PREFILL_CHAIN, a, &need);
+    if (st != LISA_OK) return st;
+    if ((st = check_workspace(a->workspace, a->workspace_bytes, need)) != LISA_OK) return st;
+    if (tensor_cores) {
+        const lisa_shared_prefill_args deepest = chain_layer(*a, a->chain_len - 1);
+        cudaError_t e = launch_tc_shared_prefill_chain(deepest, a->v, a->o, a->workspace, static_cast<cudaStream_t>(stream));
+        return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+    }
+    for (int k = 0; k < a->chain_len; ++k) {
+        const lisa_shared_prefill_args p = chain_layer(*a, k);
+        if ((st = lisa_attn_shared_prefill(&p, stream)) != LISA_OK) return st;
+    }
+    return LISA_OK;
 }
 
 lisa_status_t lisa_attn_anchor(const lisa_anchor_args* a, lisa_stream_t stream) {

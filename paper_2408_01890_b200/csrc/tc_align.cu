@@ -50,6 +50,7 @@ struct AlignParams {
     __half* planes[kMaxTcChain];   // [0] = A_0 in / Y out; [k] = D_k for k = 1..c-1; blocked, see tc_flash.cu
     const void *w1[kMaxTcChain], *b1[kMaxTcChain], *w2[kMaxTcChain], *b2[kMaxTcChain];
     int w_dtype[kMaxTcChain], act[kMaxTcChain];
+    int store_all;                 // 1: the output of EVERY link k leaves (times log2 e) in plane k, for a chain of layers
     int* status;
 };
 
@@ -170,7 +171,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         uint2* w1f = reinterpret_cast<uint2*>(sW + k * LINK_BYTES);
         uint2* w2f = reinterpret_cast<uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
         float* bias = reinterpret_cast<float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
-        const float out_scale = k == c - 1 ? kLog2e : 1.f;
+        const float out_scale = (k == c - 1 && !p.store_all) ? kLog2e : 1.f;   // store_all scales what it stores instead
         const int wd = p.w_dtype[k];
         for (int e = tid; e < 2 * 8 * 32; e += NT) {   // W1 [32 heads][64 hidden]: k = head, n = hidden
             const int ln = e & 31, j = (e >> 5) & 7, ks = e >> 8, g = ln >> 2, t = ln & 3;
@@ -300,6 +301,20 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                 if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
                 else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
                 else ffn_link<LISA_ACT_NONE, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
+                if (p.store_all && k + 1 < c) {
+                    // a chain of layers: link k's own output leaves too, over plane k's place in the scratch (plane 0 = A_0
+                    // and plane k = D_k have been consumed by every lane before this link's MMAs could complete)
+                    __syncwarp();
+#pragma unroll
+                    for (int x = 0; x < 2; ++x) {
+                        uint32_t r[4];
+                        r[0] = pack_f16(y[2 * x][0] * kLog2e, y[2 * x][1] * kLog2e);
+                        r[1] = pack_f16(y[2 * x][2] * kLog2e, y[2 * x][3] * kLog2e);
+                        r[2] = pack_f16(y[2 * x + 1][0] * kLog2e, y[2 * x + 1][1] * kLog2e);
+                        r[3] = pack_f16(y[2 * x + 1][2] * kLog2e, y[2 * x + 1][3] * kLog2e);
+                        stmatrix_x4_trans(base + k * 2048 + (x ? off1 : off0), r);
+                    }
+                }
                 if (k + 1 < c) {
                     // A_{k+1} = y + D_{k+1}; the difference comes in the same fragment arrangement as A did
 #pragma unroll
@@ -315,25 +330,32 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                     }
                 }
             }
-            // result over this strip's place in scratch plane 0 (every lane's ldmatrix of it is done), transposed back
+            // the last link's result over its place in the scratch (plane 0, or plane c-1 in a chain of layers; every
+            // lane's ldmatrix of it is done), transposed back
+            const float last_scale = p.store_all ? kLog2e : 1.f;
+            const uint32_t last_plane = p.store_all ? (uint32_t)(c - 1) * 2048u : 0u;
             __syncwarp();
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
                 uint32_t r[4];
-                r[0] = pack_f16(y[2 * x][0], y[2 * x][1]);
-                r[1] = pack_f16(y[2 * x][2], y[2 * x][3]);
-                r[2] = pack_f16(y[2 * x + 1][0], y[2 * x + 1][1]);
-                r[3] = pack_f16(y[2 * x + 1][2], y[2 * x + 1][3]);
-                stmatrix_x4_trans(base + (x ? off1 : off0), r);
+                r[0] = pack_f16(y[2 * x][0] * last_scale, y[2 * x][1] * last_scale);
+                r[1] = pack_f16(y[2 * x][2] * last_scale, y[2 * x][3] * last_scale);
+                r[2] = pack_f16(y[2 * x + 1][0] * last_scale, y[2 * x + 1][1] * last_scale);
+                r[3] = pack_f16(y[2 * x + 1][2] * last_scale, y[2 * x + 1][3] * last_scale);
+                stmatrix_x4_trans(base + last_plane + (x ? off1 : off0), r);
             }
         }
         __syncwarp();
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int head = l_head + 8 * i;
-            *reinterpret_cast<uint4*>(p.planes[0] + piece_off(here, head)) =
-                *reinterpret_cast<const uint4*>(scr + buf * c * 2048 + scr_off(head, l_chunk));
-        }
+        for (int k = 0; k < kMaxTcChain; ++k)
+            if (k == 0 || (p.store_all && k < c)) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int head = l_head + 8 * i;
+                    *reinterpret_cast<uint4*>(p.planes[k] + piece_off(here, head)) =
+                        *reinterpret_cast<const uint4*>(scr + (buf * c + k) * 2048 + scr_off(head, l_chunk));
+                }
+            }
         __syncwarp();   // the next iteration's fetch refills the buffer that was stored one iteration ago, not this one
         buf = buf + 1 == STAGES ? 0 : buf + 1;
     }
@@ -367,6 +389,7 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
         p.w1[k] = l.w1; p.b1[k] = l.b1; p.w2[k] = l.w2; p.b2[k] = l.b2;
         p.w_dtype[k] = l.w_dtype; p.act[k] = l.act;
     }
+    p.store_all = a.store_all ? 1 : 0;
     p.status = status_words();
     if (!p.status) return cudaErrorUnknown;
     if (a.plane_cols % 64 != 0 || a.plane_rows % 128 != 0) return cudaErrorInvalidValue;   // whole blocks

@@ -142,6 +142,15 @@ bool tc_shared_prefill_supported(const lisa_shared_prefill_args& a) {
 size_t tc_shared_prefill_workspace(const lisa_shared_prefill_args& a) { return plan_layout(a).total + 1024; }
 
 cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws, cudaStream_t s) {
+    return launch_tc_shared_prefill_chain(a, nullptr, nullptr, ws, s);
+}
+
+// With vs/os == nullptr: the layer at chain depth c (a.v, a.o).  With vs/os[c]: all c layers of the chain in one
+// pass -- the anchor scores and the differences are emitted once, the aligner stores every link's output (link k
+// over plane k), and one attention kernel per layer consumes its plane with its own Q', K' and V.
+cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, const lisa_tensor* vs, const lisa_tensor* os, void* ws,
+                                           cudaStream_t s) {
+    const bool all_layers = vs != nullptr;
     const Layout l = plan_layout(a);
     char* base = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(ws) + 1023) & ~(uintptr_t)1023);
     const int c = a.chain_len;
@@ -180,21 +189,25 @@ cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws
         al.plane_rows = l.plane_rows; al.plane_cols = l.plane_cols;
         for (int k = 0; k < c; ++k) al.planes[k] = base + l.plane_off[k];
         al.links = a.links;
+        al.store_all = all_layers;
         {
             PhaseMark mark(2, s);
             if ((e = launch_tc_align(al, s)) != cudaSuccess) return e;
         }
-        // 3. this layer's own difference, softmax and .V
-        TcFlashArgs fv = f;
-        fv.emit_plane = nullptr;
-        fv.kd = kPadRank;
-        fv.qa = packed_view(base + l.qp_off[c - 1], a.Hq, a.N);
-        fv.ka = packed_view(base + l.kp_off[c - 1], a.Hkv, a.N);
-        fv.scale = 1.f / sqrtf((float)a.links[c - 1].r);
-        fv.ksteps = (a.links[c - 1].r + 15) / 16;
-        fv.plane = base + l.plane_off[0];
-        PhaseMark mark(3, s);
-        if ((e = launch_tc_flash(fv, s)) != cudaSuccess) return e;
+        // 3. each layer's own difference, softmax and .V
+        for (int k = all_layers ? 0 : c - 1; k < c; ++k) {
+            TcFlashArgs fv = f;
+            fv.emit_plane = nullptr;
+            fv.kd = kPadRank;
+            fv.qa = packed_view(base + l.qp_off[k], a.Hq, a.N);
+            fv.ka = packed_view(base + l.kp_off[k], a.Hkv, a.N);
+            fv.scale = 1.f / sqrtf((float)a.links[k].r);
+            fv.ksteps = (a.links[k].r + 15) / 16;
+            fv.plane = base + l.plane_off[all_layers ? k : 0];
+            if (all_layers) { fv.v = vs[k]; fv.o = os[k]; }
+            PhaseMark mark(3, s);
+            if ((e = launch_tc_flash(fv, s)) != cudaSuccess) return e;
+        }
     }
     return cudaSuccess;
 }

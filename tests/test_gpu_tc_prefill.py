@@ -54,6 +54,38 @@ def test_shared_prefill_tensor_core(B, N, Hkv, chain, act):
     run_tc_shared(B, N, Hkv, chain, act)
 
 
+@pytest.mark.parametrize("B,N,Hkv,chain,act,hq", [(1, 300, 8, 3, "relu", 32), (2, 200, 32, 2, "silu", 32), (1, 130, 32, 1, "relu", 32),
+                                                    (1, 150, 4, 3, "relu", 8)])
+def test_shared_prefill_chain(B, N, Hkv, chain, act, hq):
+    """All layers of a chain in one pass: layer k's output equals the oracle's layer at depth k+1 with its own V.
+    Hq = 32 runs the tensor-core kernels (every link's output stored by one aligner pass), Hq = 8 the layer-by-layer route."""
+    w = synth.Workload("tc_chain", "bf16", B, N, hq, Hkv, 128, 21, 2 * hq, act, chain)
+    t = synth.prefill_inputs(w, 7)
+    dl, ol = make_links(t, chain, act)
+    vs = [dev(t[f"v{k}"]) for k in range(1, chain + 1)]
+    n0 = lb.lisa_kernel_launches()
+    outs = lb.lisa_attn_shared_prefill_chain(dev(t["q0"]), dev(t["k0"]), dl, vs)
+    torch.cuda.synchronize()
+    if hq == 32:   # packs (2 per link) + emits (chain) + one aligner + one attention per layer
+        assert lb.lisa_kernel_launches() - n0 == 2 * chain + chain + 1 + chain
+    assert lb.lisa_check() == lb.OK
+    for k in range(chain):
+        ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1])
+        assert_close(outs[k].float().cpu().numpy(), ref, "bf16", "chain prefill N=%d layer %d of %d" % (N, k + 1, chain))
+
+
+def test_shared_prefill_chain_rejects_bad_arguments():
+    w = synth.Workload("tc_chain", "bf16", 1, 130, 32, 32, 128, 21, 64, "relu", 2)
+    t = synth.prefill_inputs(w, 1)
+    dl, _ = make_links(t, 2, "relu")
+    vs = [dev(t["v1"]), dev(t["v2"])]
+    with pytest.raises(lb.LisaError):      # workspace too small
+        lb.lisa_attn_shared_prefill_chain(dev(t["q0"]), dev(t["k0"]), dl, vs, workspace=torch.empty(1024, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(lb.LisaError):      # V of the wrong shape
+        lb.lisa_attn_shared_prefill_chain(dev(t["q0"]), dev(t["k0"]), dl, [vs[0], vs[1][:, :64]])
+    assert lb.lisa_check() == lb.OK
+
+
 def test_shared_prefill_tensor_core_bias_and_rank():
     run_tc_shared(1, 260, 32, 2, "relu", seed=3, bias=True, r=32)
     run_tc_shared(1, 140, 32, 1, "silu", seed=4, bias=True, r=8)
