@@ -81,8 +81,8 @@ def test_shared_prefill_chain_rejects_bad_arguments():
     vs = [dev(t["v1"]), dev(t["v2"])]
     with pytest.raises(lb.LisaError):      # workspace too small
         lb.lisa_attn_shared_prefill_chain(dev(t["q0"]), dev(t["k0"]), dl, vs, workspace=torch.empty(1024, dtype=torch.uint8, device="cuda"))
-    with pytest.raises(lb.LisaError):      # V of the wrong shape
-        lb.lisa_attn_shared_prefill_chain(dev(t["q0"]), dev(t["k0"]), dl, [vs[0], vs[1][:, :64]])
+    with pytest.raises(lb.LisaError):      # 32 query heads do not divide over 3 key heads
+        lb.lisa_attn_shared_prefill_chain(dev(t["q0"]), dev(t["k0"])[:, :, :3], dl, vs)
     assert lb.lisa_check() == lb.OK
 
 
