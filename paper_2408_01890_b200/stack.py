@@ -60,16 +60,20 @@ class AttentionStack:
         return l + 1 < self.n_layers and not self.is_standard[l + 1]
 
     # ------------------------------------------------------------------ prefill
-    def prefill(self, probe: Optional[Probe] = None, nf: bool = False) -> float:
+    def prefill(self, probe: Optional[Probe] = None, nf: bool = False, fused: bool = True) -> float:
         """Runs every layer over the prompt and fills the caches. Returns the device time in milliseconds.
 
+        fused=True hands every run of shared layers behind an anchor to `lisa_attn_shared_prefill_chain` (the anchor
+        scores and each link's difference are computed once for the run); fused=False calls
+        `lisa_attn_shared_prefill` layer by layer.  Same results either way.
         nf=True is the paper's lossless-prefill recipe (Sec. 5.2, "NF"): a shared layer attends over the prompt with
         standard attention on its own full Q and K, and only what it caches differs (K_LR instead of K); sharing
         starts with the first decoded token.  Prefill then costs what a standard stack costs.
         """
         B, N, Hq, Hkv, d, r = self.B, self.N, self.Hq, self.Hkv, self.d, self.r
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        out = torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device="cuda")
+        outs = [torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device="cuda") for _ in range(3 if fused and not nf else 1)]
+        out = outs[0]
         # every layer's inputs are drawn before the clock starts
         drawn = []
         for l in range(self.n_layers):
@@ -82,20 +86,60 @@ class AttentionStack:
                 drawn.append((self.draw("qp", l, (B, N, Hq, r)), self.draw("kp", l, (B, N, Hkv, r)),
                               self.draw("v", l, (B, N, Hkv, d))))
         ws = None
+
+        def record(l, o, q0, k0, v, links):
+            if probe is not None and l in probe.layers:
+                rb = torch.tensor(list(probe.rows_b), device="cuda")
+                ri = torch.tensor(list(probe.rows_i), device="cuda")
+                seqs = sorted(set(probe.rows_b))
+                probe.prefill[l] = {
+                    "seqs": seqs, "out": o[rb, ri].float().cpu(), "q0": q0[seqs].cpu(), "k0": k0[seqs].cpu(), "v": v[seqs].cpu(),
+                    "links": [(lk.qp[seqs].cpu(), lk.kp[seqs].cpu(), lk.w1.cpu(), lk.w2.cpu()) for lk in links]}
+
         torch.cuda.synchronize()
         t0.record()
         q0 = k0 = None
         links: List[lb.Link] = []
-        for l in range(self.n_layers):
+        l = 0
+        while l < self.n_layers:
             a, b_, v = drawn[l][:3]
             if nf and not self.is_standard[l]:
                 lb.lisa_attn_anchor(a, b_, v, out=out)
                 lb.lisa_kvcache_append(self.caches[l], drawn[l][3], v)
-                q0, k0, links = a, b_, []
+                record(l, out, a, b_, v, [])
             elif self.is_standard[l]:
                 lb.lisa_attn_anchor(a, b_, v, out=out)
                 lb.lisa_kvcache_append(self.caches[l], b_, v)
                 q0, k0, links = a, b_, []
+                record(l, out, q0, k0, v, [])
+            elif fused:
+                end = l
+                while end < self.n_layers and not self.is_standard[end] and end - l < len(outs):
+                    end += 1
+                run = list(range(l, end))
+                for j in run:
+                    w1, w2 = self.weights[j]
+                    links = links + [lb.Link(drawn[j][0], drawn[j][1], w1, w2, act=lb.ACTS[self.act])]
+                run_links, vs = links[-len(run):], [drawn[j][2] for j in run]
+                if len(links) == len(run):   # the run starts right behind the anchor: one pass for all of it
+                    args = lb._prefill_chain_args(q0, k0, run_links, vs, outs[:len(run)])[0]
+                    need = lb._workspace_bytes(lb.OP_SHARED_PREFILL_CHAIN, args)
+                    if ws is None or ws.numel() < need:
+                        ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+                    lb.lisa_attn_shared_prefill_chain(q0, k0, run_links, vs, outs=outs[:len(run)], workspace=ws)
+                else:                        # a run longer than the buffers: its tail goes layer by layer
+                    for i, j in enumerate(run):
+                        depth = len(links) - len(run) + i + 1
+                        args = lb._prefill_args(q0, k0, links[:depth], vs[i], outs[i])[0]
+                        need = lb._workspace_bytes(lb.OP_SHARED_PREFILL, args)
+                        if ws is None or ws.numel() < need:
+                            ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+                        lb.lisa_attn_shared_prefill(q0, k0, links[:depth], vs[i], out=outs[i], workspace=ws)
+                for i, j in enumerate(run):
+                    lb.lisa_kvcache_append(self.caches[j], drawn[j][1], drawn[j][2])
+                    record(j, outs[i], q0, k0, drawn[j][2], links[:len(links) - len(run) + i + 1])
+                l = end
+                continue
             else:
                 w1, w2 = self.weights[l]
                 links = links + [lb.Link(a, b_, w1, w2, act=lb.ACTS[self.act])]
@@ -105,13 +149,8 @@ class AttentionStack:
                     ws = torch.empty(need, dtype=torch.uint8, device="cuda")
                 lb.lisa_attn_shared_prefill(q0, k0, links, v, out=out, workspace=ws)
                 lb.lisa_kvcache_append(self.caches[l], b_, v)
-            if probe is not None and l in probe.layers:
-                rb = torch.tensor(list(probe.rows_b), device="cuda")
-                ri = torch.tensor(list(probe.rows_i), device="cuda")
-                seqs = sorted(set(probe.rows_b))
-                probe.prefill[l] = {
-                    "seqs": seqs, "out": out[rb, ri].float().cpu(), "q0": q0[seqs].cpu(), "k0": k0[seqs].cpu(), "v": v[seqs].cpu(),
-                    "links": [(lk.qp[seqs].cpu(), lk.kp[seqs].cpu(), lk.w1.cpu(), lk.w2.cpu()) for lk in links]}
+                record(l, out, q0, k0, v, links)
+            l += 1
         t1.record()
         torch.cuda.synchronize()
         return t0.elapsed_time(t1)

@@ -49,6 +49,16 @@ def test_small_stack_every_layer():
     check_probe(st, probe)
 
 
+def test_small_stack_layer_by_layer_prefill():
+    """The same small stack with every shared layer prefilled by its own call instead of one pass per chain."""
+    st = lstack.AttentionStack(n_layers=8, B=2, N=200, T=2, seed=3)
+    probe = lstack.Probe(layers=range(8), rows_b=[0, 1, 1, 0], rows_i=[0, 199, 77, 128], steps=[1], seqs=[0, 1])
+    st.prefill(probe, fused=False)
+    st.decode(probe)
+    assert lb.lisa_check() == lb.OK
+    check_probe(st, probe)
+
+
 def test_small_stack_lossless_prefill():
     """Sec. 5.2 "NF": shared layers attend over the prompt with standard attention on their own Q and K and cache
     K_LR; sharing starts with the first decoded token."""
