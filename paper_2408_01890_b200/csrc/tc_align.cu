@@ -35,7 +35,7 @@ using namespace tc;
 
 constexpr int HQ = 32, MH = 64, UNIT = 128;
 constexpr int kWorkers = 384, kStages = 2;                        // weights read from shared memory: one CTA per SM
-constexpr int kRegwThreads = 128, kRegwCtas = 3, kRegwStages = 4; // weights held in registers (single link)
+constexpr int kRegwThreads = 128, kRegwCtas = 3, kRegwStages = 3, kRegwPiece = 64; // weights held in registers (single link)
 constexpr int W1F_BYTES = 2 * 8 * 32 * 8;     // B fragments of W1: [k-step][n-tile][lane] x (b0, b1)
 constexpr int W2F_BYTES = 4 * 4 * 32 * 8;     // B fragments of W2
 constexpr float kLog2e = 1.4426950408889634f; // the last link's output leaves multiplied by log2(e): the attention
@@ -156,7 +156,7 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
 //   scratch -> fragments ldmatrix.trans per 16-position strip
 //   chain in registers   (ffn_link)
 //   result               stmatrix.trans back into the scratch, then 16 bytes per lane to the plane
-template <bool REGW, int NT, int MIN_CTAS, int STAGES>
+template <bool REGW, int NT, int MIN_CTAS, int STAGES, int PP>
 __global__ void __launch_bounds__(NT, MIN_CTAS)
 tc_align_kernel(const __grid_constant__ AlignParams p) {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -195,18 +195,21 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
     }
     __syncthreads();
 
-    // ---- this warp's contiguous range of pieces; a piece is 32 positions (4 per 128-position unit) ----
-    const long long n_pieces = (long long)p.units_per_batch * p.B * 4;
+    // ---- this warp's contiguous range of pieces; a piece is PP (32 or 64) positions of a 128-position unit ----
+    constexpr int PPU = UNIT / PP;                 // pieces per unit
+    constexpr int PLANE_SCR = HQ * PP * 2;         // scratch bytes of one plane of a piece: [32 heads][PP positions]
+    constexpr int CPR = PP / 8;                    // 16-byte chunks per head row
+    const long long n_pieces = (long long)p.units_per_batch * p.B * PPU;
     const long long n_warps = (long long)gridDim.x * (NT / 32);
     const long long per_warp = (n_pieces + n_warps - 1) / n_warps;
     const long long s_begin = min(n_pieces, ((long long)blockIdx.x * (NT / 32) + warp) * per_warp);
     const long long s_end = min(n_pieces, s_begin + per_warp);
     if (s_begin >= s_end) return;
-    struct Cursor { int b, t, row, jb, sub; };   // batch, query tile, row in the tile, key block, 32-position piece in the block
+    struct Cursor { int b, t, row, jb, sub; };   // batch, query tile, row in the tile, key block, piece in the block
     Cursor cu;
     {
-        const long long u = s_begin >> 2;
-        cu.sub = (int)(s_begin & 3);
+        const long long u = s_begin / PPU;
+        cu.sub = (int)(s_begin % PPU);
         cu.b = (int)(u / p.units_per_batch);
         int rem = (int)(u - (long long)cu.b * p.units_per_batch);
         cu.t = p.qt_begin;
@@ -219,7 +222,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         cu.jb = rem - cu.row * (cu.t + 1);
     }
     auto advance = [&](Cursor& x) {
-        if (++x.sub < 4) return;
+        if (++x.sub < PPU) return;
         x.sub = 0;
         if (++x.jb <= x.t) return;
         x.jb = 0;
@@ -229,26 +232,32 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         x.t = p.qt_begin;
         ++x.b;
     };
-    // Global <-> scratch: four lanes cover the 64 bytes [head][32 positions] of one head, so one warp-wide access
-    // touches 8 heads (8 lines); four accesses move a piece.  Scratch rows are 64 bytes (one head); the 16-byte chunk
-    // index is XOR-ed with (head / 2) % 4 so that the 8 rows of an 8x8 matrix fall into distinct banks.
-    const int l_head = lane >> 2, l_chunk = lane & 3;
+    // Global <-> scratch: CPR lanes cover the PP * 2 bytes [head][PP positions] of one head, so one warp-wide access
+    // touches 32 / CPR heads; 128 / CPR... PP * 4 / 32 accesses move a piece of one plane (with PP = 64 a piece is one
+    // contiguous 4 KB run of the blocked plane).  Scratch rows are one head; the 16-byte chunk index is XOR-ed with
+    // the head index (over as many bits as there are chunks) so that the 8 rows of an 8x8 matrix fall into distinct banks.
+    constexpr int HPA = 32 / CPR;                  // heads per warp-wide access
+    constexpr int NACC = HQ / HPA;                 // accesses per plane and piece
+    const int l_head = lane / CPR, l_chunk = lane % CPR;
     auto piece_off = [&](const Cursor& x, int head) {   // element offset of [head][this piece] + this lane's chunk
         // blocked plane: [row block of 128][column block of 64][row in block][b*HQ + head][64 columns]
         const int r = x.t * UNIT + x.row - p.row0;
-        const int64_t blk = (int64_t)(r >> 7) * (p.plane_cols >> 6) + (x.jb * 2 + (x.sub >> 1));
-        return ((blk * 128 + (r & 127)) * (p.B * HQ) + (x.b * HQ + head)) * 64 + (x.sub & 1) * 32 + l_chunk * 8;
+        const int col = x.sub * PP;                // within the 128-column key block
+        const int64_t blk = (int64_t)(r >> 7) * (p.plane_cols >> 6) + (x.jb * 2 + (col >> 6));
+        return ((blk * 128 + (r & 127)) * (p.B * HQ) + (x.b * HQ + head)) * 64 + (col & 63) + l_chunk * 8;
     };
-    auto scr_off = [&](int head, int chunk) { return (uint32_t)(head * 64 + ((chunk ^ ((head >> 1) & 3)) << 4)); };
-    uint8_t* scr = sScr + warp * (STAGES * c * 2048);     // [STAGES buffers][c planes][32 heads][64 B]
+    auto scr_off = [&](int head, int chunk) {
+        return (uint32_t)(head * (PP * 2) + ((chunk ^ (PP == 64 ? (head & 7) : ((head >> 1) & 3))) << 4));
+    };
+    uint8_t* scr = sScr + warp * (STAGES * c * PLANE_SCR);   // [STAGES buffers][c planes][32 heads][PP * 2 B]
     auto fetch = [&](const Cursor& x, int buf) {          // asynchronous global -> scratch copy of a piece, all planes
 #pragma unroll
         for (int k = 0; k < kMaxTcChain; ++k)
             if (k < c) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int head = l_head + 8 * i;
-                    const uint32_t dst = smem_u32(scr + (buf * c + k) * 2048) + scr_off(head, l_chunk);
+                for (int i = 0; i < NACC; ++i) {
+                    const int head = l_head + HPA * i;
+                    const uint32_t dst = smem_u32(scr + (buf * c + k) * PLANE_SCR) + scr_off(head, l_chunk);
                     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(p.planes[k] + piece_off(x, head)) : "memory");
                 }
             }
@@ -284,9 +293,9 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         fbuf = fbuf + 1 == STAGES ? 0 : fbuf + 1;
         asm volatile("cp.async.wait_group %0;" ::"n"(STAGES - 1) : "memory");
         __syncwarp();
-        const uint32_t base = smem_u32(scr + buf * c * 2048);
+        const uint32_t base = smem_u32(scr + buf * c * PLANE_SCR);
 #pragma unroll 1
-        for (int s2 = 0; s2 < 2; ++s2) {
+        for (int s2 = 0; s2 < PP / 16; ++s2) {
             const uint32_t off0 = frag_off(s2, 0), off1 = frag_off(s2, 1);
             uint32_t afr[2][4];
             ldmatrix_x4_trans(afr[0], base + off0);
@@ -312,7 +321,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                         r[1] = pack_f16(y[2 * x][2] * kLog2e, y[2 * x][3] * kLog2e);
                         r[2] = pack_f16(y[2 * x + 1][0] * kLog2e, y[2 * x + 1][1] * kLog2e);
                         r[3] = pack_f16(y[2 * x + 1][2] * kLog2e, y[2 * x + 1][3] * kLog2e);
-                        stmatrix_x4_trans(base + k * 2048 + (x ? off1 : off0), r);
+                        stmatrix_x4_trans(base + k * PLANE_SCR + (x ? off1 : off0), r);
                     }
                 }
                 if (k + 1 < c) {
@@ -320,7 +329,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
 #pragma unroll
                     for (int x = 0; x < 2; ++x) {
                         uint32_t dfr[4];
-                        ldmatrix_x4_trans(dfr, base + (k + 1) * 2048 + (x ? off1 : off0));
+                        ldmatrix_x4_trans(dfr, base + (k + 1) * PLANE_SCR + (x ? off1 : off0));
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             const float2 dv = unpack_f16(dfr[q]);
@@ -333,7 +342,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             // the last link's result over its place in the scratch (plane 0, or plane c-1 in a chain of layers; every
             // lane's ldmatrix of it is done), transposed back
             const float last_scale = p.store_all ? kLog2e : 1.f;
-            const uint32_t last_plane = p.store_all ? (uint32_t)(c - 1) * 2048u : 0u;
+            const uint32_t last_plane = p.store_all ? (uint32_t)(c - 1) * PLANE_SCR : 0u;
             __syncwarp();
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
@@ -350,10 +359,10 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         for (int k = 0; k < kMaxTcChain; ++k)
             if (k == 0 || (p.store_all && k < c)) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int head = l_head + 8 * i;
+                for (int i = 0; i < NACC; ++i) {
+                    const int head = l_head + HPA * i;
                     *reinterpret_cast<uint4*>(p.planes[k] + piece_off(here, head)) =
-                        *reinterpret_cast<const uint4*>(scr + (buf * c + k) * 2048 + scr_off(head, l_chunk));
+                        *reinterpret_cast<const uint4*>(scr + (buf * c + k) * PLANE_SCR + scr_off(head, l_chunk));
                 }
             }
         __syncwarp();   // the next iteration's fetch refills the buffer that was stored one iteration ago, not this one
@@ -361,8 +370,8 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
     }
 }
 
-size_t align_smem_bytes(int c, int threads, int stages) {
-    return (size_t)c * (W1F_BYTES + W2F_BYTES + (MH + HQ) * 4) + (size_t)(threads / 32) * stages * c * 2048 + 16;
+size_t align_smem_bytes(int c, int threads, int stages, int piece) {
+    return (size_t)c * (W1F_BYTES + W2F_BYTES + (MH + HQ) * 4) + (size_t)(threads / 32) * stages * c * (HQ * piece * 2) + 16;
 }
 
 }  // namespace
@@ -398,8 +407,8 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     const bool regw = a.chain == 1;
     const int threads = regw ? kRegwThreads : kWorkers;
     const int ctas_per_sm = regw ? kRegwCtas : 1;
-    const size_t smem = align_smem_bytes(a.chain, threads, regw ? kRegwStages : kStages);
-    auto kernel = regw ? tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages> : tc_align_kernel<false, kWorkers, 1, kStages>;
+    const size_t smem = align_smem_bytes(a.chain, threads, regw ? kRegwStages : kStages, regw ? kRegwPiece : 32);
+    auto kernel = regw ? tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece> : tc_align_kernel<false, kWorkers, 1, kStages, 32>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const int64_t total_units = (int64_t)p.units_per_batch * a.B;
