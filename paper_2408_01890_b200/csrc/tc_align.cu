@@ -195,11 +195,21 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
     }
     __syncthreads();
 
+    // Parameter fields of the main loop, read once into registers: behind the asm statements (memory clobbers) the
+    // compiler would re-read them from the parameter bank every time, the per-link ones through a run-time index.
+    const int pB = p.B, pN = p.N, p_row0 = p.row0, p_qt0 = p.qt_begin, p_qt1 = p.qt_begin + p.qt_count;
+    const int p_ncb = (int)(p.plane_cols >> 6);
+    const bool store_all = p.store_all != 0;
+    __half* const plane0 = p.planes[0];
+    __half* const plane1 = p.planes[1];
+    __half* const plane2 = p.planes[2];
+    auto plane_ptr = [&](int k) { return k == 0 ? plane0 : (k == 1 ? plane1 : plane2); };
+    const int act0 = p.act[0], act1 = p.act[1], act2 = p.act[2];
     // ---- this warp's contiguous range of pieces; a piece is PP (32 or 64) positions of a 128-position unit ----
     constexpr int PPU = UNIT / PP;                 // pieces per unit
     constexpr int PLANE_SCR = HQ * PP * 2;         // scratch bytes of one plane of a piece: [32 heads][PP positions]
     constexpr int CPR = PP / 8;                    // 16-byte chunks per head row
-    const long long n_pieces = (long long)p.units_per_batch * p.B * PPU;
+    const long long n_pieces = (long long)p.units_per_batch * pB * PPU;
     const long long n_warps = (long long)gridDim.x * (NT / 32);
     const long long per_warp = (n_pieces + n_warps - 1) / n_warps;
     const long long s_begin = min(n_pieces, ((long long)blockIdx.x * (NT / 32) + warp) * per_warp);
@@ -212,10 +222,10 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         cu.sub = (int)(s_begin % PPU);
         cu.b = (int)(u / p.units_per_batch);
         int rem = (int)(u - (long long)cu.b * p.units_per_batch);
-        cu.t = p.qt_begin;
+        cu.t = p_qt0;
         for (;; ++cu.t) {
-            const int n_t = min(UNIT, p.N - cu.t * UNIT) * (cu.t + 1);
-            if (rem < n_t || cu.t + 1 >= p.qt_begin + p.qt_count) break;
+            const int n_t = min(UNIT, pN - cu.t * UNIT) * (cu.t + 1);
+            if (rem < n_t || cu.t + 1 >= p_qt1) break;
             rem -= n_t;
         }
         cu.row = rem / (cu.t + 1);
@@ -226,10 +236,10 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         x.sub = 0;
         if (++x.jb <= x.t) return;
         x.jb = 0;
-        if (++x.row < min(UNIT, p.N - x.t * UNIT)) return;
+        if (++x.row < min(UNIT, pN - x.t * UNIT)) return;
         x.row = 0;
-        if (++x.t < p.qt_begin + p.qt_count) return;
-        x.t = p.qt_begin;
+        if (++x.t < p_qt1) return;
+        x.t = p_qt0;
         ++x.b;
     };
     // Global <-> scratch: CPR lanes cover the PP * 2 bytes [head][PP positions] of one head, so one warp-wide access
@@ -241,10 +251,10 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
     const int l_head = lane / CPR, l_chunk = lane % CPR;
     auto piece_off = [&](const Cursor& x, int head) {   // element offset of [head][this piece] + this lane's chunk
         // blocked plane: [row block of 128][column block of 64][row in block][b*HQ + head][64 columns]
-        const int r = x.t * UNIT + x.row - p.row0;
+        const int r = x.t * UNIT + x.row - p_row0;
         const int col = x.sub * PP;                // within the 128-column key block
-        const int64_t blk = (int64_t)(r >> 7) * (p.plane_cols >> 6) + (x.jb * 2 + (col >> 6));
-        return ((blk * 128 + (r & 127)) * (p.B * HQ) + (x.b * HQ + head)) * 64 + (col & 63) + l_chunk * 8;
+        const int64_t blk = (int64_t)(r >> 7) * p_ncb + (x.jb * 2 + (col >> 6));
+        return ((blk * 128 + (r & 127)) * (pB * HQ) + (x.b * HQ + head)) * 64 + (col & 63) + l_chunk * 8;
     };
     auto scr_off = [&](int head, int chunk) {
         return (uint32_t)(head * (PP * 2) + ((chunk ^ (PP == 64 ? (head & 7) : ((head >> 1) & 3))) << 4));
@@ -258,7 +268,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                 for (int i = 0; i < NACC; ++i) {
                     const int head = l_head + HPA * i;
                     const uint32_t dst = smem_u32(scr + (buf * c + k) * PLANE_SCR) + scr_off(head, l_chunk);
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(p.planes[k] + piece_off(x, head)) : "memory");
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(plane_ptr(k) + piece_off(x, head)) : "memory");
                 }
             }
         asm volatile("cp.async.commit_group;" ::: "memory");
@@ -306,11 +316,11 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                 const uint2* w2f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
                 const float* b1 = reinterpret_cast<const float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
                 const uint32_t* b1h = reinterpret_cast<const uint32_t*>(b1);
-                const int act = p.act[k];
+                const int act = k == 0 ? act0 : (k == 1 ? act1 : act2);
                 if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
                 else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
                 else ffn_link<LISA_ACT_NONE, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
-                if (p.store_all && k + 1 < c) {
+                if (store_all && k + 1 < c) {
                     // a chain of layers: link k's own output leaves too, over plane k's place in the scratch (plane 0 = A_0
                     // and plane k = D_k have been consumed by every lane before this link's MMAs could complete)
                     __syncwarp();
@@ -341,8 +351,8 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             }
             // the last link's result over its place in the scratch (plane 0, or plane c-1 in a chain of layers; every
             // lane's ldmatrix of it is done), transposed back
-            const float last_scale = p.store_all ? kLog2e : 1.f;
-            const uint32_t last_plane = p.store_all ? (uint32_t)(c - 1) * PLANE_SCR : 0u;
+            const float last_scale = store_all ? kLog2e : 1.f;
+            const uint32_t last_plane = store_all ? (uint32_t)(c - 1) * PLANE_SCR : 0u;
             __syncwarp();
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
@@ -357,11 +367,11 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         __syncwarp();
 #pragma unroll
         for (int k = 0; k < kMaxTcChain; ++k)
-            if (k == 0 || (p.store_all && k < c)) {
+            if (k == 0 || (store_all && k < c)) {
 #pragma unroll
                 for (int i = 0; i < NACC; ++i) {
                     const int head = l_head + HPA * i;
-                    *reinterpret_cast<uint4*>(p.planes[k] + piece_off(here, head)) =
+                    *reinterpret_cast<uint4*>(plane_ptr(k) + piece_off(here, head)) =
                         *reinterpret_cast<const uint4*>(scr + (buf * c + k) * PLANE_SCR + scr_off(head, l_chunk));
                 }
             }
