@@ -249,18 +249,20 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
     constexpr int HPA = 32 / CPR;                  // heads per warp-wide access
     constexpr int NACC = HQ / HPA;                 // accesses per plane and piece
     const int l_head = lane / CPR, l_chunk = lane % CPR;
-    auto piece_off = [&](const Cursor& x, int head) {   // element offset of [head][this piece] + this lane's chunk
-        // blocked plane: [row block of 128][column block of 64][row in block][b*HQ + head][64 columns]
+    // element offset of [this lane's first head][this piece] + this lane's chunk; the lane's other heads follow every
+    // HPA * 64 elements (blocked plane: [row block of 128][column block of 64][row in block][b*HQ + head][64 columns])
+    auto piece_off = [&](const Cursor& x) {
         const int r = x.t * UNIT + x.row - p_row0;
         const int col = x.sub * PP;                // within the 128-column key block
         const int64_t blk = (int64_t)(r >> 7) * p_ncb + (x.jb * 2 + (col >> 6));
-        return ((blk * 128 + (r & 127)) * (pB * HQ) + (x.b * HQ + head)) * 64 + (col & 63) + l_chunk * 8;
+        return ((blk * 128 + (r & 127)) * (pB * HQ) + (x.b * HQ + l_head)) * 64 + (col & 63) + l_chunk * 8;
     };
     auto scr_off = [&](int head, int chunk) {
         return (uint32_t)(head * (PP * 2) + ((chunk ^ (PP == 64 ? (head & 7) : ((head >> 1) & 3))) << 4));
     };
     uint8_t* scr = sScr + warp * (STAGES * c * PLANE_SCR);   // [STAGES buffers][c planes][32 heads][PP * 2 B]
     auto fetch = [&](const Cursor& x, int buf) {          // asynchronous global -> scratch copy of a piece, all planes
+        const int64_t off = piece_off(x);
 #pragma unroll
         for (int k = 0; k < kMaxTcChain; ++k)
             if (k < c) {
@@ -268,7 +270,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                 for (int i = 0; i < NACC; ++i) {
                     const int head = l_head + HPA * i;
                     const uint32_t dst = smem_u32(scr + (buf * c + k) * PLANE_SCR) + scr_off(head, l_chunk);
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(plane_ptr(k) + piece_off(x, head)) : "memory");
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(plane_ptr(k) + off + i * (HPA * 64)) : "memory");
                 }
             }
         asm volatile("cp.async.commit_group;" ::: "memory");
@@ -365,13 +367,14 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             }
         }
         __syncwarp();
+        const int64_t here_off = piece_off(here);
 #pragma unroll
         for (int k = 0; k < kMaxTcChain; ++k)
             if (k == 0 || (store_all && k < c)) {
 #pragma unroll
                 for (int i = 0; i < NACC; ++i) {
                     const int head = l_head + HPA * i;
-                    *reinterpret_cast<uint4*>(plane_ptr(k) + piece_off(here, head)) =
+                    *reinterpret_cast<uint4*>(plane_ptr(k) + here_off + i * (HPA * 64)) =
                         *reinterpret_cast<const uint4*>(scr + (buf * c + k) * PLANE_SCR + scr_off(head, l_chunk));
                 }
             }
