@@ -17,6 +17,7 @@ namespace {
 
 constexpr int kTile = 128;
 constexpr int kPadRank = 64;
+constexpr int kMaxPackLinks = 4;   // links whose Q', K' one call packs (the aligner takes chains of up to three)
 // A wave takes query tiles until its head-partitioned kernels have at least kWaveMinCtas CTAs (four per SM: with
 // fewer, the grids do not fill the GPU and launch and tail costs dominate) and then further tiles while the causal
 // part of its score planes stays within kWaveBytes.  Measured on B200: grid fill matters far more than keeping
@@ -24,7 +25,17 @@ constexpr int kPadRank = 64;
 constexpr size_t kWaveBytes = (size_t)256 << 20;
 constexpr int kWaveMinCtas = 4 * 148;
 
-__global__ void pack_lowrank_kernel(TView src, int B, int N, int H, int r, __nv_bfloat16* dst) {
+// Every Q' and K' of a call is packed by one launch: blockIdx.y selects the tensor.
+struct PackJobs {
+    TView src[2 * kMaxPackLinks];
+    __nv_bfloat16* dst[2 * kMaxPackLinks];
+    int H[2 * kMaxPackLinks], r[2 * kMaxPackLinks];
+};
+
+__global__ void pack_lowrank_kernel(const __grid_constant__ PackJobs jobs, int B, int N) {
+    const TView src = jobs.src[blockIdx.y];
+    const int H = jobs.H[blockIdx.y], r = jobs.r[blockIdx.y];
+    __nv_bfloat16* dst = jobs.dst[blockIdx.y];
     const int64_t total = (int64_t)B * H * N * (kPadRank / 8);
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
         const int chunk = (int)(e % (kPadRank / 8));
@@ -122,9 +133,11 @@ lisa_tensor packed_view(void* ptr, int H, int N) {
 }  // namespace
 
 cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int r, void* dst, cudaStream_t s) {
+    PackJobs jobs{};
+    jobs.src[0] = make_view(src); jobs.dst[0] = reinterpret_cast<__nv_bfloat16*>(dst); jobs.H[0] = H; jobs.r[0] = r;
     const int64_t total = (int64_t)B * H * N * (kPadRank / 8);
     const int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 32);
-    pack_lowrank_kernel<<<blocks, 256, 0, s>>>(make_view(src), B, N, H, r, reinterpret_cast<__nv_bfloat16*>(dst));
+    pack_lowrank_kernel<<<dim3(blocks, 1), 256, 0, s>>>(jobs, B, N);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -155,10 +168,20 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
     char* base = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(ws) + 1023) & ~(uintptr_t)1023);
     const int c = a.chain_len;
     cudaError_t e;
-    for (int k = 0; k < c; ++k) {
+    {
         PhaseMark mark(0, s);
-        if ((e = launch_pack_lowrank(a.links[k].qp, a.B, a.N, a.Hq, a.links[k].r, base + l.qp_off[k], s)) != cudaSuccess) return e;
-        if ((e = launch_pack_lowrank(a.links[k].kp, a.B, a.N, a.Hkv, a.links[k].r, base + l.kp_off[k], s)) != cudaSuccess) return e;
+        PackJobs jobs{};
+        for (int k = 0; k < c; ++k) {
+            jobs.src[2 * k] = make_view(a.links[k].qp); jobs.dst[2 * k] = reinterpret_cast<__nv_bfloat16*>(base + l.qp_off[k]);
+            jobs.H[2 * k] = a.Hq; jobs.r[2 * k] = a.links[k].r;
+            jobs.src[2 * k + 1] = make_view(a.links[k].kp); jobs.dst[2 * k + 1] = reinterpret_cast<__nv_bfloat16*>(base + l.kp_off[k]);
+            jobs.H[2 * k + 1] = a.Hkv; jobs.r[2 * k + 1] = a.links[k].r;
+        }
+        const int64_t total = (int64_t)a.B * a.Hq * a.N * (kPadRank / 8);
+        const int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 16);
+        pack_lowrank_kernel<<<dim3(blocks, 2 * c), 256, 0, s>>>(jobs, a.B, a.N);
+        count_launches(1);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     Wave waves[1024];
     const int nw = plan_waves(a.B, a.N, a.Hq, c, waves, 1024);

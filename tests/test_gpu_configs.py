@@ -21,7 +21,7 @@ def test_cfg2_llama2_7b_prefill_all_rows():
     n0 = lb.lisa_kernel_launches()
     got = lb.lisa_attn_shared_prefill(dev(t["q0"]), dev(t["k0"]), dl, dev(t["v1"]))
     torch.cuda.synchronize()
-    assert lb.lisa_kernel_launches() - n0 >= 5 and lb.lisa_check() == lb.OK   # the tensor-core path ran
+    assert lb.lisa_kernel_launches() - n0 >= 4 and lb.lisa_check() == lb.OK   # the tensor-core path ran
     rows = np.arange(w.N, dtype=np.int32)
     ref = oracle.prefill_rows(f64(t["q0"]), f64(t["k0"]), f64(t["v1"]), ol, np.zeros_like(rows), rows)
     assert_close(got[0].float().cpu().numpy(), ref, "bf16", "cfg2 shared prefill")
