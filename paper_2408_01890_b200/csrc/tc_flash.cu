@@ -12,7 +12,7 @@
 // scores leave as fp16 tiles (staged in shared memory, stored with TMA) for the aligner kernel.
 //
 // Warp roles: warps 0-3 softmax/epilogue (thread = query row = TMEM lane), warp 4 TMA producer,
-// warp 5 MMA issuer and TMEM owner.  K and V(/Y) have their own rings: a K stage is free again as soon as its
+// warp 5 issuer of the score MMAs and TMEM owner, warp 6 issuer of the P.V MMAs.  K and V(/Y) have their own rings: a K stage is free again as soon as its
 // score MMA has run, a V stage after its P.V MMA.
 // Sizing: the softmax warps are the slow stage (one exp2 per score on the 16-lane transcendental unit) and every
 // hand-off between the roles costs a few hundred cycles of latency, so TWO CTAs share an SM and fill each other's
@@ -34,7 +34,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 
 struct FlashParams {
     int B, N, Hq, Hkv;
@@ -208,53 +208,59 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             if (++ks_next == KST) { ks_next = 0; kpar_next ^= 1; }
         }
     } else if (warp == 5) {
-        // ------------------------------ MMA issuer ------------------------------
-        // Every lane of the warp runs the loop (waits, stage counters, descriptor arithmetic: all warp-uniform);
-        // only the MMA and commit instructions themselves are predicated on lane 0.
-        {
+        // ------------------------------ MMA issuer: scores ------------------------------
+        // Issuing a tcgen05.mma holds the issuing thread for about as long as the MMAs queued before it take to run, so
+        // the score MMAs and the P.V MMAs are issued by two different warps: each waits for its own operands and the
+        // two hold-ups overlap instead of adding up.  Every lane of an issuing warp runs the loop (waits, stage
+        // counters, descriptor arithmetic: all warp-uniform); only the MMA and commit instructions themselves are
+        // predicated on lane 0.
+        const uint32_t issue = lane == 0;
+        constexpr uint32_t IDESC_QK = umma_idesc_bf16(BM, BN, 0, 0);
+        const int ksteps = p.ksteps;
+        // Descriptors are built once; per MMA only the start-address field (bits 0-13 of the low word, in
+        // 16-byte units) moves, by a compile-time constant or a stage offset: no carry can leave the field.
+        auto desc_off = [](uint64_t d, uint32_t bytes) -> uint64_t {
+            return (d & 0xffffffff00000000ull) | (uint32_t)((uint32_t)d + (bytes >> 4));
+        };
+        const uint64_t dq0 = umma_desc_sw128(smem_u32(sQ), 16, 1024);
+        const uint64_t dk0 = umma_desc_sw128(smem_u32(sK), 16, 1024);
+        // scores of tile t into buffer t&1; needs K(t) loaded and (t >= 2) the buffer read by the softmax of t-2
+        int sk = 0;
+        uint32_t kpar = 0;
+        bool ok = __all_sync(0xffffffffu, mbar_wait(q_full, 0, abort_flag));
+        for (int t = 0; ok && t < nt; ++t) {
+            const int s = t & 1;
+            ok = mbar_wait(k_full + sk, kpar, abort_flag) && mbar_wait(s_free + s, ((t >> 1) & 1) ^ 1, abort_flag);
+            if (!(ok = __all_sync(0xffffffffu, ok))) break;   // one verdict for the whole warp
+            tc_fence_after();
+            const uint64_t dk = desc_off(dk0, sk * L::K_BYTES);
+            const uint32_t dst = tmem_base + s * BN;
+#pragma unroll
+            for (int ks = 0; ks < KD / 16; ++ks) {
+                if (ks < ksteps) {
+                    umma_ss_if(issue, dst, desc_off(dq0, (ks >> 2) * (BM * 128) + (ks & 3) * 32), desc_off(dk, (ks >> 2) * (BN * 128) + (ks & 3) * 32),
+                               IDESC_QK, ks > 0);
+                }
+            }
+            umma_commit_if(issue, s_full + s);
+            if (!L::P_IN_K && t + KST < nt) umma_commit_if(issue, k_empty + sk);  // nobody waits for the last ones: do not arm them
+            if (++sk == KST) { sk = 0; kpar ^= 1; }
+        }
+    } else if (warp == 6) {
+        // ------------------------------ MMA issuer: P.V ------------------------------
+        if constexpr (!EMIT) {
             const uint32_t issue = lane == 0;
-            constexpr uint32_t IDESC_QK = umma_idesc_bf16(BM, BN, 0, 0);
             constexpr uint32_t IDESC_PV = umma_idesc_bf16(BM, D, 0, 1);
-            const int ksteps = p.ksteps;
-            // Descriptors are built once; per MMA only the start-address field (bits 0-13 of the low word, in
-            // 16-byte units) moves, by a compile-time constant or a stage offset: no carry can leave the field.
             auto desc_off = [](uint64_t d, uint32_t bytes) -> uint64_t {
                 return (d & 0xffffffff00000000ull) | (uint32_t)((uint32_t)d + (bytes >> 4));
             };
-            const uint64_t dq0 = umma_desc_sw128(smem_u32(sQ), 16, 1024);
-            const uint64_t dk0 = umma_desc_sw128(smem_u32(sK), 16, 1024);
             const uint64_t dv0 = umma_desc_sw128(smem_u32(sV), BN * 128, 1024);
             const uint64_t dp0 = umma_desc_sw128(smem_u32(p_buf(0)), 16, 1024);
             constexpr uint32_t P_STRIDE = L::P_IN_Y ? L::Y_BYTES : (L::P_IN_K ? L::K_BYTES : L::P_BYTES);
-            // scores of the next tile into buffer t&1; needs K(t) loaded and (t >= 2) the buffer read by the softmax of t-2
-            int qk_t = 0, qk_sk = 0;
-            uint32_t qk_kpar = 0;
-            auto issue_qk = [&]() -> bool {
-                const int t = qk_t, s = t & 1;
-                const bool ready = mbar_wait(k_full + qk_sk, qk_kpar, abort_flag) && mbar_wait(s_free + s, ((t >> 1) & 1) ^ 1, abort_flag);
-                if (!__all_sync(0xffffffffu, ready)) return false;   // one verdict for the whole warp
-                tc_fence_after();
-                const uint64_t dk = desc_off(dk0, qk_sk * L::K_BYTES);
-                const uint32_t dst = tmem_base + s * BN;
-#pragma unroll
-                for (int ks = 0; ks < KD / 16; ++ks) {
-                    if (ks < ksteps) {
-                        umma_ss_if(issue, dst, desc_off(dq0, (ks >> 2) * (BM * 128) + (ks & 3) * 32), desc_off(dk, (ks >> 2) * (BN * 128) + (ks & 3) * 32),
-                                IDESC_QK, ks > 0);
-                    }
-                }
-                umma_commit_if(issue, s_full + s);
-                if (!L::P_IN_K && t + KST < nt) umma_commit_if(issue, k_empty + qk_sk);  // nobody waits for the last ones: do not arm them
-                ++qk_t;
-                if (++qk_sk == KST) { qk_sk = 0; qk_kpar ^= 1; }
-                return true;
-            };
-            bool ok = __all_sync(0xffffffffu, mbar_wait(q_full, 0, abort_flag)) && issue_qk();
             int pk = 0;   // P_IN_K: K stage that holds P(t)
+            bool ok = true;
             for (int t = 0; ok && t < nt; ++t) {
                 const int s = t & 1;
-                if (t + 1 < nt && !(ok = issue_qk())) break;
-                if constexpr (EMIT) continue;
                 ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag) && mbar_wait(p_full + s, (t >> 1) & 1, abort_flag);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;
                 tc_fence_after();
