@@ -12,7 +12,7 @@
 // scores leave as fp16 tiles (staged in shared memory, stored with TMA) for the aligner kernel.
 //
 // Warp roles: warps 0-3 softmax/epilogue (thread = query row = TMEM lane), warp 4 TMA producer,
-// warp 5 issuer of the score MMAs and TMEM owner, warp 6 issuer of the P.V MMAs.  K and V(/Y) have their own rings: a K stage is free again as soon as its
+// warp 5 issuer of the score MMAs and TMEM owner, warp 6 issuer of the P.V MMAs (warp 7 only completes the warpgroup).  K and V(/Y) have their own rings: a K stage is free again as soon as its
 // score MMA has run, a V stage after its P.V MMA.
 // Sizing: the softmax warps are the slow stage (one exp2 per score on the 16-lane transcendental unit) and every
 // hand-off between the roles costs a few hundred cycles of latency, so TWO CTAs share an SM and fill each other's
@@ -34,7 +34,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-constexpr int kThreads = 224;
+constexpr int kThreads = 256;   // warpgroup 0: softmax/epilogue; warpgroup 1: producer, two MMA issuers, one idle warp
 
 struct FlashParams {
     int B, N, Hq, Hkv;
@@ -153,6 +153,11 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_O = tmem_base + 128;
 
+    // The kernel is compiled for 128 registers per thread (two CTAs of 256 threads per SM).  The three single-thread
+    // roles need few, the softmax threads (64 scores, their exponentials and a row of the accumulator in flight) more:
+    // warpgroup 1 hands registers back and warpgroup 0 takes them (2 x (128 x 72 + 128 x 184) = 64 K).
+    if (warp >= 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (warp == 4) {
         // ------------------------------ TMA producer ------------------------------
         // The two single-thread roles (this one and the MMA issuer) share their scheduler with busy softmax warps and
@@ -278,7 +283,9 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 if (++pk == KST) pk = 0;
             }
         }
+    }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 184;");
         // ------------------------------ softmax / epilogue (thread = query row) ------------------------------
         const int row = tid;                       // 0..127, TMEM lane
         const int qi = q0 + row;                   // global query index
