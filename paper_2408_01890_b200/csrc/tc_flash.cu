@@ -382,9 +382,12 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                     tmem_wait_st();
                 }
             }
-            if constexpr (L::P_OWN) {   // this buffer was the A operand of the P.V two tiles back
-                if (t >= 2 && !(ok = mbar_wait(pv_done + s, ((t - 2) >> 1) & 1, abort_flag))) break;
-            }
+            // P(t) is announced on p_full[t & 1], a barrier whose phases the P.V warp tells apart by parity alone.  Since the
+            // score MMAs no longer wait for the P.V MMAs, the softmax could finish tile t while P.V(t-2) has not even been
+            // picked up: the barrier would then run two phases ahead and the waiting warp would never see its phase end.
+            // So tile t's announcement waits until P.V(t-2) has completed (which also frees a P buffer of its own,
+            // where the layout has one); two tiles back, this has nearly always happened already.
+            if (t >= 2 && !(ok = mbar_wait(pv_done + s, ((t - 2) >> 1) & 1, abort_flag))) break;
             uint8_t* pb = p_buf(t);
             float sum = 0.f;
             const float neg_m = -m_ref;
