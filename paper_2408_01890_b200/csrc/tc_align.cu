@@ -112,9 +112,11 @@ __device__ __forceinline__ uint32_t act_h2(uint32_t x) {
 // or repacked.  The second layer accumulates in fp32.  b1h holds b1 as packed fp16 pairs, b2 is fp32.
 // The fragments of W1 and W2 come either from shared memory (w1f/w2f, one 8-byte load per MMA) or, when REGW, from
 // the register copies w1r/w2r that a warp keeps for its whole life (single-link calls).
-template <int ACT, bool REGW>
+// `side` is called once, after the first layer's MMAs have been issued: unrelated instructions placed there (the copies
+// of neighbouring pieces) issue while this warp's MMAs wait for their turn on the tensor pipe.
+template <int ACT, bool REGW, typename Side>
 __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* w1f, const uint2* w2f, const uint2* w1r, const uint2* w2r,
-                                         const uint32_t* b1h, const float* b2, int lane, float (*y)[4]) {
+                                         const uint32_t* b1h, const float* b2, int lane, float (*y)[4], Side side) {
     const int t = lane & 3;
     uint32_t h[8][2];
 #pragma unroll
@@ -128,6 +130,7 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
         const uint2 w = REGW ? w1r[8 + j] : w1f[(8 + j) * 32 + lane];
         mma_f16acc(h[j], afr[1], w.x, w.y, h[j][0], h[j][1]);
     }
+    side();
     uint32_t hfr[4][4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
@@ -287,6 +290,82 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             w2r[i] = reinterpret_cast<const uint2*>(sW + W1F_BYTES)[i * 32 + lane];
         }
     }
+    if constexpr (REGW) {
+        // One link, weights in registers.  Three scratch buffers rotate: the piece being worked on, the next one (copied
+        // in meanwhile) and the previous one (copied out meanwhile).  Both copies are cut into one part per strip and
+        // issued in the middle of the strip's FFN, between its two groups of MMAs, where the warp would otherwise only
+        // wait for its turn on the tensor pipe; done as blocks of their own before and after a piece, they cost the
+        // warp about a quarter of its time with nothing of its own on the pipe.
+        static_assert(!REGW || STAGES == 3, "previous, current and next piece");
+        constexpr int NS = PP / 16, APS = NACC / NS;   // strips per piece, accesses of each copy per strip
+        static_assert(!REGW || NACC % NS == 0, "the copies divide evenly over the strips");
+        const uint2* w1f = reinterpret_cast<const uint2*>(sW);
+        const uint2* w2f = reinterpret_cast<const uint2*>(sW + W1F_BYTES);
+        const float* b1 = reinterpret_cast<const float*>(sW + W1F_BYTES + W2F_BYTES);
+        const uint32_t* b1h = reinterpret_cast<const uint32_t*>(b1);
+        const float last_scale = store_all ? kLog2e : 1.f;
+        fetch(cu, 0);
+        Cursor here = cu, nxt = cu, prev = cu;
+        advance(nxt);
+        bool has_prev = false;
+        int b_cur = 0, b_next = 1, b_prev = 2;
+        for (long long sidx = s_begin; sidx < s_end; ++sidx) {
+            const bool has_next = sidx + 1 < s_end;
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncwarp();
+            __half* const g_next = plane0 + (has_next ? piece_off(nxt) : 0);
+            __half* const g_prev = plane0 + (has_prev ? piece_off(prev) : 0);
+            const uint32_t base = smem_u32(scr + b_cur * PLANE_SCR), s_next = smem_u32(scr + b_next * PLANE_SCR);
+            const uint8_t* s_prev = scr + b_prev * PLANE_SCR;
+#pragma unroll 1
+            for (int s2 = 0; s2 < NS; ++s2) {
+                const uint32_t off0 = frag_off(s2, 0), off1 = frag_off(s2, 1);
+                uint32_t afr[2][4];
+                ldmatrix_x4_trans(afr[0], base + off0);
+                ldmatrix_x4_trans(afr[1], base + off1);
+                float y[4][4];
+                auto side = [&] {
+#pragma unroll
+                    for (int j = 0; j < APS; ++j) {
+                        const int i = s2 * APS + j, head = l_head + HPA * i;
+                        const uint32_t so = scr_off(head, l_chunk);
+                        if (has_next) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s_next + so), "l"(g_next + i * (HPA * 64)) : "memory");
+                        if (has_prev) *reinterpret_cast<uint4*>(g_prev + i * (HPA * 64)) = *reinterpret_cast<const uint4*>(s_prev + so);
+                    }
+                };
+                if (act0 == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, true>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, side);
+                else if (act0 == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, true>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, side);
+                else ffn_link<LISA_ACT_NONE, true>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, side);
+                __syncwarp();
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    uint32_t r[4];
+                    r[0] = pack_f16(y[2 * x][0] * last_scale, y[2 * x][1] * last_scale);
+                    r[1] = pack_f16(y[2 * x][2] * last_scale, y[2 * x][3] * last_scale);
+                    r[2] = pack_f16(y[2 * x + 1][0] * last_scale, y[2 * x + 1][1] * last_scale);
+                    r[3] = pack_f16(y[2 * x + 1][2] * last_scale, y[2 * x + 1][3] * last_scale);
+                    stmatrix_x4_trans(base + (x ? off1 : off0), r);
+                }
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            __syncwarp();
+            prev = here; has_prev = true;
+            here = nxt;
+            if (has_next) advance(nxt);
+            const int b_old = b_prev;
+            b_prev = b_cur; b_cur = b_next; b_next = b_old;
+        }
+        // the last piece leaves on its own
+        {
+            const int64_t off = piece_off(prev);
+#pragma unroll
+            for (int i = 0; i < NACC; ++i) {
+                const int head = l_head + HPA * i;
+                *reinterpret_cast<uint4*>(plane0 + off + i * (HPA * 64)) = *reinterpret_cast<const uint4*>(scr + b_prev * PLANE_SCR + scr_off(head, l_chunk));
+            }
+        }
+        return;
+    }
     // STAGES - 1 pieces are in flight ahead of the one being worked on; one commit group per piece (an empty group
     // past the end keeps the count uniform), so waiting for all but the newest STAGES - 1 groups completes this one.
     Cursor ahead = cu;
@@ -319,9 +398,9 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                 const float* b1 = reinterpret_cast<const float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
                 const uint32_t* b1h = reinterpret_cast<const uint32_t*>(b1);
                 const int act = k == 0 ? act0 : (k == 1 ? act1 : act2);
-                if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
-                else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
-                else ffn_link<LISA_ACT_NONE, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y);
+                if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
+                else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
+                else ffn_link<LISA_ACT_NONE, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
                 if (store_all && k + 1 < c) {
                     // a chain of layers: link k's own output leaves too, over plane k's place in the scratch (plane 0 = A_0
                     // and plane k = D_k have been consumed by every lane before this link's MMAs could complete)
