@@ -34,7 +34,7 @@ namespace {
 using namespace tc;
 
 constexpr int HQ = 32, MH = 64, UNIT = 128;
-constexpr int kWorkers = 384, kStages = 2;                        // weights read from shared memory: one CTA per SM
+constexpr int kWorkers = 512, kStages = 2;                        // weights read from shared memory: one 16-warp CTA per SM
 constexpr int kRegwThreads = 128, kRegwCtas = 3, kRegwStages = 3, kRegwPiece = 64; // weights held in registers (single link)
 constexpr int W1F_BYTES = 2 * 8 * 32 * 8;     // B fragments of W1: [k-step][n-tile][lane] x (b0, b1)
 constexpr int W2F_BYTES = 4 * 4 * 32 * 8;     // B fragments of W2
@@ -495,7 +495,7 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     if (!p.status) return cudaErrorUnknown;
     if (a.plane_cols % 64 != 0 || a.plane_rows % 128 != 0) return cudaErrorInvalidValue;   // whole blocks
     // One link: its weight fragments live in registers, 4-warp CTAs, three per SM, three pieces in flight per warp.
-    // Longer chains: weights in shared memory, one 12-warp CTA per SM, one piece in flight per warp.
+    // Longer chains: weights in shared memory, one 16-warp CTA per SM, one piece in flight per warp.
     const bool regw = a.chain == 1;
     const int threads = regw ? kRegwThreads : kWorkers;
     const int ctas_per_sm = regw ? kRegwCtas : 1;
