@@ -156,8 +156,14 @@ class AttentionStack:
         return t0.elapsed_time(t1)
 
     # ------------------------------------------------------------------ decode
-    def decode(self, probe: Optional[Probe] = None) -> float:
-        """T decode steps through all layers (one new token per sequence and step). Returns milliseconds."""
+    def decode(self, probe: Optional[Probe] = None, graph: bool = False) -> float:
+        """T decode steps through all layers (one new token per sequence and step). Returns milliseconds.
+
+        graph=True captures ONE step (every layer's cache append and attention call) in a CUDA graph and replays it T
+        times: the context length then lives on the device (`seq_lens`, advanced inside the graph) while the calls are
+        made with the run's maximum length as the bound, so the same launches serve every step and no Python runs
+        between kernels.  Same results as the step-by-step loop; `probe` needs the loop.
+        """
         B, N, T, Hq, Hkv, d, r = self.B, self.N, self.T, self.Hq, self.Hkv, self.d, self.r
         new = []
         for l in range(self.n_layers):
@@ -166,14 +172,13 @@ class AttentionStack:
             else:
                 new.append((self.draw("dqp", l, (B, 1, Hq, r)), self.draw("dkp", l, (B, 1, Hkv, r)), self.draw("dv", l, (B, 1, Hkv, d))))
         out = torch.empty((B, 1, Hq, d), dtype=torch.bfloat16, device="cuda")
+        self.last_out = out
         ws = torch.empty(lb.decode_workspace_bytes(B, Hq, d, self.L_cap), dtype=torch.uint8, device="cuda")
         before = torch.empty((B,), dtype=torch.int32, device="cuda")
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        t0.record()
-        for t in range(T):
-            L = N + t + 1
-            before.fill_(L - 1)
+
+        def step(L, lens, probe_t=None):
+            """All layers for one new token: L bounds the context length, lens (device) gives it when not None."""
             cur = 0
             for l in range(self.n_layers):
                 a, kn, vn = new[l]
@@ -181,20 +186,57 @@ class AttentionStack:
                 lb.lisa_kvcache_append(cache, kn, vn, before)
                 row_out = self.rows[cur ^ 1] if self.next_is_shared(l) else None
                 if self.is_standard[l]:
-                    lb.lisa_attn_anchor(a, cache=cache, L=L, out=out, out_scores=row_out, workspace=ws)
+                    lb.lisa_attn_anchor(a, cache=cache, L=L, seq_lens=lens, out=out, out_scores=row_out, workspace=ws)
                 else:
                     w1, w2 = self.weights[l]
-                    lb.lisa_attn_shared_decode(self.rows[cur], lb.Link(a, None, w1, w2, act=lb.ACTS[self.act]), cache, L=L, out=out,
-                                               out_scores=row_out, workspace=ws)
-                if probe is not None and t in probe.steps and l in probe.layers:
+                    lb.lisa_attn_shared_decode(self.rows[cur], lb.Link(a, None, w1, w2, act=lb.ACTS[self.act]), cache, L=L,
+                                               seq_lens=lens, out=out, out_scores=row_out, workspace=ws)
+                if probe_t is not None and probe_t in probe.steps and l in probe.layers:
                     s = list(probe.seqs)
                     rec = {"L": L, "out": out[s, 0].float().cpu(), "a": a[s, 0].cpu(), "v": cache.v[s, :, :L].cpu(),
                            "k": cache.k[s][..., :L].cpu() if not self.is_standard[l] else cache.k[s, :, :L].cpu(),
                            "row": None if row_out is None else row_out[s, :, :L].cpu(),
                            "prev": None if self.is_standard[l] else self.rows[cur][s, :, :L].cpu()}
-                    probe.decode[(t, l)] = rec
+                    probe.decode[(probe_t, l)] = rec
                 if row_out is not None:
                     cur ^= 1
+
+        if graph:
+            assert probe is None, "probing needs the step-by-step loop"
+            lens = torch.empty((B,), dtype=torch.int32, device="cuda")
+            L_max = N + T
+
+            def graph_step():
+                before.copy_(lens)
+                lens.add_(1)
+                step(L_max, lens)
+
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):     # one plain step first: one-time set-up inside the library happens here
+                lens.fill_(N)
+                graph_step()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            lens.fill_(N)
+            with torch.cuda.graph(g):
+                graph_step()
+            lens.fill_(N)
+            torch.cuda.synchronize()
+            t0.record()
+            for _ in range(T):
+                g.replay()
+            t1.record()
+            torch.cuda.synchronize()
+            return t0.elapsed_time(t1)
+
+        torch.cuda.synchronize()
+        t0.record()
+        for t in range(T):
+            L = N + t + 1
+            before.fill_(L - 1)
+            step(L, None, t if probe is not None else None)
         t1.record()
         torch.cuda.synchronize()
         return t0.elapsed_time(t1)

@@ -59,6 +59,22 @@ def test_small_stack_layer_by_layer_prefill():
     check_probe(st, probe)
 
 
+def test_small_stack_decode_from_a_graph():
+    """One captured decode step replayed T times (context lengths on the device) ends where the step-by-step loop does."""
+    outs, caches = [], []
+    for graph in (False, True):
+        st = lstack.AttentionStack(n_layers=8, B=2, N=200, T=6, seed=9)
+        st.prefill()
+        st.decode(graph=graph)
+        torch.cuda.synchronize()
+        assert lb.lisa_check() == lb.OK
+        outs.append(st.last_out.float().cpu())
+        caches.append([(c.k.float().cpu(), c.v.float().cpu()) for c in st.caches])
+    assert torch.allclose(outs[0], outs[1], atol=1e-6, rtol=0)
+    for (k0, v0), (k1, v1) in zip(*caches):
+        assert torch.equal(k0, k1) and torch.equal(v0, v1)
+
+
 def test_small_stack_lossless_prefill():
     """Sec. 5.2 "NF": shared layers attend over the prompt with standard attention on their own Q and K and cache
     K_LR; sharing starts with the first decoded token."""
