@@ -85,6 +85,29 @@ def test_cache_bytes_reproduce_the_papers_memory_model(lib, h, l, dk, r, S):
     assert S * (std_k - sh_k) - h * l * l * 2 == pre
 
 
+def golden_lowrank_widths():
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "lowrank_widths.txt")
+    rows = []
+    for line in open(path):
+        if line.strip() and not line.startswith("#"):
+            v, m, hq, hkv, r, wq, wk = line.split()
+            rows.append((v, m, int(hq), int(hkv), int(r), int(wq), int(wk)))
+    return rows
+
+
+@pytest.mark.parametrize("variant,model,hq,hkv,r,wq,wk", golden_lowrank_widths())
+def test_cache_row_matches_the_papers_projection_widths(lib, variant, model, hq, hkv, r, wq, wk):
+    """The appendix prints the output widths of W_LR^Q and W_LR^K per model (tests/golden/lowrank_widths.txt).  A token's
+    K_LR row in a shared layer's cache must hold exactly that many values: rank per head times KV heads, with the query
+    side at rank per head times query heads (so r is per head, and grouped-query models cache Hkv heads of K_LR)."""
+    assert hq * r == wq and hkv * r == wk
+    L = 4096
+    sh_k, sh_v = lb.lisa_kvcache_bytes(lb.CACHE_SHARED, 1, hkv, L, 128, r)
+    std_k, _ = lb.lisa_kvcache_bytes(lb.CACHE_STANDARD, 1, hkv, L, 128)
+    assert sh_k == L * wk * 2                      # bf16: two bytes per cached K_LR value
+    assert std_k * wk == sh_k * hkv * 128           # the K cache shrinks by d_k / r
+
+
 def test_decode_workspace_query(lib):
     cache = lb.CCacheLayer(lb.CACHE_SHARED, lb.BF16, 64, 40, 4096, 128, 21, 0, None, None)
     a = lb.SharedDecodeArgs()
