@@ -19,7 +19,7 @@ struct AppendParams {
 
 // rows of d elements (V, or K of a STANDARD layer): one thread per 16 bytes
 template <typename Vec, int kElems>
-__global__ void append_rows_kernel(const __grid_constant__ AppendParams p, TView src, void* dst_base, bool count_drops) {
+__device__ __forceinline__ void append_rows(const AppendParams& p, const TView& src, void* dst_base, bool count_drops) {
     const int vec_per_row = p.d / kElems;
     const int64_t total = (int64_t)p.B * p.n_new * p.Hkv * vec_per_row;
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
@@ -43,7 +43,7 @@ __global__ void append_rows_kernel(const __grid_constant__ AppendParams p, TView
 
 // K' of a SHARED layer: thread per (b, g, t); consecutive threads write consecutive positions
 template <typename T>
-__global__ void append_kp_transposed_kernel(const __grid_constant__ AppendParams p) {
+__device__ __forceinline__ void append_kp_transposed(const AppendParams& p) {
     const int64_t total = (int64_t)p.B * p.Hkv * p.n_new;
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
         const int t = (int)(e % p.n_new);
@@ -58,6 +58,15 @@ __global__ void append_kp_transposed_kernel(const __grid_constant__ AppendParams
     }
 }
 
+// One launch appends both halves of a layer's cache: blockIdx.y = 0 the V rows, 1 the K rows (STANDARD) or the
+// transposed K_LR columns (SHARED).
+template <typename Vec, int kElems, typename T>
+__global__ void append_kernel(const __grid_constant__ AppendParams p) {
+    if (blockIdx.y == 0) append_rows<Vec, kElems>(p, p.v, p.vc, true);
+    else if (p.kind == LISA_CACHE_STANDARD) append_rows<Vec, kElems>(p, p.k, p.kc, false);
+    else append_kp_transposed<T>(p);
+}
+
 }  // namespace
 
 cudaError_t launch_kvcache_append(const lisa_kvcache_layer& c, const lisa_tensor& k, const lisa_tensor& v,
@@ -68,20 +77,9 @@ cudaError_t launch_kvcache_append(const lisa_kvcache_layer& c, const lisa_tensor
     const int threads = 256;
     const int64_t rows = (int64_t)c.B * n_new * c.Hkv;
     auto blocks_for = [&](int64_t n) { return (int)std::max<int64_t>(1, std::min<int64_t>((n + threads - 1) / threads, 148 * 16)); };
-    if (c.dtype == LISA_BF16) {
-        append_rows_kernel<uint4, 8><<<blocks_for(rows * (c.d / 8)), threads, 0, s>>>(p, p.v, c.v, true);
-        if (c.kind == LISA_CACHE_STANDARD)
-            append_rows_kernel<uint4, 8><<<blocks_for(rows * (c.d / 8)), threads, 0, s>>>(p, p.k, c.k, false);
-        else
-            append_kp_transposed_kernel<__nv_bfloat16><<<blocks_for(rows), threads, 0, s>>>(p);
-    } else {
-        append_rows_kernel<float4, 4><<<blocks_for(rows * (c.d / 4)), threads, 0, s>>>(p, p.v, c.v, true);
-        if (c.kind == LISA_CACHE_STANDARD)
-            append_rows_kernel<float4, 4><<<blocks_for(rows * (c.d / 4)), threads, 0, s>>>(p, p.k, c.k, false);
-        else
-            append_kp_transposed_kernel<float><<<blocks_for(rows), threads, 0, s>>>(p);
-    }
-    count_launches(2);
+    if (c.dtype == LISA_BF16) append_kernel<uint4, 8, __nv_bfloat16><<<dim3(blocks_for(rows * (c.d / 8)), 2), threads, 0, s>>>(p);
+    else append_kernel<float4, 4, float><<<dim3(blocks_for(rows * (c.d / 4)), 2), threads, 0, s>>>(p);
+    count_launches(1);
     return cudaGetLastError();
 }
 
