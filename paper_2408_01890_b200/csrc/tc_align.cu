@@ -159,7 +159,8 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
 //   scratch -> fragments ldmatrix.trans per 16-position strip
 //   chain in registers   (ffn_link)
 //   result               stmatrix.trans back into the scratch, then 16 bytes per lane to the plane
-template <bool REGW, int NT, int MIN_CTAS, int STAGES, int PP>
+// ACT0: the single link's activation as a compile-time constant (REGW), or -1 = look at the parameters.
+template <bool REGW, int NT, int MIN_CTAS, int STAGES, int PP, int ACT0>
 __global__ void __launch_bounds__(NT, MIN_CTAS)
 tc_align_kernel(const __grid_constant__ AlignParams p) {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -317,7 +318,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             __half* const g_prev = plane0 + (has_prev ? piece_off(prev) : 0);
             const uint32_t base = smem_u32(scr + b_cur * PLANE_SCR), s_next = smem_u32(scr + b_next * PLANE_SCR);
             const uint8_t* s_prev = scr + b_prev * PLANE_SCR;
-#pragma unroll 1
+#pragma unroll
             for (int s2 = 0; s2 < NS; ++s2) {
                 const uint32_t off0 = frag_off(s2, 0), off1 = frag_off(s2, 1);
                 uint32_t afr[2][4];
@@ -333,9 +334,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                         if (has_prev) *reinterpret_cast<uint4*>(g_prev + i * (HPA * 64)) = *reinterpret_cast<const uint4*>(s_prev + so);
                     }
                 };
-                if (act0 == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, true>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, side);
-                else if (act0 == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, true>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, side);
-                else ffn_link<LISA_ACT_NONE, true>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, side);
+                ffn_link<(ACT0 < 0 ? LISA_ACT_NONE : ACT0), true>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, side);
                 __syncwarp();
 #pragma unroll
                 for (int x = 0; x < 2; ++x) {
@@ -500,7 +499,13 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     const int threads = regw ? kRegwThreads : kWorkers;
     const int ctas_per_sm = regw ? kRegwCtas : 1;
     const size_t smem = align_smem_bytes(a.chain, threads, regw ? kRegwStages : kStages, regw ? kRegwPiece : 32);
-    auto kernel = regw ? tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece> : tc_align_kernel<false, kWorkers, 1, kStages, 32>;
+    auto kernel = tc_align_kernel<false, kWorkers, 1, kStages, 32, -1>;
+    if (regw) {
+        const int act = a.links[0].act;
+        kernel = act == LISA_ACT_RELU   ? tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece, LISA_ACT_RELU>
+                 : act == LISA_ACT_SILU ? tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece, LISA_ACT_SILU>
+                                        : tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece, LISA_ACT_NONE>;
+    }
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const int64_t total_units = (int64_t)p.units_per_batch * a.B;
