@@ -175,7 +175,9 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         uint2* w1f = reinterpret_cast<uint2*>(sW + k * LINK_BYTES);
         uint2* w2f = reinterpret_cast<uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
         float* bias = reinterpret_cast<float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
-        const float out_scale = (k == c - 1 && !p.store_all) ? kLog2e : 1.f;   // store_all scales what it stores instead
+        // the last link's log2(e) is folded into its W2 and b2, except where every link's output leaves (store_all with
+        // more than one link): there the stored values are scaled instead and the chain continues unscaled
+        const float out_scale = (k == c - 1 && (!p.store_all || c == 1)) ? kLog2e : 1.f;
         const int wd = p.w_dtype[k];
         for (int e = tid; e < 2 * 8 * 32; e += NT) {   // W1 [32 heads][64 hidden]: k = head, n = hidden
             const int ln = e & 31, j = (e >> 5) & 7, ks = e >> 8, g = ln >> 2, t = ln & 3;
@@ -304,7 +306,6 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         const uint2* w2f = reinterpret_cast<const uint2*>(sW + W1F_BYTES);
         const float* b1 = reinterpret_cast<const float*>(sW + W1F_BYTES + W2F_BYTES);
         const uint32_t* b1h = reinterpret_cast<const uint32_t*>(b1);
-        const float last_scale = store_all ? kLog2e : 1.f;
         fetch(cu, 0);
         Cursor here = cu, nxt = cu, prev = cu;
         advance(nxt);
@@ -339,10 +340,10 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
 #pragma unroll
                 for (int x = 0; x < 2; ++x) {
                     uint32_t r[4];
-                    r[0] = pack_f16(y[2 * x][0] * last_scale, y[2 * x][1] * last_scale);
-                    r[1] = pack_f16(y[2 * x][2] * last_scale, y[2 * x][3] * last_scale);
-                    r[2] = pack_f16(y[2 * x + 1][0] * last_scale, y[2 * x + 1][1] * last_scale);
-                    r[3] = pack_f16(y[2 * x + 1][2] * last_scale, y[2 * x + 1][3] * last_scale);
+                    r[0] = pack_f16(y[2 * x][0], y[2 * x][1]);
+                    r[1] = pack_f16(y[2 * x][2], y[2 * x][3]);
+                    r[2] = pack_f16(y[2 * x + 1][0], y[2 * x + 1][1]);
+                    r[3] = pack_f16(y[2 * x + 1][2], y[2 * x + 1][3]);
                     stmatrix_x4_trans(base + (x ? off1 : off0), r);
                 }
             }
@@ -431,7 +432,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             }
             // the last link's result over its place in the scratch (plane 0, or plane c-1 in a chain of layers; every
             // lane's ldmatrix of it is done), transposed back
-            const float last_scale = store_all ? kLog2e : 1.f;
+            const float last_scale = (store_all && c > 1) ? kLog2e : 1.f;
             const uint32_t last_plane = store_all ? (uint32_t)(c - 1) * PLANE_SCR : 0u;
             __syncwarp();
 #pragma unroll
