@@ -114,14 +114,15 @@ __device__ __forceinline__ uint32_t act_h2(uint32_t x) {
 // the register copies w1r/w2r that a warp keeps for its whole life (single-link calls).
 // `side` is called once, after the first layer's MMAs have been issued: unrelated instructions placed there (the copies
 // of neighbouring pieces) issue while this warp's MMAs wait for their turn on the tensor pipe.
-template <int ACT, bool REGW, typename Side>
+// BIAS = false: b1 and b2 are known to be absent (zero accumulator start, nothing loaded).
+template <int ACT, bool REGW, bool BIAS = true, typename Side>
 __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* w1f, const uint2* w2f, const uint2* w1r, const uint2* w2r,
                                          const uint32_t* b1h, const float* b2, int lane, float (*y)[4], Side side) {
     const int t = lane & 3;
     uint32_t h[8][2];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const uint32_t bb = b1h[j * 4 + t];
+        const uint32_t bb = BIAS ? b1h[j * 4 + t] : 0u;
         const uint2 w = REGW ? w1r[j] : w1f[j * 32 + lane];
         mma_f16acc(h[j], afr[0], w.x, w.y, bb, bb);
     }
@@ -141,7 +142,7 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
     }
 #pragma unroll
     for (int j2 = 0; j2 < 4; ++j2) {
-        const float2 bb = *reinterpret_cast<const float2*>(b2 + j2 * 8 + 2 * t);
+        const float2 bb = BIAS ? *reinterpret_cast<const float2*>(b2 + j2 * 8 + 2 * t) : make_float2(0.f, 0.f);
         const uint2 w = REGW ? w2r[j2] : w2f[j2 * 32 + lane];
         mma_f16_bias(y[j2], hfr[0], w.x, w.y, bb.x, bb.y);
     }
@@ -160,6 +161,7 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
 //   chain in registers   (ffn_link)
 //   result               stmatrix.trans back into the scratch, then 16 bytes per lane to the plane
 // ACT0: the single link's activation as a compile-time constant (REGW), or -1 = look at the parameters.
+// ACT0 >= 8: additionally, the link has no biases.
 template <bool REGW, int NT, int MIN_CTAS, int STAGES, int PP, int ACT0>
 __global__ void __launch_bounds__(NT, MIN_CTAS)
 tc_align_kernel(const __grid_constant__ AlignParams p) {
@@ -335,7 +337,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                         if (has_prev) *reinterpret_cast<uint4*>(g_prev + i * (HPA * 64)) = *reinterpret_cast<const uint4*>(s_prev + so);
                     }
                 };
-                ffn_link<(ACT0 < 0 ? LISA_ACT_NONE : ACT0), true>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, side);
+                ffn_link<(ACT0 < 0 ? LISA_ACT_NONE : (ACT0 & 7)), true, (ACT0 < 8)>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, side);
                 __syncwarp();
 #pragma unroll
                 for (int x = 0; x < 2; ++x) {
@@ -503,9 +505,11 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     auto kernel = tc_align_kernel<false, kWorkers, 1, kStages, 32, -1>;
     if (regw) {
         const int act = a.links[0].act;
-        kernel = act == LISA_ACT_RELU   ? tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece, LISA_ACT_RELU>
-                 : act == LISA_ACT_SILU ? tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece, LISA_ACT_SILU>
-                                        : tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece, LISA_ACT_NONE>;
+        const bool bias = a.links[0].b1 || a.links[0].b2;
+#define LISA_ALIGN_REGW(A_) (bias ? tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece, (A_)> \
+                                  : tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece, (A_) + 8>)
+        kernel = act == LISA_ACT_RELU ? LISA_ALIGN_REGW(LISA_ACT_RELU) : act == LISA_ACT_SILU ? LISA_ALIGN_REGW(LISA_ACT_SILU) : LISA_ALIGN_REGW(LISA_ACT_NONE);
+#undef LISA_ALIGN_REGW
     }
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
