@@ -160,7 +160,7 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
 //   scratch -> fragments ldmatrix.trans per 16-position strip
 //   chain in registers   (ffn_link)
 //   result               stmatrix.trans back into the scratch, then 16 bytes per lane to the plane
-// ACT0: the single link's activation as a compile-time constant (REGW), or -1 = look at the parameters.
+// ACT0: the activation of every link as a compile-time constant, or -1 = look at the parameters link by link.
 // ACT0 >= 8: additionally, the link has no biases.
 template <bool REGW, int NT, int MIN_CTAS, int STAGES, int PP, int ACT0>
 __global__ void __launch_bounds__(NT, MIN_CTAS)
@@ -387,7 +387,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         asm volatile("cp.async.wait_group %0;" ::"n"(STAGES - 1) : "memory");
         __syncwarp();
         const uint32_t base = smem_u32(scr + buf * c * PLANE_SCR);
-#pragma unroll 1
+#pragma unroll
         for (int s2 = 0; s2 < PP / 16; ++s2) {
             const uint32_t off0 = frag_off(s2, 0), off1 = frag_off(s2, 1);
             uint32_t afr[2][4];
@@ -400,9 +400,13 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                 const float* b1 = reinterpret_cast<const float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
                 const uint32_t* b1h = reinterpret_cast<const uint32_t*>(b1);
                 const int act = k == 0 ? act0 : (k == 1 ? act1 : act2);
-                if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
-                else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
-                else ffn_link<LISA_ACT_NONE, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
+                if constexpr (ACT0 >= 0) {   // every link has this activation (and, from 8 up, no biases)
+                    ffn_link<(ACT0 & 7), REGW, (ACT0 < 8)>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
+                } else {
+                    if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
+                    else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
+                    else ffn_link<LISA_ACT_NONE, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
+                }
                 if (store_all && k + 1 < c) {
                     // a chain of layers: link k's own output leaves too, over plane k's place in the scratch (plane 0 = A_0
                     // and plane k = D_k have been consumed by every lane before this link's MMAs could complete)
@@ -503,9 +507,18 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     const int ctas_per_sm = regw ? kRegwCtas : 1;
     const size_t smem = align_smem_bytes(a.chain, threads, regw ? kRegwStages : kStages, regw ? kRegwPiece : 32);
     auto kernel = tc_align_kernel<false, kWorkers, 1, kStages, 32, -1>;
+    const int act = a.links[0].act;
+    bool bias = false, same_act = true;
+    for (int k = 0; k < a.chain; ++k) {
+        bias = bias || a.links[k].b1 || a.links[k].b2;
+        same_act = same_act && a.links[k].act == act;
+    }
+    if (!regw && same_act) {
+#define LISA_ALIGN_CHAIN(A_) (bias ? tc_align_kernel<false, kWorkers, 1, kStages, 32, (A_)> : tc_align_kernel<false, kWorkers, 1, kStages, 32, (A_) + 8>)
+        kernel = act == LISA_ACT_RELU ? LISA_ALIGN_CHAIN(LISA_ACT_RELU) : act == LISA_ACT_SILU ? LISA_ALIGN_CHAIN(LISA_ACT_SILU) : LISA_ALIGN_CHAIN(LISA_ACT_NONE);
+#undef LISA_ALIGN_CHAIN
+    }
     if (regw) {
-        const int act = a.links[0].act;
-        const bool bias = a.links[0].b1 || a.links[0].b2;
 #define LISA_ALIGN_REGW(A_) (bias ? tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece, (A_)> \
                                   : tc_align_kernel<true, kRegwThreads, kRegwCtas, kRegwStages, kRegwPiece, (A_) + 8>)
         kernel = act == LISA_ACT_RELU ? LISA_ALIGN_REGW(LISA_ACT_RELU) : act == LISA_ACT_SILU ? LISA_ALIGN_REGW(LISA_ACT_SILU) : LISA_ALIGN_REGW(LISA_ACT_NONE);
