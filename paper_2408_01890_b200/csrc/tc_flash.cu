@@ -313,10 +313,10 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
 #pragma unroll
                 for (int c = 0; c < BN / 8; ++c) {
                     uint4 v;
-                    v.x = pack_f16(sf[c * 8 + 0] * emit_scale, sf[c * 8 + 1] * emit_scale);
-                    v.y = pack_f16(sf[c * 8 + 2] * emit_scale, sf[c * 8 + 3] * emit_scale);
-                    v.z = pack_f16(sf[c * 8 + 4] * emit_scale, sf[c * 8 + 5] * emit_scale);
-                    v.w = pack_f16(sf[c * 8 + 6] * emit_scale, sf[c * 8 + 7] * emit_scale);
+                    { const float2 t2 = __fmul2_rn(reinterpret_cast<const float2*>(sf)[c * 4 + 0], make_float2(emit_scale, emit_scale)); v.x = pack_f16(t2.x, t2.y); }
+                    { const float2 t2 = __fmul2_rn(reinterpret_cast<const float2*>(sf)[c * 4 + 1], make_float2(emit_scale, emit_scale)); v.y = pack_f16(t2.x, t2.y); }
+                    { const float2 t2 = __fmul2_rn(reinterpret_cast<const float2*>(sf)[c * 4 + 2], make_float2(emit_scale, emit_scale)); v.z = pack_f16(t2.x, t2.y); }
+                    { const float2 t2 = __fmul2_rn(reinterpret_cast<const float2*>(sf)[c * 4 + 3], make_float2(emit_scale, emit_scale)); v.w = pack_f16(t2.x, t2.y); }
                     *reinterpret_cast<uint4*>(stg + sw128_offset(lane, c)) = v;
                 }
                 fence_async_smem();
@@ -336,9 +336,8 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                     const uint32_t w[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        const float2 yv = unpack_f16(w[e]);
-                        sf[c * 8 + 2 * e] = fmaf(sf[c * 8 + 2 * e], scale_log2, yv.x);
-                        sf[c * 8 + 2 * e + 1] = fmaf(sf[c * 8 + 2 * e + 1], scale_log2, yv.y);
+                        float2* s2 = reinterpret_cast<float2*>(sf) + c * 4 + e;
+                        *s2 = __ffma2_rn(*s2, make_float2(scale_log2, scale_log2), unpack_f16(w[e]));
                     }
                 }
             }
@@ -350,10 +349,12 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             }
             float mx[4] = {sf[0], sf[1], sf[2], sf[3]};   // four independent chains instead of one of 64 dependent steps
 #pragma unroll
-            for (int j = 4; j < BN; j += 4) {
-                mx[0] = fmaxf(mx[0], sf[j]); mx[1] = fmaxf(mx[1], sf[j + 1]);
-                mx[2] = fmaxf(mx[2], sf[j + 2]); mx[3] = fmaxf(mx[3], sf[j + 3]);
+            for (int j = 4; j + 8 <= BN; j += 8) {   // two new values per step and chain: a three-input maximum where there is one
+                mx[0] = fmaxf(fmaxf(mx[0], sf[j]), sf[j + 4]); mx[1] = fmaxf(fmaxf(mx[1], sf[j + 1]), sf[j + 5]);
+                mx[2] = fmaxf(fmaxf(mx[2], sf[j + 2]), sf[j + 6]); mx[3] = fmaxf(fmaxf(mx[3], sf[j + 3]), sf[j + 7]);
             }
+            mx[0] = fmaxf(mx[0], sf[BN - 4]); mx[1] = fmaxf(mx[1], sf[BN - 3]);
+            mx[2] = fmaxf(mx[2], sf[BN - 2]); mx[3] = fmaxf(mx[3], sf[BN - 1]);
             float m_t = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             if constexpr (!PLANE) m_t *= scale_log2;
             // lazy rescale: move the reference maximum only when some row of the warp outgrew it by 2^8
@@ -376,7 +377,10 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                         tmem_ld32(tmem_O + lane_sel + c * 32, orr);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) orr[j] = __float_as_uint(__uint_as_float(orr[j]) * factor);
+                        for (int j = 0; j < 16; ++j) {
+                            float2* o2 = reinterpret_cast<float2*>(orr) + j;
+                            *o2 = __fmul2_rn(*o2, make_float2(factor, factor));
+                        }
                         tmem_st32(tmem_O + lane_sel + c * 32, orr);
                     }
                     tmem_wait_st();
@@ -389,21 +393,27 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             // where the layout has one); two tiles back, this has nearly always happened already.
             if (t >= 2 && !(ok = mbar_wait(pv_done + s, ((t - 2) >> 1) & 1, abort_flag))) break;
             uint8_t* pb = p_buf(t);
-            float sum = 0.f;
-            const float neg_m = -m_ref;
+            // The softmax warps are bound by the length of their own instruction chain, so the fp32 arithmetic around
+            // the exponentials runs two values per instruction (packed fp32 pairs; the scores of a thread sit in
+            // consecutive registers).
+            float2 sum2 = make_float2(0.f, 0.f);
+            const float2 neg_m2 = make_float2(-m_ref, -m_ref), scale2 = make_float2(scale_log2, scale_log2);
+            const float2* sf2 = reinterpret_cast<const float2*>(sf);
 #pragma unroll
             for (int c = 0; c < BN / 8; ++c) {
                 float e[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    e[j] = PLANE ? fast_exp2(sf[c * 8 + j] + neg_m) : fast_exp2(fmaf(sf[c * 8 + j], scale_log2, neg_m));
-                    sum += e[j];
+                for (int j = 0; j < 4; ++j) {
+                    const float2 x = PLANE ? __fadd2_rn(sf2[c * 4 + j], neg_m2) : __ffma2_rn(sf2[c * 4 + j], scale2, neg_m2);
+                    e[2 * j] = fast_exp2(x.x);
+                    e[2 * j + 1] = fast_exp2(x.y);
+                    sum2 = __fadd2_rn(sum2, make_float2(e[2 * j], e[2 * j + 1]));
                 }
                 uint4 v;
                 v.x = pack_bf16(e[0], e[1]); v.y = pack_bf16(e[2], e[3]); v.z = pack_bf16(e[4], e[5]); v.w = pack_bf16(e[6], e[7]);
                 *reinterpret_cast<uint4*>(pb + sw128_offset(row, c)) = v;
             }
-            l_sum = l_sum * factor + sum;
+            l_sum = l_sum * factor + (sum2.x + sum2.y);
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(p_full + s);
