@@ -31,7 +31,7 @@ DECODE = "cfg4_llama2_13b_decode"
 METRIC = "lisa_attention_tokens_per_s"
 # dram bytes (read + write) per launch from the ncu captures summarised under profiles/ (cold cache, same workload);
 # None for a kernel that has changed since its counters were taken
-PREFILL_TRAFFIC = {"align": 142642688 + 83800064, "emit_scores": 39559424 + 86833664, "attention": 186025984 + 5347328}
+PREFILL_TRAFFIC = {"align": 142642688 + 83800064, "emit_scores": 40019456 + 85420032, "attention": 186513920 + 6682368}
 DECODE_TRAFFIC_PER_SEQ = (395953152 + 5092608) / 8  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
 
 
