@@ -559,19 +559,40 @@ __global__ void __launch_bounds__(kThreads, 2) anchor_decode_chunk_kernel(const 
 
 // Merge the per-chunk (m, l, o) partials of one (b, h): o = sum_c e^{m_c - M} o_c / sum_c e^{m_c - M} l_c.
 __global__ void decode_merge_kernel(const __grid_constant__ DecodeParams p) {
+    extern __shared__ float s_w[];   // per chunk: exp(m_c - M) / sum, the weight of the chunk's partial output
     const int h = blockIdx.x, b = blockIdx.y, x = threadIdx.x;
     const int L = p.seq_lens ? p.seq_lens[b] : p.L_uniform;
     const int nc = (L + kChunk - 1) / kChunk;
     const size_t base = (size_t)b * p.n_chunks * p.Hq + h;
-    float M = -INFINITY;
-    for (int c = 0; c < nc; ++c) M = fmaxf(M, p.ws_m[base + (size_t)c * p.Hq]);
-    float num = 0.f, den = 0.f;
-    for (int c = 0; c < nc; ++c) {
-        const float w = __expf(p.ws_m[base + (size_t)c * p.Hq] - M);
-        den = fmaf(w, p.ws_l[base + (size_t)c * p.Hq], den);
-        num = fmaf(w, p.ws_o[(base + (size_t)c * p.Hq) * p.d + x], num);
+    if (x < 32) {
+        // the first warp turns the chunks' (m, l) into weights: one chunk per lane and step, reductions by shuffle
+        float M = -INFINITY;
+        for (int c = x; c < nc; c += 32) M = fmaxf(M, p.ws_m[base + (size_t)c * p.Hq]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        float den = 0.f;
+        for (int c = x; c < nc; c += 32) {
+            const float w = __expf(p.ws_m[base + (size_t)c * p.Hq] - M);
+            s_w[c] = w;
+            den = fmaf(w, p.ws_l[base + (size_t)c * p.Hq], den);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+        const float inv = 1.f / den;
+        for (int c = x; c < nc; c += 32) s_w[c] *= inv;
     }
-    st_elem(const_cast<void*>(p.o.ptr), b * p.o.sb + h * p.o.sh + x, p.o.dtype, num / den);
+    __syncthreads();
+    // every thread one output column: independent loads, four accumulators
+    const float* po = p.ws_o + base * p.d + x;
+    const size_t step = (size_t)p.Hq * p.d;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    int c = 0;
+    for (; c + 4 <= nc; c += 4) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[j] = fmaf(s_w[c + j], po[(size_t)(c + j) * step], acc[j]);
+    }
+    for (; c < nc; ++c) acc[0] = fmaf(s_w[c], po[(size_t)c * step], acc[0]);
+    st_elem(const_cast<void*>(p.o.ptr), b * p.o.sb + h * p.o.sh + x, p.o.dtype, (acc[0] + acc[1]) + (acc[2] + acc[3]));
 }
 
 void carve_workspace(DecodeParams& p, void* ws) {
@@ -630,7 +651,7 @@ cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cud
         shared_decode_chunk_kernel<0, 0><<<grid, kThreads, smem, s>>>(p);
     }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, 0, s>>>(p);
+    decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, (size_t)p.n_chunks * sizeof(float), s>>>(p);
     count_launches(2);
     return cudaGetLastError();
 }
@@ -651,7 +672,7 @@ cudaError_t launch_anchor_decode(const lisa_anchor_args& a, void* ws, cudaStream
     if ((e = set_smem(anchor_decode_chunk_kernel, smem)) != cudaSuccess) return e;
     anchor_decode_chunk_kernel<<<dim3(p.n_chunks, p.B), kThreads, smem, s>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, 0, s>>>(p);
+    decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, (size_t)p.n_chunks * sizeof(float), s>>>(p);
     count_launches(2);
     return cudaGetLastError();
 }
