@@ -181,22 +181,10 @@ def main():
     if rank == 0:
         lbuild.build()
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    from paper_2408_01890_b200.ranks import RankGroup
+    group = RankGroup("nccl", torch.device("cuda", local))   # one process per GPU; replicas over the batch, no data-path collective
     lb.load()
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-
-    def max_over_ranks(x):
-        if dist is None:
-            return x
-        tt = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        return float(tt.item())
+    barrier, max_over_ranks = group.barrier, group.max_over_ranks
 
     peaks = measured_peaks()
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
@@ -230,7 +218,7 @@ def main():
     total_ms = max_over_ranks(total_ms)
     ms_per_step = total_ms / args.steps
     tokens = w.B * w.N
-    value = world * tokens / (ms_per_step * 1e-3)
+    value = group.whole_job_per_second(tokens, ms_per_step)
     flops = prefill_flops(w, 1)
     # per-kernel device times of the same step (events recorded inside the library around each of its kernels)
     lb.lisa_prefill_phase_timing(True)
@@ -412,8 +400,7 @@ def main():
                        "step": "lisa_attn_shared_prefill + lisa_kvcache_append"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
             "decode": decode, "stack": stack}))
-    if dist is not None:
-        dist.destroy_process_group()
+    group.close()
 
 
 if __name__ == "__main__":
