@@ -9,6 +9,7 @@
 // The N x N x Hq scores of the whole prompt are never stored; only the wave's strip of rows is.
 #include <algorithm>
 #include <cmath>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -154,6 +155,34 @@ bool tc_shared_prefill_supported(const lisa_shared_prefill_args& a) {
 // + 1024: the launch aligns the caller's pointer up to the 1024 bytes the swizzled tiles need
 size_t tc_shared_prefill_workspace(const lisa_shared_prefill_args& a) { return plan_layout(a).total + 1024; }
 
+namespace {
+// The packing of Q'/K' feeds only the kernels that come after the first emit (the attention kernel; the emits of the
+// differences of deeper chains), so it runs beside that emit on a stream of the library's own: forked from the
+// caller's stream with one event and joined with another before its first consumer.  One stream and one event pair
+// per device, created on first use; the fork and the join are each enqueued under a lock, so calls from several host
+// threads cannot pair one call's wait with another call's record.
+struct SideStream {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+    bool ok = false;
+};
+SideStream g_side[64];
+std::mutex g_side_mutex;
+
+SideStream* side_stream() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    SideStream& ss = g_side[dev];
+    if (!ss.ok) {
+        if (cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        ss.ok = true;
+    }
+    return &ss;
+}
+}  // namespace
+
 cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws, cudaStream_t s) {
     return launch_tc_shared_prefill_chain(a, nullptr, nullptr, ws, s);
 }
@@ -168,6 +197,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
     char* base = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(ws) + 1023) & ~(uintptr_t)1023);
     const int c = a.chain_len;
     cudaError_t e;
+    SideStream* side = nullptr;
     {
         PhaseMark mark(0, s);
         PackJobs jobs{};
@@ -179,10 +209,29 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         }
         const int64_t total = (int64_t)a.B * a.Hq * a.N * (kPadRank / 8);
         const int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 16);
-        pack_lowrank_kernel<<<dim3(blocks, 2 * c), 256, 0, s>>>(jobs, a.B, a.N);
+        // beside the first emit, unless the per-kernel timing is on (then every kernel is timed on the caller's stream)
+        if (!g_pt.on) {
+            std::lock_guard<std::mutex> lock(g_side_mutex);
+            side = side_stream();
+            if (side) {
+                if ((e = cudaEventRecord(side->fork, s)) != cudaSuccess) return e;
+                if ((e = cudaStreamWaitEvent(side->stream, side->fork, 0)) != cudaSuccess) return e;
+                pack_lowrank_kernel<<<dim3(blocks, 2 * c), 256, 0, side->stream>>>(jobs, a.B, a.N);
+                if ((e = cudaGetLastError()) != cudaSuccess) return e;
+                if ((e = cudaEventRecord(side->join, side->stream)) != cudaSuccess) return e;
+            }
+        }
+        if (!side) pack_lowrank_kernel<<<dim3(blocks, 2 * c), 256, 0, s>>>(jobs, a.B, a.N);
         count_launches(1);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
+    bool joined = side == nullptr;
+    auto join_pack = [&]() -> cudaError_t {   // before the first kernel that reads the packed Q'/K'
+        if (joined) return cudaSuccess;
+        joined = true;
+        std::lock_guard<std::mutex> lock(g_side_mutex);
+        return cudaStreamWaitEvent(s, side->join, 0);
+    };
     Wave waves[1024];
     const int nw = plan_waves(a.B, a.N, a.Hq, c, waves, 1024);
     for (int w = 0; w < nw; ++w) {
@@ -196,6 +245,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             if ((e = launch_tc_flash(f, s)) != cudaSuccess) return e;
         }
         for (int k = 0; k + 1 < c; ++k) {
+            if ((e = join_pack()) != cudaSuccess) return e;
             PhaseMark mark(1, s);
             TcFlashArgs fd = f;
             fd.kd = kPadRank;
@@ -218,6 +268,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             if ((e = launch_tc_align(al, s)) != cudaSuccess) return e;
         }
         // 3. each layer's own difference, softmax and .V
+        if ((e = join_pack()) != cudaSuccess) return e;
         for (int k = all_layers ? 0 : c - 1; k < c; ++k) {
             TcFlashArgs fv = f;
             fv.emit_plane = nullptr;
