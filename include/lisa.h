@@ -12,7 +12,11 @@
  *   - Returns a lisa_status_t.  Never throws, never aborts.  Unless an entry
  *     point says otherwise it allocates and frees no device memory and does not
  *     synchronise: it validates on the host, then enqueues kernels on the
- *     caller's stream.  On any error nothing is launched and outputs are untouched.
+ *     caller's stream.  (The prefill of a shared layer also runs one small kernel
+ *     on a stream of the library's own, created on first use per device; it is
+ *     forked from the caller's stream and joined back into it by events inside
+ *     the same call, so to the caller all work is ordered on the stream it gave.)
+ *     On any error nothing is launched and outputs are untouched.
  *   - All data pointers are DEVICE pointers owned by the caller, 16-byte
  *     aligned, and must stay valid until the enqueued work has finished.
  *     Descriptor structs and the `links` array are HOST memory, read only
