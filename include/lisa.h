@@ -93,7 +93,7 @@ typedef struct lisa_link {
     int32_t ffn_layers; /* 1 or 2 */
 } lisa_link;
 
-/* The cache of one layer (Sec. 2.2 "KV cache"; Sec. 5.2: a shared layer stores K_LR instead of K).
+/* The cache of one layer (Sec. 2.2, KV cache; Sec. 5.2: a shared layer caches the low-rank keys K_LR in place of K).
  *   STANDARD: k = K   [B][Hkv][L_cap][d]
  *   SHARED:   k = K'^T [B][Hkv][r][L_cap]   (position contiguous, so r needs no padding)
  *   both:     v = V   [B][Hkv][L_cap][d]
@@ -110,6 +110,27 @@ typedef struct lisa_kvcache_layer {
     void* k;
     void* v;
 } lisa_kvcache_layer;
+
+/* The cache of a whole stack of layers: one lisa_kvcache_layer per layer, all carved out of ONE caller-owned device
+ * buffer (Sec. 5.2: standard layers keep K and V, shared layers K_LR and V; the layers of a model differ only in kind).
+ * lisa_kvcache_total_bytes gives the size of that buffer, lisa_kvcache_init fills in the per-layer descriptors
+ * (host-only: no device work, nothing is cleared); layer l's k and v then live at 256-byte aligned offsets of `base`.
+ * `layers[l]` can be handed to the attention entry points; lisa_kvcache_append_layer is lisa_kvcache_append on layer l. */
+#define LISA_MAX_LAYERS 128
+typedef struct lisa_kvcache_desc {
+    size_t struct_size; /* sizeof(lisa_kvcache_desc) */
+    int32_t n_layers;   /* 1..LISA_MAX_LAYERS */
+    int32_t dtype;      /* lisa_dtype_t */
+    int32_t B, Hkv, L_cap, d;
+    int32_t r;          /* low rank of the shared layers */
+    int32_t reserved;
+    const int32_t* kinds; /* host array [n_layers] of lisa_cache_kind_t */
+} lisa_kvcache_desc;
+typedef struct lisa_kvcache {
+    int32_t n_layers;
+    int32_t reserved;
+    lisa_kvcache_layer layers[LISA_MAX_LAYERS];
+} lisa_kvcache;
 
 /* ------------------------------------------------------------------------------------------------
  * lisa_attn_anchor -- standard causal attention (Eq. 1-2), the layer whose scores a chain starts from.
@@ -233,15 +254,24 @@ lisa_status_t lisa_attn_shared_decode(const lisa_shared_decode_args* args, lisa_
 lisa_status_t lisa_attn_shared_decode_static(const lisa_shared_decode_args* args, lisa_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
- * lisa_kvcache_append -- write n_new new positions into a layer's cache (Sec. 2.2; Sec. 5.2: "store K_LR
- * instead of K").  k_or_kp: [B,n_new,Hkv,d] for a STANDARD layer, [B,n_new,Hkv,r] (K') for a SHARED one,
+ * lisa_kvcache_append -- write n_new new positions into a layer's cache (Sec. 2.2; Sec. 5.2: a shared layer
+ * caches K_LR in place of K).  k_or_kp: [B,n_new,Hkv,d] for a STANDARD layer, [B,n_new,Hkv,r] (K') for a SHARED one,
  * which is stored transposed.  v: [B,n_new,Hkv,d].  Row t of sequence b lands at position
  * seq_lens_before[b] + t (device int32 [B]; NULL = position 0).  Positions that would fall at or beyond
  * L_cap are dropped and counted: lisa_check() then reports LISA_ERR_INVALID_ARG. */
 lisa_status_t lisa_kvcache_append(const lisa_kvcache_layer* layer, const lisa_tensor* k_or_kp, const lisa_tensor* v,
                                   const int32_t* seq_lens_before, int32_t n_new, lisa_stream_t stream);
 
+/* lisa_kvcache_append on layer `layer` of a multi-layer cache (LISA_ERR_INVALID_ARG if there is no such layer). */
+lisa_status_t lisa_kvcache_append_layer(const lisa_kvcache* cache, int32_t layer, const lisa_tensor* k_or_kp, const lisa_tensor* v,
+                                        const int32_t* seq_lens_before, int32_t n_new, lisa_stream_t stream);
+
 /* Host-only helpers (no device work). */
+
+/* Bytes of the one buffer that backs every layer of `desc` (each k and v rounded up to 256 bytes), and the carving of
+ * such a buffer (`base`: device memory, 256-byte aligned, at least that many bytes) into `cache`. */
+lisa_status_t lisa_kvcache_total_bytes(const lisa_kvcache_desc* desc, size_t* bytes);
+lisa_status_t lisa_kvcache_init(const lisa_kvcache_desc* desc, void* base, size_t base_bytes, lisa_kvcache* cache);
 
 /* Bytes of the k and v buffers of a cache layer (fields k, v ignored).  For one SHARED layer with 2-byte
  * elements, k_bytes is smaller than a STANDARD layer's by B*Hkv*L_cap*(d-r)*2, the saving of Sec. 5.2. */
@@ -254,21 +284,6 @@ lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes);
  * append (LISA_ERR_INVALID_ARG) or a bounded wait that ran out (LISA_ERR_TIMEOUT); LISA_ERR_CUDA if the
  * stream itself reports an error. */
 lisa_status_t lisa_check(lisa_stream_t stream);
-
-/* Measurement aid for the tensor-core path of lisa_attn_shared_prefill, which runs as several kernels (pack the
- * low-rank operands, emit score planes, align, attention).  lisa_prefill_phase_timing(1) makes every later call
- * record CUDA events around each of them on the caller's stream (it creates the events; 0 destroys them; not
- * thread-safe, single device); lisa_prefill_phase_times waits for the recorded work and returns the device time
- * in milliseconds summed per phase since the last read: ms4[0] pack, [1] emit, [2] align, [3] attention. */
-lisa_status_t lisa_prefill_phase_timing(int enable);
-lisa_status_t lisa_prefill_phase_times(float* ms4);
-
-/* on != 0: every later call in this process uses the general SIMT kernels even where a tensor-core kernel
- * exists (for cross-checking the two paths against each other); on == 0 restores the default choice. */
-void lisa_force_general_kernels(int on);
-
-/* Number of kernels this library has enqueued so far in this process (all threads). */
-uint64_t lisa_kernel_launches(void);
 
 int lisa_last_cuda_error(void);             /* the cudaError_t of the last LISA_ERR_CUDA on this thread, else 0 */
 const char* lisa_status_string(int status); /* static string */

@@ -25,9 +25,13 @@ CACHE_STANDARD, CACHE_SHARED = 0, 1
 OP_ANCHOR, OP_SHARED_PREFILL, OP_SHARED_DECODE, OP_SHARED_PREFILL_CHAIN = 0, 1, 2, 3
 ACTS = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
 
-EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_chain", "lisa_attn_shared_prefill_host", "lisa_host_arena_bytes",
-           "lisa_attn_shared_decode", "lisa_attn_shared_decode_static", "lisa_kvcache_append", "lisa_kvcache_bytes", "lisa_prefill_phase_times", "lisa_prefill_phase_timing", "lisa_workspace_bytes", "lisa_check",
-           "lisa_force_general_kernels", "lisa_kernel_launches", "lisa_last_cuda_error", "lisa_status_string", "lisa_version"]
+# include/lisa.h (the method's entry points and host helpers) and include/lisa_debug.h (test and measurement hooks)
+EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_chain", "lisa_attn_shared_prefill_host",
+           "lisa_host_arena_bytes", "lisa_attn_shared_decode", "lisa_attn_shared_decode_static", "lisa_kvcache_append",
+           "lisa_kvcache_append_layer", "lisa_kvcache_bytes", "lisa_kvcache_total_bytes", "lisa_kvcache_init",
+           "lisa_workspace_bytes", "lisa_check", "lisa_last_cuda_error", "lisa_status_string", "lisa_version",
+           "lisa_prefill_phase_times", "lisa_prefill_phase_timing", "lisa_force_general_kernels", "lisa_kernel_launches"]
+MAX_LAYERS = 128
 
 
 class LisaError(RuntimeError):
@@ -52,6 +56,15 @@ class CLink(C.Structure):
 class CCacheLayer(C.Structure):
     _fields_ = [("kind", C.c_int32), ("dtype", C.c_int32), ("B", C.c_int32), ("Hkv", C.c_int32), ("L_cap", C.c_int32),
                 ("d", C.c_int32), ("r", C.c_int32), ("reserved", C.c_int32), ("k", C.c_void_p), ("v", C.c_void_p)]
+
+
+class CCacheDesc(C.Structure):
+    _fields_ = [("struct_size", C.c_size_t), ("n_layers", C.c_int32), ("dtype", C.c_int32), ("B", C.c_int32), ("Hkv", C.c_int32),
+                ("L_cap", C.c_int32), ("d", C.c_int32), ("r", C.c_int32), ("reserved", C.c_int32), ("kinds", C.POINTER(C.c_int32))]
+
+
+class CCache(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("reserved", C.c_int32), ("layers", CCacheLayer * MAX_LAYERS)]
 
 
 class AnchorArgs(C.Structure):
@@ -108,6 +121,10 @@ def load():
         lib.lisa_kvcache_append.argtypes = [C.POINTER(CCacheLayer), C.POINTER(Tensor), C.POINTER(Tensor), C.c_void_p,
                                             C.c_int32, C.c_void_p]
         lib.lisa_kvcache_bytes.argtypes = [C.POINTER(CCacheLayer), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+        lib.lisa_kvcache_total_bytes.argtypes = [C.POINTER(CCacheDesc), C.POINTER(C.c_size_t)]
+        lib.lisa_kvcache_init.argtypes = [C.POINTER(CCacheDesc), C.c_void_p, C.c_size_t, C.POINTER(CCache)]
+        lib.lisa_kvcache_append_layer.argtypes = [C.POINTER(CCache), C.c_int32, C.POINTER(Tensor), C.POINTER(Tensor), C.c_void_p,
+                                                  C.c_int32, C.c_void_p]
         lib.lisa_workspace_bytes.argtypes = [C.c_int32, C.c_void_p, C.POINTER(C.c_size_t)]
         lib.lisa_check.argtypes = [C.c_void_p]
         lib.lisa_kernel_launches.restype = C.c_uint64
@@ -182,6 +199,50 @@ class KVCacheLayer:
         assert self.k.numel() * es == kb.value and self.v.numel() * es == vb.value
         desc.k, desc.v = self.k.data_ptr(), self.v.data_ptr()
         self.desc = desc
+
+
+class _LayerView:
+    """A layer of a KVCache, with the attributes the attention wrappers read from a KVCacheLayer."""
+
+    def __init__(self, owner, index, desc, k, v):
+        self.owner, self.index, self.desc, self.k, self.v = owner, index, desc, k, v
+        self.kind, self.B, self.Hkv, self.L_cap, self.d, self.r = desc.kind, desc.B, desc.Hkv, desc.L_cap, desc.d, desc.r
+
+
+class KVCache:
+    """The caches of a stack of layers in ONE torch buffer, carved by lisa_kvcache_init; kinds[l] is CACHE_STANDARD or
+    CACHE_SHARED.  layer(l) is accepted wherever a KVCacheLayer is; append(l, ...) is lisa_kvcache_append_layer."""
+
+    def __init__(self, kinds: Sequence[int], B: int, Hkv: int, L_cap: int, d: int, r: int = 0, dtype=torch.bfloat16, device="cuda"):
+        self.kinds = (C.c_int32 * len(kinds))(*kinds)
+        self.cdesc = CCacheDesc(C.sizeof(CCacheDesc), len(kinds), BF16 if dtype == torch.bfloat16 else F32, B, Hkv, L_cap, d, r, 0,
+                                C.cast(self.kinds, C.POINTER(C.c_int32)))
+        n = C.c_size_t()
+        _check(load().lisa_kvcache_total_bytes(C.byref(self.cdesc), C.byref(n)), "lisa_kvcache_total_bytes")
+        self.buffer = torch.zeros(n.value, dtype=torch.uint8, device=device)
+        self.c = CCache()
+        _check(load().lisa_kvcache_init(C.byref(self.cdesc), self.buffer.data_ptr(), n.value, C.byref(self.c)), "lisa_kvcache_init")
+        es = 2 if dtype == torch.bfloat16 else 4
+        self.layers = []
+        for l, kind in enumerate(kinds):
+            desc = self.c.layers[l]
+            kshape = (B, Hkv, r, L_cap) if kind == CACHE_SHARED else (B, Hkv, L_cap, d)
+            views = []
+            for ptr, shape in ((desc.k, kshape), (desc.v, (B, Hkv, L_cap, d))):
+                off = ptr - self.buffer.data_ptr()
+                numel = 1
+                for x in shape:
+                    numel *= x
+                views.append(self.buffer[off:off + numel * es].view(dtype).view(shape))
+            self.layers.append(_LayerView(self, l, desc, views[0], views[1]))
+
+    def layer(self, l: int) -> "_LayerView":
+        return self.layers[l]
+
+    def append(self, l: int, k_or_kp: torch.Tensor, v: torch.Tensor, seq_lens_before: Optional[torch.Tensor] = None):
+        kt, vt = _tensor4(k_or_kp), _tensor4(v)
+        _check(load().lisa_kvcache_append_layer(C.byref(self.c), int(l), C.byref(kt), C.byref(vt), _ptr(seq_lens_before),
+                                                int(v.shape[1]), _stream()), "lisa_kvcache_append_layer")
 
 
 def lisa_kvcache_bytes(kind: int, B: int, Hkv: int, L_cap: int, d: int, r: int = 0, dtype: int = BF16):

@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "lisa.h"
+#include "lisa_debug.h"
 
 namespace lisa {
 
@@ -56,6 +57,9 @@ __device__ __forceinline__ float act_apply(float x, int act) {
 // Host function; returns the device address to hand to kernels, or nullptr if the lookup failed.
 int* status_words();
 
+// Streaming multiprocessors of the current device (cached per device; 1 if the query fails).
+int sm_count();
+
 // Adds n to the process-wide count of kernels enqueued by the library.
 void count_launches(int n);
 
@@ -65,6 +69,7 @@ cudaError_t launch_generic_prefill(const lisa_shared_prefill_args& a, cudaStream
 cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cudaStream_t s);
 cudaError_t launch_anchor_decode(const lisa_anchor_args& a, void* ws, cudaStream_t s);
 size_t decode_workspace(int B, int Hq, int d, int L);
+size_t shared_decode_smem(int Hq, int m, int integrate);   // dynamic shared memory the shared-layer decode kernel asks for
 
 // Tensor-core flash kernel (head width 128, bf16): O = softmax_causal(QA.KA^T * scale [+ plane]) . V for query tiles
 // [qt_begin, qt_begin + qt_count).  qa [B,N,Hq,kd], ka [B,N,Hkv,kd] with kd in {64,128}; plane (optional) holds

@@ -220,7 +220,7 @@ template <int HQ_C, int M_C>
 __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(16) float smem[];
     const int b = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x;
-    const int L = p.seq_lens ? p.seq_lens[b] : p.L_uniform;
+    const int L = p.seq_lens ? min(p.seq_lens[b], p.L_uniform) : p.L_uniform;   // never beyond the chunks the launch covers
     const int j0 = chunk * kChunk;
     if (j0 >= L) return;
     const int nrows = min(kChunk, L - j0);
@@ -230,8 +230,7 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
     const int h_in = p.integrate == LISA_INTEGRATE_CONCAT ? 2 * Hq : Hq;
 
     float* s_s = smem;                      // [Hq][kChunk]  delta, then scores, then exp
-    float* part_s = s_s + Hq * kChunk;      // [Hq][kChunk]  partial FFN output of the upper half
-    float* qp_s = part_s + Hq * kChunk;     // [Hq][kMaxRank]
+    float* qp_s = s_s + Hq * kChunk;        // [Hq][kMaxRank]
     // weight rows are padded in the tensor-core path (strides m + 8 and Hq + 4) so that the fragment loads of a
     // warp spread over all shared-memory banks
     const int w1_ld = HQ_C ? m + 8 : m, w2_ld = HQ_C ? Hq + 4 : Hq;
@@ -306,7 +305,7 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
         // after bias and activation, ARE the A fragments of layer 2 when hidden unit 8j + 2t / 8j + 2t + 1 is taken
         // as k-index t / t + 4 of k-step j (the order of the hidden units inside the sum is free), so nothing moves
         // between lanes.  bf16 weights are exact in tf32; the fp32 score row is rounded to tf32 (2^-11 relative).
-        constexpr int KS1 = HQ_C / 8, NT1 = M_C / 8, KS2 = M_C / 8, NT2 = HQ_C / 8;
+        constexpr int KS1 = HQ_C / 8, NT1 = M_C / 8, NT2 = HQ_C / 8;   // the second layer has NT1 k-steps
         const int lane = tid & 31, warp = tid >> 5;
         const int g = lane >> 2, t = lane & 3;
         const int p0 = warp * 16 + g, p1 = p0 + 8;              // this lane's two position rows
@@ -486,7 +485,7 @@ __device__ __forceinline__ void anchor_qk_full_chunk(const DecodeParams& p, floa
 __global__ void __launch_bounds__(kThreads, 2) anchor_decode_chunk_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(16) float smem[];
     const int b = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int L = p.seq_lens ? p.seq_lens[b] : p.L_uniform;
+    const int L = p.seq_lens ? min(p.seq_lens[b], p.L_uniform) : p.L_uniform;   // never beyond the chunks the launch covers
     const int j0 = chunk * kChunk;
     if (j0 >= L) return;
     const int nrows = min(kChunk, L - j0);
@@ -561,7 +560,7 @@ __global__ void __launch_bounds__(kThreads, 2) anchor_decode_chunk_kernel(const 
 __global__ void decode_merge_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ float s_w[];   // per chunk: exp(m_c - M) / sum, the weight of the chunk's partial output
     const int h = blockIdx.x, b = blockIdx.y, x = threadIdx.x;
-    const int L = p.seq_lens ? p.seq_lens[b] : p.L_uniform;
+    const int L = p.seq_lens ? min(p.seq_lens[b], p.L_uniform) : p.L_uniform;   // never beyond the chunks the launch covers
     const int nc = (L + kChunk - 1) / kChunk;
     const size_t base = (size_t)b * p.n_chunks * p.Hq + h;
     if (x < 32) {
@@ -610,6 +609,14 @@ cudaError_t set_smem(K kernel, size_t smem) {
 
 }  // namespace
 
+// Dynamic shared memory of the shared-layer chunk kernel: scores [Hq][kChunk], q' [Hq][kMaxRank], W1 and W2 (rows padded
+// by 8 and 4 floats on the tensor-core path; the same bound is used for every path), b1, b2.
+size_t shared_decode_smem(int Hq, int m_link, int integrate) {
+    const int h_in = integrate == LISA_INTEGRATE_CONCAT ? 2 * Hq : Hq;
+    const int m = integrate == LISA_INTEGRATE_PLUS ? 0 : m_link;
+    return sizeof(float) * ((size_t)Hq * kChunk + (size_t)Hq * kMaxRank + (size_t)h_in * (m + 8) + (size_t)m * (Hq + 4) + m + Hq + 8);
+}
+
 size_t decode_workspace(int B, int Hq, int d, int L) {
     const size_t nc = (size_t)(L + kChunk - 1) / kChunk;
     const size_t n = (size_t)B * nc * Hq;
@@ -633,10 +640,7 @@ cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cud
     p.out_scores = a.out_scores; p.sc_sb = a.scores_stride_b; p.sc_sh = a.scores_stride_h;
     p.o = make_view(a.o);
     carve_workspace(p, ws);
-    const int h_in = p.integrate == LISA_INTEGRATE_CONCAT ? 2 * p.Hq : p.Hq;
-    const int m = p.integrate == LISA_INTEGRATE_PLUS ? 0 : p.m;
-    const size_t smem = sizeof(float) * ((size_t)2 * p.Hq * kChunk + (size_t)p.Hq * kMaxRank + (size_t)h_in * m +
-                                         (size_t)m * p.Hq + m + p.Hq + 8 + (size_t)h_in * 8 + (size_t)m * 4);
+    const size_t smem = shared_decode_smem(p.Hq, p.m, p.integrate);
     dim3 grid(p.n_chunks, p.B);
     const bool fast = p.integrate == LISA_INTEGRATE_ADD && p.ffn_layers == 2 && c.dtype == LISA_BF16;
     cudaError_t e;

@@ -76,7 +76,7 @@ cudaError_t launch_kvcache_append(const lisa_kvcache_layer& c, const lisa_tensor
     if (!p.status) return cudaErrorUnknown;
     const int threads = 256;
     const int64_t rows = (int64_t)c.B * n_new * c.Hkv;
-    auto blocks_for = [&](int64_t n) { return (int)std::max<int64_t>(1, std::min<int64_t>((n + threads - 1) / threads, 148 * 16)); };
+    auto blocks_for = [&](int64_t n) { return (int)std::max<int64_t>(1, std::min<int64_t>((n + threads - 1) / threads, sm_count() * 16)); };
     if (c.dtype == LISA_BF16) append_kernel<uint4, 8, __nv_bfloat16><<<dim3(blocks_for(rows * (c.d / 8)), 2), threads, 0, s>>>(p);
     else append_kernel<float4, 4, float><<<dim3(blocks_for(rows * (c.d / 4)), 2), threads, 0, s>>>(p);
     count_launches(1);

@@ -26,6 +26,18 @@ int* status_words() {
     return cached[dev];
 }
 
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 1;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 namespace {
 
 lisa_status_t cuda_fail(cudaError_t e) {
@@ -80,6 +92,17 @@ lisa_status_t check_cache(const lisa_kvcache_layer* c, int kind, bool need_ptrs)
     return LISA_OK;
 }
 
+// Largest dynamic shared memory a CTA may opt into on the current device (B200: 227 KB, also the answer when the
+// query fails, e.g. with no device present).
+size_t max_optin_smem() {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess || v <= 0) {
+        (void)cudaGetLastError();
+        return 232448;
+    }
+    return (size_t)v;
+}
+
 lisa_status_t check_workspace(const void* ws, size_t have, size_t need) {
     if (need == 0) return LISA_OK;
     if (!ws || have < need || !aligned16(ws)) return LISA_ERR_WORKSPACE;
@@ -123,6 +146,8 @@ lisa_status_t validate_shared_decode(const lisa_shared_decode_args* a) {
     if (!a->prev_scores || (reinterpret_cast<uintptr_t>(a->prev_scores) & 3u)) return LISA_ERR_INVALID_ARG;
     if (a->out_scores && a->out_scores == a->prev_scores) return LISA_ERR_INVALID_ARG;
     if ((st = check_tensor(a->o)) != LISA_OK) return st;
+    // a head count and FFN width whose weights do not fit one CTA's shared memory are outside the kernel's range
+    if (shared_decode_smem(a->Hq, a->link.m, a->link.integrate) > max_optin_smem()) return LISA_ERR_UNSUPPORTED;
     return LISA_OK;
 }
 
@@ -299,17 +324,15 @@ lisa_status_t lisa_attn_shared_decode(const lisa_shared_decode_args* a, lisa_str
 // a host-side handle: kernels get the device address that cudaGetSymbolAddress returns for the current device.
 static __device__ __align__(256) unsigned char g_static_scratch[LISA_STATIC_SCRATCH_BYTES];
 
-static void* static_scratch_address() {
+// Device address of the array on the current device (looked up once per device); on failure *err holds the CUDA code.
+static void* static_scratch_address(cudaError_t* err) {
     static void* cached[64] = {nullptr};
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if ((*err = cudaGetDevice(&dev)) != cudaSuccess) return nullptr;
+    if (dev < 0 || dev >= 64) { *err = cudaErrorInvalidDevice; return nullptr; }
     if (!cached[dev]) {
         void* p = nullptr;
-        cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
-        if (e != cudaSuccess) {
-            t_last_cuda_error = (int)e;
-            return nullptr;
-        }
+        if ((*err = cudaGetSymbolAddress(&p, g_static_scratch)) != cudaSuccess) return nullptr;
         cached[dev] = p;
     }
     return cached[dev];
@@ -320,8 +343,9 @@ lisa_status_t lisa_attn_shared_decode_static(const lisa_shared_decode_args* a, l
     if (st != LISA_OK) return st;
     const size_t need = decode_workspace(a->B, a->Hq, a->cache->d, a->L);
     if (need > (size_t)LISA_STATIC_SCRATCH_BYTES) return LISA_ERR_WORKSPACE;
-    void* scratch = static_scratch_address();
-    if (!scratch) return LISA_ERR_CUDA;
+    cudaError_t lookup = cudaSuccess;
+    void* scratch = static_scratch_address(&lookup);
+    if (!scratch) return cuda_fail(lookup);
     cudaError_t e = launch_shared_decode(*a, scratch, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? LISA_OK : cuda_fail(e);
 }
@@ -339,6 +363,50 @@ lisa_status_t lisa_kvcache_append(const lisa_kvcache_layer* layer, const lisa_te
     if (layer->kind == LISA_CACHE_STANDARD && !rows_ok(*k_or_kp)) return LISA_ERR_INVALID_ARG;
     cudaError_t e = launch_kvcache_append(*layer, *k_or_kp, *v, seq_lens_before, n_new, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+}
+
+namespace {
+// Walks the layers of a multi-layer cache: per-layer descriptor and 256-byte aligned offsets of k and v.
+lisa_status_t walk_cache(const lisa_kvcache_desc* d, char* base, lisa_kvcache* out, size_t* total) {
+    if (!d || d->struct_size != sizeof(lisa_kvcache_desc) || !d->kinds) return LISA_ERR_INVALID_ARG;
+    if (d->n_layers < 1 || d->n_layers > LISA_MAX_LAYERS) return LISA_ERR_INVALID_ARG;
+    size_t off = 0;
+    for (int l = 0; l < d->n_layers; ++l) {
+        lisa_kvcache_layer layer{d->kinds[l], d->dtype, d->B, d->Hkv, d->L_cap, d->d, d->kinds[l] == LISA_CACHE_SHARED ? d->r : 0, 0, nullptr, nullptr};
+        if (layer.kind != LISA_CACHE_STANDARD && layer.kind != LISA_CACHE_SHARED) return LISA_ERR_INVALID_ARG;
+        size_t kb = 0, vb = 0;
+        lisa_status_t st = lisa_kvcache_bytes(&layer, &kb, &vb);
+        if (st != LISA_OK) return st;
+        if (base) { layer.k = base + off; }
+        off += (kb + 255) & ~(size_t)255;
+        if (base) { layer.v = base + off; }
+        off += (vb + 255) & ~(size_t)255;
+        if (out) out->layers[l] = layer;
+    }
+    if (out) { out->n_layers = d->n_layers; out->reserved = 0; }
+    if (total) *total = off;
+    return LISA_OK;
+}
+}  // namespace
+
+lisa_status_t lisa_kvcache_total_bytes(const lisa_kvcache_desc* desc, size_t* bytes) {
+    if (!bytes) return LISA_ERR_INVALID_ARG;
+    return walk_cache(desc, nullptr, nullptr, bytes);
+}
+
+lisa_status_t lisa_kvcache_init(const lisa_kvcache_desc* desc, void* base, size_t base_bytes, lisa_kvcache* cache) {
+    if (!cache || !base || (reinterpret_cast<uintptr_t>(base) & 255u)) return LISA_ERR_INVALID_ARG;
+    size_t need = 0;
+    lisa_status_t st = walk_cache(desc, nullptr, nullptr, &need);
+    if (st != LISA_OK) return st;
+    if (base_bytes < need) return LISA_ERR_WORKSPACE;
+    return walk_cache(desc, static_cast<char*>(base), cache, nullptr);
+}
+
+lisa_status_t lisa_kvcache_append_layer(const lisa_kvcache* cache, int32_t layer, const lisa_tensor* k_or_kp, const lisa_tensor* v,
+                                        const int32_t* seq_lens_before, int32_t n_new, lisa_stream_t stream) {
+    if (!cache || layer < 0 || layer >= cache->n_layers || cache->n_layers > LISA_MAX_LAYERS) return LISA_ERR_INVALID_ARG;
+    return lisa_kvcache_append(&cache->layers[layer], k_or_kp, v, seq_lens_before, n_new, stream);
 }
 
 lisa_status_t lisa_prefill_phase_timing(int enable) {
@@ -445,12 +513,27 @@ lisa_status_t validate_host_args(const lisa_shared_prefill_args* a) {
 }
 }  // namespace
 
+namespace {
+// Scratch bytes of the staged call.  The host descriptors' strides are ignored by contract, so the question is put
+// to the dense device-side descriptors the call will actually run with (laid out from a 256-byte aligned dummy base:
+// only strides and alignment matter to the answer, the pointers are not read).
+lisa_status_t staged_workspace_bytes(const lisa_shared_prefill_args& h, size_t* ws) {
+    lisa_shared_prefill_args dev = h;
+    lisa_link dlinks[kMaxChain];
+    Copy copies[3 + 6 * kMaxChain];
+    int nc = 0;
+    plan_host_call(h, reinterpret_cast<char*>(uintptr_t(1) << 20), &dev, dlinks, copies, &nc, nullptr);
+    dev.links = dlinks;
+    return lisa_workspace_bytes(LISA_OP_SHARED_PREFILL, &dev, ws);
+}
+}  // namespace
+
 lisa_status_t lisa_host_arena_bytes(const lisa_shared_prefill_args* host_args, size_t* bytes) {
     if (!bytes) return LISA_ERR_INVALID_ARG;
     lisa_status_t st = validate_host_args(host_args);
     if (st != LISA_OK) return st;
     size_t ws = 0;
-    if ((st = lisa_workspace_bytes(LISA_OP_SHARED_PREFILL, host_args, &ws)) != LISA_OK) return st;
+    if ((st = staged_workspace_bytes(*host_args, &ws)) != LISA_OK) return st;
     *bytes = plan_host_call(*host_args, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr) + ((ws + 255) & ~(size_t)255);
     return LISA_OK;
 }
@@ -469,10 +552,12 @@ lisa_status_t lisa_attn_shared_prefill_host(const lisa_shared_prefill_args* host
     const size_t used = plan_host_call(*host_args, static_cast<char*>(device_arena), &dev, dlinks, copies, &nc, &o_bytes);
     dev.links = dlinks;
     size_t ws = 0;
-    lisa_workspace_bytes(LISA_OP_SHARED_PREFILL, host_args, &ws);
+    if ((st = lisa_workspace_bytes(LISA_OP_SHARED_PREFILL, &dev, &ws)) != LISA_OK) return st;
     dev.workspace = ws ? static_cast<char*>(device_arena) + used : nullptr;
     dev.workspace_bytes = ws;
+    // everything that can refuse the call is checked before the first copy is enqueued
     if ((st = validate_prefill(&dev)) != LISA_OK) return st;
+    if (used + ((ws + 255) & ~(size_t)255) > arena_bytes) return LISA_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     for (int i = 0; i < nc; ++i)

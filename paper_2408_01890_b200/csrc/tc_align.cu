@@ -25,21 +25,18 @@
 // position and head for one link), not by its arithmetic.
 #include <algorithm>
 
-#include "common.cuh"
-#include "tc_common.cuh"
+#include "tc_align_mma.cuh"
 
 namespace lisa {
 namespace {
 
 using namespace tc;
+using namespace alignmma;
 
-constexpr int HQ = 32, MH = 64, UNIT = 128;
+constexpr int UNIT = 128;
 constexpr int kWorkers = 512, kStages = 2;                        // weights read from shared memory: one 16-warp CTA per SM
 constexpr int kRegwThreads = 128, kRegwCtas = 3, kRegwStages = 3, kRegwPiece = 64; // weights held in registers (single link)
-constexpr int W1F_BYTES = 2 * 8 * 32 * 8;     // B fragments of W1: [k-step][n-tile][lane] x (b0, b1)
-constexpr int W2F_BYTES = 4 * 4 * 32 * 8;     // B fragments of W2
-constexpr float kLog2e = 1.4426950408889634f; // the last link's output leaves multiplied by log2(e): the attention
-                                              // kernel that adds it to its logits works in the exp2 domain
+// the last link's output leaves multiplied by log2(e): the attention kernel that adds it to its logits works in the exp2 domain
 constexpr int kMaxTcChain = 3;
 
 struct AlignParams {
@@ -54,107 +51,6 @@ struct AlignParams {
     int* status;
 };
 
-__device__ __forceinline__ float ldw(const void* p, int idx, int dtype) { return p ? ld_elem(p, idx, dtype) : 0.f; }
-
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, uint32_t saddr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr) : "memory");
-}
-__device__ __forceinline__ void stmatrix_x4_trans(uint32_t saddr, const uint32_t* r) {
-    asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1,%2,%3,%4};"
-                 ::"r"(saddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
-}
-// d += a (16x16, row) . b (16x8, col), fp16 in, fp32 accumulate
-__device__ __forceinline__ void mma_f16(float* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// d = a (16x16, row) . b (16x8, col) + c with fp16 accumulators: the two result registers hold rows g and g+8 as
-// packed pairs of columns (2t, 2t+1), which is exactly the A-fragment arrangement of a following MMA.
-__device__ __forceinline__ void mma_f16acc(uint32_t* d, const uint32_t* a, uint32_t b0, uint32_t b1, uint32_t c0, uint32_t c1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f16.f16.f16.f16 {%0,%1}, {%2,%3,%4,%5}, {%6,%7}, {%8,%9};"
-                 : "=r"(d[0]), "=r"(d[1])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(c0), "r"(c1));
-}
-// d = a . b + c, fp32 accumulators, c given separately (a bias pair repeated for both rows)
-__device__ __forceinline__ void mma_f16_bias(float* d, const uint32_t* a, uint32_t b0, uint32_t b1, float c0, float c1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%10,%11};"
-                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(c0), "f"(c1));
-}
-
-// Activation of two hidden units held as a packed fp16 pair; the result is again a packed pair (an A-fragment
-// register of the second layer's MMA).
-template <int ACT>
-__device__ __forceinline__ uint32_t act_h2(uint32_t x) {
-    if constexpr (ACT == LISA_ACT_RELU) {
-        uint32_t r;
-        asm("max.f16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(0u));
-        return r;
-    }
-    if constexpr (ACT == LISA_ACT_SILU) {
-        // x * sigmoid(x) = (x/2) tanh(x/2) + x/2: one packed multiply, one packed tanh, one packed fused multiply-add
-        uint32_t hx, th, r;
-        asm("mul.f16x2 %0, %1, %2;" : "=r"(hx) : "r"(x), "r"(0x38003800u));   // 0.5, 0.5
-        asm("tanh.approx.f16x2 %0, %1;" : "=r"(th) : "r"(hx));
-        asm("fma.rn.f16x2 %0, %1, %2, %1;" : "=r"(r) : "r"(hx), "r"(th));
-        return r;
-    }
-    return x;
-}
-
-// One link on a warp's 16 positions: afr = A fragments (2 k-steps of 16 heads) -> y = W2^T act(W1^T a + b1) + b2
-// as four accumulator tiles of 8 heads.  The first layer accumulates in fp16 (32 products per hidden unit, the
-// result is rounded to fp16 for the second layer's operand in any case): its accumulator registers ARE the second
-// layer's A fragments, so the activation is one to three packed instructions per register and nothing is converted
-// or repacked.  The second layer accumulates in fp32.  b1h holds b1 as packed fp16 pairs, b2 is fp32.
-// The fragments of W1 and W2 come either from shared memory (w1f/w2f, one 8-byte load per MMA) or, when REGW, from
-// the register copies w1r/w2r that a warp keeps for its whole life (single-link calls).
-// `side` is called once, after the first layer's MMAs have been issued: unrelated instructions placed there (the copies
-// of neighbouring pieces) issue while this warp's MMAs wait for their turn on the tensor pipe.
-// BIAS = false: b1 and b2 are known to be absent (zero accumulator start, nothing loaded).
-template <int ACT, bool REGW, bool BIAS = true, typename Side>
-__device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* w1f, const uint2* w2f, const uint2* w1r, const uint2* w2r,
-                                         const uint32_t* b1h, const float* b2, int lane, float (*y)[4], Side side) {
-    const int t = lane & 3;
-    uint32_t h[8][2];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const uint32_t bb = BIAS ? b1h[j * 4 + t] : 0u;
-        const uint2 w = REGW ? w1r[j] : w1f[j * 32 + lane];
-        mma_f16acc(h[j], afr[0], w.x, w.y, bb, bb);
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const uint2 w = REGW ? w1r[8 + j] : w1f[(8 + j) * 32 + lane];
-        mma_f16acc(h[j], afr[1], w.x, w.y, h[j][0], h[j][1]);
-    }
-    side();
-    uint32_t hfr[4][4];
-#pragma unroll
-    for (int s = 0; s < 4; ++s) {
-        hfr[s][0] = act_h2<ACT>(h[2 * s][0]);
-        hfr[s][1] = act_h2<ACT>(h[2 * s][1]);
-        hfr[s][2] = act_h2<ACT>(h[2 * s + 1][0]);
-        hfr[s][3] = act_h2<ACT>(h[2 * s + 1][1]);
-    }
-#pragma unroll
-    for (int j2 = 0; j2 < 4; ++j2) {
-        const float2 bb = BIAS ? *reinterpret_cast<const float2*>(b2 + j2 * 8 + 2 * t) : make_float2(0.f, 0.f);
-        const uint2 w = REGW ? w2r[j2] : w2f[j2 * 32 + lane];
-        mma_f16_bias(y[j2], hfr[0], w.x, w.y, bb.x, bb.y);
-    }
-#pragma unroll
-    for (int s = 1; s < 4; ++s)
-#pragma unroll
-        for (int j2 = 0; j2 < 4; ++j2) {
-            const uint2 w = REGW ? w2r[s * 4 + j2] : w2f[(s * 4 + j2) * 32 + lane];
-            mma_f16(y[j2], hfr[s], w.x, w.y);
-        }
-}
-
 // Each warp works alone on pieces of 32 key positions of one query row: no block-wide barrier, no producer warp.
 //   global -> scratch    cp.async, 16 bytes per lane, four lanes per head (64 contiguous bytes), one piece ahead
 //   scratch -> fragments ldmatrix.trans per 16-position strip
@@ -167,39 +63,16 @@ __global__ void __launch_bounds__(NT, MIN_CTAS)
 tc_align_kernel(const __grid_constant__ AlignParams p) {
     extern __shared__ __align__(16) uint8_t smem[];
     const int c = p.chain;
-    constexpr int LINK_BYTES = W1F_BYTES + W2F_BYTES + (MH + HQ) * 4;
     uint8_t* sW = smem;                               // per link: W1 fragments, W2 fragments, b1[64], b2[32]
     uint8_t* sScr = sW + c * LINK_BYTES;              // per warp: STAGES buffers of c planes x [32 heads][64 B]
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // ---- one-time set-up: weights as ready-made B fragments (fp16, the last link's W2/b2 times log2 e) ----
     for (int k = 0; k < c; ++k) {
-        uint2* w1f = reinterpret_cast<uint2*>(sW + k * LINK_BYTES);
-        uint2* w2f = reinterpret_cast<uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
-        float* bias = reinterpret_cast<float*>(sW + k * LINK_BYTES + W1F_BYTES + W2F_BYTES);
         // the last link's log2(e) is folded into its W2 and b2, except where every link's output leaves (store_all with
         // more than one link): there the stored values are scaled instead and the chain continues unscaled
         const float out_scale = (k == c - 1 && (!p.store_all || c == 1)) ? kLog2e : 1.f;
-        const int wd = p.w_dtype[k];
-        for (int e = tid; e < 2 * 8 * 32; e += NT) {   // W1 [32 heads][64 hidden]: k = head, n = hidden
-            const int ln = e & 31, j = (e >> 5) & 7, ks = e >> 8, g = ln >> 2, t = ln & 3;
-            const int k0 = ks * 16 + 2 * t, n = j * 8 + g;
-            uint2 w;
-            w.x = pack_f16(ld_elem(p.w1[k], k0 * MH + n, wd), ld_elem(p.w1[k], (k0 + 1) * MH + n, wd));
-            w.y = pack_f16(ld_elem(p.w1[k], (k0 + 8) * MH + n, wd), ld_elem(p.w1[k], (k0 + 9) * MH + n, wd));
-            w1f[e] = w;
-        }
-        for (int e = tid; e < 4 * 4 * 32; e += NT) {   // W2 [64 hidden][32 heads]: k = hidden, n = head
-            const int ln = e & 31, j2 = (e >> 5) & 3, s2 = e >> 7, g = ln >> 2, t = ln & 3;
-            const int k0 = s2 * 16 + 2 * t, n = j2 * 8 + g;
-            uint2 w;
-            w.x = pack_f16(ld_elem(p.w2[k], k0 * HQ + n, wd) * out_scale, ld_elem(p.w2[k], (k0 + 1) * HQ + n, wd) * out_scale);
-            w.y = pack_f16(ld_elem(p.w2[k], (k0 + 8) * HQ + n, wd) * out_scale, ld_elem(p.w2[k], (k0 + 9) * HQ + n, wd) * out_scale);
-            w2f[e] = w;
-        }
-        for (int e = tid; e < MH / 2; e += NT)   // b1 as packed fp16 pairs (the first layer's accumulator format)
-            reinterpret_cast<uint32_t*>(bias)[e] = pack_f16(ldw(p.b1[k], 2 * e, wd), ldw(p.b1[k], 2 * e + 1, wd));
-        for (int e = tid; e < HQ; e += NT) bias[MH + e] = ldw(p.b2[k], e, wd) * out_scale;
+        stage_link_fragments(sW + k * LINK_BYTES, p.w1[k], p.b1[k], p.w2[k], p.b2[k], p.w_dtype[k], out_scale, tid, NT);
     }
     __syncthreads();
 
@@ -528,7 +401,10 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
     const int64_t total_units = (int64_t)p.units_per_batch * a.B;
     if (total_units <= 0 || total_units > 0x7fffffff) return cudaErrorInvalidValue;
-    const int max_ctas = a.ctas > 0 ? a.ctas : 148 * ctas_per_sm;
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const int max_ctas = a.ctas > 0 ? a.ctas : sms * ctas_per_sm;
     dim3 grid((unsigned)std::min<int64_t>((total_units + 3) / 4, max_ctas));  // at least a unit per warp
     kernel<<<grid, threads, smem, stream>>>(p);
     count_launches(1);

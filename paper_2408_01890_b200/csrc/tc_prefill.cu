@@ -19,12 +19,12 @@ namespace {
 constexpr int kTile = 128;
 constexpr int kPadRank = 64;
 constexpr int kMaxPackLinks = 4;   // links whose Q', K' one call packs (the aligner takes chains of up to three)
-// A wave takes query tiles until its head-partitioned kernels have at least kWaveMinCtas CTAs (four per SM: with
+// A wave takes query tiles until its head-partitioned kernels have at least kWaveCtasPerSm CTAs per SM (with
 // fewer, the grids do not fill the GPU and launch and tail costs dominate) and then further tiles while the causal
 // part of its score planes stays within kWaveBytes.  Measured on B200: grid fill matters far more than keeping
 // the planes inside the 126 MB L2.
 constexpr size_t kWaveBytes = (size_t)256 << 20;
-constexpr int kWaveMinCtas = 4 * 148;
+constexpr int kWaveCtasPerSm = 4;
 
 // Every Q' and K' of a call is packed by one launch: blockIdx.y selects the tensor.
 struct PackJobs {
@@ -84,13 +84,14 @@ struct PhaseMark {
 struct Wave { int begin, count; };
 
 int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves) {
+    const int min_ctas = kWaveCtasPerSm * sm_count();
     const int n_qt = (N + kTile - 1) / kTile;
     const size_t per_col_tile = (size_t)B * Hq * kTile * kTile * 2 * c;
     int n = 0, qt = 0;
     while (qt < n_qt) {
         size_t bytes = 0;
         int cnt = 0;
-        while (qt + cnt < n_qt && (B * Hq * cnt < kWaveMinCtas || bytes + per_col_tile * (qt + cnt + 1) <= kWaveBytes)) {
+        while (qt + cnt < n_qt && (B * Hq * cnt < min_ctas || bytes + per_col_tile * (qt + cnt + 1) <= kWaveBytes)) {
             bytes += per_col_tile * (qt + cnt + 1);
             ++cnt;
         }
@@ -137,7 +138,7 @@ cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int
     PackJobs jobs{};
     jobs.src[0] = make_view(src); jobs.dst[0] = reinterpret_cast<__nv_bfloat16*>(dst); jobs.H[0] = H; jobs.r[0] = r;
     const int64_t total = (int64_t)B * H * N * (kPadRank / 8);
-    const int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 32);
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, sm_count() * 32);
     pack_lowrank_kernel<<<dim3(blocks, 1), 256, 0, s>>>(jobs, B, N);
     count_launches(1);
     return cudaGetLastError();
@@ -208,7 +209,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             jobs.H[2 * k + 1] = a.Hkv; jobs.r[2 * k + 1] = a.links[k].r;
         }
         const int64_t total = (int64_t)a.B * a.Hq * a.N * (kPadRank / 8);
-        const int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 16);
+        const int blocks = (int)std::min<int64_t>((total + 255) / 256, sm_count() * 16);
         // beside the first emit, unless the per-kernel timing is on (then every kernel is timed on the caller's stream)
         if (!g_pt.on) {
             std::lock_guard<std::mutex> lock(g_side_mutex);

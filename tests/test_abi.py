@@ -19,10 +19,15 @@ def lib():
     return lb.load()
 
 
-def declared_functions():
-    text = open(os.path.join(ROOT, "include", "lisa.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(lisa_[a-z_0-9]+)\s*\(", text)))
+def declared_functions(header=None):
+    """Function names declared in include/<header> (comments stripped); every header when none is named."""
+    headers = [header] if header else sorted(f for f in os.listdir(os.path.join(ROOT, "include")) if f.endswith(".h"))
+    names = set()
+    for h in headers:
+        text = open(os.path.join(ROOT, "include", h)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names.update(re.findall(r"\b(lisa_[a-z_0-9]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_exports_every_declared_symbol(lib):
@@ -31,7 +36,12 @@ def test_library_exports_every_declared_symbol(lib):
     assert "lisa_attn_shared_decode" in names and "lisa_kvcache_append" in names
     for n in names:
         assert hasattr(lib, n), "missing export %s" % n
-    assert sorted(lb.EXPORTS) == [n for n in names if n in lb.EXPORTS]
+    assert sorted(lb.EXPORTS) == names, "the binding's export list and the two headers disagree"
+    # the product header carries the method's entry points only; test and measurement hooks live in lisa_debug.h
+    product, debug = declared_functions("lisa.h"), declared_functions("lisa_debug.h")
+    assert not set(product) & set(debug)
+    for hook in ("lisa_force_general_kernels", "lisa_kernel_launches", "lisa_prefill_phase_timing", "lisa_prefill_phase_times"):
+        assert hook in debug and hook not in product
     assert lib.lisa_version() >= 1000
     assert lib.lisa_status_string(0) == b"ok"
 
@@ -117,3 +127,54 @@ def test_decode_workspace_query(lib):
     n = C.c_size_t()
     assert lib.lisa_workspace_bytes(lb.OP_SHARED_DECODE, C.byref(a), C.byref(n)) == lb.OK
     assert n.value >= 64 * 32 * 40 * (128 + 2) * 4 and n.value % 256 == 0
+
+
+def test_multi_layer_cache_is_carved_from_one_buffer(lib):
+    """lisa_kvcache_init (host-only): per-layer descriptors at 256-byte aligned, non-overlapping offsets of one base, sizes as
+    lisa_kvcache_bytes gives them; a shared layer's k region is smaller by the factor d/r (Sec. 5.2)."""
+    kinds = [lb.CACHE_STANDARD, lb.CACHE_SHARED, lb.CACHE_SHARED, lb.CACHE_STANDARD]
+    arr = (C.c_int32 * 4)(*kinds)
+    desc = lb.CCacheDesc(C.sizeof(lb.CCacheDesc), 4, lb.BF16, 2, 8, 64, 128, 21, 0, C.cast(arr, C.POINTER(C.c_int32)))
+    n = C.c_size_t()
+    assert lib.lisa_kvcache_total_bytes(C.byref(desc), C.byref(n)) == lb.OK
+    std_k, v = lb.lisa_kvcache_bytes(lb.CACHE_STANDARD, 2, 8, 64, 128)
+    sh_k, _ = lb.lisa_kvcache_bytes(lb.CACHE_SHARED, 2, 8, 64, 128, 21)
+    up = lambda x: (x + 255) // 256 * 256
+    assert n.value == 2 * (up(std_k) + up(v)) + 2 * (up(sh_k) + up(v))
+    cache = lb.CCache()
+    base = 1 << 30                                     # any 256-byte aligned address: nothing is dereferenced
+    assert lib.lisa_kvcache_init(C.byref(desc), base, n.value - 1, C.byref(cache)) == lb.ERR_WORKSPACE
+    assert lib.lisa_kvcache_init(C.byref(desc), base + 8, n.value, C.byref(cache)) == lb.ERR_INVALID_ARG
+    assert lib.lisa_kvcache_init(C.byref(desc), base, n.value, C.byref(cache)) == lb.OK
+    assert cache.n_layers == 4
+    spans = []
+    for l, kind in enumerate(kinds):
+        layer = cache.layers[l]
+        assert layer.kind == kind and layer.r == (21 if kind == lb.CACHE_SHARED else 0)
+        assert layer.k % 256 == 0 and layer.v % 256 == 0
+        spans += [(layer.k, sh_k if kind == lb.CACHE_SHARED else std_k), (layer.v, v)]
+    for (a, na), (b, nb) in zip(spans, spans[1:]):
+        assert a + na <= b
+    assert spans[0][0] == base and spans[-1][0] + spans[-1][1] <= base + n.value
+    assert lib.lisa_kvcache_append_layer(C.byref(cache), 4, None, None, None, 1, None) == lb.ERR_INVALID_ARG
+    desc.n_layers = 0
+    assert lib.lisa_kvcache_total_bytes(C.byref(desc), C.byref(n)) == lb.ERR_INVALID_ARG
+
+
+def test_host_arena_ignores_host_strides(lib):
+    """The host-memory entry point takes dense host tensors and ignores their strides: the arena it asks for (and with it
+    the workspace of the tensor-core path) must not depend on them."""
+    def arena(strided):
+        t = lambda H, x: lb.Tensor(1 << 20, lb.BF16, 0, (256 * H * x) if strided else 0, (H * x) if strided else 0, x if strided else 0)
+        link = lb.CLink(t(32, 21), t(32, 21), 1 << 20, None, 1 << 20, None, lb.BF16, 21, 64, lb.ACT_RELU, lb.INTEGRATE_ADD, 2)
+        a = lb.SharedPrefillArgs()
+        a.struct_size = C.sizeof(lb.SharedPrefillArgs)
+        a.B, a.N, a.Hq, a.Hkv, a.d, a.chain_len = 1, 256, 32, 32, 128, 1
+        a.q0, a.k0, a.v, a.o = t(32, 128), t(32, 128), t(32, 128), t(32, 128)
+        a.links = C.pointer(link)
+        n = C.c_size_t()
+        assert lib.lisa_host_arena_bytes(C.byref(a), C.byref(n)) == lb.OK
+        return n.value
+    dense, zero = arena(True), arena(False)
+    tensors = 4 * 256 * 32 * 128 * 2
+    assert dense == zero and dense > tensors + (1 << 20)     # inputs + output + a score-plane workspace
