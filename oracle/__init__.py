@@ -202,3 +202,15 @@ def memory_saving(n_shared: int, h: int, l: int, d_k: int, r: int):
     f.argtypes = [ctypes.c_long] * 5 + [ctypes.POINTER(ctypes.c_long)]
     f(n_shared, h, l, d_k, r, out)
     return int(out[0]), int(out[1])
+
+
+def project(x, w):
+    """Eq. 1 / Eq. 3 projections: x [..., d_in] times w [d_in, n_out] (row = input unit). Returns [..., n_out]."""
+    x, w = _f64(x, "x"), _f64(w, "w")
+    d_in, n_out = w.shape
+    rows = int(np.prod(x.shape[:-1]))
+    out = np.empty(x.shape[:-1] + (n_out,), dtype=np.float64)
+    f = _load().oracle_project
+    f.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_long, ctypes.c_long, ctypes.c_long, ctypes.c_void_p]
+    f(_ptr(x), _ptr(w), rows, d_in, n_out, _ptr(out))
+    return out

@@ -21,6 +21,8 @@
  *            before the FFN
  *   Sec. 5.2 decode stage: the previous layer's score row (h x l) is kept and
  *            K_LR replaces K in the cache
+ *   Eq. 1, 3 the projections H W^V_i, H W^Q_LR, H W^K_LR and the product with W^O
+ *            (oracle_project: a plain matrix product)
  *
  * Readings taken where the paper is silent (each is listed in the design
  * document as well): the aligner acts on pre-softmax scores that already carry
@@ -388,4 +390,17 @@ void oracle_memory_saving(long n_shared, long h, long l, long d_k, long r, long*
     const long k_saved = n_shared * h * l * (d_k - r) * 2;
     out[0] = k_saved - h * l * l * 2;
     out[1] = k_saved - h * l * 2;
+}
+
+/* Projection either side of the attention: C[row, col] = sum_k X[row, k] * W[k, col], X [rows, d_in], W [d_in, n_out]
+ * row-major (row = input unit, as the paper writes H W).  Eq. 1: the per-head H W^V_i are column blocks of one such
+ * product and W^O multiplies the concatenated heads; Eq. 3: H W^Q_LR and H W^K_LR.  Plain triple loop, fp64. */
+void oracle_project(const double* X, const double* W, long rows, long d_in, long n_out, double* C) {
+#pragma omp parallel for schedule(static)
+    for (long i = 0; i < rows; ++i)
+        for (long j = 0; j < n_out; ++j) {
+            double acc = 0.0;
+            for (long k = 0; k < d_in; ++k) acc += X[i * d_in + k] * W[k * n_out + j];
+            C[i * n_out + j] = acc;
+        }
 }

@@ -222,6 +222,22 @@ def test_concat_reduces_to_add_free_form():
     np.testing.assert_allclose(A_bot, A_bot2, rtol=0, atol=1e-12)
 
 
+@pytest.mark.parametrize("act,fn", [(ACT_SILU, torch.nn.functional.silu), (ACT_RELU, torch.nn.functional.relu)])
+def test_activation_against_torch(act, fn):
+    """The oracle's activation through link_apply against torch's fp64 silu / relu (a library routine, not the formula
+    retyped): with W1 = I (m = h), W2 = I and zero Q'/K', Eq. 4 (ADD) reduces to A_out = act(A_in + b1) element by element.
+    Values span both signs and the range where SiLU is far from linear."""
+    B, N, Hq = 1, 5, 6
+    A_in = rnd(61, B, Hq, N, N, std=3.0)
+    b1 = rnd(62, Hq)
+    eye = np.eye(Hq)
+    lk = Link(qp=np.zeros((B, N, Hq, 2)), kp=np.zeros((B, N, Hq, 2)), w1=eye, w2=eye, b1=b1, b2=None, r=2, act=act)
+    got = oracle.link_apply(A_in, lk, Hkv=Hq)
+    want = fn(torch.from_numpy(A_in + b1[None, :, None, None])).numpy()
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-13)
+    assert np.abs(want - (A_in + b1[None, :, None, None])).max() > 1.0     # the activation is not the identity on this data
+
+
 def test_rows_mode_equals_full_mode():
     q0, k0, v, links = make_case(31, B=2, N=13, c=3)
     O, A = oracle.prefill_full(q0, k0, v, links, want_scores=True)
@@ -300,3 +316,27 @@ def test_memory_model_closed_forms():
     pre_long, dec_long = oracle.memory_saving(S, h, 4096, dk, r)
     assert pre_long < 0 < dec_long
     assert oracle.memory_saving(S, h, S * (dk - r), dk, r)[0] == 0
+
+
+def test_projection_is_a_plain_matrix_product():
+    """oracle.project against numpy's matmul (a library routine) and a scalar loop, on shapes where every dimension differs
+    (a transposed operand or swapped index fails), and the column blocks of [W_Q | W_K | W_V] against separate products
+    (Eq. 1: the per-head H W^V_i are column blocks; Eq. 3: H W_LR)."""
+    x = rnd(71, 2, 5, 7)
+    w = rnd(72, 7, 11)
+    got = oracle.project(x, w)
+    np.testing.assert_allclose(got, x @ w, rtol=0, atol=1e-13)
+    slow = np.zeros((2, 5, 11))
+    for b in range(2):
+        for n in range(5):
+            for j in range(11):
+                slow[b, n, j] = sum(x[b, n, k] * w[k, j] for k in range(7))
+    np.testing.assert_allclose(got, slow, rtol=0, atol=1e-13)
+    wq, wk, wv = w[:, :3], w[:, 3:5], w[:, 5:]
+    np.testing.assert_allclose(got[..., 3:5], oracle.project(x, np.ascontiguousarray(wk)), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(got[..., 5:], x @ wv, rtol=0, atol=1e-13)
+    # the low-rank difference built from projected operands equals Eq. 3 written out: (H W_Q)(H W_K)^T / sqrt(r)
+    h = rnd(73, 1, 4, 7)
+    q, k = oracle.project(h, np.ascontiguousarray(wq)), oracle.project(h, np.ascontiguousarray(wq))
+    A = oracle.scores(q.reshape(1, 4, 1, 3), k.reshape(1, 4, 1, 3))
+    np.testing.assert_allclose(A[0, 0], (h[0] @ wq) @ (h[0] @ wq).T / math.sqrt(3), rtol=0, atol=1e-12)
