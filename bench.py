@@ -1,11 +1,12 @@
 """Benchmark of the LiSA shared-layer attention hot path on B200.
 
-One step = one pass of the hot path over one batch of seeded synthetic input:
-  prefill step: lisa_attn_shared_prefill (scores chain, mask, softmax, .V) + lisa_kvcache_append (K', V)
-  decode step : lisa_kvcache_append (one token) + lisa_attn_shared_decode (reads the previous layer's
-                score row, writes its own)
-The JSON line's headline is the prefill step on the LLaMA2-7B-shaped workload; the decode step on the
-LLaMA2-13B-shaped workload and the library's own standard-attention decode are reported in "decode".
+One step = one pass of the hot path over one batch of seeded synthetic input.  Headline workload: the
+LLaMA3-8B-shaped grouped-query prefill (B 4, N 8192, 32 query / 8 KV heads, an anchor followed by a chain of three
+shared layers): a step computes the three shared layers, each by its own lisa_attn_shared_prefill call at chain
+depth 1, 2, 3 (score chain, mask, softmax, .V) followed by lisa_kvcache_append of its K', V.  The same three layers
+through one lisa_attn_shared_prefill_chain call are reported beside it ("chain_call"), the LLaMA2-7B-shaped prefill
+under "cfg2", the LLaMA2-13B-shaped decode step and the library's own standard-attention decode under "decode", the
+32-layer stack under "stack".
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 Under torchrun (N > 1) every rank runs the same step on its own batch (weak scaling, no data exchange).
@@ -26,12 +27,17 @@ sys.path.insert(0, ROOT)
 
 from paper_2408_01890_b200 import synth  # noqa: E402
 
-PREFILL = "cfg2_llama2_7b_prefill"
+HEADLINE = "cfg3_llama3_8b_gqa_prefill"
+SECOND = "cfg2_llama2_7b_prefill"
 DECODE = "cfg4_llama2_13b_decode"
 METRIC = "lisa_attention_tokens_per_s"
-# dram bytes (read + write) per launch from the ncu captures summarised under profiles/ (cold cache, same workload);
-# None for a kernel that has changed since its counters were taken
-PREFILL_TRAFFIC = {"align": 142642688 + 83800064, "emit_scores": 40019456 + 85420032, "attention": 186513920 + 6682368}
+# DRAM bytes (read + write) per causal position and head of each prefill kernel, from the ncu captures of the cfg2 launch
+# summarised under profiles/ (cold cache); every kernel streams its planes once, so traffic grows in proportion to
+# the causal positions and the figures are scaled by them for other workloads.  None for a kernel that has changed since.
+CFG2_POSITIONS_HEADS = 2098176 * 32
+PREFILL_TRAFFIC_PER_PH = {"emit_scores": (40019456 + 85420032) / CFG2_POSITIONS_HEADS,
+                          "align": (142642688 + 83800064) / CFG2_POSITIONS_HEADS,
+                          "attention": (186513920 + 6682368) / CFG2_POSITIONS_HEADS}
 DECODE_TRAFFIC_PER_SEQ = (395953152 + 5092608) / 8  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
 
 
@@ -43,11 +49,23 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
 
 
+def positions(w):
+    return w.B * w.N * (w.N + 1) // 2
+
+
+def flops_per_position(w, c):
+    """QK^T + c * (difference + aligner FFN) + P.V of a layer at chain depth c, per causal (query, key) position."""
+    return 2 * w.Hq * w.d + c * (2 * w.Hq * w.r + 4 * w.Hq * w.m) + 2 * w.Hq * w.d
+
+
 def prefill_flops(w, c):
-    """Algorithmic flops of one shared layer at chain depth c: causal positions x (QK^T + c*(delta + FFN) + PV)."""
-    positions = w.B * w.N * (w.N + 1) // 2
-    per_pos = 2 * w.Hq * w.d + c * (2 * w.Hq * w.r + 4 * w.Hq * w.m) + 2 * w.Hq * w.d
-    return positions * per_pos
+    return positions(w) * flops_per_position(w, c)
+
+
+def prefill_algorithmic_bytes(w, c):
+    """What a layer at depth c must read and write: Q0, K0, the Q', K' of its c links, its V and its output."""
+    e = 2
+    return w.B * w.N * e * (w.Hq * w.d + w.Hkv * w.d + c * (w.Hq + w.Hkv) * w.r + w.Hkv * w.d + w.Hq * w.d)
 
 
 def decode_bytes(w, shared=True, B=None):
@@ -97,44 +115,64 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def oracle_links(t, w, c):
+    import oracle
+    act = {"relu": oracle.ACT_RELU, "silu": oracle.ACT_SILU, "none": oracle.ACT_NONE}[w.act]
+    return [oracle.Link(synth.to_f64(t[f"qp{k}"]), synth.to_f64(t[f"kp{k}"]), synth.to_f64(t[f"w1_{k}"]), synth.to_f64(t[f"w2_{k}"]),
+                        r=w.r, act=act) for k in range(1, c + 1)]
 
-def flush_l2(buf):
-    buf.zero_()
+
+def sample_rows(w, n):
+    """n query rows spread evenly over the batch and the prompt (unbiased for the mean row cost, which grows with the row index)."""
+    idx = (np.arange(n, dtype=np.int64) * (w.B * w.N) // n + (w.B * w.N) // (2 * n)) % (w.B * w.N)
+    return (idx % w.B).astype(np.int32), (idx // w.B).astype(np.int32)
 
 
 def run_reference(args, rank):
-    """The CPU oracle as it stands, on the host cores, on a bounded sample of the prefill workload."""
+    """The CPU oracle as it stands, on the host cores, on a bounded sample of the headline workload: per step, a fixed set
+    of query rows through each of the three shared layers."""
     if rank != 0:
         return
     import oracle
-    w = synth.WORKLOADS[PREFILL]
+    w = synth.WORKLOADS[HEADLINE]
     t = synth.prefill_inputs(w, 0)
-    links = [oracle.Link(synth.to_f64(t["qp1"]), synth.to_f64(t["kp1"]), synth.to_f64(t["w1_1"]), synth.to_f64(t["w2_1"]),
-                         r=w.r, act=oracle.ACT_SILU)]
-    q0, k0, v = synth.to_f64(t["q0"]), synth.to_f64(t["k0"]), synth.to_f64(t["v1"])
-    rows = np.arange(3, w.N, 8, dtype=np.int32)  # 256 evenly spaced query rows: unbiased for the mean row cost
-    rb = np.zeros_like(rows)
+    q0, k0 = synth.to_f64(t["q0"]), synth.to_f64(t["k0"])
+    links = oracle_links(t, w, w.chain)
+    vs = [synth.to_f64(t[f"v{c}"]) for c in range(1, w.chain + 1)]
+    n = 48
+    rb, ri = sample_rows(w, n)
+
+    def step():
+        for c in range(1, w.chain + 1):
+            oracle.prefill_rows(q0, k0, vs[c - 1], links[:c], rb, ri)
+
     for _ in range(args.warmup):
-        oracle.prefill_rows(q0, k0, v, links, rb, rows)
+        step()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.prefill_rows(q0, k0, v, links, rb, rows)
+        step()
     dt = (time.perf_counter() - t0) / args.steps
-    val = len(rows) / dt
-    sample = "%d evenly spaced query rows of N=%d per step, all heads, chain depth 1" % (len(rows), w.N)
+    val = n / dt   # a token is through when its row has passed all three layers
+    sample = "%d query rows spread evenly over B=%d x N=%d per step, each through the shared layers at chain depth 1, 2, 3 (all heads); extrapolated linearly to all rows" % (n, w.B, w.N)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic",
-        "config": {"workload": PREFILL, "B": w.B, "N": w.N, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "r": w.r, "m": w.m,
-                   "act": w.act, "chain_len": 1},
+        "dtype": "f64", "data": "synthetic", "config": workload_config(w),
         "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+def workload_config(w):
+    """The same dictionary in both arms (the reference arm runs the same step, on a row sample, on the host)."""
+    return {"workload": w.name, "B": w.B, "N": w.N, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "r": w.r, "m": w.m, "act": w.act,
+            "chain_len": w.chain, "l2": "GPU arm: 256 MiB buffer written between timed iterations",
+            "step": "per shared layer of the chain: the layer at its chain depth (lisa_attn_shared_prefill) + the append of its K', V "
+                    "(lisa_kvcache_append); a token counts once it is through all %d layers" % w.chain}
+
+
 def time_steps(step, n, flush, barrier):
     """Times n calls of step() with CUDA events on the current stream, L2 flushed (untimed) before each.
-    step() returns extra events it recorded; returns (total_ms, [per-step extra intervals])."""
+    step() returns the events it recorded between its calls; returns (total_ms, start events, per-step marks)."""
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
     ends = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
     marks = []
@@ -151,6 +189,173 @@ def time_steps(step, n, flush, barrier):
     return total, starts, marks
 
 
+def mark():
+    ev = torch.cuda.Event(enable_timing=True)
+    ev.record()
+    return ev
+
+
+def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
+    """The prefill step of workload `name`: one lisa_attn_shared_prefill + lisa_kvcache_append per shared layer of the chain."""
+    flush, barrier, max_over_ranks, peaks, world = env
+    w = synth.WORKLOADS[name]
+    C = w.chain
+    t = synth.prefill_inputs(w, seed=rank)
+    d = {k: v.cuda() for k, v in t.items()}
+    links = [lb.Link(d[f"qp{k}"], d[f"kp{k}"], d[f"w1_{k}"], d[f"w2_{k}"], act=lb.ACTS[w.act]) for k in range(1, C + 1)]
+    vs = [d[f"v{k}"] for k in range(1, C + 1)]
+    outs = [torch.empty_like(d["q0"]) for _ in range(C)]
+    caches = [lb.KVCacheLayer(lb.CACHE_SHARED, w.B, w.Hkv, w.N, w.d, w.r) for _ in range(C)]
+    ws = lb.prefill_workspace(d["q0"], d["k0"], links, vs[-1], outs[-1])   # the deepest layer needs the most
+
+    def layer_call(c):
+        lb.lisa_attn_shared_prefill(d["q0"], d["k0"], links[:c], vs[c - 1], out=outs[c - 1], workspace=ws)
+
+    def step():
+        evs = []
+        for c in range(1, C + 1):
+            layer_call(c)
+            evs.append(mark())
+            lb.lisa_kvcache_append(caches[c - 1], d[f"kp{c}"], vs[c - 1])
+            evs.append(mark())
+        return evs
+
+    for _ in range(args.warmup):
+        flush(); step()
+    l0 = lb.lisa_kernel_launches()
+    total_ms, starts, marks = time_steps(step, args.steps, flush, barrier)
+    launches = lb.lisa_kernel_launches() - l0
+    ms_per_step = max_over_ranks(total_ms) / args.steps
+    # device time of each layer's attention call (without its append), averaged over the steps
+    call_ms = []
+    for c in range(C):
+        tot = 0.0
+        for s, evs in zip(starts, marks):
+            tot += (s if c == 0 else evs[2 * c - 1]).elapsed_time(evs[2 * c])
+        call_ms.append(tot / args.steps)
+    tokens = w.B * w.N
+
+    # per-kernel device times of each call (events recorded inside the library around each of its kernels)
+    names = ["pack", "emit_scores", "align", "attention"]
+    P, ph = positions(w), positions(w) * w.Hq
+    qk_lr = w.B * w.N * (w.Hq + w.Hkv) * 2
+    per_layer = []
+    lb.lisa_prefill_phase_timing(True)
+    for c in range(1, C + 1):
+        for _ in range(args.steps):
+            flush(); layer_call(c)
+        phase_ms = [x / args.steps for x in lb.lisa_prefill_phase_times()]
+        # algorithmic work of each kernel at depth c.  The kernels hand the scores of every causal position to one another as
+        # fp16 planes (2 bytes per position and head); emit writes A_0 and the c-1 inner differences, the aligner reads
+        # those c planes and writes one, the attention kernel reads one.
+        kflops = {"pack": 0, "emit_scores": P * (2 * w.Hq * w.d + (c - 1) * 2 * w.Hq * w.r), "align": P * c * 4 * w.Hq * w.m,
+                  "attention": P * (2 * w.Hq * w.r + 2 * w.Hq * w.d)}
+        kbytes = {"pack": c * qk_lr * (w.r + 64), "emit_scores": qk_lr * w.d + c * ph * 2, "align": (c + 1) * ph * 2,
+                  "attention": ph * 2 + qk_lr * 64 + w.B * w.N * (w.Hkv + w.Hq) * w.d * 2}
+        ktraffic = {"emit_scores": PREFILL_TRAFFIC_PER_PH["emit_scores"], "align": PREFILL_TRAFFIC_PER_PH["align"],
+                    "attention": PREFILL_TRAFFIC_PER_PH["attention"]}
+        kernels = {}
+        for i, n in enumerate(names):
+            sec = phase_ms[i] * 1e-3
+            t_tensor, t_hbm = kflops[n] / (peaks["bf16_tflops"] * 1e12), kbytes[n] / (peaks["hbm_gbs"] * 1e9)
+            tr = ktraffic.get(n)
+            kernels[n] = {"ms": phase_ms[i], "share": phase_ms[i] / max(sum(phase_ms), 1e-9), "flops": kflops[n], "bytes": kbytes[n],
+                          "tflops": kflops[n] / sec / 1e12 if sec > 0 else None, "gbs": kbytes[n] / sec / 1e9 if sec > 0 else None,
+                          "bound": "hbm" if t_hbm >= t_tensor else "tensor", "frac": max(t_tensor, t_hbm) / sec if sec > 0 else None,
+                          "traffic": tr * ph if (tr and c == 1) else None}
+        fl = prefill_flops(w, c)
+        tf = fl / (call_ms[c - 1] * 1e-3) / 1e12
+        traffic = sum(k["traffic"] for k in kernels.values() if k["traffic"]) if c == 1 else None
+        per_layer.append({"chain_depth": c, "ms": call_ms[c - 1], "flops": fl, "flops_per_position": flops_per_position(w, c),
+                          "achieved": tf, "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
+                          "algorithmic_bytes": prefill_algorithmic_bytes(w, c),
+                          "traffic_over_algorithmic": traffic / prefill_algorithmic_bytes(w, c) if traffic else None,
+                          "kernels": kernels})
+    lb.lisa_prefill_phase_timing(False)
+
+    flops = sum(prefill_flops(w, c) for c in range(1, C + 1))
+    calls_ms = sum(call_ms)
+    tf = flops / (calls_ms * 1e-3) / 1e12
+    # the kernel with the largest share of the step, over all three calls
+    dom_name = max(names, key=lambda n: sum(pl["kernels"][n]["ms"] for pl in per_layer))
+    dom_ms = sum(pl["kernels"][dom_name]["ms"] for pl in per_layer)
+    dom_bytes = sum(pl["kernels"][dom_name]["bytes"] for pl in per_layer)
+    dom_flops = sum(pl["kernels"][dom_name]["flops"] for pl in per_layer)
+    dom_hbm = dom_bytes / (peaks["hbm_gbs"] * 1e9) >= dom_flops / (peaks["bf16_tflops"] * 1e12)
+    roofline = {
+        "bound": "tensor", "kernel": "lisa_attn_shared_prefill, chain depth 1..%d (the %d calls of a step, appends excluded)" % (C, C),
+        "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
+        "peak_source": peaks["source"] + " (burst)", "ms": calls_ms, "flops_per_step": flops,
+        "formula": "causal positions B*N*(N+1)/2 x sum over c of (2hd + c(2hr + 4hm) + 2hd)",
+        "traffic": per_layer[0]["kernels"][dom_name]["traffic"],
+        "traffic_note": "ncu DRAM bytes of the dominant kernel at chain depth 1, the cfg2 capture scaled by causal positions",
+        "traffic_over_algorithmic": per_layer[0]["traffic_over_algorithmic"],
+        "dominant_kernel": {"name": dom_name, "ms_per_step": dom_ms, "bound": "hbm" if dom_hbm else "tensor",
+                            "achieved": dom_bytes / (dom_ms * 1e-3) / 1e9 if dom_hbm else dom_flops / (dom_ms * 1e-3) / 1e12,
+                            "unit": "GB/s" if dom_hbm else "TFLOP/s",
+                            "frac": (dom_bytes / (dom_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]) if dom_hbm else (dom_flops / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]),
+                            "tensor_frac": dom_flops / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]},
+        "per_layer": per_layer}
+
+    res = {"workload": w.name, "ms_per_step": ms_per_step, "value": world * tokens / (ms_per_step * 1e-3), "launches": launches,
+           "roofline": roofline, "tokens": tokens, "outs": outs, "inputs": t}
+
+    # ---------------- the same layers through one lisa_attn_shared_prefill_chain call ----------------
+    if with_chain and C > 1:
+        cws = lb.prefill_chain_workspace(d["q0"], d["k0"], links, vs, outs)
+
+        def chain_step():
+            lb.lisa_attn_shared_prefill_chain(d["q0"], d["k0"], links, vs, outs=outs, workspace=cws)
+            ev = mark()
+            for c in range(C):
+                lb.lisa_kvcache_append(caches[c], d[f"kp{c + 1}"], vs[c])
+            return [ev]
+
+        for _ in range(args.warmup):
+            flush(); chain_step()
+        l1 = lb.lisa_kernel_launches()
+        ctot, cst, cmk = time_steps(chain_step, args.steps, flush, barrier)
+        res["launches"] += lb.lisa_kernel_launches() - l1
+        cms = max_over_ranks(ctot) / args.steps
+        call = sum(s.elapsed_time(m[0]) for s, m in zip(cst, cmk)) / args.steps
+        executed = P * (2 * w.Hq * w.d + C * (2 * w.Hq * w.r + 4 * w.Hq * w.m + 2 * w.Hq * w.d))
+        res["chain_call"] = {"ms_per_step": cms, "value": world * tokens / (cms * 1e-3), "unit": "tokens/s", "call_ms": call,
+                             "frac_by_layer_formula": flops / (call * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                             "flops_needed_once": executed,
+                             "frac_by_flops_needed_once": executed / (call * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                             "note": "one pass computes A_0 and every link once; the per-layer formula counts what three separate calls recompute"}
+        del cws
+
+    # ---------------- end to end through the host-memory entry point ----------------
+    if with_e2e:
+        hp = {k: v.pin_memory() for k, v in t.items() if k != "v0"}
+        hlinks = [lb.Link(hp[f"qp{k}"], hp[f"kp{k}"], hp[f"w1_{k}"], hp[f"w2_{k}"], act=lb.ACTS[w.act]) for k in range(1, C + 1)]
+        houts = [torch.empty_like(t["q0"]).pin_memory() for _ in range(C)]
+        arena = torch.empty(lb.lisa_host_arena_bytes(hp["q0"], hp["k0"], hlinks, hp[f"v{C}"], houts[-1]), dtype=torch.uint8, device="cuda")
+        nbytes = lambda x: x.numel() * x.element_size()
+        h2d = sum(nbytes(hp["q0"]) + nbytes(hp["k0"]) + nbytes(hp[f"v{c}"]) +
+                  sum(nbytes(hp[f"qp{k}"]) + nbytes(hp[f"kp{k}"]) + nbytes(hp[f"w1_{k}"]) + nbytes(hp[f"w2_{k}"]) for k in range(1, c + 1))
+                  for c in range(1, C + 1))
+        d2h = sum(nbytes(o) for o in houts)
+
+        def e2e_step():
+            for c in range(1, C + 1):
+                lb.lisa_attn_shared_prefill_host(hp["q0"], hp["k0"], hlinks[:c], hp[f"v{c}"], houts[c - 1], arena)
+            return []
+
+        for _ in range(3):
+            e2e_step()
+        n_e2e = min(args.steps, 10) if tokens > 8192 else args.steps
+        e2e_total, _, _ = time_steps(e2e_step, n_e2e, flush, barrier)
+        e2e_ms = max_over_ranks(e2e_total) / n_e2e
+        res["e2e"] = {"value": world * tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms, "steps": n_e2e,
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                      "call": "lisa_attn_shared_prefill_host per layer: pinned host tensors in, pinned host output back, every step"}
+        del arena, hp, houts
+    del d, caches, ws
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -159,13 +364,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-decode", action="store_true", help="skip the decode section")
     ap.add_argument("--no-stack", action="store_true", help="skip the 32-layer stack section")
-    ap.add_argument("--only", choices=["prefill", "decode"], default=None,
-                    help="profiling aid: run just that section (prefill: no end-to-end, decode, stack or CPU legs)")
+    ap.add_argument("--only", choices=["prefill", "cfg2", "decode"], default=None,
+                    help="profiling aid: run just that section (prefill: the headline step; cfg2: the LLaMA2-7B-shaped layer; "
+                         "neither runs the end-to-end, decode, stack or CPU legs)")
     ap.add_argument("--decode-batch", type=int, default=0, help="profiling aid: decode batch size (default: the workload's 64)")
     args = ap.parse_args()
     if args.only is None:
         args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.only == "prefill":
+    if args.only in ("prefill", "cfg2"):
         args.no_decode = args.no_stack = True
     if args.only == "decode":
         args.no_stack = True
@@ -188,99 +394,21 @@ def main():
 
     peaks = measured_peaks()
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    flush = lambda: flush_l2(flush_buf)
+    flush = lambda: flush_buf.zero_()
+    env = (flush, barrier, max_over_ranks, peaks, world)
 
-    # ---------------- prefill step (headline) ----------------
-    w = synth.WORKLOADS[PREFILL]
-    t = synth.prefill_inputs(w, seed=rank)
-    d = {k: v.cuda() for k, v in t.items()}
-    link = lb.Link(d["qp1"], d["kp1"], d["w1_1"], d["w2_1"], act=lb.ACTS[w.act])
-    out = torch.empty_like(d["q0"])
-    cache = lb.KVCacheLayer(lb.CACHE_SHARED, w.B, w.Hkv, w.N, w.d, w.r)
-
-    pws = lb._workspace(lb.OP_SHARED_PREFILL, lb._prefill_args(d["q0"], d["k0"], [link], d["v1"], out)[0])
-
-    def prefill_step():
-        lb.lisa_attn_shared_prefill(d["q0"], d["k0"], [link], d["v1"], out=out, workspace=pws)
-        ev = torch.cuda.Event(enable_timing=True)
-        ev.record()
-        lb.lisa_kvcache_append(cache, d["kp1"], d["v1"])
-        return ev
-
-    sampler = ClockSampler(local)   # runs from the warm-up to the end of the last timed region
+    sampler = ClockSampler(local)   # runs from the first warm-up to the end of the last timed region
     sampler.start()
-    for _ in range(args.warmup):
-        flush(); prefill_step()
-    l0 = lb.lisa_kernel_launches()
-    total_ms, starts, marks = time_steps(prefill_step, args.steps, flush, barrier)
-    launches = lb.lisa_kernel_launches() - l0
-    kernel_ms = sum(s.elapsed_time(m) for s, m in zip(starts, marks)) / args.steps
-    total_ms = max_over_ranks(total_ms)
-    ms_per_step = total_ms / args.steps
-    tokens = w.B * w.N
-    value = group.whole_job_per_second(tokens, ms_per_step)
-    flops = prefill_flops(w, 1)
-    # per-kernel device times of the same step (events recorded inside the library around each of its kernels)
-    lb.lisa_prefill_phase_timing(True)
-    for _ in range(args.steps):
-        flush(); prefill_step()
-    phase_ms = [x / args.steps for x in lb.lisa_prefill_phase_times()]
-    lb.lisa_prefill_phase_timing(False)
-    positions = w.B * w.N * (w.N + 1) // 2
-    phase_flops = {"pack": 0, "emit_scores": positions * 2 * w.Hq * w.d, "align": positions * 4 * w.Hq * w.m,
-                   "attention": positions * (2 * w.Hq * w.r + 2 * w.Hq * w.d)}
-    # Algorithmic HBM bytes of each kernel.  The three kernels hand the scores of every causal position to one
-    # another as fp16 planes (2 bytes per position and head); those planes, not the flops, set each kernel's floor:
-    # at 60 flop per plane byte every one of them sits far left of the ridge (about 250 flop/byte).
-    plane = positions * w.Hq * 2
-    qk_lr = w.B * w.N * (w.Hq + w.Hkv) * 2
-    phase_bytes = {"pack": qk_lr * (w.r + 64), "emit_scores": qk_lr * w.d + plane, "align": 2 * plane,
-                   "attention": plane + qk_lr * 64 + w.B * w.N * (w.Hkv + w.Hq) * w.d * 2}
-    names = ["pack", "emit_scores", "align", "attention"]
-    kernels = {}
-    for i, n in enumerate(names):
-        sec = phase_ms[i] * 1e-3
-        t_tensor, t_hbm = phase_flops[n] / (peaks["bf16_tflops"] * 1e12), phase_bytes[n] / (peaks["hbm_gbs"] * 1e9)
-        kernels[n] = {"ms": phase_ms[i], "share": phase_ms[i] / max(sum(phase_ms), 1e-9), "flops": phase_flops[n],
-                      "bytes": phase_bytes[n], "tflops": phase_flops[n] / sec / 1e12 if sec > 0 else None,
-                      "gbs": phase_bytes[n] / sec / 1e9 if sec > 0 else None, "bound": "hbm" if t_hbm >= t_tensor else "tensor",
-                      "frac": max(t_tensor, t_hbm) / sec if sec > 0 else None, "traffic": PREFILL_TRAFFIC.get(n)}
-    dom = max(names, key=lambda n: kernels[n]["ms"])
-    kd = kernels[dom]
-    call_tflops = flops / (kernel_ms * 1e-3) / 1e12
-    if kd["bound"] == "hbm":
-        roofline = {"bound": "hbm", "kernel": "lisa_attn_shared_prefill/" + dom, "achieved": kd["gbs"], "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "frac": kd["gbs"] / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                    "bytes_per_launch": kd["bytes"]}
-    else:
-        roofline = {"bound": "tensor", "kernel": "lisa_attn_shared_prefill/" + dom, "achieved": kd["tflops"], "peak": peaks["bf16_tflops"],
-                    "unit": "TFLOP/s", "frac": kd["tflops"] / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst)",
-                    "flops_per_launch": kd["flops"]}
-    roofline.update({"traffic": kd["traffic"], "kernel_ms": kd["ms"], "kernels": kernels,
-                     "whole_call": {"bound": "tensor", "ms": kernel_ms, "flops": flops, "achieved": call_tflops, "unit": "TFLOP/s",
-                                    "frac": call_tflops / peaks["bf16_tflops"]}})
+    launches = 0
 
-
-    # ---------------- end to end through the host-memory entry point ----------------
-    def measure_e2e():
-        hp = {k: t[k].pin_memory() for k in ("q0", "k0", "v1", "qp1", "kp1", "w1_1", "w2_1")}
-        hlink = lb.Link(hp["qp1"], hp["kp1"], hp["w1_1"], hp["w2_1"], act=lb.ACTS[w.act])
-        hout = torch.empty_like(t["q0"]).pin_memory()
-        arena = torch.empty(lb.lisa_host_arena_bytes(hp["q0"], hp["k0"], [hlink], hp["v1"], hout), dtype=torch.uint8, device="cuda")
-        h2d = sum(x.numel() * x.element_size() for x in hp.values())
-        d2h = hout.numel() * hout.element_size()
-
-        def e2e_step():
-            lb.lisa_attn_shared_prefill_host(hp["q0"], hp["k0"], [hlink], hp["v1"], hout, arena)
-
-        for _ in range(3):
-            e2e_step()
-        e2e_total, _, _ = time_steps(e2e_step, args.steps, flush, barrier)
-        e2e_ms = max_over_ranks(e2e_total) / args.steps
-        return {"value": world * tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
-
-    e2e = measure_e2e() if args.only is None else None
+    # ---------------- prefill: the headline step, and the LLaMA2-7B-shaped layer beside it ----------------
+    head = second = None
+    if args.only in (None, "prefill"):
+        head = bench_prefill(lb, HEADLINE, rank, args, env, with_chain=True, with_e2e=args.only is None)
+        launches += head["launches"]
+    if args.only in (None, "cfg2"):
+        second = bench_prefill(lb, SECOND, rank, args, env, with_chain=False, with_e2e=args.only is None)
+        launches += second["launches"]
 
     # ---------------- decode step and the library's own standard-attention decode ----------------
     decode = None
@@ -308,13 +436,13 @@ def main():
 
         def shared_step():
             lb.lisa_kvcache_append(sh, new_kp, new_v, before)
-            ev = torch.cuda.Event(enable_timing=True); ev.record()
+            ev = mark()
             lb.lisa_attn_shared_decode(prev, dlink, sh, L=L, out=o_sh, out_scores=row, workspace=ws)
             return ev
 
         def standard_step():
             lb.lisa_kvcache_append(st, new_k, new_v, before)
-            ev = torch.cuda.Event(enable_timing=True); ev.record()
+            ev = mark()
             lb.lisa_attn_anchor(q0, cache=st, L=L, out=o_st, out_scores=row, workspace=ws)
             return ev
 
@@ -375,31 +503,44 @@ def main():
 
     clocks = sampler.stop()  # sampled across all timed regions above (prefill, end-to-end, decode, stack)
 
-    # ---------------- the CPU oracle on the host cores (rank 0, N = 1 only) ----------------
+    # ---------------- the CPU oracle on the host cores (rank 0, N = 1 only): a row sample of the headline workload ----------------
     cpu = None
-    if rank == 0 and world == 1 and args.only is None:
+    if rank == 0 and world == 1 and args.only is None and head is not None:
         import oracle
-        ol = [oracle.Link(synth.to_f64(t["qp1"]), synth.to_f64(t["kp1"]), synth.to_f64(t["w1_1"]), synth.to_f64(t["w2_1"]),
-                          r=w.r, act={"relu": oracle.ACT_RELU, "silu": oracle.ACT_SILU, "none": oracle.ACT_NONE}[w.act])]
-        rows = np.arange(0, w.N, dtype=np.int32)
-        t0 = time.perf_counter()
-        ref = oracle.prefill_rows(synth.to_f64(t["q0"]), synth.to_f64(t["k0"]), synth.to_f64(t["v1"]), ol,
-                                  np.zeros_like(rows), rows)
-        dt = time.perf_counter() - t0
-        err = float(np.abs(out[0].float().cpu().numpy() - ref).max())
-        cpu = {"value": len(rows) / dt, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
-               "sample": "all %d query rows of the workload, once (%.1f s)" % (len(rows), dt), "max_abs_err_vs_gpu": err}
+        w = synth.WORKLOADS[HEADLINE]
+        t = head["inputs"]
+        q0, k0 = synth.to_f64(t["q0"]), synth.to_f64(t["k0"])
+        ol = oracle_links(t, w, w.chain)
+        n = 768
+        rb, ri = sample_rows(w, n)
+        secs, err = 0.0, 0.0
+        for c in range(1, w.chain + 1):
+            v = synth.to_f64(t[f"v{c}"])
+            t0 = time.perf_counter()
+            ref = oracle.prefill_rows(q0, k0, v, ol[:c], rb, ri)
+            secs += time.perf_counter() - t0
+            got = head["outs"][c - 1][torch.from_numpy(rb).long().cuda(), torch.from_numpy(ri).long().cuda()].float().cpu().numpy()
+            err = max(err, float(np.abs(got - ref).max()))
+        cpu = {"value": n / secs, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": "%d query rows spread evenly over B=%d x N=%d, each through the three shared layers (chain depth 1, 2, 3), once "
+                         "(%.1f s); extrapolated linearly to all %d rows" % (n, w.B, w.N, secs, w.B * w.N),
+               "max_abs_err_vs_gpu": err}
 
     if rank == 0:
-        print(json.dumps({
-            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-            "data": "synthetic",
-            "config": {"workload": PREFILL, "B": w.B, "N": w.N, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "r": w.r, "m": w.m,
-                       "act": w.act, "chain_len": 1, "l2": "256 MiB buffer written between timed iterations",
-                       "step": "lisa_attn_shared_prefill + lisa_kvcache_append"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
-            "decode": decode, "stack": stack}))
+        line = {"metric": METRIC, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "clocks": clocks, "gpu_launches": int(launches)}
+        main_res = head or second
+        if main_res is not None:
+            w = synth.WORKLOADS[main_res["workload"]]
+            cfg = workload_config(w)
+            line.update({"value": main_res["value"], "ms_per_step": main_res["ms_per_step"], "config": cfg,
+                         "e2e": main_res.get("e2e"), "roofline": main_res["roofline"], "chain_call": main_res.get("chain_call")})
+        if head is not None and second is not None:
+            line["cfg2"] = {"workload": second["workload"], "value": second["value"], "unit": "tokens/s", "ms_per_step": second["ms_per_step"],
+                            "e2e": second.get("e2e"), "roofline": second["roofline"]}
+        line.update({"cpu_baseline": cpu, "decode": decode, "stack": stack})
+        print(json.dumps(line))
     group.close()
 
 

@@ -22,7 +22,7 @@
  *     Descriptor structs and the `links` array are HOST memory, read only
  *     during the call.
  *   - Activations are [B, N, H, x] with x (d or r) contiguous; strides are in
- *     elements.  Scores handed between decode layers are fp32 [B, Hq, L_cap].
+ *     elements.  Scores handed between decode layers are [B, Hq, L_cap], fp32 unless the call says bf16.
  *   - Grouped-query attention: query head h reads key/value head h / (Hq/Hkv).
  *   - Scratch memory comes from the caller: ask lisa_workspace_bytes() for the
  *     size and pass a buffer of at least that size (may be NULL when 0).
@@ -138,8 +138,8 @@ typedef struct lisa_kvcache {
  * Decode  (cache != NULL, Nq == 1): the new token's q against a STANDARD cache that already holds the
  *   new token's K and V.  The context length of sequence b is seq_lens[b] (device int32 [B]) with
  *   1 <= seq_lens[b] <= L, or L for every sequence when seq_lens is NULL; L <= L_cap.
- *   If out_scores != NULL the pre-softmax row q.k_j/sqrt(d), j < length, is written there in fp32 for
- *   the following shared layer (entries beyond the length are left untouched).
+ *   If out_scores != NULL the pre-softmax row q.k_j/sqrt(d), j < length, is written there (fp32, or bf16 when
+ *   scores_dtype says so) for the following shared layer (entries beyond the length are left untouched).
  * o has q's shape.  Workspace: lisa_workspace_bytes(LISA_OP_ANCHOR, args, &n). */
 typedef struct lisa_anchor_args {
     size_t struct_size; /* sizeof(lisa_anchor_args) */
@@ -148,10 +148,12 @@ typedef struct lisa_anchor_args {
     lisa_tensor q, k, v, o;
     const lisa_kvcache_layer* cache;
     const int32_t* seq_lens;
-    float* out_scores; /* decode only; [B, Hq, >= length] */
+    void* out_scores; /* decode only; [B, Hq, >= length], fp32 or (scores_dtype == LISA_BF16) bf16 */
     int64_t scores_stride_b, scores_stride_h;
     void* workspace;
     size_t workspace_bytes;
+    int32_t scores_dtype; /* lisa_dtype_t of out_scores: LISA_F32 (0, the default) or LISA_BF16 */
+    int32_t reserved;
 } lisa_anchor_args;
 lisa_status_t lisa_attn_anchor(const lisa_anchor_args* args, lisa_stream_t stream);
 
@@ -208,19 +210,22 @@ lisa_status_t lisa_host_arena_bytes(const lisa_shared_prefill_args* host_args, s
  * prev_scores: the previous layer's fp32 score row [B,Hq,>=length]; link.qp the new token's Q' [B,1,Hq,r];
  * cache: a SHARED layer already holding the new token's K' and V; length = seq_lens[b] (<= L) or L.
  * For each cached position j < length: A[:,j] = Integrate(Align(prev[:,j]), q'.K'_j/sqrt(r)); then softmax
- * over j and the product with V.  o [B,1,Hq,d].  out_scores (fp32 [B,Hq,>=length], may be NULL, must not
- * alias prev_scores) receives A for the next shared layer. */
+ * over j and the product with V.  o [B,1,Hq,d].  out_scores ([B,Hq,>=length], may be NULL, must not alias prev_scores)
+ * receives A for the next shared layer.
+ * Score rows are fp32 by default.  With scores_dtype == LISA_BF16 both rows are bf16 (2 bytes per entry, the size
+ * Sec. 5.2 counts for the row): every hand-off between layers then rounds the scores to 8 mantissa bits (relative
+ * 2^-9), on top of which the layer computes exactly as before. */
 typedef struct lisa_shared_decode_args {
     size_t struct_size;
     int32_t B, Hq, L;
-    int32_t reserved;
-    const float* prev_scores;
+    int32_t scores_dtype; /* lisa_dtype_t of prev_scores AND out_scores: LISA_F32 (0, the default) or LISA_BF16 */
+    const void* prev_scores;
     int64_t prev_stride_b, prev_stride_h;
     lisa_link link;
     const lisa_kvcache_layer* cache;
     const int32_t* seq_lens; /* device int32 [B] or NULL */
     lisa_tensor o;
-    float* out_scores;
+    void* out_scores;
     int64_t scores_stride_b, scores_stride_h;
     void* workspace;
     size_t workspace_bytes;
@@ -252,6 +257,32 @@ lisa_status_t lisa_attn_shared_decode(const lisa_shared_decode_args* args, lisa_
  * wrong results; order them on one stream or with events. */
 #define LISA_STATIC_SCRATCH_BYTES (8u << 20)
 lisa_status_t lisa_attn_shared_decode_static(const lisa_shared_decode_args* args, lisa_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * lisa_project -- the projections either side of the attention (Eq. 1: H W^V_i per head, and Concat(.) W^O; Eq. 3:
+ * H W^Q_LR, H W^K_LR): C = X . W with X [B,N,1,d_in] (rows of d_in contiguous values; stride_h is ignored) and
+ * W [d_in, n_out] row-major (row = input unit, as the paper writes H W), fp32 accumulation.  The n_out columns of C are
+ * the concatenation [outputs[0] | outputs[1] | ...]: output o receives H_o * x_o consecutive columns, column h*x_o + j
+ * of its block going to element [b, n, h, j] of its tensor (any strides, so a block can be written straight into the
+ * layout its consumer reads: Q' and K' for lisa_attn_shared_prefill, K'/V rows for lisa_kvcache_append, a flat
+ * [B,N,1,d_model] row for W^O).  One call with W = [W^Q_LR | W^K_LR | W^V] projects a shared layer's three operands at once.
+ * bf16 X, W and outputs with 16-byte aligned rows run on the tensor cores; fp32 and odd shapes on a general kernel.
+ * No workspace.  1 <= n_outputs <= 4. */
+typedef struct lisa_project_output {
+    lisa_tensor t; /* [B, N, H, x] */
+    int32_t H;
+    int32_t x;
+} lisa_project_output;
+typedef struct lisa_project_args {
+    size_t struct_size;
+    int32_t B, N, d_in, n_outputs;
+    lisa_tensor x;   /* [B, N, 1, d_in] */
+    const void* w;   /* [d_in, sum_o H_o * x_o], row-major, device */
+    int32_t w_dtype; /* lisa_dtype_t; must equal x.dtype */
+    int32_t reserved;
+    lisa_project_output outputs[4];
+} lisa_project_args;
+lisa_status_t lisa_project(const lisa_project_args* args, lisa_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
  * lisa_kvcache_append -- write n_new new positions into a layer's cache (Sec. 2.2; Sec. 5.2: a shared layer

@@ -24,6 +24,12 @@ lisa_status_t lisa_prefill_phase_times(float* ms4);
  * exists (for cross-checking the two paths against each other); on == 0 restores the default choice. */
 void lisa_force_general_kernels(int on);
 
+/* Enqueues a one-warp kernel whose only thread waits, with the library's bounded wait, for an arrival that never
+ * comes; after limit_cycles SM cycles (1 .. 1e8) the wait gives up and records it, so the next lisa_check() on the
+ * stream returns LISA_ERR_TIMEOUT and the one after that LISA_OK.  Nothing else is touched: the device context stays
+ * usable.  This is the path a tensor-core kernel takes when one of its hand-offs stalls. */
+lisa_status_t lisa_debug_wait_timeout(int64_t limit_cycles, lisa_stream_t stream);
+
 /* Number of kernels this library has enqueued so far in this process (all threads). */
 uint64_t lisa_kernel_launches(void);
 

@@ -28,9 +28,10 @@ ACTS = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
 # include/lisa.h (the method's entry points and host helpers) and include/lisa_debug.h (test and measurement hooks)
 EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_chain", "lisa_attn_shared_prefill_host",
            "lisa_host_arena_bytes", "lisa_attn_shared_decode", "lisa_attn_shared_decode_static", "lisa_kvcache_append",
-           "lisa_kvcache_append_layer", "lisa_kvcache_bytes", "lisa_kvcache_total_bytes", "lisa_kvcache_init",
+           "lisa_kvcache_append_layer", "lisa_project", "lisa_kvcache_bytes", "lisa_kvcache_total_bytes", "lisa_kvcache_init",
            "lisa_workspace_bytes", "lisa_check", "lisa_last_cuda_error", "lisa_status_string", "lisa_version",
-           "lisa_prefill_phase_times", "lisa_prefill_phase_timing", "lisa_force_general_kernels", "lisa_kernel_launches"]
+           "lisa_prefill_phase_times", "lisa_prefill_phase_timing", "lisa_force_general_kernels", "lisa_kernel_launches",
+           "lisa_debug_wait_timeout"]
 MAX_LAYERS = 128
 
 
@@ -67,12 +68,21 @@ class CCache(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("reserved", C.c_int32), ("layers", CCacheLayer * MAX_LAYERS)]
 
 
+class CProjectOutput(C.Structure):
+    _fields_ = [("t", Tensor), ("H", C.c_int32), ("x", C.c_int32)]
+
+
+class ProjectArgs(C.Structure):
+    _fields_ = [("struct_size", C.c_size_t), ("B", C.c_int32), ("N", C.c_int32), ("d_in", C.c_int32), ("n_outputs", C.c_int32),
+                ("x", Tensor), ("w", C.c_void_p), ("w_dtype", C.c_int32), ("reserved", C.c_int32), ("outputs", CProjectOutput * 4)]
+
+
 class AnchorArgs(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("B", C.c_int32), ("Nq", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32),
                 ("d", C.c_int32), ("L", C.c_int32), ("q", Tensor), ("k", Tensor), ("v", Tensor), ("o", Tensor),
                 ("cache", C.POINTER(CCacheLayer)), ("seq_lens", C.c_void_p), ("out_scores", C.c_void_p),
                 ("scores_stride_b", C.c_int64), ("scores_stride_h", C.c_int64), ("workspace", C.c_void_p),
-                ("workspace_bytes", C.c_size_t)]
+                ("workspace_bytes", C.c_size_t), ("scores_dtype", C.c_int32), ("reserved", C.c_int32)]
 
 
 class SharedPrefillArgs(C.Structure):
@@ -89,7 +99,7 @@ class SharedPrefillChainArgs(C.Structure):
 
 class SharedDecodeArgs(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("B", C.c_int32), ("Hq", C.c_int32), ("L", C.c_int32),
-                ("reserved", C.c_int32), ("prev_scores", C.c_void_p), ("prev_stride_b", C.c_int64),
+                ("scores_dtype", C.c_int32), ("prev_scores", C.c_void_p), ("prev_stride_b", C.c_int64),
                 ("prev_stride_h", C.c_int64), ("link", CLink), ("cache", C.POINTER(CCacheLayer)),
                 ("seq_lens", C.c_void_p), ("o", Tensor), ("out_scores", C.c_void_p), ("scores_stride_b", C.c_int64),
                 ("scores_stride_h", C.c_int64), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
@@ -120,6 +130,7 @@ def load():
         lib.lisa_attn_shared_decode_static.restype = C.c_int
         lib.lisa_kvcache_append.argtypes = [C.POINTER(CCacheLayer), C.POINTER(Tensor), C.POINTER(Tensor), C.c_void_p,
                                             C.c_int32, C.c_void_p]
+        lib.lisa_project.argtypes = [C.POINTER(ProjectArgs), C.c_void_p]
         lib.lisa_kvcache_bytes.argtypes = [C.POINTER(CCacheLayer), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
         lib.lisa_kvcache_total_bytes.argtypes = [C.POINTER(CCacheDesc), C.POINTER(C.c_size_t)]
         lib.lisa_kvcache_init.argtypes = [C.POINTER(CCacheDesc), C.c_void_p, C.c_size_t, C.POINTER(CCache)]
@@ -128,6 +139,7 @@ def load():
         lib.lisa_workspace_bytes.argtypes = [C.c_int32, C.c_void_p, C.POINTER(C.c_size_t)]
         lib.lisa_check.argtypes = [C.c_void_p]
         lib.lisa_kernel_launches.restype = C.c_uint64
+        lib.lisa_debug_wait_timeout.argtypes = [C.c_int64, C.c_void_p]
         _lib = lib
     return _lib
 
@@ -260,6 +272,23 @@ def lisa_kvcache_append(cache: KVCacheLayer, k_or_kp: torch.Tensor, v: torch.Ten
                                       int(v.shape[1]), _stream()), "lisa_kvcache_append")
 
 
+def lisa_project(x: torch.Tensor, w: torch.Tensor, outs: Sequence[torch.Tensor]) -> Sequence[torch.Tensor]:
+    """C = x . w scattered into outs: x [B,N,d_in] (rows contiguous), w [d_in, n_out] row-major, outs[o] a [B,N,H_o,x_o] tensor
+    (any strides, innermost contiguous) that receives the next H_o*x_o columns of C."""
+    B, N, d_in = x.shape
+    assert x.stride(2) == 1 and w.is_contiguous() and w.shape[0] == d_in and w.shape[1] == sum(o.shape[2] * o.shape[3] for o in outs)
+    assert 1 <= len(outs) <= 4
+    a = ProjectArgs()
+    a.struct_size = C.sizeof(ProjectArgs)
+    a.B, a.N, a.d_in, a.n_outputs = B, N, d_in, len(outs)
+    a.x = Tensor(x.data_ptr(), _dt(x), 0, x.stride(0), x.stride(1), 0)
+    a.w, a.w_dtype = w.data_ptr(), _dt(w)
+    for i, o in enumerate(outs):
+        a.outputs[i] = CProjectOutput(_tensor4(o), int(o.shape[2]), int(o.shape[3]))
+    _check(load().lisa_project(C.byref(a), _stream()), "lisa_project")
+    return outs
+
+
 def _workspace_bytes(op: int, args) -> int:
     n = C.c_size_t()
     _check(load().lisa_workspace_bytes(op, C.byref(args), C.byref(n)), "lisa_workspace_bytes")
@@ -302,8 +331,9 @@ def lisa_attn_anchor(q: torch.Tensor, k: Optional[torch.Tensor] = None, v: Optio
         a.cache = C.pointer(cache.desc)
         a.seq_lens = _ptr(seq_lens)
         if out_scores is not None:
-            assert out_scores.dtype == torch.float32 and out_scores.stride(2) == 1
+            assert out_scores.stride(2) == 1
             a.out_scores, a.scores_stride_b, a.scores_stride_h = out_scores.data_ptr(), out_scores.stride(0), out_scores.stride(1)
+            a.scores_dtype = _dt(out_scores)
     ws = workspace if workspace is not None else _workspace(OP_ANCHOR, a)
     a.workspace, a.workspace_bytes = _ptr(ws), (ws.numel() if ws is not None else 0)
     _check(load().lisa_attn_anchor(C.byref(a), _stream()), "lisa_attn_anchor")
@@ -330,6 +360,19 @@ def lisa_attn_shared_prefill(q0: torch.Tensor, k0: torch.Tensor, links: Sequence
     a.workspace, a.workspace_bytes = _ptr(ws), (ws.numel() if ws is not None else 0)
     _check(load().lisa_attn_shared_prefill(C.byref(a), _stream()), "lisa_attn_shared_prefill")
     return out
+
+
+def prefill_workspace(q0, k0, links: Sequence[Link], v, out) -> Optional[torch.Tensor]:
+    """Scratch buffer of the size lisa_workspace_bytes reports for this lisa_attn_shared_prefill call (None when it needs none);
+    callers that repeat a call pass it back as `workspace` instead of allocating every time."""
+    a, keep = _prefill_args(q0, k0, links, v, out)
+    return _workspace(OP_SHARED_PREFILL, a)
+
+
+def prefill_chain_workspace(q0, k0, links: Sequence[Link], vs, outs) -> Optional[torch.Tensor]:
+    """The same for lisa_attn_shared_prefill_chain."""
+    a, keep = _prefill_chain_args(q0, k0, links, vs, outs)
+    return _workspace(OP_SHARED_PREFILL_CHAIN, a)
 
 
 def _prefill_chain_args(q0, k0, links: Sequence[Link], vs, outs):
@@ -377,21 +420,22 @@ def lisa_attn_shared_decode(prev_scores: torch.Tensor, link: Link, cache: KVCach
                             seq_lens: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
                             out_scores: Optional[torch.Tensor] = None,
                             workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """One decode step of a shared layer. prev_scores fp32 [B,Hq,>=L]; link.qp [B,1,Hq,r]; returns o [B,1,Hq,d]."""
+    """One decode step of a shared layer. prev_scores [B,Hq,>=L] fp32 or bf16 (out_scores then has the same type);
+    link.qp [B,1,Hq,r]; returns o [B,1,Hq,d]."""
     B, Hq = prev_scores.shape[0], prev_scores.shape[1]
-    assert prev_scores.dtype == torch.float32 and prev_scores.stride(2) == 1
+    assert prev_scores.stride(2) == 1
     if out is None:
         out = torch.empty((B, 1, Hq, cache.d), dtype=cache.v.dtype, device=prev_scores.device)
     a = SharedDecodeArgs()
     a.struct_size = C.sizeof(SharedDecodeArgs)
-    a.B, a.Hq, a.L = B, Hq, int(L)
+    a.B, a.Hq, a.L, a.scores_dtype = B, Hq, int(L), _dt(prev_scores)
     a.prev_scores, a.prev_stride_b, a.prev_stride_h = prev_scores.data_ptr(), prev_scores.stride(0), prev_scores.stride(1)
     a.link = link.to_c()
     a.cache = C.pointer(cache.desc)
     a.seq_lens = _ptr(seq_lens)
     a.o = _tensor4(out)
     if out_scores is not None:
-        assert out_scores.dtype == torch.float32 and out_scores.stride(2) == 1
+        assert out_scores.dtype == prev_scores.dtype and out_scores.stride(2) == 1
         a.out_scores, a.scores_stride_b, a.scores_stride_h = out_scores.data_ptr(), out_scores.stride(0), out_scores.stride(1)
     ws = workspace if workspace is not None else _workspace(OP_SHARED_DECODE, a)
     a.workspace, a.workspace_bytes = _ptr(ws), (ws.numel() if ws is not None else 0)
@@ -410,17 +454,17 @@ def lisa_attn_shared_decode_static(prev_scores: torch.Tensor, link: Link, cache:
     ([B,1,Hq,d]) must be passed in.  Steps that need more scratch raise LisaError(ERR_WORKSPACE).  Calls share
     that array: keep them ordered on one stream."""
     B, Hq = prev_scores.shape[0], prev_scores.shape[1]
-    assert prev_scores.dtype == torch.float32 and prev_scores.stride(2) == 1
+    assert prev_scores.stride(2) == 1
     a = SharedDecodeArgs()
     a.struct_size = C.sizeof(SharedDecodeArgs)
-    a.B, a.Hq, a.L = B, Hq, int(L)
+    a.B, a.Hq, a.L, a.scores_dtype = B, Hq, int(L), _dt(prev_scores)
     a.prev_scores, a.prev_stride_b, a.prev_stride_h = prev_scores.data_ptr(), prev_scores.stride(0), prev_scores.stride(1)
     a.link = link.to_c()
     a.cache = C.pointer(cache.desc)
     a.seq_lens = _ptr(seq_lens)
     a.o = _tensor4(out)
     if out_scores is not None:
-        assert out_scores.dtype == torch.float32 and out_scores.stride(2) == 1
+        assert out_scores.dtype == prev_scores.dtype and out_scores.stride(2) == 1
         a.out_scores, a.scores_stride_b, a.scores_stride_h = out_scores.data_ptr(), out_scores.stride(0), out_scores.stride(1)
     _check(load().lisa_attn_shared_decode_static(C.byref(a), _stream()), "lisa_attn_shared_decode_static")
     return out
@@ -439,6 +483,11 @@ def lisa_kernel_launches() -> int:
 def lisa_force_general_kernels(on: bool) -> None:
     """Route every later call through the general SIMT kernels (True) or restore the default choice (False)."""
     load().lisa_force_general_kernels(1 if on else 0)
+
+
+def lisa_debug_wait_timeout(limit_cycles: int = 1000000) -> None:
+    """Enqueues the test kernel whose bounded wait runs out after limit_cycles SM cycles (see lisa_debug.h)."""
+    _check(load().lisa_debug_wait_timeout(int(limit_cycles), _stream()), "lisa_debug_wait_timeout")
 
 
 def lisa_prefill_phase_timing(enable: bool) -> None:

@@ -115,6 +115,11 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
 cudaError_t prefill_phase_timing(bool enable);
 cudaError_t prefill_phase_times(float* ms4);
 
+// Projection GEMM (tc_project.cu): tensor-core kernel for aligned bf16, general kernel otherwise.
+bool tc_project_supported(const lisa_project_args& a);
+cudaError_t launch_tc_project(const lisa_project_args& a, cudaStream_t s);
+cudaError_t launch_generic_project(const lisa_project_args& a, cudaStream_t s);
+
 cudaError_t launch_kvcache_append(const lisa_kvcache_layer& c, const lisa_tensor& k, const lisa_tensor& v,
                                   const int32_t* lens_before, int n_new, cudaStream_t s);
 

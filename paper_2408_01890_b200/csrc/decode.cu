@@ -23,7 +23,7 @@ struct DecodeParams {
     int B, Hq, Hkv, d, L_cap, L_uniform, n_chunks;
     const int32_t* seq_lens;
     // shared layer
-    const float* prev;
+    const void* prev;       // fp32, or bf16 when row_bf16
     int64_t prev_sb, prev_sh;
     TView qp;
     const void* kpT;
@@ -35,11 +35,24 @@ struct DecodeParams {
     // common
     const void* vcache;
     int cache_dtype;
-    float* out_scores;
+    void* out_scores;       // fp32, or bf16 when row_bf16
     int64_t sc_sb, sc_sh;
+    int row_bf16;           // the score rows handed between layers are bf16 (Sec. 5.2 counts them at 2 bytes) instead of fp32
     float *ws_m, *ws_l, *ws_o;
     TView o;
 };
+
+// Score-row access: RB = rows are bf16.
+template <bool RB>
+__device__ __forceinline__ float ld_row(const void* p, int64_t i) {
+    if constexpr (RB) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i]);
+    else return reinterpret_cast<const float*>(p)[i];
+}
+template <bool RB>
+__device__ __forceinline__ void st_row(void* p, int64_t i, float v) {
+    if constexpr (RB) reinterpret_cast<__nv_bfloat16*>(p)[i] = __float2bfloat16_rn(v);
+    else reinterpret_cast<float*>(p)[i] = v;
+}
 
 __device__ __forceinline__ uint4 ld_stream16(const void* p) {
     uint4 v;
@@ -216,7 +229,7 @@ __device__ __forceinline__ void softmax_pv_chunk(const DecodeParams& p, float* s
 // Shared layer.  HQ_C/M_C > 0: compile-time sizes, aligner on the tensor cores (ADD, two layers, bf16 cache,
 // M_C % 8 == 0, HQ_C % 8 == 0).  HQ_C == 0: any supported mode and size, per-thread scratch arrays.
 // ---------------------------------------------------------------------------------------------
-template <int HQ_C, int M_C>
+template <int HQ_C, int M_C, bool RB>
 __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(16) float smem[];
     const int b = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x;
@@ -296,8 +309,8 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
 
     const int pos = tid & (kChunk - 1), half = tid / kChunk;
     const bool valid = pos < nrows;
-    const float* prev = p.prev + b * p.prev_sb + j0 + pos;
-    float* outrow = p.out_scores ? p.out_scores + b * p.sc_sb + j0 + pos : nullptr;
+    const int64_t prev_i = b * p.prev_sb + j0 + pos;     // this thread's position in the previous layer's row of head 0
+    const int64_t out_i = b * p.sc_sb + j0 + pos;
 
     if constexpr (HQ_C > 0) {
         // ADD, two-layer FFN on the tensor cores (mma.sync m16n8k8, tf32 operands, fp32 accumulation): a warp owns
@@ -310,16 +323,16 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
         const int g = lane >> 2, t = lane & 3;
         const int p0 = warp * 16 + g, p1 = p0 + 8;              // this lane's two position rows
         const bool ok0 = p0 < nrows, ok1 = p1 < nrows;
-        const float* prow = p.prev + b * p.prev_sb + j0;
+        const int64_t prow = b * p.prev_sb + j0;
         uint32_t afr[KS1][4];
 #pragma unroll
         for (int ks = 0; ks < KS1; ++ks) {
-            const float* r0 = prow + (int64_t)(ks * 8 + t) * p.prev_sh;
-            const float* r1 = prow + (int64_t)(ks * 8 + t + 4) * p.prev_sh;
-            afr[ks][0] = f32_to_tf32(ok0 ? r0[p0] : 0.f);
-            afr[ks][1] = f32_to_tf32(ok1 ? r0[p1] : 0.f);
-            afr[ks][2] = f32_to_tf32(ok0 ? r1[p0] : 0.f);
-            afr[ks][3] = f32_to_tf32(ok1 ? r1[p1] : 0.f);
+            const int64_t r0 = prow + (int64_t)(ks * 8 + t) * p.prev_sh;
+            const int64_t r1 = prow + (int64_t)(ks * 8 + t + 4) * p.prev_sh;
+            afr[ks][0] = f32_to_tf32(ok0 ? ld_row<RB>(p.prev, r0 + p0) : 0.f);
+            afr[ks][1] = f32_to_tf32(ok1 ? ld_row<RB>(p.prev, r0 + p1) : 0.f);
+            afr[ks][2] = f32_to_tf32(ok0 ? ld_row<RB>(p.prev, r1 + p0) : 0.f);
+            afr[ks][3] = f32_to_tf32(ok1 ? ld_row<RB>(p.prev, r1 + p1) : 0.f);
         }
         float yacc[NT2][4];
 #pragma unroll
@@ -352,7 +365,7 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
             }
         }
         // scores = FFN + A_Delta; yacc[j2]: [0] (p0, head 8 j2 + 2t), [1] (p0, +1), [2] (p1, 2t), [3] (p1, +1)
-        float* out0 = p.out_scores ? p.out_scores + b * p.sc_sb + j0 : nullptr;
+        const int64_t out0 = b * p.sc_sb + j0;
 #pragma unroll
         for (int j2 = 0; j2 < NT2; ++j2) {
 #pragma unroll
@@ -362,14 +375,14 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
                 const bool okp = (e & 2) ? ok1 : ok0;
                 const float sc = yacc[j2][e] + s_s[hh * kChunk + pp];
                 s_s[hh * kChunk + pp] = okp ? sc : -INFINITY;
-                if (okp && out0) out0[(int64_t)hh * p.sc_sh + pp] = sc;
+                if (okp && p.out_scores) st_row<RB>(p.out_scores, out0 + (int64_t)hh * p.sc_sh + pp, sc);
             }
         }
     } else {
         if (half == 0) {
             float a[kMaxHeads], dl[kMaxHeads], hid[kMaxHidden];
             for (int h = 0; h < Hq; ++h) {
-                a[h] = valid ? prev[h * p.prev_sh] : 0.f;
+                a[h] = valid ? ld_row<RB>(p.prev, prev_i + h * p.prev_sh) : 0.f;
                 dl[h] = s_s[h * kChunk + pos];
             }
             if (p.integrate == LISA_INTEGRATE_PLUS) {
@@ -397,7 +410,7 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
             }
             for (int g = 0; g < Hq; ++g) {
                 s_s[g * kChunk + pos] = valid ? a[g] : -INFINITY;
-                if (valid && outrow) outrow[g * p.sc_sh] = a[g];
+                if (valid && p.out_scores) st_row<RB>(p.out_scores, out_i + g * p.sc_sh, a[g]);
             }
         }
     }
@@ -550,7 +563,10 @@ __global__ void __launch_bounds__(kThreads, 2) anchor_decode_chunk_kernel(const 
     if (p.out_scores) {
         for (int u = tid; u < Hq * kChunk; u += kThreads) {
             const int h = u / kChunk, jj = u % kChunk;
-            if (jj < nrows) p.out_scores[b * p.sc_sb + h * p.sc_sh + j0 + jj] = s_s[u];
+            if (jj < nrows) {
+                if (p.row_bf16) st_row<true>(p.out_scores, b * p.sc_sb + h * p.sc_sh + j0 + jj, s_s[u]);
+                else st_row<false>(p.out_scores, b * p.sc_sb + h * p.sc_sh + j0 + jj, s_s[u]);
+            }
         }
     }
     softmax_pv_chunk(p, s_s, b, chunk, nrows);
@@ -638,22 +654,27 @@ cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cud
     p.w_dtype = a.link.w_dtype;
     p.w1 = a.link.w1; p.b1 = a.link.b1; p.w2 = a.link.w2; p.b2 = a.link.b2;
     p.out_scores = a.out_scores; p.sc_sb = a.scores_stride_b; p.sc_sh = a.scores_stride_h;
+    p.row_bf16 = a.scores_dtype == LISA_BF16;
     p.o = make_view(a.o);
     carve_workspace(p, ws);
     const size_t smem = shared_decode_smem(p.Hq, p.m, p.integrate);
     dim3 grid(p.n_chunks, p.B);
     const bool fast = p.integrate == LISA_INTEGRATE_ADD && p.ffn_layers == 2 && c.dtype == LISA_BF16;
     cudaError_t e;
-    if (fast && p.Hq == 40 && p.m == 80) {
-        if ((e = set_smem(shared_decode_chunk_kernel<40, 80>, smem)) != cudaSuccess) return e;
-        shared_decode_chunk_kernel<40, 80><<<grid, kThreads, smem, s>>>(p);
-    } else if (fast && p.Hq == 32 && p.m == 64) {
-        if ((e = set_smem(shared_decode_chunk_kernel<32, 64>, smem)) != cudaSuccess) return e;
-        shared_decode_chunk_kernel<32, 64><<<grid, kThreads, smem, s>>>(p);
-    } else {
-        if ((e = set_smem(shared_decode_chunk_kernel<0, 0>, smem)) != cudaSuccess) return e;
-        shared_decode_chunk_kernel<0, 0><<<grid, kThreads, smem, s>>>(p);
-    }
+#define LISA_LAUNCH_CHUNK(HQ_, M_)                                                                                 \
+    do {                                                                                                           \
+        if (p.row_bf16) {                                                                                          \
+            if ((e = set_smem(shared_decode_chunk_kernel<HQ_, M_, true>, smem)) != cudaSuccess) return e;          \
+            shared_decode_chunk_kernel<HQ_, M_, true><<<grid, kThreads, smem, s>>>(p);                             \
+        } else {                                                                                                   \
+            if ((e = set_smem(shared_decode_chunk_kernel<HQ_, M_, false>, smem)) != cudaSuccess) return e;         \
+            shared_decode_chunk_kernel<HQ_, M_, false><<<grid, kThreads, smem, s>>>(p);                            \
+        }                                                                                                          \
+    } while (0)
+    if (fast && p.Hq == 40 && p.m == 80) LISA_LAUNCH_CHUNK(40, 80);
+    else if (fast && p.Hq == 32 && p.m == 64) LISA_LAUNCH_CHUNK(32, 64);
+    else LISA_LAUNCH_CHUNK(0, 0);
+#undef LISA_LAUNCH_CHUNK
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, (size_t)p.n_chunks * sizeof(float), s>>>(p);
     count_launches(2);
@@ -669,6 +690,7 @@ cudaError_t launch_anchor_decode(const lisa_anchor_args& a, void* ws, cudaStream
     p.q = make_view(a.q);
     p.kcache = c.k; p.vcache = c.v; p.cache_dtype = c.dtype;
     p.out_scores = a.out_scores; p.sc_sb = a.scores_stride_b; p.sc_sh = a.scores_stride_h;
+    p.row_bf16 = a.scores_dtype == LISA_BF16;
     p.o = make_view(a.o);
     carve_workspace(p, ws);
     const size_t smem = sizeof(float) * ((size_t)p.Hq * kChunk + (size_t)p.Hq * p.d);

@@ -131,6 +131,8 @@ lisa_status_t validate_anchor_decode(const lisa_anchor_args* a) {
     if (a->Nq != 1 || a->B > c.B || a->Hkv != c.Hkv || a->d != c.d) return LISA_ERR_INVALID_ARG;
     if (a->L < 1 || a->L > c.L_cap) return LISA_ERR_INVALID_ARG;
     if ((st = check_tensor(a->q)) != LISA_OK || (st = check_tensor(a->o)) != LISA_OK) return st;
+    if (a->scores_dtype != LISA_F32 && a->scores_dtype != LISA_BF16) return LISA_ERR_INVALID_ARG;
+    if (a->out_scores && (reinterpret_cast<uintptr_t>(a->out_scores) & (a->scores_dtype == LISA_BF16 ? 1u : 3u))) return LISA_ERR_INVALID_ARG;
     return LISA_OK;
 }
 
@@ -143,7 +145,10 @@ lisa_status_t validate_shared_decode(const lisa_shared_decode_args* a) {
     if (a->B > c.B || a->L < 1 || a->L > c.L_cap) return LISA_ERR_INVALID_ARG;
     if (a->link.r != c.r) return LISA_ERR_INVALID_ARG;
     if ((st = check_link(a->link, a->Hq, false)) != LISA_OK) return st;
-    if (!a->prev_scores || (reinterpret_cast<uintptr_t>(a->prev_scores) & 3u)) return LISA_ERR_INVALID_ARG;
+    if (a->scores_dtype != LISA_F32 && a->scores_dtype != LISA_BF16) return LISA_ERR_INVALID_ARG;
+    const uintptr_t row_align = a->scores_dtype == LISA_BF16 ? 1u : 3u;
+    if (!a->prev_scores || (reinterpret_cast<uintptr_t>(a->prev_scores) & row_align)) return LISA_ERR_INVALID_ARG;
+    if (a->out_scores && (reinterpret_cast<uintptr_t>(a->out_scores) & row_align)) return LISA_ERR_INVALID_ARG;
     if (a->out_scores && a->out_scores == a->prev_scores) return LISA_ERR_INVALID_ARG;
     if ((st = check_tensor(a->o)) != LISA_OK) return st;
     // a head count and FFN width whose weights do not fit one CTA's shared memory are outside the kernel's range
@@ -347,6 +352,21 @@ lisa_status_t lisa_attn_shared_decode_static(const lisa_shared_decode_args* a, l
     void* scratch = static_scratch_address(&lookup);
     if (!scratch) return cuda_fail(lookup);
     cudaError_t e = launch_shared_decode(*a, scratch, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+}
+
+lisa_status_t lisa_project(const lisa_project_args* a, lisa_stream_t stream) {
+    if (!a || a->struct_size != sizeof(lisa_project_args)) return LISA_ERR_INVALID_ARG;
+    if (a->B < 1 || a->N < 1 || a->d_in < 1 || a->n_outputs < 1 || a->n_outputs > 4) return LISA_ERR_INVALID_ARG;
+    lisa_status_t st = check_tensor(a->x);
+    if (st != LISA_OK) return st;
+    if (!a->w || !aligned16(a->w) || !dtype_ok(a->w_dtype) || a->w_dtype != a->x.dtype) return LISA_ERR_INVALID_ARG;
+    for (int o = 0; o < a->n_outputs; ++o) {
+        if ((st = check_tensor(a->outputs[o].t)) != LISA_OK) return st;
+        if (a->outputs[o].H < 1 || a->outputs[o].x < 1) return LISA_ERR_INVALID_ARG;
+    }
+    cudaError_t e = (!g_force_general.load() && tc_project_supported(*a)) ? launch_tc_project(*a, static_cast<cudaStream_t>(stream))
+                                                                          : launch_generic_project(*a, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? LISA_OK : cuda_fail(e);
 }
 

@@ -46,7 +46,7 @@ struct AlignParams {
     int64_t plane_rows, plane_cols;
     __half* planes[kMaxTcChain];   // [0] = A_0 in / Y out; [k] = D_k for k = 1..c-1; blocked, see tc_flash.cu
     const void *w1[kMaxTcChain], *b1[kMaxTcChain], *w2[kMaxTcChain], *b2[kMaxTcChain];
-    int w_dtype[kMaxTcChain], act[kMaxTcChain];
+    int w_dtype[kMaxTcChain], act[kMaxTcChain], kind[kMaxTcChain];   // kind: KIND_FFN / KIND_SINGLE / KIND_PLUS
     int store_all;                 // 1: the output of EVERY link k leaves (times log2 e) in plane k, for a chain of layers
     int* status;
 };
@@ -72,7 +72,7 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         // the last link's log2(e) is folded into its W2 and b2, except where every link's output leaves (store_all with
         // more than one link): there the stored values are scaled instead and the chain continues unscaled
         const float out_scale = (k == c - 1 && (!p.store_all || c == 1)) ? kLog2e : 1.f;
-        stage_link_fragments(sW + k * LINK_BYTES, p.w1[k], p.b1[k], p.w2[k], p.b2[k], p.w_dtype[k], out_scale, tid, NT);
+        stage_link_fragments(sW + k * LINK_BYTES, p.w1[k], p.b1[k], p.w2[k], p.b2[k], p.w_dtype[k], p.kind[k], out_scale, tid, NT);
     }
     __syncthreads();
 
@@ -351,7 +351,10 @@ bool tc_align_supported(int Hq, const lisa_link* links, int chain) {
     if (Hq != HQ || chain < 1 || chain > kMaxTcChain) return false;
     for (int k = 0; k < chain; ++k) {
         const lisa_link& l = links[k];
-        if (l.integrate != LISA_INTEGRATE_ADD || l.ffn_layers != 2 || l.m != MH) return false;
+        // ADD with the two-layer 32 -> 64 -> 32 FFN or with one linear 32 x 32 layer; PLUS (no FFN).  CONCAT runs on the general kernel.
+        const bool ffn2 = l.integrate == LISA_INTEGRATE_ADD && l.ffn_layers == 2 && l.m == MH;
+        const bool single = l.integrate == LISA_INTEGRATE_ADD && l.ffn_layers == 1 && l.m == HQ;
+        if (!ffn2 && !single && l.integrate != LISA_INTEGRATE_PLUS) return false;
     }
     return true;
 }
@@ -367,7 +370,8 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
         p.planes[k] = reinterpret_cast<__half*>(a.planes[k]);
         const lisa_link& l = a.links[k];
         p.w1[k] = l.w1; p.b1[k] = l.b1; p.w2[k] = l.w2; p.b2[k] = l.b2;
-        p.w_dtype[k] = l.w_dtype; p.act[k] = l.act;
+        p.kind[k] = link_kind(l.integrate, l.ffn_layers);
+        p.w_dtype[k] = l.w_dtype; p.act[k] = p.kind[k] == KIND_FFN ? l.act : LISA_ACT_NONE;   // only a hidden layer has an activation
     }
     p.store_all = a.store_all ? 1 : 0;
     p.status = status_words();
@@ -380,11 +384,11 @@ cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     const int ctas_per_sm = regw ? kRegwCtas : 1;
     const size_t smem = align_smem_bytes(a.chain, threads, regw ? kRegwStages : kStages, regw ? kRegwPiece : 32);
     auto kernel = tc_align_kernel<false, kWorkers, 1, kStages, 32, -1>;
-    const int act = a.links[0].act;
+    const int act = p.act[0];
     bool bias = false, same_act = true;
     for (int k = 0; k < a.chain; ++k) {
-        bias = bias || a.links[k].b1 || a.links[k].b2;
-        same_act = same_act && a.links[k].act == act;
+        bias = bias || (p.kind[k] != KIND_PLUS && (a.links[k].b1 || (p.kind[k] == KIND_FFN && a.links[k].b2)));
+        same_act = same_act && p.act[k] == act;
     }
     if (!regw && same_act) {
 #define LISA_ALIGN_CHAIN(A_) (bias ? tc_align_kernel<false, kWorkers, 1, kStages, 32, (A_)> : tc_align_kernel<false, kWorkers, 1, kStages, 32, (A_) + 8>)

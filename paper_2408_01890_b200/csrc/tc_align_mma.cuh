@@ -118,32 +118,51 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
 }
 
 
+// What a link's FFN is, as far as this 32 -> 64 -> 32 two-layer engine is concerned.  The variants without a hidden
+// layer run on the same engine with an identity first layer (exact: every hidden unit is one fp16 input times one):
+//   KIND_FFN     y = W2^T act(W1^T a + b1) + b2                       (Sec. 5.1, two-layer FFN, m = 64)
+//   KIND_SINGLE  y = W1^T a + b1, W1 [32, 32]                         (one linear layer, no activation)
+//   KIND_PLUS    y = a                                                 (no FFN: A_n = A_{n-1} + A_Delta)
+constexpr int KIND_FFN = 0, KIND_SINGLE = 1, KIND_PLUS = 2;
+
+__host__ __device__ inline int link_kind(int integrate, int ffn_layers) {
+    return integrate == LISA_INTEGRATE_PLUS ? KIND_PLUS : (ffn_layers == 1 ? KIND_SINGLE : KIND_FFN);
+}
+
 // All nthreads threads of a CTA: one link's weights as ready-made B fragments in shared memory at `dst` (LINK_BYTES):
 // W1 fragments, W2 fragments (times out_scale), b1 as packed fp16 pairs, b2 (times out_scale) as fp32.
 __device__ __forceinline__ void stage_link_fragments(uint8_t* dst, const void* w1, const void* b1, const void* w2, const void* b2, int wd,
-                                                     float out_scale, int tid, int nthreads) {
+                                                     int kind, float out_scale, int tid, int nthreads) {
     uint2* w1f = reinterpret_cast<uint2*>(dst);
     uint2* w2f = reinterpret_cast<uint2*>(dst + W1F_BYTES);
     float* bias = reinterpret_cast<float*>(dst + W1F_BYTES + W2F_BYTES);
-    for (int e = tid; e < 2 * 8 * 32; e += nthreads) {   // W1 [32 heads][64 hidden]: k = head, n = hidden
+    // first layer [32 heads][64 hidden] and second layer [64 hidden][32 heads] as this link's kind defines them
+    auto first = [&](int k, int n) -> float { return kind == KIND_FFN ? ld_elem(w1, k * MH + n, wd) : (k == n ? 1.f : 0.f); };
+    auto second = [&](int k, int n) -> float {
+        if (kind == KIND_FFN) return ld_elem(w2, k * HQ + n, wd);
+        if (kind == KIND_SINGLE) return k < HQ ? ld_elem(w1, k * HQ + n, wd) : 0.f;
+        return k == n ? 1.f : 0.f;
+    };
+    for (int e = tid; e < 2 * 8 * 32; e += nthreads) {   // k = head, n = hidden
         const int ln = e & 31, j = (e >> 5) & 7, ks = e >> 8, g = ln >> 2, t = ln & 3;
         const int k0 = ks * 16 + 2 * t, n = j * 8 + g;
         uint2 w;
-        w.x = pack_f16(ld_elem(w1, k0 * MH + n, wd), ld_elem(w1, (k0 + 1) * MH + n, wd));
-        w.y = pack_f16(ld_elem(w1, (k0 + 8) * MH + n, wd), ld_elem(w1, (k0 + 9) * MH + n, wd));
+        w.x = pack_f16(first(k0, n), first(k0 + 1, n));
+        w.y = pack_f16(first(k0 + 8, n), first(k0 + 9, n));
         w1f[e] = w;
     }
-    for (int e = tid; e < 4 * 4 * 32; e += nthreads) {   // W2 [64 hidden][32 heads]: k = hidden, n = head
+    for (int e = tid; e < 4 * 4 * 32; e += nthreads) {   // k = hidden, n = head
         const int ln = e & 31, j2 = (e >> 5) & 3, s2 = e >> 7, g = ln >> 2, t = ln & 3;
         const int k0 = s2 * 16 + 2 * t, n = j2 * 8 + g;
         uint2 w;
-        w.x = pack_f16(ld_elem(w2, k0 * HQ + n, wd) * out_scale, ld_elem(w2, (k0 + 1) * HQ + n, wd) * out_scale);
-        w.y = pack_f16(ld_elem(w2, (k0 + 8) * HQ + n, wd) * out_scale, ld_elem(w2, (k0 + 9) * HQ + n, wd) * out_scale);
+        w.x = pack_f16(second(k0, n) * out_scale, second(k0 + 1, n) * out_scale);
+        w.y = pack_f16(second(k0 + 8, n) * out_scale, second(k0 + 9, n) * out_scale);
         w2f[e] = w;
     }
     for (int e = tid; e < MH / 2; e += nthreads)   // b1 as packed fp16 pairs (the first layer's accumulator format)
-        reinterpret_cast<uint32_t*>(bias)[e] = pack_f16(ldw(b1, 2 * e, wd), ldw(b1, 2 * e + 1, wd));
-    for (int e = tid; e < HQ; e += nthreads) bias[MH + e] = ldw(b2, e, wd) * out_scale;
+        reinterpret_cast<uint32_t*>(bias)[e] = kind == KIND_FFN ? pack_f16(ldw(b1, 2 * e, wd), ldw(b1, 2 * e + 1, wd)) : 0u;
+    for (int e = tid; e < HQ; e += nthreads)
+        bias[MH + e] = (kind == KIND_FFN ? ldw(b2, e, wd) : (kind == KIND_SINGLE ? ldw(b1, e, wd) : 0.f)) * out_scale;
 }
 
 // Byte offset of 16-byte chunk `chunk` (0..7) of head `head` inside a [32 heads][64 positions] fp16 piece (one 128-byte line

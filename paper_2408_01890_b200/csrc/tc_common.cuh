@@ -40,12 +40,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Waits for the phase with the given parity to complete.  Bounded: gives up after about 4e9 SM cycles (two
-// seconds), or as soon as another thread of the CTA has given up (*abort_flag != 0); then sets the flag and
-// returns false.  Callers leave their loops on false and fall through to the CTA's common teardown.
+// Waits for the phase with the given parity to complete.  Bounded: gives up after `limit_cycles` SM cycles (by
+// default about 4e9, two seconds), or as soon as another thread of the CTA has given up (*abort_flag != 0); then
+// sets the flag and returns false.  Callers leave their loops on false and fall through to the CTA's common teardown.
 // The limit is kept on the SM-local cycle counter, read only every 1024 failed polls: the global nanosecond
 // timer is far too slow to read inside a wait that normally lasts a few hundred cycles.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+constexpr long long kWaitLimitCycles = 4000000000ll;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, long long limit_cycles = kWaitLimitCycles) {
     uint32_t spins = 0;
     long long t0 = 0;
     while (true) {
@@ -54,7 +55,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > 4000000000ll) {
+            else if (now - t0 > limit_cycles) {
                 *abort_flag = 1;
                 return false;
             }

@@ -8,7 +8,10 @@ from paper_2408_01890_b200 import synth
 
 # Tolerances: bf16 inputs with fp32 accumulation (the stated bar); fp32 inputs (from fp32 rounding of
 # ~1e2..1e4-term sums of O(1) values: a few 1e-6 relative; one decade of margin).
-TOL = {"bf16": dict(max_abs=2e-2, rel_rms=5e-3), "f32": dict(max_abs=1e-4, rel_rms=1e-5)}
+# "row_tf32": an fp32 score row that went through the decode kernel's FFN on tf32 tensor-core operands (10 mantissa
+# bits: relative rounding 2^-11 uniform, i.e. 2.8e-4 rms, on the row and again on the hidden activations; the two layers sum
+# 40..80 such terms of total variance ~1 each, so the row's error is ~4e-4 rms and ~2e-3 at the 5-sigma tail of 1e6 entries).
+TOL = {"bf16": dict(max_abs=2e-2, rel_rms=5e-3), "f32": dict(max_abs=1e-4, rel_rms=1e-5), "row_tf32": dict(max_abs=3e-3, rel_rms=6e-4)}
 ACT = {"none": (lb.ACT_NONE, oracle.ACT_NONE), "relu": (lb.ACT_RELU, oracle.ACT_RELU), "silu": (lb.ACT_SILU, oracle.ACT_SILU)}
 
 

@@ -141,3 +141,45 @@ def test_decode_rejects_bad_arguments():
     with pytest.raises(lb.LisaError) as e:
         lb.lisa_attn_shared_decode(prev, link, cache, L=16, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
     assert e.value.status == lb.ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("Hq,Hkv,d,r,m,L", [(40, 40, 128, 21, 80, 700), (8, 2, 64, 21, 16, 300)])
+def test_bf16_score_rows(Hq, Hkv, d, r, m, L):
+    """Score rows handed between decode layers as bf16 (2 bytes per entry, the size Sec. 5.2 counts).  The layer reads the
+    bf16 row exactly (the oracle gets the same rounded values), so its output stays within the usual bar; the row it writes
+    is the oracle's row rounded to bf16 once more: relative 2^-8 at worst (half an ulp of 8 mantissa bits is 2^-9; the kernel's
+    own fp32/tf32 arithmetic can move a value across a rounding boundary), which is what the hand-off costs per layer.
+    The standard layer's row is checked the same way."""
+    B = 2
+    w = synth.Workload("rows16", "bf16", B, L, Hq, Hkv, d, r, m, "relu", 1, True)
+    t = synth.decode_inputs(w, 8, B=B, L=L)
+    L_cap = (L + 7) // 8 * 8
+    lens_h = np.array([L, L // 2 + 1], dtype=np.int32)
+    lens_d = torch.from_numpy(lens_h).cuda()
+    prev16 = t["prev"].to(torch.bfloat16)
+    cache = fill_shared_cache(w, t, B, L, L_cap, torch.bfloat16)
+    link = lb.Link(dev(t["qp"]), None, dev(t["w1"]), dev(t["w2"]), act=lb.ACT_RELU)
+    row = torch.full((B, Hq, L_cap), -7.0, dtype=torch.bfloat16, device="cuda")
+    out = lb.lisa_attn_shared_decode(dev(prev16), link, cache, L=L, seq_lens=lens_d, out_scores=row)
+    torch.cuda.synchronize()
+    olink = oracle.Link(None, None, f64(t["w1"]), f64(t["w2"]), r=r, act=oracle.ACT_RELU)
+    O, R = oracle.decode_shared(f64(prev16), f64(t["qp"])[:, 0], f64(t["kp"]), f64(t["v"]), olink, lens_h)
+    assert_close(out[:, 0].float().cpu().numpy(), O, "bf16", "decode O from a bf16 row")
+    row_h = row.float().cpu().numpy()
+    for b in range(B):
+        got, ref = row_h[b, :, :lens_h[b]], R[b, :, :lens_h[b]]
+        assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 3e-3), "bf16 row beyond one rounding of the oracle's row"
+        assert np.all(row_h[b, :, lens_h[b]:] == -7.0), "row written beyond the sequence length"
+    # standard layer emitting a bf16 row
+    st = lb.KVCacheLayer(lb.CACHE_STANDARD, B, Hkv, L_cap, d)
+    lb.lisa_kvcache_append(st, dev(t["k"]), dev(t["v"]))
+    row0 = torch.full((B, Hq, L_cap), -7.0, dtype=torch.bfloat16, device="cuda")
+    out0 = lb.lisa_attn_anchor(dev(t["q0"]), cache=st, L=L, seq_lens=lens_d, out_scores=row0)
+    O0, R0 = oracle.decode_anchor(f64(t["q0"])[:, 0], f64(t["k"]), f64(t["v"]), lens_h)
+    assert_close(out0[:, 0].float().cpu().numpy(), O0, "bf16", "standard decode O with a bf16 row")
+    r0 = row0.float().cpu().numpy()
+    for b in range(B):
+        got, ref = r0[b, :, :lens_h[b]], R0[b, :, :lens_h[b]]
+        assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-4)
+        assert np.all(r0[b, :, lens_h[b]:] == -7.0)
+    assert lb.lisa_check() == lb.OK

@@ -89,3 +89,15 @@ def test_shared_prefill_chain_rejects_bad_arguments():
 def test_shared_prefill_tensor_core_bias_and_rank():
     run_tc_shared(1, 260, 32, 2, "relu", seed=3, bias=True, r=32)
     run_tc_shared(1, 140, 32, 1, "silu", seed=4, bias=True, r=8)
+
+
+def test_bounded_wait_runs_out_and_the_context_survives():
+    """A device-side wait that nothing satisfies gives up by itself: the status word reports it once (LISA_ERR_TIMEOUT),
+    the next check is clean, and a tensor-core prefill launched right after still matches the oracle."""
+    assert lb.lisa_check() == lb.OK
+    lb.lisa_debug_wait_timeout(1000000)          # about half a millisecond of waiting, then the kernel returns
+    assert lb.lisa_check() == lb.ERR_TIMEOUT
+    assert lb.lisa_check() == lb.OK
+    run_tc_shared(1, 256, 32, 1, "relu", seed=5)
+    with pytest.raises(lb.LisaError):
+        lb.lisa_debug_wait_timeout(10 ** 12)     # limits beyond 1e8 cycles are refused before anything is launched
