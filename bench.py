@@ -364,14 +364,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-decode", action="store_true", help="skip the decode section")
     ap.add_argument("--no-stack", action="store_true", help="skip the 32-layer stack section")
-    ap.add_argument("--only", choices=["prefill", "cfg2", "decode"], default=None,
+    ap.add_argument("--only", choices=["prefill", "cfg2", "decode", "project"], default=None,
                     help="profiling aid: run just that section (prefill: the headline step; cfg2: the LLaMA2-7B-shaped layer; "
                          "neither runs the end-to-end, decode, stack or CPU legs)")
     ap.add_argument("--decode-batch", type=int, default=0, help="profiling aid: decode batch size (default: the workload's 64)")
     args = ap.parse_args()
     if args.only is None:
         args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.only in ("prefill", "cfg2"):
+    if args.only in ("prefill", "cfg2", "project"):
         args.no_decode = args.no_stack = True
     if args.only == "decode":
         args.no_stack = True
@@ -409,6 +409,35 @@ def main():
     if args.only in (None, "cfg2"):
         second = bench_prefill(lb, SECOND, rank, args, env, with_chain=False, with_e2e=args.only is None)
         launches += second["launches"]
+
+    # ---------------- the fused projection H.[W_Q' | W_K' | W_V] of a shared layer (LLaMA2-7B widths) ----------------
+    project = None
+    if args.only in (None, "project"):
+        Bp, Np, dm, Hh, rr, dd = 8, 2048, 4096, 32, 21, 128
+        g = torch.Generator(device="cuda"); g.manual_seed(1234 + rank)
+        xh = torch.randn((Bp, Np, dm), generator=g, device="cuda").to(torch.bfloat16)
+        n_out = Hh * rr + Hh * rr + Hh * dd
+        wp = (torch.randn((dm, n_out), generator=g, device="cuda") * dm ** -0.5).to(torch.bfloat16)
+        pouts = [torch.empty((Bp, Np, Hh, rr), dtype=torch.bfloat16, device="cuda"), torch.empty((Bp, Np, Hh, rr), dtype=torch.bfloat16, device="cuda"),
+                 torch.empty((Bp, Np, Hh, dd), dtype=torch.bfloat16, device="cuda")]
+
+        def project_step():
+            lb.lisa_project(xh, wp, pouts)
+            return []
+
+        for _ in range(args.warmup):
+            flush(); project_step()
+        l1 = lb.lisa_kernel_launches()
+        ptot, _, _ = time_steps(project_step, args.steps, flush, barrier)
+        launches += lb.lisa_kernel_launches() - l1
+        pms = max_over_ranks(ptot) / args.steps
+        pflops = 2.0 * Bp * Np * dm * n_out
+        ptf = pflops / (pms * 1e-3) / 1e12
+        project = {"call": "lisa_project", "rows": Bp * Np, "d_in": dm, "n_out": n_out, "outputs": "Q' [%d x %d], K' [%d x %d], V [%d x %d]" % (Hh, rr, Hh, rr, Hh, dd),
+                   "ms": pms, "value": world * Bp * Np / (pms * 1e-3), "unit": "tokens/s",
+                   "roofline": {"bound": "tensor", "achieved": ptf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ptf / peaks["bf16_tflops"],
+                                "peak_source": peaks["source"] + " (burst)", "flops_per_launch": pflops, "traffic": None}}
+        del xh, wp, pouts
 
     # ---------------- decode step and the library's own standard-attention decode ----------------
     decode = None
@@ -531,6 +560,9 @@ def main():
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "clocks": clocks, "gpu_launches": int(launches)}
         main_res = head or second
+        if main_res is None and project is not None:
+            line.update({"value": project["value"], "ms_per_step": project["ms"], "config": {"workload": "projection " + project["outputs"]},
+                         "roofline": project["roofline"]})
         if main_res is not None:
             w = synth.WORKLOADS[main_res["workload"]]
             cfg = workload_config(w)
@@ -539,7 +571,7 @@ def main():
         if head is not None and second is not None:
             line["cfg2"] = {"workload": second["workload"], "value": second["value"], "unit": "tokens/s", "ms_per_step": second["ms_per_step"],
                             "e2e": second.get("e2e"), "roofline": second["roofline"]}
-        line.update({"cpu_baseline": cpu, "decode": decode, "stack": stack})
+        line.update({"cpu_baseline": cpu, "project": project, "decode": decode, "stack": stack})
         print(json.dumps(line))
     group.close()
 

@@ -65,10 +65,7 @@ struct Smem {
     static constexpr bool P_IN_Y = PLANE;
     static constexpr bool P_IN_K = !EMIT && !PLANE && KD == 128;
     static constexpr bool P_OWN = !EMIT && !P_IN_Y && !P_IN_K;
-    static constexpr int KST = (EMIT || P_IN_K) ? 3 : 2;  // K ring depth (V: two stages)
-    // The plane tiles Y come straight from HBM and are needed at the very start of a tile's softmax, so they travel in a
-    // ring of their own, three deep, loaded two tiles ahead (a V stage, by contrast, is needed only by the P.V MMA).
-    static constexpr int YST = 3;
+    static constexpr int KST = (EMIT || P_IN_K) ? 3 : 2;  // K ring depth (V/Y: two stages)
     static constexpr int Q_BYTES = BM * KD * 2;
     static constexpr int K_BYTES = BN * KD * 2;
     static constexpr int V_BYTES = EMIT ? 0 : BN * D * 2;
@@ -81,7 +78,7 @@ struct Smem {
     static constexpr int OFF_V = OFF_K + KST * K_BYTES;
     static constexpr int OFF_P = OFF_V + 2 * V_BYTES;
     static constexpr int OFF_Y = OFF_P + P_OWN_BYTES;
-    static constexpr int OFF_STG = OFF_Y + YST * Y_BYTES;
+    static constexpr int OFF_STG = OFF_Y + 2 * Y_BYTES;
     static constexpr int OFF_BAR = OFF_STG + STG_BYTES;
     static constexpr int TOTAL = OFF_BAR + 256;
     static constexpr uint32_t TMEM_COLS = EMIT ? 128 : 256;   // S[2]: [0,128), O: [128,256)
@@ -120,13 +117,11 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     uint64_t* s_free = bars + 13;   // [2] score buffer copied to registers by all 128 rows
     uint64_t* p_full = bars + 15;   // [2]
     uint64_t* pv_done = bars + 17;  // [2]
-    uint64_t* y_full = bars + 19;   // [YST] plane tile landed
-    uint64_t* y_empty = bars + 22;  // [YST] the P.V MMA that read P out of this stage has completed
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 25);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 26);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 19);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 20);
     // P of tile t
     auto p_buf = [&](int t) -> uint8_t* {
-        if constexpr (L::P_IN_Y) return sY + (t % L::YST) * L::Y_BYTES;
+        if constexpr (L::P_IN_Y) return sY + (t & 1) * L::Y_BYTES;
         else if constexpr (L::P_IN_K) return sK + (t % KST) * L::K_BYTES;
         else return sP + (t & 1) * L::P_BYTES;
     };
@@ -148,7 +143,6 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             mbar_init(s_full + i, 1); mbar_init(s_free + i, 128);
             mbar_init(p_full + i, 128); mbar_init(pv_done + i, 1);
         }
-        for (int i = 0; i < L::YST; ++i) { mbar_init(y_full + i, 1); mbar_init(y_empty + i, 1); }
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -170,8 +164,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         // get an instruction slot every several cycles, so their loops are kept to a few dozen instructions per tile:
         // running stage counters instead of divisions, one wait/arm section by lane 0 per tile, then every copy of
         // the tile issued by different lanes (one 64-column box each).
-        // V(t) travels together with K(t+1): both wait for the P.V of tile t-2 at the latest.  Y(t+2) follows them: its
-        // stage is the one tile t-1 used, free once the P.V of tile t-1 has completed.
+        // V(t) (with Y(t)) travels together with K(t+1): both wait for the P.V of tile t-2 at the latest.
         constexpr int NQ = KD / 64, NK = KD / 64, NV = EMIT ? 0 : D / 64;
         if (lane == 0) {
             tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
@@ -187,16 +180,6 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
         __syncwarp();
         if (lane < NK) tma_load_4d(sK + lane * (BN * 128), &tmK, k_full, lane * 64, g, 0, b);
         __syncwarp();
-        const int y_rb = (q0 - p.plane_row0) / BM;
-        if constexpr (PLANE) {
-            if (lane < 2 && lane < nt) {     // Y(0) and Y(1): their stages are fresh
-                mbar_expect_tx(y_full + lane, L::Y_BYTES);
-                tma_load_5d(sY + lane * L::Y_BYTES, &tmY, y_full + lane, 0, b * p.Hq + h, 0, lane, y_rb);
-            }
-            __syncwarp();
-        }
-        int ys_next = 2 % L::YST;           // Y stage of tile t+2
-        uint32_t ypar_next = 1;             // its "empty" parity (first pass over the ring: passes at once)
         int ks_next = 1 % KST;              // K stage of tile t+1
         uint32_t kpar_next = 1;             // parity to wait for on its "empty" barrier (first pass: passes at once)
         for (int t = 0; t < nt; ++t) {
@@ -206,7 +189,7 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             if (lane == 0) {
                 if constexpr (!EMIT) {
                     okp = mbar_wait(v_empty + sv, ((t >> 1) & 1) ^ 1, abort_flag);
-                    if (okp) mbar_expect_tx(v_full + sv, L::V_BYTES);
+                    if (okp) mbar_expect_tx(v_full + sv, L::V_BYTES + L::Y_BYTES);
                 }
                 if (okp && more_k) {
                     okp = mbar_wait(k_empty + ks_next, kpar_next, abort_flag);
@@ -219,26 +202,15 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 if (lane < NV) tma_load_4d(sV + sv * L::V_BYTES + lane * (BN * 128), &tmV, v_full + sv, lane * 64, g, t * BN, b);
                 __syncwarp();
             }
+            if constexpr (PLANE) {
+                if (lane == 0) tma_load_5d(sY + sv * L::Y_BYTES, &tmY, v_full + sv, 0, b * p.Hq + h, 0, t, (q0 - p.plane_row0) / BM);
+                __syncwarp();
+            }
             if (more_k) {
                 if (lane < NK) tma_load_4d(sK + ks_next * L::K_BYTES + lane * (BN * 128), &tmK, k_full + ks_next, lane * 64, g, (t + 1) * BN, b);
                 __syncwarp();
             }
             if (++ks_next == KST) { ks_next = 0; kpar_next ^= 1; }
-            if constexpr (PLANE) {
-                if (t + 2 < nt) {
-                    bool oky = true;
-                    if (lane == 0) {
-                        oky = mbar_wait(y_empty + ys_next, ypar_next, abort_flag);
-                        if (oky) {
-                            mbar_expect_tx(y_full + ys_next, L::Y_BYTES);
-                            tma_load_5d(sY + ys_next * L::Y_BYTES, &tmY, y_full + ys_next, 0, b * p.Hq + h, 0, t + 2, y_rb);
-                        }
-                    }
-                    oky = __shfl_sync(0xffffffffu, oky, 0);
-                    if (!oky) break;
-                }
-                if (++ys_next == L::YST) { ys_next = 0; ypar_next ^= 1; }
-            }
         }
     } else if (warp == 5) {
         // ------------------------------ MMA issuer: scores ------------------------------
@@ -291,14 +263,13 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             const uint64_t dp0 = umma_desc_sw128(smem_u32(p_buf(0)), 16, 1024);
             constexpr uint32_t P_STRIDE = L::P_IN_Y ? L::Y_BYTES : (L::P_IN_K ? L::K_BYTES : L::P_BYTES);
             int pk = 0;   // P_IN_K: K stage that holds P(t)
-            int py = 0;   // P_IN_Y: Y stage that holds P(t)
             bool ok = true;
             for (int t = 0; ok && t < nt; ++t) {
                 const int s = t & 1;
                 ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag) && mbar_wait(p_full + s, (t >> 1) & 1, abort_flag);
                 if (!(ok = __all_sync(0xffffffffu, ok))) break;
                 tc_fence_after();
-                const uint64_t dp = desc_off(dp0, (L::P_IN_K ? pk : (L::P_IN_Y ? py : s)) * P_STRIDE);
+                const uint64_t dp = desc_off(dp0, (L::P_IN_K ? pk : s) * P_STRIDE);
                 const uint64_t dv = desc_off(dv0, s * L::V_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < BN / 16; ++ks) {
@@ -310,8 +281,6 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 if (t + 2 < nt) umma_commit_if(issue, v_empty + s);
                 if (L::P_IN_K && t + KST < nt) umma_commit_if(issue, k_empty + pk);
                 if (++pk == KST) pk = 0;
-                if (L::P_IN_Y && t + L::YST < nt) umma_commit_if(issue, y_empty + py);
-                if (++py == L::YST) py = 0;
             }
         }
     }
@@ -359,8 +328,8 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                 continue;
             }
             if constexpr (PLANE) {
-                if (!(ok = mbar_wait(y_full + t % L::YST, (uint32_t)(t / L::YST) & 1u, abort_flag))) break;  // Y(t) has landed
-                const uint8_t* yb = sY + (t % L::YST) * L::Y_BYTES;
+                if (!(ok = mbar_wait(v_full + s, (t >> 1) & 1, abort_flag))) break;  // Y of this stage has landed
+                const uint8_t* yb = sY + s * L::Y_BYTES;
 #pragma unroll
                 for (int c = 0; c < BN / 8; ++c) {
                     const uint4 y = *reinterpret_cast<const uint4*>(yb + sw128_offset(row, c));

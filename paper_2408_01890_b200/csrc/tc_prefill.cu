@@ -102,8 +102,13 @@ int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves) {
     return n;
 }
 
+// The concatenating Integrate feeds every link's difference to its FFN as a plane of its own, the top link's included:
+// one plane more than the adding forms, where the attention kernel adds the top link's difference itself.
+bool concat_chain(const lisa_shared_prefill_args& a) { return a.chain_len > 0 && a.links[0].integrate == LISA_INTEGRATE_CONCAT; }
+int plane_count(const lisa_shared_prefill_args& a) { return a.chain_len + (concat_chain(a) ? 1 : 0); }
+
 struct Layout {
-    size_t qp_off[kMaxChain], kp_off[kMaxChain], plane_off[kMaxChain];
+    size_t qp_off[kMaxChain], kp_off[kMaxChain], plane_off[kMaxChain + 1];
     int64_t plane_rows, plane_cols;
     size_t total;
 };
@@ -118,12 +123,12 @@ Layout plan_layout(const lisa_shared_prefill_args& a) {
     }
     const int n_qt = (a.N + kTile - 1) / kTile;
     Wave waves[1024];
-    const int nw = plan_waves(a.B, a.N, a.Hq, a.chain_len, waves, 1024);
+    const int nw = plan_waves(a.B, a.N, a.Hq, plane_count(a), waves, 1024);
     int max_cnt = 1;
     for (int i = 0; i < std::min(nw, 1024); ++i) max_cnt = std::max(max_cnt, waves[i].count);
     l.plane_rows = (int64_t)max_cnt * kTile;
     l.plane_cols = (int64_t)n_qt * kTile;
-    for (int k = 0; k < a.chain_len; ++k) l.plane_off[k] = take((size_t)a.B * a.Hq * l.plane_rows * l.plane_cols * 2);
+    for (int k = 0; k < plane_count(a); ++k) l.plane_off[k] = take((size_t)a.B * a.Hq * l.plane_rows * l.plane_cols * 2);
     l.total = off;
     return l;
 }
@@ -146,7 +151,7 @@ cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int
 
 bool tc_shared_prefill_supported(const lisa_shared_prefill_args& a) {
     if (a.d != 128 || a.chain_len < 1 || a.N > kTile * 1024) return false;
-    if (!tc_align_supported(a.Hq, a.links, a.chain_len)) return false;
+    if (!tc_align_supported(a.Hq, a.links, a.chain_len) && !tc_align_concat_supported(a.Hq, a.links, a.chain_len)) return false;
     for (int k = 0; k < a.chain_len; ++k)
         if (a.links[k].qp.dtype != LISA_BF16 || a.links[k].kp.dtype != LISA_BF16 || a.links[k].r > 32) return false;
     TcFlashArgs f{a.B, a.N, a.Hq, a.Hkv, 128, a.q0, a.k0, a.v, a.o, 1.f, nullptr, 0, 0, 0, 1};
@@ -233,8 +238,9 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         std::lock_guard<std::mutex> lock(g_side_mutex);
         return cudaStreamWaitEvent(s, side->join, 0);
     };
+    const bool concat = concat_chain(a);
     Wave waves[1024];
-    const int nw = plan_waves(a.B, a.N, a.Hq, c, waves, 1024);
+    const int nw = plan_waves(a.B, a.N, a.Hq, plane_count(a), waves, 1024);
     for (int w = 0; w < nw; ++w) {
         const Wave wv = waves[w];
         // 1. anchor scores and the differences of the links below the top one
@@ -245,7 +251,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             PhaseMark mark(1, s);
             if ((e = launch_tc_flash(f, s)) != cudaSuccess) return e;
         }
-        for (int k = 0; k + 1 < c; ++k) {
+        for (int k = 0; k + (concat ? 0 : 1) < c; ++k) {   // the concatenating form also needs the top link's difference as a plane
             if ((e = join_pack()) != cudaSuccess) return e;
             PhaseMark mark(1, s);
             TcFlashArgs fd = f;
@@ -256,6 +262,31 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             fd.ksteps = (a.links[k].r + 15) / 16;
             fd.emit_plane = base + l.plane_off[k + 1];
             if ((e = launch_tc_flash(fd, s)) != cudaSuccess) return e;
+        }
+        if (concat) {
+            // 2c. link by link: A_k = FFN_k([A_{k-1}; D_k]) over plane 0; log2(e) * A_k over D_k's plane where a layer's
+            // attention consumes it (the top link's; every link's when all layers of the chain are computed)
+            for (int k = 0; k < c; ++k) {
+                TcAlignConcatArgs ac{a.B, a.N, wv.begin, wv.count, l.plane_rows, l.plane_cols, base + l.plane_off[0], base + l.plane_off[k + 1],
+                                     &a.links[k], k + 1 < c, all_layers || k == c - 1};
+                PhaseMark mark(2, s);
+                if ((e = launch_tc_align_concat(ac, s)) != cudaSuccess) return e;
+            }
+            // 3c. softmax and .V on the finished scores: the attention kernel's own difference is switched off (scale 0)
+            for (int k = all_layers ? 0 : c - 1; k < c; ++k) {
+                TcFlashArgs fv = f;
+                fv.emit_plane = nullptr;
+                fv.kd = kPadRank;
+                fv.qa = packed_view(base + l.qp_off[k], a.Hq, a.N);
+                fv.ka = packed_view(base + l.kp_off[k], a.Hkv, a.N);
+                fv.scale = 0.f;
+                fv.ksteps = 1;
+                fv.plane = base + l.plane_off[k + 1];
+                if (all_layers) { fv.v = vs[k]; fv.o = os[k]; }
+                PhaseMark mark(3, s);
+                if ((e = launch_tc_flash(fv, s)) != cudaSuccess) return e;
+            }
+            continue;
         }
         // 2. the FFN chain over the head axis, in place
         TcAlignArgs al{};

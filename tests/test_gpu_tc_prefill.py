@@ -101,3 +101,75 @@ def test_bounded_wait_runs_out_and_the_context_survives():
     run_tc_shared(1, 256, 32, 1, "relu", seed=5)
     with pytest.raises(lb.LisaError):
         lb.lisa_debug_wait_timeout(10 ** 12)     # limits beyond 1e8 cycles are refused before anything is launched
+
+
+@pytest.mark.parametrize("integrate,layers,chain,r,bias", [
+    (lb.INTEGRATE_ADD, 1, 1, 32, True),       # one linear 32 x 32 layer over the heads, r = 32
+    (lb.INTEGRATE_ADD, 1, 3, 21, False),
+    (lb.INTEGRATE_PLUS, 2, 1, 20, False),     # no FFN: A_n = A_{n-1} + A_Delta (Sec. 6.3's variant for pre-trained sharing)
+    (lb.INTEGRATE_PLUS, 2, 3, 21, False)])
+def test_variants_without_a_hidden_layer_run_on_the_tensor_cores(integrate, layers, chain, r, bias):
+    """32 heads, d = 128: the one-layer aligner and the FFN-free variant take the tensor-core path (seen in the launch count:
+    pack, one emit per plane, align, attention) and match the oracle like the two-layer FFN does."""
+    B, N, Hkv = 1, 300, 8
+    w = synth.Workload("tc_variant", "bf16", B, N, 32, Hkv, 128, r, 32, "none", chain)
+    t = synth.prefill_inputs(w, 13)
+    for k in range(1, chain + 1):
+        t[f"w1_{k}"] = synth.as_dtype(synth.normal(f"w1_{k}", (32, 32), 13, std=32 ** -0.5), "bf16")
+        t[f"b1_{k}"] = synth.as_dtype(synth.normal(f"b1_{k}", (32,), 13, std=0.5), "bf16")
+    dl, ol = make_links(t, chain, "none", integrate, layers, bias)
+    n0 = lb.lisa_kernel_launches()
+    got = lb.lisa_attn_shared_prefill(dev(t["q0"]), dev(t["k0"]), dl, dev(t[f"v{chain}"]))
+    torch.cuda.synchronize()
+    assert lb.lisa_kernel_launches() - n0 == chain + 3
+    assert lb.lisa_check() == lb.OK
+    ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{chain}"]), ol)
+    assert_close(got.float().cpu().numpy(), ref, "bf16", "tensor-core prefill, variant without a hidden layer")
+
+
+def concat_inputs(B, N, Hkv, chain, m, act, layers, r, seed, bias):
+    w = synth.Workload("tc_concat", "bf16", B, N, 32, Hkv, 128, r, m, act, chain)
+    t = synth.prefill_inputs(w, seed)
+    mm = 32 if layers == 1 else m
+    for k in range(1, chain + 1):
+        t[f"w1_{k}"] = synth.as_dtype(synth.normal(f"w1_{k}", (64, mm), seed, std=64 ** -0.5), "bf16")
+        t[f"w2_{k}"] = synth.as_dtype(synth.normal(f"w2_{k}", (mm, 32), seed, std=mm ** -0.5), "bf16")
+        t[f"b1_{k}"] = synth.as_dtype(synth.normal(f"b1_{k}", (mm,), seed, std=0.5), "bf16")
+        t[f"b2_{k}"] = synth.as_dtype(synth.normal(f"b2_{k}", (32,), seed, std=0.5), "bf16")
+    return t
+
+
+@pytest.mark.parametrize("B,N,Hkv,chain,m,act,layers,r,bias", [
+    (1, 300, 32, 1, 256, "relu", 2, 20, False),    # the paper's complete model: FFN 64 x 256, 256 x 32, ReLU, r = 20
+    (2, 200, 8, 2, 64, "silu", 2, 21, True),
+    (1, 260, 32, 3, 200, "relu", 2, 21, True),     # hidden width that is not a multiple of 64
+    (1, 300, 8, 1, 32, "none", 1, 32, True),       # one linear 64 x 32 layer, r = 32
+    (1, 150, 32, 2, 32, "none", 1, 21, False)])
+def test_concatenating_integrate_runs_on_the_tensor_cores(B, N, Hkv, chain, m, act, layers, r, bias):
+    """Integrate by concatenation (Sec. 5.1, the overview's complete model): [A_{n-1}; A_Delta] through the FFN, 32 heads,
+    d = 128, on the tensor-core path (launches: pack, A_0 and one difference plane per link, one aligner pass per link,
+    attention) against the oracle."""
+    t = concat_inputs(B, N, Hkv, chain, m, act, layers, r, 17, bias)
+    dl, ol = make_links(t, chain, act, lb.INTEGRATE_CONCAT, layers, bias)
+    n0 = lb.lisa_kernel_launches()
+    got = lb.lisa_attn_shared_prefill(dev(t["q0"]), dev(t["k0"]), dl, dev(t[f"v{chain}"]))
+    torch.cuda.synchronize()
+    assert lb.lisa_kernel_launches() - n0 == 2 * chain + 3
+    assert lb.lisa_check() == lb.OK
+    ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{chain}"]), ol)
+    assert_close(got.float().cpu().numpy(), ref, "bf16", "tensor-core prefill, concatenating integrate")
+
+
+def test_concatenating_chain_in_one_pass():
+    """lisa_attn_shared_prefill_chain with the concatenating Integrate: every layer of the chain against the oracle."""
+    B, N, Hkv, chain = 1, 300, 8, 3
+    t = concat_inputs(B, N, Hkv, chain, 256, "relu", 2, 20, 19, False)
+    dl, ol = make_links(t, chain, "relu", lb.INTEGRATE_CONCAT, 2, False)
+    n0 = lb.lisa_kernel_launches()
+    outs = lb.lisa_attn_shared_prefill_chain(dev(t["q0"]), dev(t["k0"]), dl, [dev(t[f"v{k}"]) for k in range(1, chain + 1)])
+    torch.cuda.synchronize()
+    assert lb.lisa_kernel_launches() - n0 == 1 + (1 + chain) + chain + chain   # pack, planes, aligner passes, one attention per layer
+    for k in range(chain):
+        ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1])
+        assert_close(outs[k].float().cpu().numpy(), ref, "bf16", "concatenating chain, layer %d" % (k + 1))
+    assert lb.lisa_check() == lb.OK
