@@ -7,12 +7,9 @@
 //            standard: A[h,j] = q_h.K_j/sqrt(d)                                           (Eq. 2)
 //            and, if asked, the fp32 row handed to the next shared layer
 //   phase B  chunk-local softmax statistics (max, sum) per head and the partial product with V
-// The per-chunk partials (m, l, o) are merged into the output (split-K softmax) by the sequence's last chunk CTA to
-// finish (merge_if_last); batches beyond the ticket words' capacity fall back to a merge kernel of their own.
+// A second kernel merges the per-chunk partials (m, l, o) into the output (split-K softmax).
 // K' is cached transposed ([r][L_cap], position contiguous) so that r = 21 needs no padding and every
 // load is a full 16-byte vector along the position axis; V rows are 256 contiguous bytes.
-#include <atomic>
-
 #include "common.cuh"
 
 namespace lisa {
@@ -42,7 +39,6 @@ struct DecodeParams {
     int64_t sc_sb, sc_sh;
     int row_bf16;           // the score rows handed between layers are bf16 (Sec. 5.2 counts them at 2 bytes) instead of fp32
     float *ws_m, *ws_l, *ws_o;
-    unsigned* tickets;      // per sequence: chunk CTAs that have finished (nullptr: the merge runs as a kernel of its own)
     TView o;
 };
 
@@ -226,66 +222,6 @@ __device__ __forceinline__ void softmax_pv_chunk(const DecodeParams& p, float* s
             for (int jj = 0; jj < nrows; ++jj) acc = fmaf(s_s[h * kChunk + jj], vb[(size_t)jj * d], acc);
             p.ws_o[(part + h) * d + x] = acc;
         }
-    }
-}
-
-// Split-K merge folded into the chunk kernels: every chunk CTA of a sequence takes a ticket when its partials are written;
-// the one that draws the last ticket combines the (m, l, o) partials of all chunks, for every head of the sequence:
-//   o = sum_c e^{m_c - M} o_c / sum_c e^{m_c - M} l_c.
-// Nobody waits for anybody.  The ticket word returns to zero for the next call.  A thread owns four output columns of one
-// head (16-byte loads of the partials, all chunks' loads independent of one another).
-__device__ __forceinline__ void merge_if_last(const DecodeParams& p, int b, int L) {
-    __shared__ int s_last;
-    __threadfence();   // this thread's partials are visible device-wide before the CTA's ticket is drawn
-    __syncthreads();
-    const int nc = (L + kChunk - 1) / kChunk;
-    if (threadIdx.x == 0) {
-        const unsigned t = atomicAdd(p.tickets + b, 1u);
-        s_last = t == (unsigned)(nc - 1);
-        if (s_last) p.tickets[b] = 0u;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();   // the other CTAs' partials, published before their tickets
-    const int d = p.d, Hq = p.Hq, q4 = d / 4;          // q4 threads per head
-    const int hs = threadIdx.x / q4, c4 = threadIdx.x % q4, heads_per_pass = kThreads / q4;
-    const size_t stride = (size_t)p.Hq;                 // partial index step from one chunk to the next
-    for (int h = hs; h < Hq; h += heads_per_pass) {
-        const size_t base = (size_t)b * p.n_chunks * Hq + h;
-        float M = -INFINITY;
-        for (int c = 0; c < nc; ++c) M = fmaxf(M, __ldcg(p.ws_m + base + c * stride));
-        float den = 0.f;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float4* po = reinterpret_cast<const float4*>(p.ws_o + base * d) + c4;
-        const size_t ostep = stride * d / 4;
-        int c = 0;
-        for (; c + 4 <= nc; c += 4) {
-            float w[4];
-            float4 o[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                w[j] = __expf(__ldcg(p.ws_m + base + (c + j) * stride) - M);
-                o[j] = __ldcg(po + (size_t)(c + j) * ostep);
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                den = fmaf(w[j], __ldcg(p.ws_l + base + (c + j) * stride), den);
-                acc.x = fmaf(w[j], o[j].x, acc.x); acc.y = fmaf(w[j], o[j].y, acc.y);
-                acc.z = fmaf(w[j], o[j].z, acc.z); acc.w = fmaf(w[j], o[j].w, acc.w);
-            }
-        }
-        for (; c < nc; ++c) {
-            const float w = __expf(__ldcg(p.ws_m + base + c * stride) - M);
-            const float4 o = __ldcg(po + (size_t)c * ostep);
-            den = fmaf(w, __ldcg(p.ws_l + base + c * stride), den);
-            acc.x = fmaf(w, o.x, acc.x); acc.y = fmaf(w, o.y, acc.y); acc.z = fmaf(w, o.z, acc.z); acc.w = fmaf(w, o.w, acc.w);
-        }
-        const float inv = 1.f / den;
-        const int64_t oi = b * p.o.sb + h * p.o.sh + c4 * 4;
-        st_elem(const_cast<void*>(p.o.ptr), oi + 0, p.o.dtype, acc.x * inv);
-        st_elem(const_cast<void*>(p.o.ptr), oi + 1, p.o.dtype, acc.y * inv);
-        st_elem(const_cast<void*>(p.o.ptr), oi + 2, p.o.dtype, acc.z * inv);
-        st_elem(const_cast<void*>(p.o.ptr), oi + 3, p.o.dtype, acc.w * inv);
     }
 }
 
@@ -480,7 +416,6 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
     }
     __syncthreads();
     softmax_pv_chunk(p, s_s, b, chunk, nrows);
-    if (p.tickets) merge_if_last(p, b, L);
 }
 
 // Scores of a FULL chunk for a standard layer, d = 128, bf16 cache: s_s[h][j] = q_h . K_j / sqrt(d).  Same streaming
@@ -635,7 +570,6 @@ __global__ void __launch_bounds__(kThreads, 2) anchor_decode_chunk_kernel(const 
         }
     }
     softmax_pv_chunk(p, s_s, b, chunk, nrows);
-    if (p.tickets) merge_if_last(p, b, L);
 }
 
 // Merge the per-chunk (m, l, o) partials of one (b, h): o = sum_c e^{m_c - M} o_c / sum_c e^{m_c - M} l_c.
@@ -674,26 +608,6 @@ __global__ void decode_merge_kernel(const __grid_constant__ DecodeParams p) {
     }
     for (; c < nc; ++c) acc[0] = fmaf(s_w[c], po[(size_t)c * step], acc[0]);
     st_elem(const_cast<void*>(p.o.ptr), b * p.o.sb + h * p.o.sh + x, p.o.dtype, (acc[0] + acc[1]) + (acc[2] + acc[3]));
-}
-
-// Ticket words of the folded merge: kTicketSlots independent sets of kTicketSeqs sequences, zero when the library is
-// loaded and returned to zero by every launch that uses them.  Successive calls rotate through the sets, so launches
-// that overlap on a device (different streams) do not share words unless 64 of them are in flight at once.
-constexpr int kTicketSlots = 64, kTicketSeqs = 1024;
-__device__ unsigned g_merge_tickets[kTicketSlots * kTicketSeqs];
-
-unsigned* ticket_words(int B) {
-    if (B > kTicketSeqs) return nullptr;   // larger batches keep the merge as a kernel of its own
-    static unsigned* cached[64] = {nullptr};
-    static std::atomic<unsigned> next{0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-    if (!cached[dev]) {
-        void* q = nullptr;
-        if (cudaGetSymbolAddress(&q, g_merge_tickets) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
-        cached[dev] = reinterpret_cast<unsigned*>(q);
-    }
-    return cached[dev] + (size_t)(next.fetch_add(1u) % kTicketSlots) * kTicketSeqs;
 }
 
 void carve_workspace(DecodeParams& p, void* ws) {
@@ -743,7 +657,6 @@ cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cud
     p.row_bf16 = a.scores_dtype == LISA_BF16;
     p.o = make_view(a.o);
     carve_workspace(p, ws);
-    p.tickets = (p.d % 4 == 0 && kThreads % (p.d / 4) == 0) ? ticket_words(p.B) : nullptr;
     const size_t smem = shared_decode_smem(p.Hq, p.m, p.integrate);
     dim3 grid(p.n_chunks, p.B);
     const bool fast = p.integrate == LISA_INTEGRATE_ADD && p.ffn_layers == 2 && c.dtype == LISA_BF16;
@@ -763,7 +676,6 @@ cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cud
     else LISA_LAUNCH_CHUNK(0, 0);
 #undef LISA_LAUNCH_CHUNK
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    if (p.tickets) { count_launches(1); return cudaSuccess; }
     decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, (size_t)p.n_chunks * sizeof(float), s>>>(p);
     count_launches(2);
     return cudaGetLastError();
@@ -781,13 +693,11 @@ cudaError_t launch_anchor_decode(const lisa_anchor_args& a, void* ws, cudaStream
     p.row_bf16 = a.scores_dtype == LISA_BF16;
     p.o = make_view(a.o);
     carve_workspace(p, ws);
-    p.tickets = (p.d % 4 == 0 && kThreads % (p.d / 4) == 0) ? ticket_words(p.B) : nullptr;
     const size_t smem = sizeof(float) * ((size_t)p.Hq * kChunk + (size_t)p.Hq * p.d);
     cudaError_t e;
     if ((e = set_smem(anchor_decode_chunk_kernel, smem)) != cudaSuccess) return e;
     anchor_decode_chunk_kernel<<<dim3(p.n_chunks, p.B), kThreads, smem, s>>>(p);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    if (p.tickets) { count_launches(1); return cudaSuccess; }
     decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, (size_t)p.n_chunks * sizeof(float), s>>>(p);
     count_launches(2);
     return cudaGetLastError();
