@@ -67,7 +67,7 @@ class AttentionStack:
         scores and each link's difference are computed once for the run); fused=False calls
         `lisa_attn_shared_prefill` layer by layer.  Same results either way.
         nf=True is the paper's lossless-prefill recipe (Sec. 5.2, "NF"): a shared layer attends over the prompt with
-        standard attention on its own full Q and K, and only what it caches differs (K_LR instead of K); sharing
+        standard attention on its own full Q and K, and only what it caches differs (the low-rank keys K_LR take the place of K); sharing
         starts with the first decoded token.  Prefill then costs what a standard stack costs.
         """
         B, N, Hq, Hkv, d, r = self.B, self.N, self.Hq, self.Hkv, self.d, self.r
