@@ -107,9 +107,16 @@ int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves) {
 bool concat_chain(const lisa_shared_prefill_args& a) { return a.chain_len > 0 && a.links[0].integrate == LISA_INTEGRATE_CONCAT; }
 int plane_count(const lisa_shared_prefill_args& a) { return a.chain_len + (concat_chain(a) ? 1 : 0); }
 
+// Waves are independent of one another, and the three kernels of a wave stress different things (the emit kernel only
+// writes HBM, the attention kernel mostly reads it, the aligner is bound by its MMA rate), so up to kWaveSets waves are
+// in flight at a time, each on a stream and a set of planes of its own: wave w uses set w % sets, and set reuse is
+// ordered by the stream the set belongs to.
+constexpr int kWaveSets = 3;
+
 struct Layout {
-    size_t qp_off[kMaxChain], kp_off[kMaxChain], plane_off[kMaxChain + 1];
+    size_t qp_off[kMaxChain], kp_off[kMaxChain], plane_off[kWaveSets][kMaxChain + 1];
     int64_t plane_rows, plane_cols;
+    int sets;
     size_t total;
 };
 
@@ -128,7 +135,9 @@ Layout plan_layout(const lisa_shared_prefill_args& a) {
     for (int i = 0; i < std::min(nw, 1024); ++i) max_cnt = std::max(max_cnt, waves[i].count);
     l.plane_rows = (int64_t)max_cnt * kTile;
     l.plane_cols = (int64_t)n_qt * kTile;
-    for (int k = 0; k < plane_count(a); ++k) l.plane_off[k] = take((size_t)a.B * a.Hq * l.plane_rows * l.plane_cols * 2);
+    l.sets = std::max(1, std::min(kWaveSets, nw));
+    for (int set = 0; set < l.sets; ++set)
+        for (int k = 0; k < plane_count(a); ++k) l.plane_off[set][k] = take((size_t)a.B * a.Hq * l.plane_rows * l.plane_cols * 2);
     l.total = off;
     return l;
 }
@@ -168,8 +177,10 @@ namespace {
 // per device, created on first use; the fork and the join are each enqueued under a lock, so calls from several host
 // threads cannot pair one call's wait with another call's record.
 struct SideStream {
-    cudaStream_t stream = nullptr;
+    cudaStream_t stream = nullptr;                 // packing of Q'/K'
     cudaEvent_t fork = nullptr, join = nullptr;
+    cudaStream_t wave[kWaveSets - 1] = {};         // waves beside the caller's stream
+    cudaEvent_t wave_done[kWaveSets - 1] = {};
     bool ok = false;
 };
 SideStream g_side[64];
@@ -183,6 +194,10 @@ SideStream* side_stream() {
         if (cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
         if (cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         if (cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        for (int i = 0; i < kWaveSets - 1; ++i) {
+            if (cudaStreamCreateWithFlags(&ss.wave[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&ss.wave_done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        }
         ss.ok = true;
     }
     return &ss;
@@ -241,36 +256,52 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
     const bool concat = concat_chain(a);
     Wave waves[1024];
     const int nw = plan_waves(a.B, a.N, a.Hq, plane_count(a), waves, 1024);
+    // Several waves in flight (see kWaveSets): wave w runs on stream w % sets (0 = the caller's) with plane set w % sets.
+    // All of it is forked from and joined back into the caller's stream inside this call, under the lock that keeps
+    // another host thread's call from interleaving its event records with these waits.
+    const int sets = (side && nw >= 2) ? l.sets : 1;
+    std::unique_lock<std::mutex> wave_lock(g_side_mutex, std::defer_lock);
+    if (sets > 1) {
+        wave_lock.lock();
+        if ((e = cudaStreamWaitEvent(s, side->join, 0)) != cudaSuccess) return e;   // every wave stream starts with the packed Q'/K' ready
+        joined = true;
+        if ((e = cudaEventRecord(side->fork, s)) != cudaSuccess) return e;
+        for (int i = 0; i + 1 < sets; ++i)
+            if ((e = cudaStreamWaitEvent(side->wave[i], side->fork, 0)) != cudaSuccess) return e;
+    }
     for (int w = 0; w < nw; ++w) {
         const Wave wv = waves[w];
+        const int set = w % sets;
+        cudaStream_t st = set == 0 ? s : side->wave[set - 1];
+        const size_t* po = l.plane_off[set];
         // 1. anchor scores and the differences of the links below the top one
         TcFlashArgs f{a.B, a.N, a.Hq, a.Hkv, 128, a.q0, a.k0, a.v, a.o, 1.f / sqrtf((float)a.d), nullptr, l.plane_rows, l.plane_cols,
                       wv.begin, wv.count};
-        f.emit_plane = base + l.plane_off[0];
+        f.emit_plane = base + po[0];
         {
-            PhaseMark mark(1, s);
-            if ((e = launch_tc_flash(f, s)) != cudaSuccess) return e;
+            PhaseMark mark(1, st);
+            if ((e = launch_tc_flash(f, st)) != cudaSuccess) return e;
         }
         for (int k = 0; k + (concat ? 0 : 1) < c; ++k) {   // the concatenating form also needs the top link's difference as a plane
             if ((e = join_pack()) != cudaSuccess) return e;
-            PhaseMark mark(1, s);
+            PhaseMark mark(1, st);
             TcFlashArgs fd = f;
             fd.kd = kPadRank;
             fd.qa = packed_view(base + l.qp_off[k], a.Hq, a.N);
             fd.ka = packed_view(base + l.kp_off[k], a.Hkv, a.N);
             fd.scale = 1.f / sqrtf((float)a.links[k].r);
             fd.ksteps = (a.links[k].r + 15) / 16;
-            fd.emit_plane = base + l.plane_off[k + 1];
-            if ((e = launch_tc_flash(fd, s)) != cudaSuccess) return e;
+            fd.emit_plane = base + po[k + 1];
+            if ((e = launch_tc_flash(fd, st)) != cudaSuccess) return e;
         }
         if (concat) {
             // 2c. link by link: A_k = FFN_k([A_{k-1}; D_k]) over plane 0; log2(e) * A_k over D_k's plane where a layer's
             // attention consumes it (the top link's; every link's when all layers of the chain are computed)
             for (int k = 0; k < c; ++k) {
-                TcAlignConcatArgs ac{a.B, a.N, wv.begin, wv.count, l.plane_rows, l.plane_cols, base + l.plane_off[0], base + l.plane_off[k + 1],
+                TcAlignConcatArgs ac{a.B, a.N, wv.begin, wv.count, l.plane_rows, l.plane_cols, base + po[0], base + po[k + 1],
                                      &a.links[k], k + 1 < c, all_layers || k == c - 1};
-                PhaseMark mark(2, s);
-                if ((e = launch_tc_align_concat(ac, s)) != cudaSuccess) return e;
+                PhaseMark mark(2, st);
+                if ((e = launch_tc_align_concat(ac, st)) != cudaSuccess) return e;
             }
             // 3c. softmax and .V on the finished scores: the attention kernel's own difference is switched off (scale 0)
             for (int k = all_layers ? 0 : c - 1; k < c; ++k) {
@@ -281,10 +312,10 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
                 fv.ka = packed_view(base + l.kp_off[k], a.Hkv, a.N);
                 fv.scale = 0.f;
                 fv.ksteps = 1;
-                fv.plane = base + l.plane_off[k + 1];
+                fv.plane = base + po[k + 1];
                 if (all_layers) { fv.v = vs[k]; fv.o = os[k]; }
-                PhaseMark mark(3, s);
-                if ((e = launch_tc_flash(fv, s)) != cudaSuccess) return e;
+                PhaseMark mark(3, st);
+                if ((e = launch_tc_flash(fv, st)) != cudaSuccess) return e;
             }
             continue;
         }
@@ -292,12 +323,12 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         TcAlignArgs al{};
         al.B = a.B; al.N = a.N; al.chain = c; al.qt_begin = wv.begin; al.qt_count = wv.count;
         al.plane_rows = l.plane_rows; al.plane_cols = l.plane_cols;
-        for (int k = 0; k < c; ++k) al.planes[k] = base + l.plane_off[k];
+        for (int k = 0; k < c; ++k) al.planes[k] = base + po[k];
         al.links = a.links;
         al.store_all = all_layers;
         {
-            PhaseMark mark(2, s);
-            if ((e = launch_tc_align(al, s)) != cudaSuccess) return e;
+            PhaseMark mark(2, st);
+            if ((e = launch_tc_align(al, st)) != cudaSuccess) return e;
         }
         // 3. each layer's own difference, softmax and .V
         if ((e = join_pack()) != cudaSuccess) return e;
@@ -309,11 +340,15 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             fv.ka = packed_view(base + l.kp_off[k], a.Hkv, a.N);
             fv.scale = 1.f / sqrtf((float)a.links[k].r);
             fv.ksteps = (a.links[k].r + 15) / 16;
-            fv.plane = base + l.plane_off[all_layers ? k : 0];
+            fv.plane = base + po[all_layers ? k : 0];
             if (all_layers) { fv.v = vs[k]; fv.o = os[k]; }
-            PhaseMark mark(3, s);
-            if ((e = launch_tc_flash(fv, s)) != cudaSuccess) return e;
+            PhaseMark mark(3, st);
+            if ((e = launch_tc_flash(fv, st)) != cudaSuccess) return e;
         }
+    }
+    for (int i = 0; i + 1 < sets; ++i) {
+        if ((e = cudaEventRecord(side->wave_done[i], side->wave[i])) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(s, side->wave_done[i], 0)) != cudaSuccess) return e;
     }
     return cudaSuccess;
 }

@@ -183,3 +183,34 @@ def test_bf16_score_rows(Hq, Hkv, d, r, m, L):
         assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-4)
         assert np.all(r0[b, :, lens_h[b]:] == -7.0)
     assert lb.lisa_check() == lb.OK
+
+
+def test_multi_layer_cache_handle_matches_per_layer_caches():
+    """lisa_kvcache_init carves one buffer into per-layer caches; lisa_kvcache_append_layer on it and a decode step on one of its
+    layers give bit for bit what separately allocated per-layer caches give."""
+    B, L, Hq, Hkv, d, r, m = 2, 200, 8, 2, 64, 21, 16
+    w = synth.Workload("handle", "bf16", B, L, Hq, Hkv, d, r, m, "relu", 1, True)
+    t = synth.decode_inputs(w, 12, B=B, L=L)
+    L_cap = 208
+    whole = lb.KVCache([lb.CACHE_STANDARD, lb.CACHE_SHARED, lb.CACHE_SHARED], B, Hkv, L_cap, d, r)
+    whole.append(0, dev(t["k"]), dev(t["v"]))
+    whole.append(1, dev(t["kp"]), dev(t["v"]))
+    first = 152                                                  # layer 2 in two pieces, the second at an offset (its rows start 16-byte aligned)
+    whole.append(2, dev(t["kp"])[:, :first], dev(t["v"])[:, :first])
+    before = torch.full((B,), first, dtype=torch.int32, device="cuda")
+    whole.append(2, dev(t["kp"])[:, first:], dev(t["v"])[:, first:], before)
+    std = lb.KVCacheLayer(lb.CACHE_STANDARD, B, Hkv, L_cap, d)
+    sh = lb.KVCacheLayer(lb.CACHE_SHARED, B, Hkv, L_cap, d, r)
+    lb.lisa_kvcache_append(std, dev(t["k"]), dev(t["v"]))
+    lb.lisa_kvcache_append(sh, dev(t["kp"]), dev(t["v"]))
+    torch.cuda.synchronize()
+    assert torch.equal(whole.layer(0).k, std.k) and torch.equal(whole.layer(0).v, std.v)
+    for l in (1, 2):
+        assert torch.equal(whole.layer(l).k, sh.k) and torch.equal(whole.layer(l).v, sh.v)
+    link = lb.Link(dev(t["qp"]), None, dev(t["w1"]), dev(t["w2"]), act=lb.ACT_RELU)
+    a = lb.lisa_attn_shared_decode(dev(t["prev"]), link, whole.layer(2), L=L)
+    b = lb.lisa_attn_shared_decode(dev(t["prev"]), link, sh, L=L)
+    assert torch.equal(a, b)
+    with pytest.raises(lb.LisaError):
+        whole.append(3, dev(t["kp"]), dev(t["v"]))               # no such layer
+    assert lb.lisa_check() == lb.OK
