@@ -35,10 +35,11 @@ METRIC = "lisa_attention_tokens_per_s"
 # summarised under profiles/ (cold cache); every kernel streams its planes once, so traffic grows in proportion to
 # the causal positions and the figures are scaled by them for other workloads.  None for a kernel that has changed since.
 CFG2_POSITIONS_HEADS = 2098176 * 32
-PREFILL_TRAFFIC_PER_PH = {"emit_scores": (40019456 + 85420032) / CFG2_POSITIONS_HEADS,
-                          "align": (142642688 + 83800064) / CFG2_POSITIONS_HEADS,
-                          "attention": (186513920 + 6682368) / CFG2_POSITIONS_HEADS}
-DECODE_TRAFFIC_PER_SEQ = (395953152 + 5092608) / 8  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
+PREFILL_TRAFFIC_PER_PH = {"emit_scores": (39902464 + 85123840) / CFG2_POSITIONS_HEADS,
+                          "align": (142643200 + 83262464) / CFG2_POSITIONS_HEADS,
+                          "attention": (186194944 + 5540864) / CFG2_POSITIONS_HEADS}
+DECODE_TRAFFIC_PER_SEQ = (395952128 + 4544512) / 8  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
+PROJECT_TRAFFIC = 220900096 + 163201024             # projection kernel at the benchmark's own size
 
 
 def measured_peaks():
@@ -467,7 +468,7 @@ def main():
         project = {"call": "lisa_project", "rows": Bp * Np, "d_in": dm, "n_out": n_out, "outputs": "Q' [%d x %d], K' [%d x %d], V [%d x %d]" % (Hh, rr, Hh, rr, Hh, dd),
                    "ms": pms, "value": world * Bp * Np / (pms * 1e-3), "unit": "tokens/s",
                    "roofline": {"bound": "tensor", "achieved": ptf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ptf / peaks["bf16_tflops"],
-                                "peak_source": peaks["source"] + " (burst)", "flops_per_launch": pflops, "traffic": None}}
+                                "peak_source": peaks["source"] + " (burst)", "flops_per_launch": pflops, "traffic": PROJECT_TRAFFIC}}
         del xh, wp, pouts
 
     # ---------------- decode step and the library's own standard-attention decode ----------------
