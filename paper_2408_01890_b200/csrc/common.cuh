@@ -102,17 +102,20 @@ struct TcAlignArgs {
 bool tc_align_supported(int Hq, const lisa_link* links, int chain);
 cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t s);
 
-// Tensor-core aligner for the concatenating Integrate, one link per launch (tc_align_concat.cu): reads plane_a = A_{k-1} and
-// plane_d = D_k, writes A_k over plane_a (write_next) and/or log2(e) * A_k over plane_d (write_scaled).
-struct TcAlignConcatArgs {
-    int B, N, qt_begin, qt_count;
+// Tensor-core aligner, one link per launch (tc_align_link.cu): the concatenating Integrate at 32 heads, and the adding forms
+// at 32 or 40 heads with a hidden layer of up to 256 units.  Reads plane_x = the link's input scores and plane_d = D_k
+// (adding forms: may be null, then nothing is added); writes the next link's input (unscaled; the adding forms include
+// D_k) and/or log2(e) times the FFN's output, each over plane_x (0) or plane_d (1), or nowhere (-1).
+struct TcAlignLinkArgs {
+    int B, N, Hq, qt_begin, qt_count;
     int64_t plane_rows, plane_cols;
-    void *plane_a, *plane_d;
+    void *plane_x, *plane_d;
     const lisa_link* link;
-    bool write_next, write_scaled;
+    int dst_next, dst_scaled;
 };
 bool tc_align_concat_supported(int Hq, const lisa_link* links, int chain);
-cudaError_t launch_tc_align_concat(const TcAlignConcatArgs& a, cudaStream_t s);
+bool tc_align_link_supported(int Hq, const lisa_link* links, int chain);
+cudaError_t launch_tc_align_link(const TcAlignLinkArgs& a, cudaStream_t s);
 
 // Packs Q' or K' ([B,N,H,r], any strides) into zero-padded bf16 [B][H][N][64] rows for the tensor-core kernels.
 cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int r, void* dst, cudaStream_t s);

@@ -160,7 +160,9 @@ cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int
 
 bool tc_shared_prefill_supported(const lisa_shared_prefill_args& a) {
     if (a.d != 128 || a.chain_len < 1 || a.N > kTile * 1024) return false;
-    if (!tc_align_supported(a.Hq, a.links, a.chain_len) && !tc_align_concat_supported(a.Hq, a.links, a.chain_len)) return false;
+    if (!tc_align_supported(a.Hq, a.links, a.chain_len) && !tc_align_concat_supported(a.Hq, a.links, a.chain_len) &&
+        !tc_align_link_supported(a.Hq, a.links, a.chain_len))
+        return false;
     for (int k = 0; k < a.chain_len; ++k)
         if (a.links[k].qp.dtype != LISA_BF16 || a.links[k].kp.dtype != LISA_BF16 || a.links[k].r > 32) return false;
     TcFlashArgs f{a.B, a.N, a.Hq, a.Hkv, 128, a.q0, a.k0, a.v, a.o, 1.f, nullptr, 0, 0, 0, 1};
@@ -298,10 +300,10 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             // 2c. link by link: A_k = FFN_k([A_{k-1}; D_k]) over plane 0; log2(e) * A_k over D_k's plane where a layer's
             // attention consumes it (the top link's; every link's when all layers of the chain are computed)
             for (int k = 0; k < c; ++k) {
-                TcAlignConcatArgs ac{a.B, a.N, wv.begin, wv.count, l.plane_rows, l.plane_cols, base + po[0], base + po[k + 1],
-                                     &a.links[k], k + 1 < c, all_layers || k == c - 1};
+                TcAlignLinkArgs ac{a.B, a.N, a.Hq, wv.begin, wv.count, l.plane_rows, l.plane_cols, base + po[0], base + po[k + 1],
+                                   &a.links[k], k + 1 < c ? 0 : -1, (all_layers || k == c - 1) ? 1 : -1};
                 PhaseMark mark(2, st);
-                if ((e = launch_tc_align_concat(ac, st)) != cudaSuccess) return e;
+                if ((e = launch_tc_align_link(ac, st)) != cudaSuccess) return e;
             }
             // 3c. softmax and .V on the finished scores: the attention kernel's own difference is switched off (scale 0)
             for (int k = all_layers ? 0 : c - 1; k < c; ++k) {
@@ -319,6 +321,19 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             }
             continue;
         }
+        const bool per_link = !tc_align_supported(a.Hq, a.links, c);
+        if (per_link) {
+            // 2l. shapes the chain kernel does not take (40 heads, wider hidden layers): one launch per link.  Link k reads
+            // plane k, writes A_k = FFN_k(A_{k-1}) + D_k over plane k + 1 (which held D_k) and, where a layer's attention
+            // consumes it, log2(e) * FFN_k(A_{k-1}) over plane k.
+            for (int k = 0; k < c; ++k) {
+                TcAlignLinkArgs al{a.B, a.N, a.Hq, wv.begin, wv.count, l.plane_rows, l.plane_cols, base + po[k],
+                                   k + 1 < c ? base + po[k + 1] : nullptr, &a.links[k], k + 1 < c ? 1 : -1,
+                                   (all_layers || k == c - 1) ? 0 : -1};
+                PhaseMark mark(2, st);
+                if ((e = launch_tc_align_link(al, st)) != cudaSuccess) return e;
+            }
+        }
         // 2. the FFN chain over the head axis, in place
         TcAlignArgs al{};
         al.B = a.B; al.N = a.N; al.chain = c; al.qt_begin = wv.begin; al.qt_count = wv.count;
@@ -326,7 +341,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         for (int k = 0; k < c; ++k) al.planes[k] = base + po[k];
         al.links = a.links;
         al.store_all = all_layers;
-        {
+        if (!per_link) {
             PhaseMark mark(2, st);
             if ((e = launch_tc_align(al, st)) != cudaSuccess) return e;
         }
@@ -340,7 +355,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             fv.ka = packed_view(base + l.kp_off[k], a.Hkv, a.N);
             fv.scale = 1.f / sqrtf((float)a.links[k].r);
             fv.ksteps = (a.links[k].r + 15) / 16;
-            fv.plane = base + po[all_layers ? k : 0];
+            fv.plane = base + po[all_layers ? k : (per_link ? c - 1 : 0)];
             if (all_layers) { fv.v = vs[k]; fv.o = os[k]; }
             PhaseMark mark(3, st);
             if ((e = launch_tc_flash(fv, st)) != cudaSuccess) return e;

@@ -173,3 +173,54 @@ def test_concatenating_chain_in_one_pass():
         ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1])
         assert_close(outs[k].float().cpu().numpy(), ref, "bf16", "concatenating chain, layer %d" % (k + 1))
     assert lb.lisa_check() == lb.OK
+
+
+def link_inputs(B, N, Hq, Hkv, chain, m, act, layers, r, seed, bias):
+    w = synth.Workload("tc_link", "bf16", B, N, Hq, Hkv, 128, r, m, act, chain)
+    t = synth.prefill_inputs(w, seed)
+    mm = Hq if layers == 1 else m
+    for k in range(1, chain + 1):
+        t[f"w1_{k}"] = synth.as_dtype(synth.normal(f"w1_{k}", (Hq, mm), seed, std=Hq ** -0.5), "bf16")
+        t[f"w2_{k}"] = synth.as_dtype(synth.normal(f"w2_{k}", (mm, Hq), seed, std=mm ** -0.5), "bf16")
+        t[f"b1_{k}"] = synth.as_dtype(synth.normal(f"b1_{k}", (mm,), seed, std=0.5), "bf16")
+        t[f"b2_{k}"] = synth.as_dtype(synth.normal(f"b2_{k}", (Hq,), seed, std=0.5), "bf16")
+    return t
+
+
+@pytest.mark.parametrize("B,N,Hq,Hkv,chain,m,act,integrate,layers,r,bias", [
+    (1, 300, 40, 40, 1, 80, "relu", lb.INTEGRATE_ADD, 2, 21, False),    # the LLaMA2-13B layer: 40 heads, FFN 40 -> 80 -> 40
+    (2, 200, 40, 8, 2, 80, "silu", lb.INTEGRATE_ADD, 2, 20, True),
+    (1, 260, 40, 40, 3, 200, "relu", lb.INTEGRATE_ADD, 2, 21, True),     # hidden width over several chunks, not a multiple of 64
+    (1, 150, 40, 40, 2, 48, "relu", lb.INTEGRATE_ADD, 2, 32, True),      # hidden width within one 64-unit chunk
+    (1, 300, 40, 8, 2, 40, "none", lb.INTEGRATE_ADD, 1, 21, True),       # one linear 40 x 40 layer
+    (1, 200, 40, 40, 3, 40, "none", lb.INTEGRATE_PLUS, 2, 21, False),    # no FFN
+    (1, 300, 32, 8, 2, 128, "relu", lb.INTEGRATE_ADD, 2, 21, True),      # 32 heads with a hidden layer wider than 64
+    (1, 513, 32, 32, 1, 256, "silu", lb.INTEGRATE_ADD, 2, 21, False)])
+def test_link_by_link_aligner_runs_on_the_tensor_cores(B, N, Hq, Hkv, chain, m, act, integrate, layers, r, bias):
+    """Adding links at 40 heads, or at 32 heads with a hidden layer wider than 64: one aligner launch per link on the
+    tensor-core path (launches: pack, A_0 and one difference plane per link below the top, one aligner pass per link,
+    attention) against the oracle."""
+    t = link_inputs(B, N, Hq, Hkv, chain, m, act, layers, r, 23, bias)
+    dl, ol = make_links(t, chain, act, integrate, layers, bias)
+    n0 = lb.lisa_kernel_launches()
+    got = lb.lisa_attn_shared_prefill(dev(t["q0"]), dev(t["k0"]), dl, dev(t[f"v{chain}"]))
+    torch.cuda.synchronize()
+    assert lb.lisa_kernel_launches() - n0 == 2 * chain + 2
+    assert lb.lisa_check() == lb.OK
+    ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{chain}"]), ol)
+    assert_close(got.float().cpu().numpy(), ref, "bf16", "tensor-core prefill, link-by-link aligner, %d heads" % Hq)
+
+
+def test_link_by_link_chain_in_one_pass():
+    """lisa_attn_shared_prefill_chain at the LLaMA2-13B layer shape (40 heads, 40 -> 80 -> 40): every layer of the chain."""
+    B, N, Hq, Hkv, chain = 1, 300, 40, 40, 3
+    t = link_inputs(B, N, Hq, Hkv, chain, 80, "relu", 2, 21, 29, True)
+    dl, ol = make_links(t, chain, "relu", lb.INTEGRATE_ADD, 2, True)
+    n0 = lb.lisa_kernel_launches()
+    outs = lb.lisa_attn_shared_prefill_chain(dev(t["q0"]), dev(t["k0"]), dl, [dev(t[f"v{k}"]) for k in range(1, chain + 1)])
+    torch.cuda.synchronize()
+    assert lb.lisa_kernel_launches() - n0 == 1 + chain + chain + chain   # pack, planes, aligner passes, one attention per layer
+    for k in range(chain):
+        ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1])
+        assert_close(outs[k].float().cpu().numpy(), ref, "bf16", "link-by-link chain at 40 heads, layer %d" % (k + 1))
+    assert lb.lisa_check() == lb.OK
