@@ -357,16 +357,18 @@ def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
     return res
 
 
-def bench_paper_default_layer(lb, rank, args, env):
-    """The layer the paper ships (Sec. 5.1 overview; appendix): Integrate by concatenation, FFN 64 x 256, 256 x 32, ReLU, r = 20, at
-    the LLaMA2-7B-shaped prompt (B 1, N 2048, 32 heads); device time of one lisa_attn_shared_prefill call."""
+def bench_single_layer(lb, rank, args, env, H, r, m, concat, label):
+    """Device time of one lisa_attn_shared_prefill call at B 1, N 2048, d 128 for a layer shape beside the headline's:
+    the layer the paper ships (Sec. 5.1 overview; appendix: Integrate by concatenation, FFN 64 x 256, 256 x 32, ReLU, r = 20),
+    and the LLaMA2-13B-shaped adding layer (40 heads, FFN 40 -> 80 -> 40)."""
     flush, barrier, max_over_ranks, peaks, world = env
-    B, N, H, d, r, m = 1, 2048, 32, 128, 20, 256
+    B, N, d = 1, 2048, 128
     g = torch.Generator(device="cuda"); g.manual_seed(77 + rank)
     rn = lambda *shape: torch.randn(*shape, generator=g, device="cuda")
     q0, k0, v = (rn(B, N, H, d).to(torch.bfloat16) for _ in range(3))
-    link = lb.Link(rn(B, N, H, r).to(torch.bfloat16), rn(B, N, H, r).to(torch.bfloat16), (rn(2 * H, m) * (2 * H) ** -0.5).to(torch.bfloat16),
-                   (rn(m, H) * m ** -0.5).to(torch.bfloat16), act=lb.ACT_RELU, integrate=lb.INTEGRATE_CONCAT)
+    h_in = 2 * H if concat else H
+    link = lb.Link(rn(B, N, H, r).to(torch.bfloat16), rn(B, N, H, r).to(torch.bfloat16), (rn(h_in, m) * h_in ** -0.5).to(torch.bfloat16),
+                   (rn(m, H) * m ** -0.5).to(torch.bfloat16), act=lb.ACT_RELU, integrate=lb.INTEGRATE_CONCAT if concat else lb.INTEGRATE_ADD)
     out = torch.empty_like(q0)
     ws = lb.prefill_workspace(q0, k0, [link], v, out)
 
@@ -380,8 +382,8 @@ def bench_paper_default_layer(lb, rank, args, env):
     tot, _, _ = time_steps(step, args.steps, flush, barrier)
     ms = max_over_ranks(tot) / args.steps
     P = B * N * (N + 1) // 2
-    fl = P * (2 * H * d + 2 * H * r + 2 * (2 * H) * m + 2 * m * H + 2 * H * d)
-    return {"layer": "CONCAT, FFN 64x256 + 256x32, ReLU, r=20, B=1 N=2048 32 heads", "ms": ms, "value": world * B * N / (ms * 1e-3), "unit": "tokens/s",
+    fl = P * (2 * H * d + 2 * H * r + 2 * h_in * m + 2 * m * H + 2 * H * d)
+    return {"layer": label, "ms": ms, "value": world * B * N / (ms * 1e-3), "unit": "tokens/s",
             "flops": fl, "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_tensor_peak": fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
             "launches": lb.lisa_kernel_launches() - l0}
 
@@ -439,8 +441,12 @@ def main():
     if args.only in (None, "cfg2"):
         second = bench_prefill(lb, SECOND, rank, args, env, with_chain=False, with_e2e=args.only is None)
         launches += second["launches"]
-        second["paper_default_layer"] = bench_paper_default_layer(lb, rank, args, env)
+        second["paper_default_layer"] = bench_single_layer(lb, rank, args, env, 32, 20, 256, True,
+                                                           "CONCAT, FFN 64x256 + 256x32, ReLU, r=20, B=1 N=2048 32 heads")
         launches += second["paper_default_layer"].pop("launches")
+        second["llama2_13b_layer"] = bench_single_layer(lb, rank, args, env, 40, 21, 80, False,
+                                                        "ADD, FFN 40x80 + 80x40, ReLU, r=21, B=1 N=2048 40 heads")
+        launches += second["llama2_13b_layer"].pop("launches")
 
     # ---------------- the fused projection H.[W_Q' | W_K' | W_V] of a shared layer (LLaMA2-7B widths) ----------------
     project = None
@@ -602,9 +608,11 @@ def main():
                          "e2e": main_res.get("e2e"), "roofline": main_res["roofline"], "chain_call": main_res.get("chain_call")})
             if head is None:
                 line["paper_default_layer"] = main_res.get("paper_default_layer")
+                line["llama2_13b_layer"] = main_res.get("llama2_13b_layer")
         if head is not None and second is not None:
             line["cfg2"] = {"workload": second["workload"], "value": second["value"], "unit": "tokens/s", "ms_per_step": second["ms_per_step"],
-                            "e2e": second.get("e2e"), "roofline": second["roofline"], "paper_default_layer": second["paper_default_layer"]}
+                            "e2e": second.get("e2e"), "roofline": second["roofline"], "paper_default_layer": second["paper_default_layer"],
+                            "llama2_13b_layer": second["llama2_13b_layer"]}
         line.update({"cpu_baseline": cpu, "project": project, "decode": decode, "stack": stack})
         print(json.dumps(line))
     group.close()
