@@ -260,13 +260,18 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
         asm volatile("cp.async.wait_group %0;" ::"n"(STAGES - 1) : "memory");
         __syncwarp();
         const uint32_t base = smem_u32(scr + buf * c * PLANE_SCR);
+        // both 16-position strips of the piece go through the chain together: every weight fragment read from shared
+        // memory feeds two MMAs
+        constexpr int NS = PP / 16;
+        static_assert(REGW || NS == 2, "the chain path works on two strips at a time");
+        {
+            uint32_t afr[NS][2][4];
 #pragma unroll
-        for (int s2 = 0; s2 < PP / 16; ++s2) {
-            const uint32_t off0 = frag_off(s2, 0), off1 = frag_off(s2, 1);
-            uint32_t afr[2][4];
-            ldmatrix_x4_trans(afr[0], base + off0);
-            ldmatrix_x4_trans(afr[1], base + off1);
-            float y[4][4];
+            for (int s2 = 0; s2 < NS; ++s2) {
+                ldmatrix_x4_trans(afr[s2][0], base + frag_off(s2, 0));
+                ldmatrix_x4_trans(afr[s2][1], base + frag_off(s2, 1));
+            }
+            float y[NS][4][4];
             for (int k = 0; k < c; ++k) {
                 const uint2* w1f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES);
                 const uint2* w2f = reinterpret_cast<const uint2*>(sW + k * LINK_BYTES + W1F_BYTES);
@@ -274,39 +279,43 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
                 const uint32_t* b1h = reinterpret_cast<const uint32_t*>(b1);
                 const int act = k == 0 ? act0 : (k == 1 ? act1 : act2);
                 if constexpr (ACT0 >= 0) {   // every link has this activation (and, from 8 up, no biases)
-                    ffn_link<(ACT0 & 7), REGW, (ACT0 < 8)>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
+                    ffn_link_strips<(ACT0 & 7), (ACT0 < 8), NS>(afr, w1f, w2f, b1h, b1 + MH, lane, y);
                 } else {
-                    if (act == LISA_ACT_RELU) ffn_link<LISA_ACT_RELU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
-                    else if (act == LISA_ACT_SILU) ffn_link<LISA_ACT_SILU, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
-                    else ffn_link<LISA_ACT_NONE, REGW>(afr, w1f, w2f, w1r, w2r, b1h, b1 + MH, lane, y, [] {});
+                    if (act == LISA_ACT_RELU) ffn_link_strips<LISA_ACT_RELU, true, NS>(afr, w1f, w2f, b1h, b1 + MH, lane, y);
+                    else if (act == LISA_ACT_SILU) ffn_link_strips<LISA_ACT_SILU, true, NS>(afr, w1f, w2f, b1h, b1 + MH, lane, y);
+                    else ffn_link_strips<LISA_ACT_NONE, true, NS>(afr, w1f, w2f, b1h, b1 + MH, lane, y);
                 }
                 if (store_all && k + 1 < c) {
                     // a chain of layers: link k's own output leaves too, over plane k's place in the scratch (plane 0 = A_0
                     // and plane k = D_k have been consumed by every lane before this link's MMAs could complete)
                     __syncwarp();
 #pragma unroll
-                    for (int x = 0; x < 2; ++x) {
-                        uint32_t r[4];
-                        r[0] = pack_f16(y[2 * x][0] * kLog2e, y[2 * x][1] * kLog2e);
-                        r[1] = pack_f16(y[2 * x][2] * kLog2e, y[2 * x][3] * kLog2e);
-                        r[2] = pack_f16(y[2 * x + 1][0] * kLog2e, y[2 * x + 1][1] * kLog2e);
-                        r[3] = pack_f16(y[2 * x + 1][2] * kLog2e, y[2 * x + 1][3] * kLog2e);
-                        stmatrix_x4_trans(base + k * PLANE_SCR + (x ? off1 : off0), r);
-                    }
+                    for (int s2 = 0; s2 < NS; ++s2)
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) {
+                            uint32_t r[4];
+                            r[0] = pack_f16(y[s2][2 * x][0] * kLog2e, y[s2][2 * x][1] * kLog2e);
+                            r[1] = pack_f16(y[s2][2 * x][2] * kLog2e, y[s2][2 * x][3] * kLog2e);
+                            r[2] = pack_f16(y[s2][2 * x + 1][0] * kLog2e, y[s2][2 * x + 1][1] * kLog2e);
+                            r[3] = pack_f16(y[s2][2 * x + 1][2] * kLog2e, y[s2][2 * x + 1][3] * kLog2e);
+                            stmatrix_x4_trans(base + k * PLANE_SCR + frag_off(s2, x), r);
+                        }
                 }
                 if (k + 1 < c) {
                     // A_{k+1} = y + D_{k+1}; the difference comes in the same fragment arrangement as A did
 #pragma unroll
-                    for (int x = 0; x < 2; ++x) {
-                        uint32_t dfr[4];
-                        ldmatrix_x4_trans(dfr, base + (k + 1) * PLANE_SCR + (x ? off1 : off0));
+                    for (int s2 = 0; s2 < NS; ++s2)
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float2 dv = unpack_f16(dfr[q]);
-                            float* yy = y[2 * x + (q >> 1)] + 2 * (q & 1);
-                            afr[x][q] = pack_f16(yy[0] + dv.x, yy[1] + dv.y);
+                        for (int x = 0; x < 2; ++x) {
+                            uint32_t dfr[4];
+                            ldmatrix_x4_trans(dfr, base + (k + 1) * PLANE_SCR + frag_off(s2, x));
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float2 dv = unpack_f16(dfr[q]);
+                                float* yy = y[s2][2 * x + (q >> 1)] + 2 * (q & 1);
+                                afr[s2][x][q] = pack_f16(yy[0] + dv.x, yy[1] + dv.y);
+                            }
                         }
-                    }
                 }
             }
             // the last link's result over its place in the scratch (plane 0, or plane c-1 in a chain of layers; every
@@ -315,14 +324,16 @@ tc_align_kernel(const __grid_constant__ AlignParams p) {
             const uint32_t last_plane = store_all ? (uint32_t)(c - 1) * PLANE_SCR : 0u;
             __syncwarp();
 #pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                uint32_t r[4];
-                r[0] = pack_f16(y[2 * x][0] * last_scale, y[2 * x][1] * last_scale);
-                r[1] = pack_f16(y[2 * x][2] * last_scale, y[2 * x][3] * last_scale);
-                r[2] = pack_f16(y[2 * x + 1][0] * last_scale, y[2 * x + 1][1] * last_scale);
-                r[3] = pack_f16(y[2 * x + 1][2] * last_scale, y[2 * x + 1][3] * last_scale);
-                stmatrix_x4_trans(base + last_plane + (x ? off1 : off0), r);
-            }
+            for (int s2 = 0; s2 < NS; ++s2)
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    uint32_t r[4];
+                    r[0] = pack_f16(y[s2][2 * x][0] * last_scale, y[s2][2 * x][1] * last_scale);
+                    r[1] = pack_f16(y[s2][2 * x][2] * last_scale, y[s2][2 * x][3] * last_scale);
+                    r[2] = pack_f16(y[s2][2 * x + 1][0] * last_scale, y[s2][2 * x + 1][1] * last_scale);
+                    r[3] = pack_f16(y[s2][2 * x + 1][2] * last_scale, y[s2][2 * x + 1][3] * last_scale);
+                    stmatrix_x4_trans(base + last_plane + frag_off(s2, x), r);
+                }
         }
         __syncwarp();
         const int64_t here_off = piece_off(here);

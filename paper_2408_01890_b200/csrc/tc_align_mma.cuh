@@ -118,6 +118,53 @@ __device__ __forceinline__ void ffn_link(const uint32_t (*afr)[4], const uint2* 
 }
 
 
+// The same link on NSTR strips of 16 positions at once, weights from shared memory: each 8-byte weight fragment is
+// loaded once and feeds NSTR MMAs.  With one strip the shared-memory pipe moves 256 bytes per MMA, which at the MMA
+// rate of the SM is about all it can deliver; two strips halve that.
+template <int ACT, bool BIAS, int NSTR>
+__device__ __forceinline__ void ffn_link_strips(const uint32_t (*afr)[2][4], const uint2* w1f, const uint2* w2f, const uint32_t* b1h,
+                                                const float* b2, int lane, float (*y)[4][4]) {
+    const int t = lane & 3;
+    uint32_t h[NSTR][8][2];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint32_t bb = BIAS ? b1h[j * 4 + t] : 0u;
+        const uint2 w = w1f[j * 32 + lane];
+#pragma unroll
+        for (int s = 0; s < NSTR; ++s) mma_f16acc(h[s][j], afr[s][0], w.x, w.y, bb, bb);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint2 w = w1f[(8 + j) * 32 + lane];
+#pragma unroll
+        for (int s = 0; s < NSTR; ++s) mma_f16acc(h[s][j], afr[s][1], w.x, w.y, h[s][j][0], h[s][j][1]);
+    }
+#pragma unroll
+    for (int s = 0; s < NSTR; ++s)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            h[s][j][0] = act_h2<ACT>(h[s][j][0]);
+            h[s][j][1] = act_h2<ACT>(h[s][j][1]);
+        }
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+        for (int j2 = 0; j2 < 4; ++j2) {
+            const uint2 w = w2f[(ks * 4 + j2) * 32 + lane];
+#pragma unroll
+            for (int s = 0; s < NSTR; ++s) {
+                const uint32_t hfr[4] = {h[s][2 * ks][0], h[s][2 * ks][1], h[s][2 * ks + 1][0], h[s][2 * ks + 1][1]};
+                if (ks == 0) {
+                    const float2 bb = BIAS ? *reinterpret_cast<const float2*>(b2 + j2 * 8 + 2 * t) : make_float2(0.f, 0.f);
+                    mma_f16_bias(y[s][j2], hfr, w.x, w.y, bb.x, bb.y);
+                } else {
+                    mma_f16(y[s][j2], hfr, w.x, w.y);
+                }
+            }
+        }
+}
+
+
 // What a link's FFN is, as far as this 32 -> 64 -> 32 two-layer engine is concerned.  The variants without a hidden
 // layer run on the same engine with an identity first layer (exact: every hidden unit is one fp16 input times one):
 //   KIND_FFN     y = W2^T act(W1^T a + b1) + b2                       (Sec. 5.1, two-layer FFN, m = 64)
