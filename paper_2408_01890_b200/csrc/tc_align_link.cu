@@ -192,91 +192,109 @@ __global__ void __launch_bounds__(NTHREADS, 1) tc_align_link_kernel(const __grid
         asm volatile("cp.async.wait_group 1;" ::: "memory");
         __syncwarp();
         const uint32_t base_x = smem_u32(scr + (buf * 2) * PLANE_SCR), base_d = base_x + PLANE_SCR;
+        // both 16-position strips of the piece go through the FFN together: every weight fragment read from shared memory
+        // feeds two MMAs (with one, the shared-memory pipe moves 256 bytes per MMA, about all it delivers at the MMA rate)
+        constexpr int NS = PP / 16;
+        {
+            uint32_t afr[NS][KS_IN][4];      // CONCAT: the first HB k-steps are the heads of the scores, the others the heads of D_k
 #pragma unroll
-        for (int s2 = 0; s2 < PP / 16; ++s2) {
-            uint32_t afr[KS_IN][4];      // CONCAT: the first HB k-steps are the heads of the scores, the others the heads of D_k
+            for (int s2 = 0; s2 < NS; ++s2)
 #pragma unroll
-            for (int x = 0; x < HB; ++x) {
-                ldmatrix_x4_trans(afr[x], base_x + frag_off(s2, x));
-                if constexpr (CONCAT) ldmatrix_x4_trans(afr[HB + x], base_d + frag_off(s2, x));
-            }
-            float y[2 * HB][4];
+                for (int x = 0; x < HB; ++x) {
+                    ldmatrix_x4_trans(afr[s2][x], base_x + frag_off(s2, x));
+                    if constexpr (CONCAT) ldmatrix_x4_trans(afr[s2][HB + x], base_d + frag_off(s2, x));
+                }
+            float y[NS][2 * HB][4];
 #pragma unroll
             for (int j2 = 0; j2 < 2 * HB; ++j2) {
                 const float2 bb = *reinterpret_cast<const float2*>(b2 + j2 * 8 + 2 * t4);
-                y[j2][0] = bb.x; y[j2][1] = bb.y; y[j2][2] = bb.x; y[j2][3] = bb.y;
+#pragma unroll
+                for (int s2 = 0; s2 < NS; ++s2) { y[s2][j2][0] = bb.x; y[s2][j2][1] = bb.y; y[s2][j2][2] = bb.x; y[s2][j2][3] = bb.y; }
             }
 #pragma unroll 1
             for (int q = 0; q < NCHUNK; ++q) {
-                uint32_t h[CHUNK / 8][2];
+                uint32_t h[NS][CHUNK / 8][2];
 #pragma unroll
                 for (int j = 0; j < CHUNK / 8; ++j) {
                     const uint32_t bb = b1h[(q * (CHUNK / 8) + j) * 4 + t4];
                     const uint2 w = w1f[(q * (CHUNK / 8) + j) * 32 + lane];
-                    mma_f16acc(h[j], afr[0], w.x, w.y, bb, bb);
+#pragma unroll
+                    for (int s2 = 0; s2 < NS; ++s2) mma_f16acc(h[s2][j], afr[s2][0], w.x, w.y, bb, bb);
                 }
 #pragma unroll
                 for (int ks = 1; ks < KS_IN; ++ks)
 #pragma unroll
                     for (int j = 0; j < CHUNK / 8; ++j) {
                         const uint2 w = w1f[(ks * (MHID / 8) + q * (CHUNK / 8) + j) * 32 + lane];
-                        mma_f16acc(h[j], afr[ks], w.x, w.y, h[j][0], h[j][1]);
+#pragma unroll
+                        for (int s2 = 0; s2 < NS; ++s2) mma_f16acc(h[s2][j], afr[s2][ks], w.x, w.y, h[s2][j][0], h[s2][j][1]);
                     }
 #pragma unroll
-                for (int s = 0; s < CHUNK / 16; ++s) {
-                    uint32_t hfr[4];
-                    hfr[0] = act_h2<ACT>(h[2 * s][0]);
-                    hfr[1] = act_h2<ACT>(h[2 * s][1]);
-                    hfr[2] = act_h2<ACT>(h[2 * s + 1][0]);
-                    hfr[3] = act_h2<ACT>(h[2 * s + 1][1]);
+                for (int s2 = 0; s2 < NS; ++s2)
+#pragma unroll
+                    for (int j = 0; j < CHUNK / 8; ++j) {
+                        h[s2][j][0] = act_h2<ACT>(h[s2][j][0]);
+                        h[s2][j][1] = act_h2<ACT>(h[s2][j][1]);
+                    }
+#pragma unroll
+                for (int s = 0; s < CHUNK / 16; ++s)
 #pragma unroll
                     for (int j2 = 0; j2 < NT_OUT; ++j2) {
                         const uint2 w = w2f[((q * (CHUNK / 16) + s) * NT_OUT + j2) * 32 + lane];
-                        mma_f16(y[j2], hfr, w.x, w.y);
+#pragma unroll
+                        for (int s2 = 0; s2 < NS; ++s2) {
+                            const uint32_t hfr[4] = {h[s2][2 * s][0], h[s2][2 * s][1], h[s2][2 * s + 1][0], h[s2][2 * s + 1][1]};
+                            mma_f16(y[s2][j2], hfr, w.x, w.y);
+                        }
                     }
-                }
             }
             // every lane has read its fragments of the scores (the MMAs that consumed them have completed): results go back transposed
             __syncwarp();
             if (dst_scaled >= 0) {
                 const uint32_t base = dst_scaled == 0 ? base_x : base_d;
 #pragma unroll
-                for (int x = 0; x < HB; ++x) {
-                    uint32_t r[4];
-                    r[0] = pack_f16(y[2 * x][0] * kLog2e, y[2 * x][1] * kLog2e);
-                    r[1] = pack_f16(y[2 * x][2] * kLog2e, y[2 * x][3] * kLog2e);
-                    r[2] = pack_f16(y[2 * x + 1][0] * kLog2e, y[2 * x + 1][1] * kLog2e);
-                    r[3] = pack_f16(y[2 * x + 1][2] * kLog2e, y[2 * x + 1][3] * kLog2e);
-                    stmatrix_x4_trans(base + frag_off(s2, x), r);
-                }
+                for (int s2 = 0; s2 < NS; ++s2)
+#pragma unroll
+                    for (int x = 0; x < HB; ++x) {
+                        uint32_t r[4];
+                        r[0] = pack_f16(y[s2][2 * x][0] * kLog2e, y[s2][2 * x][1] * kLog2e);
+                        r[1] = pack_f16(y[s2][2 * x][2] * kLog2e, y[s2][2 * x][3] * kLog2e);
+                        r[2] = pack_f16(y[s2][2 * x + 1][0] * kLog2e, y[s2][2 * x + 1][1] * kLog2e);
+                        r[3] = pack_f16(y[s2][2 * x + 1][2] * kLog2e, y[s2][2 * x + 1][3] * kLog2e);
+                        stmatrix_x4_trans(base + frag_off(s2, x), r);
+                    }
             }
             if (dst_next >= 0) {
                 if constexpr (!CONCAT) {
                     if (has_d) {   // A_k = FFN(A_{k-1}) + D_k: the difference in the fragment arrangement the scores came in
 #pragma unroll
-                        for (int x = 0; x < HB; ++x) {
-                            uint32_t dfr[4];
-                            ldmatrix_x4_trans(dfr, base_d + frag_off(s2, x));
+                        for (int s2 = 0; s2 < NS; ++s2)
 #pragma unroll
-                            for (int qq = 0; qq < 4; ++qq) {
-                                const float2 dv = unpack_f16(dfr[qq]);
-                                y[2 * x + (qq >> 1)][2 * (qq & 1)] += dv.x;
-                                y[2 * x + (qq >> 1)][2 * (qq & 1) + 1] += dv.y;
+                            for (int x = 0; x < HB; ++x) {
+                                uint32_t dfr[4];
+                                ldmatrix_x4_trans(dfr, base_d + frag_off(s2, x));
+#pragma unroll
+                                for (int qq = 0; qq < 4; ++qq) {
+                                    const float2 dv = unpack_f16(dfr[qq]);
+                                    y[s2][2 * x + (qq >> 1)][2 * (qq & 1)] += dv.x;
+                                    y[s2][2 * x + (qq >> 1)][2 * (qq & 1) + 1] += dv.y;
+                                }
                             }
-                        }
                         __syncwarp();   // all lanes hold their part of D_k before it is overwritten
                     }
                 }
                 const uint32_t base = dst_next == 0 ? base_x : base_d;
 #pragma unroll
-                for (int x = 0; x < HB; ++x) {
-                    uint32_t r[4];
-                    r[0] = pack_f16(y[2 * x][0], y[2 * x][1]);
-                    r[1] = pack_f16(y[2 * x][2], y[2 * x][3]);
-                    r[2] = pack_f16(y[2 * x + 1][0], y[2 * x + 1][1]);
-                    r[3] = pack_f16(y[2 * x + 1][2], y[2 * x + 1][3]);
-                    stmatrix_x4_trans(base + frag_off(s2, x), r);
-                }
+                for (int s2 = 0; s2 < NS; ++s2)
+#pragma unroll
+                    for (int x = 0; x < HB; ++x) {
+                        uint32_t r[4];
+                        r[0] = pack_f16(y[s2][2 * x][0], y[s2][2 * x][1]);
+                        r[1] = pack_f16(y[s2][2 * x][2], y[s2][2 * x][3]);
+                        r[2] = pack_f16(y[s2][2 * x + 1][0], y[s2][2 * x + 1][1]);
+                        r[3] = pack_f16(y[s2][2 * x + 1][2], y[s2][2 * x + 1][3]);
+                        stmatrix_x4_trans(base + frag_off(s2, x), r);
+                    }
             }
         }
         __syncwarp();
