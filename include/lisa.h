@@ -59,7 +59,10 @@ typedef enum lisa_act_t { LISA_ACT_NONE = 0, LISA_ACT_RELU = 1, LISA_ACT_SILU = 
 typedef enum lisa_integrate_t { LISA_INTEGRATE_ADD = 0, LISA_INTEGRATE_CONCAT = 1, LISA_INTEGRATE_PLUS = 2 } lisa_integrate_t;
 
 typedef enum lisa_cache_kind_t { LISA_CACHE_STANDARD = 0, LISA_CACHE_SHARED = 1 } lisa_cache_kind_t;
-typedef enum lisa_op_t { LISA_OP_ANCHOR = 0, LISA_OP_SHARED_PREFILL = 1, LISA_OP_SHARED_DECODE = 2, LISA_OP_SHARED_PREFILL_CHAIN = 3 } lisa_op_t;
+typedef enum lisa_op_t {
+    LISA_OP_ANCHOR = 0, LISA_OP_SHARED_PREFILL = 1, LISA_OP_SHARED_DECODE = 2, LISA_OP_SHARED_PREFILL_CHAIN = 3,
+    LISA_OP_SHARED_PREFILL_CARRY = 4
+} lisa_op_t;
 
 /* A strided view of an activation tensor [B, N, H, x]; x contiguous. */
 typedef struct lisa_tensor {
@@ -196,6 +199,34 @@ typedef struct lisa_shared_prefill_chain_args {
     size_t workspace_bytes;
 } lisa_shared_prefill_chain_args;
 lisa_status_t lisa_attn_shared_prefill_chain(const lisa_shared_prefill_chain_args* args, lisa_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * lisa_attn_shared_prefill_carry -- a shared layer over a whole prompt that takes the scores of the layer before it
+ * from memory, as Sec. 5.1 states the method (layer n aligns A_{n-1} "from the adjacent front layer"), instead of
+ * recomputing them from the anchor: the cost of a layer no longer grows with its depth in the chain, so runs of many
+ * consecutive shared layers (the appendix's configurations have runs of 15 and 27) cost the same per layer as the first.
+ * The price is memory: `scores` holds A_n for the whole prompt, lisa_prefill_scores_bytes(B, N, Hq) =
+ * B * Hq * ceil128(N)^2 * 2 bytes (fp16, a blocked layout private to the library; 17.2 GB for B 4, N 8192, 32 heads).
+ *   layer   the layer as for lisa_attn_shared_prefill with chain_len == 1: links[0] is this layer's own link, v and o its
+ *           own; q0 and k0 are read only when `first` (otherwise they may be zeroed descriptors)
+ *   first   1: this is the shared layer right after the anchor: A_0 = q0.k0^T/sqrt(d) is written into `scores` first;
+ *           0: `scores` holds A_{n-1} as the previous call left it (same B, N, Hq)
+ *   keep    1: A_n = Integrate(Align(A_{n-1}), D_n), unmasked, is left in `scores` for the next shared layer;
+ *           0: last layer of its chain, the contents of `scores` are unspecified afterwards
+ * o is exactly what lisa_attn_shared_prefill returns for the whole chain up to this layer, up to the rounding of the
+ * carried scores to fp16 (which the recomputing path applies between links as well).
+ * Tensor-core shapes only (d = 128, bf16, 32 or 40 heads, adding Integrate or no FFN, r <= 32): others
+ * LISA_ERR_UNSUPPORTED.  Workspace: lisa_workspace_bytes(LISA_OP_SHARED_PREFILL_CARRY, args, &n).  `scores` must be
+ * 256-byte aligned.  On error nothing is launched. */
+typedef struct lisa_shared_prefill_carry_args {
+    size_t struct_size;
+    lisa_shared_prefill_args layer;
+    void* scores;
+    size_t scores_bytes;
+    int32_t first, keep;
+} lisa_shared_prefill_carry_args;
+size_t lisa_prefill_scores_bytes(int32_t B, int32_t N, int32_t Hq);
+lisa_status_t lisa_attn_shared_prefill_carry(const lisa_shared_prefill_carry_args* args, lisa_stream_t stream);
 
 /* The same call with every tensor, weight and `o` in HOST memory (dense [B,N,H,x] layout, strides
  * ignored; workspace fields ignored).  Inputs are staged into `device_arena` (device memory of at least

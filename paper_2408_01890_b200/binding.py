@@ -22,11 +22,12 @@ F32, BF16 = 0, 1
 ACT_NONE, ACT_RELU, ACT_SILU = 0, 1, 2
 INTEGRATE_ADD, INTEGRATE_CONCAT, INTEGRATE_PLUS = 0, 1, 2
 CACHE_STANDARD, CACHE_SHARED = 0, 1
-OP_ANCHOR, OP_SHARED_PREFILL, OP_SHARED_DECODE, OP_SHARED_PREFILL_CHAIN = 0, 1, 2, 3
+OP_ANCHOR, OP_SHARED_PREFILL, OP_SHARED_DECODE, OP_SHARED_PREFILL_CHAIN, OP_SHARED_PREFILL_CARRY = 0, 1, 2, 3, 4
 ACTS = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
 
 # include/lisa.h (the method's entry points and host helpers) and include/lisa_debug.h (test and measurement hooks)
 EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_chain", "lisa_attn_shared_prefill_host",
+           "lisa_attn_shared_prefill_carry", "lisa_prefill_scores_bytes",
            "lisa_host_arena_bytes", "lisa_attn_shared_decode", "lisa_attn_shared_decode_static", "lisa_kvcache_append",
            "lisa_kvcache_append_layer", "lisa_project", "lisa_kvcache_bytes", "lisa_kvcache_total_bytes", "lisa_kvcache_init",
            "lisa_workspace_bytes", "lisa_check", "lisa_last_cuda_error", "lisa_status_string", "lisa_version",
@@ -91,6 +92,11 @@ class SharedPrefillArgs(C.Structure):
                 ("links", C.POINTER(CLink)), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
 
+class SharedPrefillCarryArgs(C.Structure):
+    _fields_ = [("struct_size", C.c_size_t), ("layer", SharedPrefillArgs), ("scores", C.c_void_p), ("scores_bytes", C.c_size_t),
+                ("first", C.c_int32), ("keep", C.c_int32)]
+
+
 class SharedPrefillChainArgs(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("B", C.c_int32), ("N", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32),
                 ("d", C.c_int32), ("chain_len", C.c_int32), ("q0", Tensor), ("k0", Tensor), ("links", C.POINTER(CLink)),
@@ -123,6 +129,9 @@ def load():
         lib.lisa_attn_shared_prefill.argtypes = [C.POINTER(SharedPrefillArgs), C.c_void_p]
         lib.lisa_attn_shared_prefill_chain.argtypes = [C.POINTER(SharedPrefillChainArgs), C.c_void_p]
         lib.lisa_attn_shared_prefill_chain.restype = C.c_int
+        lib.lisa_attn_shared_prefill_carry.argtypes = [C.POINTER(SharedPrefillCarryArgs), C.c_void_p]
+        lib.lisa_prefill_scores_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
+        lib.lisa_prefill_scores_bytes.restype = C.c_size_t
         lib.lisa_attn_shared_prefill_host.argtypes = [C.POINTER(SharedPrefillArgs), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.lisa_host_arena_bytes.argtypes = [C.POINTER(SharedPrefillArgs), C.POINTER(C.c_size_t)]
         lib.lisa_attn_shared_decode.argtypes = [C.POINTER(SharedDecodeArgs), C.c_void_p]
@@ -360,6 +369,50 @@ def lisa_attn_shared_prefill(q0: torch.Tensor, k0: torch.Tensor, links: Sequence
     a.workspace, a.workspace_bytes = _ptr(ws), (ws.numel() if ws is not None else 0)
     _check(load().lisa_attn_shared_prefill(C.byref(a), _stream()), "lisa_attn_shared_prefill")
     return out
+
+
+def lisa_prefill_scores_bytes(B: int, N: int, Hq: int) -> int:
+    """Bytes of the carried-scores buffer of lisa_attn_shared_prefill_carry."""
+    return int(load().lisa_prefill_scores_bytes(B, N, Hq))
+
+
+def _carry_args(q0, k0, link: Link, v, out, scores, first: bool, keep: bool):
+    if q0 is None:   # not read unless first: zeroed descriptors
+        B, N, Hq, d = out.shape
+        a = SharedPrefillArgs()
+        a.struct_size = C.sizeof(SharedPrefillArgs)
+        a.B, a.N, a.Hq, a.Hkv, a.d, a.chain_len = B, N, Hq, v.shape[2], d, 1
+        a.v, a.o = _tensor4(v), _tensor4(out)
+        arr = (CLink * 1)(link.to_c())
+        a.links = C.cast(arr, C.POINTER(CLink))
+    else:
+        a, arr = _prefill_args(q0, k0, [link], v, out)
+    c = SharedPrefillCarryArgs()
+    c.struct_size = C.sizeof(SharedPrefillCarryArgs)
+    c.layer = a
+    c.scores, c.scores_bytes = _ptr(scores), scores.numel() * scores.element_size()
+    c.first, c.keep = int(first), int(keep)
+    return c, arr
+
+
+def lisa_attn_shared_prefill_carry(q0: Optional[torch.Tensor], k0: Optional[torch.Tensor], link: Link, v: torch.Tensor,
+                                   scores: torch.Tensor, *, first: bool, keep: bool, out: torch.Tensor = None,
+                                   workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """A shared layer that aligns the scores the previous layer left in `scores` (or, when first, the anchor's q0.k0^T) and,
+    when keep, leaves its own there for the next one.  q0, k0 may be None unless first (then pass `out`)."""
+    if out is None:
+        out = torch.empty_like(q0)
+    c, keepalive = _carry_args(q0, k0, link, v, out, scores, first, keep)
+    ws = workspace if workspace is not None else _workspace(OP_SHARED_PREFILL_CARRY, c)
+    c.layer.workspace, c.layer.workspace_bytes = _ptr(ws), (ws.numel() if ws is not None else 0)
+    _check(load().lisa_attn_shared_prefill_carry(C.byref(c), _stream()), "lisa_attn_shared_prefill_carry")
+    return out
+
+
+def prefill_carry_workspace(q0, k0, link: Link, v, out, scores) -> Optional[torch.Tensor]:
+    """Scratch buffer for lisa_attn_shared_prefill_carry calls of this shape."""
+    c, keepalive = _carry_args(q0, k0, link, v, out, scores, q0 is not None, True)
+    return _workspace(OP_SHARED_PREFILL_CARRY, c)
 
 
 def prefill_workspace(q0, k0, links: Sequence[Link], v, out) -> Optional[torch.Tensor]:

@@ -85,6 +85,11 @@ struct TcFlashArgs {
     // (blocked [rows/128][cols/64][128][B*Hq][64], rows relative to qt_begin*128); v, o and plane are then ignored.
     void* emit_plane = nullptr;
     int ksteps = 0;  // 16-wide k-steps to issue (0 = kd/16); the columns beyond are zero padding
+    // carry != nullptr (with plane): the finished pre-softmax logits (scores * scale + plane, unmasked, fp16) of the covered
+    // tiles are written there, same blocked layout and geometry as plane; may be the plane itself (each tile is stored
+    // after it was read).
+    void* carry = nullptr;
+    int plane_row0 = -1;  // first query row the plane / emit_plane / carry buffers hold (-1: qt_begin * 128)
 };
 bool tc_flash_supported(const TcFlashArgs& a);
 cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t s);
@@ -97,6 +102,7 @@ struct TcAlignArgs {
     void* planes[4];
     const lisa_link* links;
     int ctas = 0;  // grid size (0 = three per SM)
+    int row0 = -1;  // first query row the planes hold (-1: qt_begin * 128)
     bool store_all = false;  // every link's output is stored (times log2 e): link k (0-based) into planes[k]
 };
 bool tc_align_supported(int Hq, const lisa_link* links, int chain);
@@ -112,6 +118,7 @@ struct TcAlignLinkArgs {
     void *plane_x, *plane_d;
     const lisa_link* link;
     int dst_next, dst_scaled;
+    int row0 = -1;  // first query row the planes hold (-1: qt_begin * 128)
 };
 bool tc_align_concat_supported(int Hq, const lisa_link* links, int chain);
 bool tc_align_link_supported(int Hq, const lisa_link* links, int chain);
@@ -123,10 +130,20 @@ cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int
 // Tensor-core prefill of a shared layer (tc_prefill.cu): emit planes -> align -> attention, wave by wave.
 bool tc_shared_prefill_supported(const lisa_shared_prefill_args& a);
 size_t tc_shared_prefill_workspace(const lisa_shared_prefill_args& a);
+// Carried scores (lisa_attn_shared_prefill_carry): the chain's running scores A_n of the whole prompt live in a caller's
+// buffer, blocked like the planes with N rounded up to 128 in both directions.  With `carry` set, a one-link call works
+// in place on that buffer: `first` emits A_0 there, the aligner runs over it, and the attention kernel writes A_n back
+// when `keep`.
+struct TcCarry {
+    void* scores;
+    bool first, keep;
+};
+size_t tc_carry_bytes(int B, int N, int Hq);
+size_t tc_shared_prefill_carry_workspace(const lisa_shared_prefill_args& a);
 cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws, cudaStream_t s);
 // vs/os: per-layer V and O of a chain of a.chain_len layers (nullptr: only the deepest layer, a.v / a.o)
 cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, const lisa_tensor* vs, const lisa_tensor* os, void* ws,
-                                           cudaStream_t s);
+                                           cudaStream_t s, const TcCarry* carry = nullptr);
 cudaError_t prefill_phase_timing(bool enable);
 cudaError_t prefill_phase_times(float* ms4);
 

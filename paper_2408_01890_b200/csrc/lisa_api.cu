@@ -204,7 +204,36 @@ lisa_shared_prefill_args chain_layer(const lisa_shared_prefill_chain_args& a, in
     p.workspace = a.workspace; p.workspace_bytes = a.workspace_bytes;
     return p;
 }
+
+// The one-link layer a carried call runs, validated; where the anchor's q0, k0 are not read (every layer but the first
+// of a chain) descriptors of the right shape stand in for them so that the common checks apply unchanged.
+lisa_status_t carried_layer(const lisa_shared_prefill_carry_args& a, lisa_shared_prefill_args* out) {
+    lisa_shared_prefill_args p = a.layer;
+    if (p.struct_size != sizeof(lisa_shared_prefill_args) || p.chain_len != 1 || !p.links) return LISA_ERR_INVALID_ARG;
+    if (!a.first) { p.q0 = p.o; p.k0 = p.v; }
+    lisa_status_t st = validate_prefill(&p);
+    if (st != LISA_OK) return st;
+    if (p.links[0].integrate == LISA_INTEGRATE_CONCAT || !tc_shared_prefill_supported(p)) return LISA_ERR_UNSUPPORTED;
+    *out = p;
+    return LISA_OK;
+}
 }  // namespace
+
+size_t lisa_prefill_scores_bytes(int32_t B, int32_t N, int32_t Hq) {
+    return (B < 1 || N < 1 || Hq < 1) ? 0 : tc_carry_bytes(B, N, Hq);
+}
+
+lisa_status_t lisa_attn_shared_prefill_carry(const lisa_shared_prefill_carry_args* a, lisa_stream_t stream) {
+    if (!a || a->struct_size != sizeof(lisa_shared_prefill_carry_args)) return LISA_ERR_INVALID_ARG;
+    lisa_shared_prefill_args p;
+    lisa_status_t st = carried_layer(*a, &p);
+    if (st != LISA_OK) return st;
+    if (!a->scores || (reinterpret_cast<uintptr_t>(a->scores) & 255u) || a->scores_bytes < tc_carry_bytes(p.B, p.N, p.Hq)) return LISA_ERR_INVALID_ARG;
+    if ((st = check_workspace(p.workspace, p.workspace_bytes, tc_shared_prefill_carry_workspace(p))) != LISA_OK) return st;
+    const TcCarry cy{a->scores, a->first != 0, a->keep != 0};
+    cudaError_t e = launch_tc_shared_prefill_chain(p, nullptr, nullptr, p.workspace, static_cast<cudaStream_t>(stream), &cy);
+    return e == cudaSuccess ? LISA_OK : cuda_fail(e);
+}
 
 lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes) {
     if (!args || !bytes) return LISA_ERR_INVALID_ARG;
@@ -235,6 +264,15 @@ lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes) 
             need = n > need ? n : need;
         }
         *bytes = need;
+        return LISA_OK;
+    }
+    if (op == LISA_OP_SHARED_PREFILL_CARRY) {
+        const lisa_shared_prefill_carry_args* a = static_cast<const lisa_shared_prefill_carry_args*>(args);
+        if (a->struct_size != sizeof(lisa_shared_prefill_carry_args)) return LISA_ERR_INVALID_ARG;
+        lisa_shared_prefill_args p;
+        lisa_status_t st = carried_layer(*a, &p);
+        if (st != LISA_OK) return st;
+        *bytes = tc_shared_prefill_carry_workspace(p);
         return LISA_OK;
     }
     if (op == LISA_OP_SHARED_DECODE) {

@@ -373,7 +373,8 @@ bool tc_align_supported(int Hq, const lisa_link* links, int chain) {
 cudaError_t launch_tc_align(const TcAlignArgs& a, cudaStream_t stream) {
     AlignParams p{};
     p.B = a.B; p.N = a.N; p.chain = a.chain;
-    p.row0 = a.qt_begin * UNIT; p.qt_begin = a.qt_begin; p.qt_count = a.qt_count;
+    p.row0 = a.row0 >= 0 ? a.row0 : a.qt_begin * UNIT; p.qt_begin = a.qt_begin; p.qt_count = a.qt_count;
+    if (p.row0 % UNIT != 0 || p.row0 > a.qt_begin * UNIT) return cudaErrorInvalidValue;
     p.plane_rows = a.plane_rows; p.plane_cols = a.plane_cols;
     p.units_per_batch = 0;
     for (int t = a.qt_begin; t < a.qt_begin + a.qt_count; ++t) p.units_per_batch += std::min(UNIT, a.N - t * UNIT) * (t + 1);

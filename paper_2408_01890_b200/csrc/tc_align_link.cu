@@ -361,7 +361,8 @@ cudaError_t launch_tc_align_link(const TcAlignLinkArgs& a, cudaStream_t stream) 
     const bool concat = l.integrate == LISA_INTEGRATE_CONCAT;
     if (concat && !a.plane_d) return cudaErrorInvalidValue;
     LinkParams p{};
-    p.B = a.B; p.N = a.N; p.row0 = a.qt_begin * UNIT; p.qt_begin = a.qt_begin; p.qt_count = a.qt_count;
+    p.B = a.B; p.N = a.N; p.row0 = a.row0 >= 0 ? a.row0 : a.qt_begin * UNIT; p.qt_begin = a.qt_begin; p.qt_count = a.qt_count;
+    if (p.row0 % UNIT != 0 || p.row0 > a.qt_begin * UNIT) return cudaErrorInvalidValue;
     p.plane_cols = a.plane_cols;
     for (int t = a.qt_begin; t < a.qt_begin + a.qt_count; ++t) p.units_per_batch += std::min(UNIT, a.N - t * UNIT) * (t + 1);
     p.plane_x = reinterpret_cast<__half*>(a.plane_x); p.plane_d = reinterpret_cast<__half*>(a.plane_d);

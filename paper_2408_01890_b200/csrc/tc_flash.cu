@@ -9,7 +9,9 @@
 //   row), P as bf16
 //   O += P . V                       tcgen05.mma (M 128, N 128, K 64), V read MN-major straight from its [key][d] tile
 // With QA/KA = Q/K and no Y this is standard attention (Eq. 1-2).  In MODE_EMIT there is no softmax: the scaled
-// scores leave as fp16 tiles (staged in shared memory, stored with TMA) for the aligner kernel.
+// scores leave as fp16 tiles (staged in shared memory, stored with TMA) for the aligner kernel.  In MODE_ATTN_CARRY the
+// attention also writes its finished pre-softmax logits A = S * scale + Y (unmasked, Eq. 4's A_n) back as fp16 tiles: the
+// next shared layer of a chain aligns those instead of recomputing the chain from the anchor's scores.
 //
 // Warp roles: warps 0-3 softmax/epilogue (thread = query row = TMEM lane), warp 4 TMA producer,
 // warp 5 issuer of the score MMAs and TMEM owner, warp 6 issuer of the P.V MMAs (warp 7 only completes the warpgroup).  K and V(/Y) have their own rings: a K stage is free again as soon as its
@@ -49,13 +51,15 @@ struct FlashParams {
 };
 
 // MODE_ATTN: softmax(QA.KA^T).V;  MODE_ATTN_PLANE: the same with the pre-computed tile Y added to the logits
-// (Y arrives already multiplied by log2(e));  MODE_EMIT: no softmax, the scaled scores go to the plane workspace.
-constexpr int MODE_ATTN = 0, MODE_ATTN_PLANE = 1, MODE_EMIT = 2;
+// (Y arrives already multiplied by log2(e));  MODE_EMIT: no softmax, the scaled scores go to the plane workspace;
+// MODE_ATTN_CARRY: MODE_ATTN_PLANE that also stores the logits (divided by log2(e) again) through the fifth tensor map.
+constexpr int MODE_ATTN = 0, MODE_ATTN_PLANE = 1, MODE_EMIT = 2, MODE_ATTN_CARRY = 3;
 
 template <int KD, int MODE>
 struct Smem {
-    static constexpr bool PLANE = MODE == MODE_ATTN_PLANE;
+    static constexpr bool PLANE = MODE == MODE_ATTN_PLANE || MODE == MODE_ATTN_CARRY;
     static constexpr bool EMIT = MODE == MODE_EMIT;
+    static constexpr bool CARRY = MODE == MODE_ATTN_CARRY;
     // P (the bf16 probabilities, A operand of P.V) is double-buffered so that the softmax of tile t+1 never waits
     // for the P.V of tile t.  To stay inside half an SM's shared memory it borrows a buffer whose content is dead
     // by then: with a plane, the Y tile of the same stage (each thread has read its own row of Y and overwrites just
@@ -72,7 +76,8 @@ struct Smem {
     static constexpr int P_BYTES = BM * BN * 2;
     static constexpr int P_OWN_BYTES = P_OWN ? 2 * P_BYTES : 0;
     static constexpr int Y_BYTES = PLANE ? BM * BN * 2 : 0;
-    static constexpr int STG_BYTES = EMIT ? 4 * 2 * 4096 : 0;  // per epilogue warp: two buffers of [32 rows][128 B]
+    // per epilogue warp: two buffers of [32 rows][128 B] (emit), one (carry)
+    static constexpr int STG_BYTES = EMIT ? 4 * 2 * 4096 : (CARRY ? 4 * 4096 : 0);
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = OFF_Q + Q_BYTES;
     static constexpr int OFF_V = OFF_K + KST * K_BYTES;
@@ -90,9 +95,9 @@ template <int KD, int MODE>
 __global__ void __launch_bounds__(kThreads, 2)
 tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ CUtensorMap tmQ,
                 const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-                const __grid_constant__ CUtensorMap tmY) {
+                const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmC) {
     using L = Smem<KD, MODE>;
-    constexpr bool PLANE = L::PLANE, EMIT = L::EMIT;
+    constexpr bool PLANE = L::PLANE, EMIT = L::EMIT, CARRY = L::CARRY;
     constexpr int KST = L::KST;
     extern __shared__ __align__(1024) uint8_t smem[];
     // 128-byte-swizzled tiles need 1024-byte aligned bases; the dynamic window starts on such a boundary (there is no
@@ -341,6 +346,29 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
                     }
                 }
             }
+            if constexpr (CARRY) {
+                // the finished logits of this warp's 32 rows x 64 columns leave as fp16 (back in the natural-log domain,
+                // before the mask: the next layer's aligner sees finite values everywhere) through the warp's staging buffer
+                uint8_t* stg = sStg + warp * 4096;
+                if (t >= 1 && lane == 0) tma_store_wait_read<0>();  // the store of the previous tile has read the buffer
+                __syncwarp();
+                constexpr float kLn2 = 0.6931471805599453f;
+#pragma unroll
+                for (int c = 0; c < BN / 8; ++c) {
+                    uint4 v;
+                    { const float2 t2 = __fmul2_rn(reinterpret_cast<const float2*>(sf)[c * 4 + 0], make_float2(kLn2, kLn2)); v.x = pack_f16(t2.x, t2.y); }
+                    { const float2 t2 = __fmul2_rn(reinterpret_cast<const float2*>(sf)[c * 4 + 1], make_float2(kLn2, kLn2)); v.y = pack_f16(t2.x, t2.y); }
+                    { const float2 t2 = __fmul2_rn(reinterpret_cast<const float2*>(sf)[c * 4 + 2], make_float2(kLn2, kLn2)); v.z = pack_f16(t2.x, t2.y); }
+                    { const float2 t2 = __fmul2_rn(reinterpret_cast<const float2*>(sf)[c * 4 + 3], make_float2(kLn2, kLn2)); v.w = pack_f16(t2.x, t2.y); }
+                    *reinterpret_cast<uint4*>(stg + sw128_offset(lane, c)) = v;
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_5d(&tmC, stg, 0, b * p.Hq + h, warp * 32, t, (q0 - p.plane_row0) / BM);
+                    tma_store_commit();
+                }
+            }
             // from here on: PLANE -> sf holds log2-domain logits; otherwise raw scores, scaled inside the exp
             if (t * BN + BN - 1 > q0) {   // the tile reaches past the CTA's first query row: mask keys after each row
 #pragma unroll
@@ -418,8 +446,10 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             tc_fence_before();
             mbar_arrive(p_full + s);
         }
-        if constexpr (EMIT) {
+        if constexpr (EMIT || CARRY) {
             if (lane == 0) tma_store_wait_all<0>();
+        }
+        if constexpr (EMIT) {
         } else if (ok && mbar_wait(pv_done + ((nt - 1) & 1), ((nt - 1) >> 1) & 1, abort_flag)) {
             tc_fence_after();
             const float inv_l = 1.f / l_sum;
@@ -509,6 +539,7 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     tmV = tmQ;
     if (!a.emit_plane && !map_bnhx(&tmV, a.v, a.B, a.N, a.Hkv, D, BN)) return cudaErrorInvalidValue;
     tmY = tmQ;
+    CUtensorMap tmC = tmQ;
     // Score planes are blocked [row block of 128][column block of 64][row in block][b*Hq + h][64 columns]: the 32
     // heads of a position lie 128 bytes apart (the aligner gathers them), and a head's 128 x 64 tile is 128 rows of 128
     // bytes spread over one 128 * B*Hq * 128-byte block, which the CTAs of all heads fill or drain at about the same time.
@@ -520,6 +551,11 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
         // emit: one epilogue warp's 32 rows x 64 columns per copy; attention: the CTA's 128 rows x 64 columns
         const uint32_t box[5] = {(uint32_t)BN, 1, a.emit_plane ? 32u : (uint32_t)BM, 1, 1};
         if (!make_tensor_map_bf16(&tmY, a.emit_plane ? a.emit_plane : a.plane, 5, dims, str, box, true)) return cudaErrorInvalidValue;
+        if (a.carry) {   // the logits leave one epilogue warp's 32 rows at a time
+            if (a.emit_plane || !a.plane) return cudaErrorInvalidValue;
+            const uint32_t cbox[5] = {(uint32_t)BN, 1, 32u, 1, 1};
+            if (!make_tensor_map_bf16(&tmC, a.carry, 5, dims, str, cbox, true)) return cudaErrorInvalidValue;
+        }
     }
     FlashParams p;
     p.B = a.B; p.N = a.N; p.Hq = a.Hq; p.Hkv = a.Hkv;
@@ -528,7 +564,8 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     p.o_sb = a.o.stride_b; p.o_sn = a.o.stride_n; p.o_sh = a.o.stride_h;
     p.status = status_words();
     if (!p.status) return cudaErrorUnknown;
-    p.plane_row0 = a.qt_begin * BM;
+    p.plane_row0 = a.plane_row0 >= 0 ? a.plane_row0 : a.qt_begin * BM;
+    if (p.plane_row0 % BM != 0 || p.plane_row0 > a.qt_begin * BM) return cudaErrorInvalidValue;
     p.qt_begin = a.qt_begin;
     p.ksteps = a.ksteps > 0 ? a.ksteps : a.kd / 16;
     p.scale = a.scale;
@@ -543,12 +580,13 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
             return e;                                                                                                      \
         if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared)) != cudaSuccess) \
             return e;                                                                                                      \
-        kern<<<grid, kThreads, Smem<KD_, PL_>::TOTAL, stream>>>(p, tmQ, tmK, tmV, tmY);                                    \
+        kern<<<grid, kThreads, Smem<KD_, PL_>::TOTAL, stream>>>(p, tmQ, tmK, tmV, tmY, tmC);                                    \
     } while (0)
     if (a.emit_plane) {
         if (a.kd == 128) LISA_LAUNCH_FLASH(128, MODE_EMIT);
         else LISA_LAUNCH_FLASH(64, MODE_EMIT);
     } else if (a.kd == 128 && !a.plane) LISA_LAUNCH_FLASH(128, MODE_ATTN);
+    else if (a.kd == 64 && a.plane && a.carry) LISA_LAUNCH_FLASH(64, MODE_ATTN_CARRY);
     else if (a.kd == 64 && a.plane) LISA_LAUNCH_FLASH(64, MODE_ATTN_PLANE);
     else if (a.kd == 64 && !a.plane) LISA_LAUNCH_FLASH(64, MODE_ATTN);
     else return cudaErrorInvalidValue;  // 128-wide scores plus a plane do not fit shared memory

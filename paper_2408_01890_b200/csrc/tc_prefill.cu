@@ -120,7 +120,8 @@ struct Layout {
     size_t total;
 };
 
-Layout plan_layout(const lisa_shared_prefill_args& a) {
+// carried: the scores live in the caller's buffer, the workspace holds only the packed Q', K'
+Layout plan_layout(const lisa_shared_prefill_args& a, bool carried = false) {
     Layout l{};
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 1023) & ~(size_t)1023; return o; };
@@ -136,7 +137,7 @@ Layout plan_layout(const lisa_shared_prefill_args& a) {
     l.plane_rows = (int64_t)max_cnt * kTile;
     l.plane_cols = (int64_t)n_qt * kTile;
     l.sets = std::max(1, std::min(kWaveSets, nw));
-    for (int set = 0; set < l.sets; ++set)
+    for (int set = 0; set < l.sets && !carried; ++set)
         for (int k = 0; k < plane_count(a); ++k) l.plane_off[set][k] = take((size_t)a.B * a.Hq * l.plane_rows * l.plane_cols * 2);
     l.total = off;
     return l;
@@ -171,6 +172,11 @@ bool tc_shared_prefill_supported(const lisa_shared_prefill_args& a) {
 
 // + 1024: the launch aligns the caller's pointer up to the 1024 bytes the swizzled tiles need
 size_t tc_shared_prefill_workspace(const lisa_shared_prefill_args& a) { return plan_layout(a).total + 1024; }
+size_t tc_shared_prefill_carry_workspace(const lisa_shared_prefill_args& a) { return plan_layout(a, true).total + 1024; }
+size_t tc_carry_bytes(int B, int N, int Hq) {
+    const size_t n = (size_t)(N + kTile - 1) / kTile * kTile;
+    return (size_t)B * Hq * n * n * 2;
+}
 
 namespace {
 // The packing of Q'/K' feeds only the kernels that come after the first emit (the attention kernel; the emits of the
@@ -213,10 +219,19 @@ cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws
 // With vs/os == nullptr: the layer at chain depth c (a.v, a.o).  With vs/os[c]: all c layers of the chain in one
 // pass -- the anchor scores and the differences are emitted once, the aligner stores every link's output (link k
 // over plane k), and one attention kernel per layer consumes its plane with its own Q', K' and V.
+// With cy: one link, in place on the caller's carried scores (rows from 0, N rounded up to whole tiles both ways): no A_0
+// unless this is the first layer of its chain, no wave planes, and the attention kernel leaves A_n behind when asked.
 cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, const lisa_tensor* vs, const lisa_tensor* os, void* ws,
-                                           cudaStream_t s) {
+                                           cudaStream_t s, const TcCarry* cy) {
     const bool all_layers = vs != nullptr;
-    const Layout l = plan_layout(a);
+    if (cy && (all_layers || a.chain_len != 1 || concat_chain(a) || !cy->scores)) return cudaErrorInvalidValue;
+    Layout l = plan_layout(a, cy != nullptr);
+    if (cy) {
+        l.plane_rows = l.plane_cols = (int64_t)(a.N + kTile - 1) / kTile * kTile;
+        for (int set = 0; set < kWaveSets; ++set) l.plane_off[set][0] = 0;
+    }
+    char* const plane_base = cy ? reinterpret_cast<char*>(cy->scores) : nullptr;
+    const int row0 = cy ? 0 : -1;
     char* base = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(ws) + 1023) & ~(uintptr_t)1023);
     const int c = a.chain_len;
     cudaError_t e;
@@ -279,8 +294,9 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         // 1. anchor scores and the differences of the links below the top one
         TcFlashArgs f{a.B, a.N, a.Hq, a.Hkv, 128, a.q0, a.k0, a.v, a.o, 1.f / sqrtf((float)a.d), nullptr, l.plane_rows, l.plane_cols,
                       wv.begin, wv.count};
-        f.emit_plane = base + po[0];
-        {
+        f.plane_row0 = row0;
+        f.emit_plane = cy ? plane_base : base + po[0];
+        if (!cy || cy->first) {
             PhaseMark mark(1, st);
             if ((e = launch_tc_flash(f, st)) != cudaSuccess) return e;
         }
@@ -327,9 +343,9 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             // plane k, writes A_k = FFN_k(A_{k-1}) + D_k over plane k + 1 (which held D_k) and, where a layer's attention
             // consumes it, log2(e) * FFN_k(A_{k-1}) over plane k.
             for (int k = 0; k < c; ++k) {
-                TcAlignLinkArgs al{a.B, a.N, a.Hq, wv.begin, wv.count, l.plane_rows, l.plane_cols, base + po[k],
+                TcAlignLinkArgs al{a.B, a.N, a.Hq, wv.begin, wv.count, l.plane_rows, l.plane_cols, cy ? plane_base : base + po[k],
                                    k + 1 < c ? base + po[k + 1] : nullptr, &a.links[k], k + 1 < c ? 1 : -1,
-                                   (all_layers || k == c - 1) ? 0 : -1};
+                                   (all_layers || k == c - 1) ? 0 : -1, row0};
                 PhaseMark mark(2, st);
                 if ((e = launch_tc_align_link(al, st)) != cudaSuccess) return e;
             }
@@ -338,8 +354,9 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         TcAlignArgs al{};
         al.B = a.B; al.N = a.N; al.chain = c; al.qt_begin = wv.begin; al.qt_count = wv.count;
         al.plane_rows = l.plane_rows; al.plane_cols = l.plane_cols;
-        for (int k = 0; k < c; ++k) al.planes[k] = base + po[k];
+        for (int k = 0; k < c; ++k) al.planes[k] = cy ? plane_base : base + po[k];
         al.links = a.links;
+        al.row0 = row0;
         al.store_all = all_layers;
         if (!per_link) {
             PhaseMark mark(2, st);
@@ -355,7 +372,8 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             fv.ka = packed_view(base + l.kp_off[k], a.Hkv, a.N);
             fv.scale = 1.f / sqrtf((float)a.links[k].r);
             fv.ksteps = (a.links[k].r + 15) / 16;
-            fv.plane = base + po[all_layers ? k : (per_link ? c - 1 : 0)];
+            fv.plane = cy ? plane_base : base + po[all_layers ? k : (per_link ? c - 1 : 0)];
+            if (cy && cy->keep) fv.carry = plane_base;
             if (all_layers) { fv.v = vs[k]; fv.o = os[k]; }
             PhaseMark mark(3, st);
             if ((e = launch_tc_flash(fv, st)) != cudaSuccess) return e;

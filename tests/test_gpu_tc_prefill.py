@@ -224,3 +224,51 @@ def test_link_by_link_chain_in_one_pass():
         ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1])
         assert_close(outs[k].float().cpu().numpy(), ref, "bf16", "link-by-link chain at 40 heads, layer %d" % (k + 1))
     assert lb.lisa_check() == lb.OK
+
+
+@pytest.mark.parametrize("B,N,Hq,Hkv,chain,m,act,integrate,layers,bias", [
+    (2, 300, 32, 8, 3, 64, "relu", lb.INTEGRATE_ADD, 2, False),     # the cfg3 layer shape
+    (1, 513, 32, 32, 6, 64, "silu", lb.INTEGRATE_ADD, 2, True),     # a run of six shared layers: deeper than the recomputing kernels take
+    (1, 200, 40, 40, 3, 80, "relu", lb.INTEGRATE_ADD, 2, True),     # LLaMA2-13B layer shape (link-by-link aligner)
+    (1, 260, 32, 8, 2, 32, "none", lb.INTEGRATE_ADD, 1, True),      # one linear layer
+    (1, 130, 32, 32, 3, 64, "none", lb.INTEGRATE_PLUS, 2, False)])  # no FFN
+def test_carried_scores_layer_by_layer(B, N, Hq, Hkv, chain, m, act, integrate, layers, bias):
+    """lisa_attn_shared_prefill_carry: every layer of a chain takes A_{n-1} from the scores buffer the layer before left
+    (Sec. 5.1) and must equal the oracle's layer at that depth; only the first layer computes the anchor's scores (seen in
+    the launch counts: pack, emit, align, attention for the first layer; pack, align, attention afterwards)."""
+    t = link_inputs(B, N, Hq, Hkv, chain, m, act, layers, 21, 31, bias)
+    dl, ol = make_links(t, chain, act, integrate, layers, bias)
+    scores = torch.full((lb.lisa_prefill_scores_bytes(B, N, Hq),), 0xFF, dtype=torch.uint8, device="cuda")   # NaN patterns where nothing was written
+    q0, k0 = dev(t["q0"]), dev(t["k0"])
+    for k in range(chain):
+        v = dev(t[f"v{k + 1}"])
+        n0 = lb.lisa_kernel_launches()
+        if k == 0:
+            got = lb.lisa_attn_shared_prefill_carry(q0, k0, dl[0], v, scores, first=True, keep=chain > 1)
+        else:
+            got = lb.lisa_attn_shared_prefill_carry(None, None, dl[k], v, scores, first=False, keep=k + 1 < chain, out=torch.empty_like(q0))
+        torch.cuda.synchronize()
+        assert lb.lisa_kernel_launches() - n0 == (4 if k == 0 else 3)
+        assert lb.lisa_check() == lb.OK
+        ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1])
+        assert_close(got.float().cpu().numpy(), ref, "bf16", "carried scores, layer %d of %d, %d heads" % (k + 1, chain, Hq))
+
+
+def test_carried_scores_rejects_bad_arguments():
+    B, N, Hq, Hkv = 1, 130, 32, 32
+    t = link_inputs(B, N, Hq, Hkv, 1, 64, "relu", 2, 21, 33, False)
+    dl, _ = make_links(t, 1, "relu")
+    q0, k0, v = dev(t["q0"]), dev(t["k0"]), dev(t["v1"])
+    need = lb.lisa_prefill_scores_bytes(B, N, Hq)
+    assert need == B * Hq * 256 * 256 * 2
+    small = torch.empty(need - 1, dtype=torch.uint8, device="cuda")
+    with pytest.raises(lb.LisaError) as ei:
+        lb.lisa_attn_shared_prefill_carry(q0, k0, dl[0], v, small, first=True, keep=True)
+    assert ei.value.status == lb.ERR_INVALID_ARG
+    scores = torch.empty(need, dtype=torch.uint8, device="cuda")
+    cat = concat_inputs(B, N, Hkv, 1, 64, "relu", 2, 21, 33, False)
+    dc, _ = make_links(cat, 1, "relu", lb.INTEGRATE_CONCAT, 2, False)
+    with pytest.raises(lb.LisaError) as ei:   # the concatenating Integrate has no carried form
+        lb.lisa_attn_shared_prefill_carry(q0, k0, dc[0], v, scores, first=True, keep=True)
+    assert ei.value.status == lb.ERR_UNSUPPORTED
+    assert lb.lisa_check() == lb.OK
