@@ -167,8 +167,9 @@ def workload_config(w):
     """The same dictionary in both arms (the reference arm runs the same step, on a row sample, on the host)."""
     return {"workload": w.name, "B": w.B, "N": w.N, "Hq": w.Hq, "Hkv": w.Hkv, "d": w.d, "r": w.r, "m": w.m, "act": w.act,
             "chain_len": w.chain, "l2": "GPU arm: 256 MiB buffer written between timed iterations",
-            "step": "per shared layer of the chain: the layer at its chain depth (lisa_attn_shared_prefill) + the append of its K', V "
-                    "(lisa_kvcache_append); a token counts once it is through all %d layers" % w.chain}
+            "step": "per shared layer of the chain: the layer's attention (%s) + the append of its K', V "
+                    "(lisa_kvcache_append); a token counts once it is through all %d layers"
+                    % ("lisa_attn_shared_prefill_carry, scores carried from the layer before" if w.chain > 1 else "lisa_attn_shared_prefill", w.chain)}
 
 
 def time_steps(step, n, flush, barrier):
@@ -197,10 +198,14 @@ def mark():
 
 
 def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
-    """The prefill step of workload `name`: one lisa_attn_shared_prefill + lisa_kvcache_append per shared layer of the chain."""
+    """The prefill step of workload `name`: per shared layer of the chain, the layer's attention call + lisa_kvcache_append.
+    A chain of several layers runs with the scores carried from layer to layer (lisa_attn_shared_prefill_carry: Sec. 5.1's
+    A_{n-1} from the layer before); the same layers recomputed from the anchor per layer (lisa_attn_shared_prefill at depth
+    1..C) and in one fused call (lisa_attn_shared_prefill_chain) are timed beside it.  A single layer has nothing to carry."""
     flush, barrier, max_over_ranks, peaks, world = env
     w = synth.WORKLOADS[name]
     C = w.chain
+    carried = C > 1
     t = synth.prefill_inputs(w, seed=rank)
     d = {k: v.cuda() for k, v in t.items()}
     links = [lb.Link(d[f"qp{k}"], d[f"kp{k}"], d[f"w1_{k}"], d[f"w2_{k}"], act=lb.ACTS[w.act]) for k in range(1, C + 1)]
@@ -208,88 +213,113 @@ def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
     outs = [torch.empty_like(d["q0"]) for _ in range(C)]
     caches = [lb.KVCacheLayer(lb.CACHE_SHARED, w.B, w.Hkv, w.N, w.d, w.r) for _ in range(C)]
     ws = lb.prefill_workspace(d["q0"], d["k0"], links, vs[-1], outs[-1])   # the deepest layer needs the most
+    scores = yws = None
+    if carried:
+        scores = torch.empty(lb.lisa_prefill_scores_bytes(w.B, w.N, w.Hq), dtype=torch.uint8, device="cuda")
+        yws = lb.prefill_carry_workspace(d["q0"], d["k0"], links[0], vs[0], outs[0], scores)
 
-    def layer_call(c):
-        lb.lisa_attn_shared_prefill(d["q0"], d["k0"], links[:c], vs[c - 1], out=outs[c - 1], workspace=ws)
+    def layer_call(c, carry):
+        if carry:
+            lb.lisa_attn_shared_prefill_carry(d["q0"], d["k0"], links[c - 1], vs[c - 1], scores, first=c == 1, keep=c < C,
+                                              out=outs[c - 1], workspace=yws)
+        else:
+            lb.lisa_attn_shared_prefill(d["q0"], d["k0"], links[:c], vs[c - 1], out=outs[c - 1], workspace=ws)
 
-    def step():
-        evs = []
-        for c in range(1, C + 1):
-            layer_call(c)
-            evs.append(mark())
-            lb.lisa_kvcache_append(caches[c - 1], d[f"kp{c}"], vs[c - 1])
-            evs.append(mark())
-        return evs
+    def make_step(carry):
+        def step():
+            evs = []
+            for c in range(1, C + 1):
+                layer_call(c, carry)
+                evs.append(mark())
+                lb.lisa_kvcache_append(caches[c - 1], d[f"kp{c}"], vs[c - 1])
+                evs.append(mark())
+            return evs
+        return step
 
-    for _ in range(args.warmup):
-        flush(); step()
-    l0 = lb.lisa_kernel_launches()
-    total_ms, starts, marks = time_steps(step, args.steps, flush, barrier)
-    launches = lb.lisa_kernel_launches() - l0
-    ms_per_step = max_over_ranks(total_ms) / args.steps
-    # device time of each layer's attention call (without its append), averaged over the steps
-    call_ms = []
-    for c in range(C):
-        tot = 0.0
-        for s, evs in zip(starts, marks):
-            tot += (s if c == 0 else evs[2 * c - 1]).elapsed_time(evs[2 * c])
-        call_ms.append(tot / args.steps)
+    def measure(step):
+        """(ms per step, device ms of each layer's attention call without its append, launches)"""
+        for _ in range(args.warmup):
+            flush(); step()
+        l0 = lb.lisa_kernel_launches()
+        total_ms, starts, marks = time_steps(step, args.steps, flush, barrier)
+        n_launch = lb.lisa_kernel_launches() - l0
+        call_ms = [sum((s0 if c == 0 else evs[2 * c - 1]).elapsed_time(evs[2 * c]) for s0, evs in zip(starts, marks)) / args.steps
+                   for c in range(C)]
+        return max_over_ranks(total_ms) / args.steps, call_ms, n_launch
+
+    ms_per_step, call_ms, launches = measure(make_step(carried))
     tokens = w.B * w.N
 
     # per-kernel device times of each call (events recorded inside the library around each of its kernels)
     names = ["pack", "emit_scores", "align", "attention"]
     P, ph = positions(w), positions(w) * w.Hq
     qk_lr = w.B * w.N * (w.Hq + w.Hkv) * 2
-    per_layer = []
+    phase_ms = [[0.0] * 4 for _ in range(C)]
     lb.lisa_prefill_phase_timing(True)
+    for _ in range(args.steps):
+        for c in range(1, C + 1):   # in chain order: a carried layer needs the scores the one before left
+            flush(); layer_call(c, carried)
+            for i, x in enumerate(lb.lisa_prefill_phase_times()):
+                phase_ms[c - 1][i] += x / args.steps
+    lb.lisa_prefill_phase_timing(False)
+    per_layer = []
     for c in range(1, C + 1):
-        for _ in range(args.steps):
-            flush(); layer_call(c)
-        phase_ms = [x / args.steps for x in lb.lisa_prefill_phase_times()]
-        # algorithmic work of each kernel at depth c.  The kernels hand the scores of every causal position to one another as
-        # fp16 planes (2 bytes per position and head); emit writes A_0 and the c-1 inner differences, the aligner reads
-        # those c planes and writes one, the attention kernel reads one.
-        kflops = {"pack": 0, "emit_scores": P * (2 * w.Hq * w.d + (c - 1) * 2 * w.Hq * w.r), "align": P * c * 4 * w.Hq * w.m,
-                  "attention": P * (2 * w.Hq * w.r + 2 * w.Hq * w.d)}
-        kbytes = {"pack": c * qk_lr * (w.r + 64), "emit_scores": qk_lr * w.d + c * ph * 2, "align": (c + 1) * ph * 2,
-                  "attention": ph * 2 + qk_lr * 64 + w.B * w.N * (w.Hkv + w.Hq) * w.d * 2}
-        ktraffic = {"emit_scores": PREFILL_TRAFFIC_PER_PH["emit_scores"], "align": PREFILL_TRAFFIC_PER_PH["align"],
-                    "attention": PREFILL_TRAFFIC_PER_PH["attention"]}
+        # What each kernel of the layer at depth c executes.  The kernels hand the scores of every causal position to one
+        # another as fp16 planes (2 bytes per position and head).  Recomputing: emit writes A_0 and the c-1 inner differences,
+        # the aligner reads those c planes and writes one, the attention kernel reads one.  Carried: only the first layer
+        # emits A_0; the aligner reads and writes one plane; the attention kernel reads one and (unless last) writes one.
+        if carried:
+            kflops = {"pack": 0, "emit_scores": P * 2 * w.Hq * w.d if c == 1 else 0, "align": P * 4 * w.Hq * w.m,
+                      "attention": P * (2 * w.Hq * w.r + 2 * w.Hq * w.d)}
+            kbytes = {"pack": qk_lr * (w.r + 64), "emit_scores": (qk_lr * w.d + ph * 2) if c == 1 else 0, "align": 2 * ph * 2,
+                      "attention": ph * 2 * (2 if c < C else 1) + qk_lr * 64 + w.B * w.N * (w.Hkv + w.Hq) * w.d * 2}
+        else:
+            kflops = {"pack": 0, "emit_scores": P * (2 * w.Hq * w.d + (c - 1) * 2 * w.Hq * w.r), "align": P * c * 4 * w.Hq * w.m,
+                      "attention": P * (2 * w.Hq * w.r + 2 * w.Hq * w.d)}
+            kbytes = {"pack": c * qk_lr * (w.r + 64), "emit_scores": qk_lr * w.d + c * ph * 2, "align": (c + 1) * ph * 2,
+                      "attention": ph * 2 + qk_lr * 64 + w.B * w.N * (w.Hkv + w.Hq) * w.d * 2}
+        ktraffic = PREFILL_TRAFFIC_PER_PH if (c == 1 and not carried) else {}   # the captures are of the recomputing layer at depth 1
         kernels = {}
         for i, n in enumerate(names):
-            sec = phase_ms[i] * 1e-3
+            sec = phase_ms[c - 1][i] * 1e-3
             t_tensor, t_hbm = kflops[n] / (peaks["bf16_tflops"] * 1e12), kbytes[n] / (peaks["hbm_gbs"] * 1e9)
             tr = ktraffic.get(n)
-            kernels[n] = {"ms": phase_ms[i], "share": phase_ms[i] / max(sum(phase_ms), 1e-9), "flops": kflops[n], "bytes": kbytes[n],
-                          "tflops": kflops[n] / sec / 1e12 if sec > 0 else None, "gbs": kbytes[n] / sec / 1e9 if sec > 0 else None,
+            kernels[n] = {"ms": phase_ms[c - 1][i], "share": phase_ms[c - 1][i] / max(sum(phase_ms[c - 1]), 1e-9), "flops": kflops[n],
+                          "bytes": kbytes[n], "tflops": kflops[n] / sec / 1e12 if sec > 0 else None,
+                          "gbs": kbytes[n] / sec / 1e9 if sec > 0 else None,
                           "bound": "hbm" if t_hbm >= t_tensor else "tensor", "frac": max(t_tensor, t_hbm) / sec if sec > 0 else None,
-                          "traffic": tr * ph if (tr and c == 1) else None}
-        fl = prefill_flops(w, c)
+                          "traffic": tr * ph if tr else None}
+        fl = sum(kflops.values())
         tf = fl / (call_ms[c - 1] * 1e-3) / 1e12
-        traffic = sum(k["traffic"] for k in kernels.values() if k["traffic"]) if c == 1 else None
-        per_layer.append({"chain_depth": c, "ms": call_ms[c - 1], "flops": fl, "flops_per_position": flops_per_position(w, c),
+        traffic = sum(k["traffic"] for k in kernels.values() if k["traffic"]) if ktraffic else None
+        per_layer.append({"chain_depth": c, "ms": call_ms[c - 1], "flops": fl, "flops_per_position": fl // P,
                           "achieved": tf, "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
-                          "algorithmic_bytes": prefill_algorithmic_bytes(w, c),
+                          "algorithmic_bytes": prefill_algorithmic_bytes(w, 1 if carried else c),
                           "traffic_over_algorithmic": traffic / prefill_algorithmic_bytes(w, c) if traffic else None,
                           "kernels": kernels})
-    lb.lisa_prefill_phase_timing(False)
 
-    flops = sum(prefill_flops(w, c) for c in range(1, C + 1))
+    flops = sum(pl["flops"] for pl in per_layer)                        # executed
+    formula_flops = sum(prefill_flops(w, c) for c in range(1, C + 1))   # what C layers recomputed from the anchor would execute
     calls_ms = sum(call_ms)
     tf = flops / (calls_ms * 1e-3) / 1e12
-    # the kernel with the largest share of the step, over all three calls
+    # the kernel with the largest share of the step, over all calls
     dom_name = max(names, key=lambda n: sum(pl["kernels"][n]["ms"] for pl in per_layer))
     dom_ms = sum(pl["kernels"][dom_name]["ms"] for pl in per_layer)
     dom_bytes = sum(pl["kernels"][dom_name]["bytes"] for pl in per_layer)
     dom_flops = sum(pl["kernels"][dom_name]["flops"] for pl in per_layer)
     dom_hbm = dom_bytes / (peaks["hbm_gbs"] * 1e9) >= dom_flops / (peaks["bf16_tflops"] * 1e12)
+    call_name = "lisa_attn_shared_prefill_carry" if carried else "lisa_attn_shared_prefill"
     roofline = {
-        "bound": "tensor", "kernel": "lisa_attn_shared_prefill, chain depth 1..%d (the %d calls of a step, appends excluded)" % (C, C),
+        "bound": "tensor", "kernel": "%s, chain depth 1..%d (the %d calls of a step, appends excluded)" % (call_name, C, C),
         "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
         "peak_source": peaks["source"] + " (burst)", "ms": calls_ms, "flops_per_step": flops,
-        "formula": "causal positions B*N*(N+1)/2 x sum over c of (2hd + c(2hr + 4hm) + 2hd)",
+        "formula": ("causal positions B*N*(N+1)/2 x (2hd + C(2hr + 4hm + 2hd)): the anchor's scores once, every link once, P.V per layer"
+                    if carried else "causal positions B*N*(N+1)/2 x sum over c of (2hd + c(2hr + 4hm) + 2hd)"),
+        "frac_by_recompute_formula": formula_flops / (calls_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "recompute_formula": "causal positions x sum over c = 1..C of (2hd + c(2hr + 4hm) + 2hd): what layers recomputed from the anchor execute",
         "traffic": per_layer[0]["kernels"][dom_name]["traffic"],
-        "traffic_note": "ncu DRAM bytes of the dominant kernel at chain depth 1, the cfg2 capture scaled by causal positions",
+        "traffic_note": ("none: the kernels' DRAM counters were captured on the recomputing layer at depth 1 (see cfg2)" if carried else
+                         "ncu DRAM bytes of the dominant kernel at chain depth 1, the cfg2 capture scaled by causal positions"),
         "traffic_over_algorithmic": per_layer[0]["traffic_over_algorithmic"],
         "dominant_kernel": {"name": dom_name, "ms_per_step": dom_ms, "bound": "hbm" if dom_hbm else "tensor",
                             "achieved": dom_bytes / (dom_ms * 1e-3) / 1e9 if dom_hbm else dom_flops / (dom_ms * 1e-3) / 1e12,
@@ -299,10 +329,18 @@ def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
         "per_layer": per_layer}
 
     res = {"workload": w.name, "ms_per_step": ms_per_step, "value": world * tokens / (ms_per_step * 1e-3), "launches": launches,
-           "roofline": roofline, "tokens": tokens, "outs": outs, "inputs": t}
+           "roofline": roofline, "tokens": tokens, "outs": outs, "inputs": t, "carried": carried,
+           "scores_buffer_bytes": scores.numel() if carried else 0}
 
-    # ---------------- the same layers through one lisa_attn_shared_prefill_chain call ----------------
-    if with_chain and C > 1:
+    if carried and with_chain:
+        # ---------------- the same layers, each recomputed from the anchor (lisa_attn_shared_prefill at depth 1..C) ----------------
+        rms, rcalls, rl = measure(make_step(False))
+        res["launches"] += rl
+        res["recompute"] = {"ms_per_step": rms, "value": world * tokens / (rms * 1e-3), "unit": "tokens/s", "call_ms_by_depth": rcalls,
+                            "flops_per_step": formula_flops, "frac": formula_flops / (sum(rcalls) * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                            "note": "every layer recomputes the chain from the anchor's q0, k0: workspace of a wave of rows instead of the "
+                                    "whole prompt's scores; frac counts the recomputed flops it executes"}
+        # ---------------- the same layers through one lisa_attn_shared_prefill_chain call ----------------
         cws = lb.prefill_chain_workspace(d["q0"], d["k0"], links, vs, outs)
 
         def chain_step():
@@ -318,14 +356,13 @@ def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
         ctot, cst, cmk = time_steps(chain_step, args.steps, flush, barrier)
         res["launches"] += lb.lisa_kernel_launches() - l1
         cms = max_over_ranks(ctot) / args.steps
-        call = sum(s.elapsed_time(m[0]) for s, m in zip(cst, cmk)) / args.steps
-        executed = P * (2 * w.Hq * w.d + C * (2 * w.Hq * w.r + 4 * w.Hq * w.m + 2 * w.Hq * w.d))
+        call = sum(s0.elapsed_time(m[0]) for s0, m in zip(cst, cmk)) / args.steps
         res["chain_call"] = {"ms_per_step": cms, "value": world * tokens / (cms * 1e-3), "unit": "tokens/s", "call_ms": call,
-                             "frac_by_layer_formula": flops / (call * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                             "flops_needed_once": executed,
-                             "frac_by_flops_needed_once": executed / (call * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                             "note": "one pass computes A_0 and every link once; the per-layer formula counts what three separate calls recompute"}
+                             "frac": flops / (call * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                             "frac_by_recompute_formula": formula_flops / (call * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                             "note": "one call for all layers of the chain (needs every layer's Q', K', V at once)"}
         del cws
+    del scores, yws
 
     # ---------------- end to end through the host-memory entry point ----------------
     if with_e2e:
@@ -605,7 +642,9 @@ def main():
             w = synth.WORKLOADS[main_res["workload"]]
             cfg = workload_config(w)
             line.update({"value": main_res["value"], "ms_per_step": main_res["ms_per_step"], "config": cfg,
-                         "e2e": main_res.get("e2e"), "roofline": main_res["roofline"], "chain_call": main_res.get("chain_call")})
+                         "e2e": main_res.get("e2e"), "roofline": main_res["roofline"], "recompute": main_res.get("recompute"),
+                         "chain_call": main_res.get("chain_call")})
+            line["scores_buffer_bytes"] = main_res["scores_buffer_bytes"]
             if head is None:
                 line["paper_default_layer"] = main_res.get("paper_default_layer")
                 line["llama2_13b_layer"] = main_res.get("llama2_13b_layer")
