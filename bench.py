@@ -579,7 +579,7 @@ def main():
         from paper_2408_01890_b200 import stack as lstack
         ws5 = synth.WORKLOADS["cfg5_llama2_7b_stack"]
         res5 = {}
-        # lisa: shared layers prefilled through the shared path, one pass per chain of three; lisa_nf: the paper's lossless-prefill recipe
+        # lisa: shared layers prefilled layer by layer with the scores carried along each chain of three; lisa_nf: the paper's lossless-prefill recipe
         # (Sec. 5.2), shared layers prefilled with standard attention and only their cache differing
         for name, std_layers, nf in (("lisa", None, False), ("lisa_nf", None, True), ("standard", list(range(32)), False)):
             torch.cuda.empty_cache()

@@ -60,19 +60,27 @@ class AttentionStack:
         return l + 1 < self.n_layers and not self.is_standard[l + 1]
 
     # ------------------------------------------------------------------ prefill
-    def prefill(self, probe: Optional[Probe] = None, nf: bool = False, fused: bool = True) -> float:
+    def prefill(self, probe: Optional[Probe] = None, nf: bool = False, mode: str = "carried") -> float:
         """Runs every layer over the prompt and fills the caches. Returns the device time in milliseconds.
 
-        fused=True hands every run of shared layers behind an anchor to `lisa_attn_shared_prefill_chain` (the anchor
-        scores and each link's difference are computed once for the run); fused=False calls
-        `lisa_attn_shared_prefill` layer by layer.  Same results either way.
+        mode="carried" (the order a model runs in: layer by layer, each shared layer aligning the scores the layer before
+        left in a buffer, `lisa_attn_shared_prefill_carry`); "fused" hands every run of shared layers behind an anchor to
+        `lisa_attn_shared_prefill_chain` (possible here because the stack's inputs do not depend on its outputs);
+        "recompute" calls `lisa_attn_shared_prefill` layer by layer, each recomputing its chain from the anchor.  Same
+        results every way.
         nf=True is the paper's lossless-prefill recipe (Sec. 5.2, "NF"): a shared layer attends over the prompt with
         standard attention on its own full Q and K, and only what it caches differs (the low-rank keys K_LR take the place of K); sharing
         starts with the first decoded token.  Prefill then costs what a standard stack costs.
         """
         B, N, Hq, Hkv, d, r = self.B, self.N, self.Hq, self.Hkv, self.d, self.r
         t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if mode not in ("carried", "fused", "recompute"):
+            raise ValueError("mode: carried, fused or recompute")
+        fused = mode == "fused"
         outs = [torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device="cuda") for _ in range(3 if fused and not nf else 1)]
+        scores = None
+        if mode == "carried" and not nf and not all(self.is_standard):
+            scores = torch.empty(lb.lisa_prefill_scores_bytes(B, N, Hq), dtype=torch.uint8, device="cuda")
         out = outs[0]
         # every layer's inputs are drawn before the clock starts
         drawn = []
@@ -140,6 +148,15 @@ class AttentionStack:
                     record(j, outs[i], q0, k0, drawn[j][2], links[:len(links) - len(run) + i + 1])
                 l = end
                 continue
+            elif mode == "carried":
+                w1, w2 = self.weights[l]
+                links = links + [lb.Link(a, b_, w1, w2, act=lb.ACTS[self.act])]
+                if ws is None:
+                    ws = lb.prefill_carry_workspace(q0, k0, links[-1], v, out, scores)
+                lb.lisa_attn_shared_prefill_carry(q0, k0, links[-1], v, scores, first=len(links) == 1, keep=self.next_is_shared(l),
+                                                  out=out, workspace=ws)
+                lb.lisa_kvcache_append(self.caches[l], b_, v)
+                record(l, out, q0, k0, v, links)
             else:
                 w1, w2 = self.weights[l]
                 links = links + [lb.Link(a, b_, w1, w2, act=lb.ACTS[self.act])]

@@ -49,11 +49,13 @@ def test_small_stack_every_layer():
     check_probe(st, probe)
 
 
-def test_small_stack_layer_by_layer_prefill():
-    """The same small stack with every shared layer prefilled by its own call instead of one pass per chain."""
+@pytest.mark.parametrize("mode", ["recompute", "fused"])
+def test_small_stack_other_prefill_modes(mode):
+    """The same small stack with every shared layer recomputing its chain from the anchor, and with one pass per chain,
+    instead of the scores carried from layer to layer."""
     st = lstack.AttentionStack(n_layers=8, B=2, N=200, T=2, seed=3)
     probe = lstack.Probe(layers=range(8), rows_b=[0, 1, 1, 0], rows_i=[0, 199, 77, 128], steps=[1], seqs=[0, 1])
-    st.prefill(probe, fused=False)
+    st.prefill(probe, mode=mode)
     st.decode(probe)
     assert lb.lisa_check() == lb.OK
     check_probe(st, probe)
