@@ -56,6 +56,16 @@ def test_cfg3_llama3_8b_gqa_prefill_chain_sampled_rows():
         del got
         ref = oracle.prefill_rows(q0h, k0h, f64(v), ol[:c], rb, ri)
         assert_close(sel, ref, "bf16", "cfg3 chain depth %d" % c)
+        if c >= 1:
+            # the same layer with the scores carried from the layer before (the form the benchmark times)
+            if c == 1:
+                scores = torch.empty(lb.lisa_prefill_scores_bytes(w.B, w.N, w.Hq), dtype=torch.uint8, device="cuda")
+            got = lb.lisa_attn_shared_prefill_carry(q0d, k0d, dl[c - 1], dev(v), scores, first=c == 1, keep=c < w.chain)
+            torch.cuda.synchronize()
+            assert lb.lisa_check() == lb.OK
+            sel = got[torch.from_numpy(rb).long().cuda(), torch.from_numpy(ri).long().cuda()].float().cpu().numpy()
+            del got
+            assert_close(sel, ref, "bf16", "cfg3 carried scores, layer %d" % c)
 
 
 def test_cfg4_llama2_13b_decode_sampled_sequences():
