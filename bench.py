@@ -364,22 +364,38 @@ def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
         del cws
     del scores, yws
 
-    # ---------------- end to end through the host-memory entry point ----------------
+    # ---------------- end to end through the host-memory entry points ----------------
     if with_e2e:
         hp = {k: v.pin_memory() for k, v in t.items() if k != "v0"}
         hlinks = [lb.Link(hp[f"qp{k}"], hp[f"kp{k}"], hp[f"w1_{k}"], hp[f"w2_{k}"], act=lb.ACTS[w.act]) for k in range(1, C + 1)]
         houts = [torch.empty_like(t["q0"]).pin_memory() for _ in range(C)]
-        arena = torch.empty(lb.lisa_host_arena_bytes(hp["q0"], hp["k0"], hlinks, hp[f"v{C}"], houts[-1]), dtype=torch.uint8, device="cuda")
         nbytes = lambda x: x.numel() * x.element_size()
-        h2d = sum(nbytes(hp["q0"]) + nbytes(hp["k0"]) + nbytes(hp[f"v{c}"]) +
-                  sum(nbytes(hp[f"qp{k}"]) + nbytes(hp[f"kp{k}"]) + nbytes(hp[f"w1_{k}"]) + nbytes(hp[f"w2_{k}"]) for k in range(1, c + 1))
-                  for c in range(1, C + 1))
-        d2h = sum(nbytes(o) for o in houts)
+        per_link = lambda k: nbytes(hp[f"qp{k}"]) + nbytes(hp[f"kp{k}"]) + nbytes(hp[f"w1_{k}"]) + nbytes(hp[f"w2_{k}"])
+        if carried:
+            scores = torch.empty(lb.lisa_prefill_scores_bytes(w.B, w.N, w.Hq), dtype=torch.uint8, device="cuda")
+            arena = torch.empty(lb.lisa_carry_host_arena_bytes(hp["q0"], hp["k0"], hlinks[0], hp["v1"], houts[0], scores, first=True),
+                                dtype=torch.uint8, device="cuda")
+            h2d = nbytes(hp["q0"]) + nbytes(hp["k0"]) + sum(nbytes(hp[f"v{c}"]) + per_link(c) for c in range(1, C + 1))
 
-        def e2e_step():
-            for c in range(1, C + 1):
-                lb.lisa_attn_shared_prefill_host(hp["q0"], hp["k0"], hlinks[:c], hp[f"v{c}"], houts[c - 1], arena)
-            return []
+            def e2e_step():
+                for c in range(1, C + 1):
+                    lb.lisa_attn_shared_prefill_carry_host(hp["q0"], hp["k0"], hlinks[c - 1], hp[f"v{c}"], houts[c - 1], scores, arena,
+                                                           first=c == 1, keep=c < C)
+                return []
+            e2e_call = ("lisa_attn_shared_prefill_carry_host per layer: pinned host tensors in (the anchor's q0, k0 with the first layer "
+                        "only), pinned host output back, every step; the carried scores stay on the device")
+        else:
+            scores = None
+            arena = torch.empty(lb.lisa_host_arena_bytes(hp["q0"], hp["k0"], hlinks, hp[f"v{C}"], houts[-1]), dtype=torch.uint8, device="cuda")
+            h2d = sum(nbytes(hp["q0"]) + nbytes(hp["k0"]) + nbytes(hp[f"v{c}"]) + sum(per_link(k) for k in range(1, c + 1))
+                      for c in range(1, C + 1))
+
+            def e2e_step():
+                for c in range(1, C + 1):
+                    lb.lisa_attn_shared_prefill_host(hp["q0"], hp["k0"], hlinks[:c], hp[f"v{c}"], houts[c - 1], arena)
+                return []
+            e2e_call = "lisa_attn_shared_prefill_host per layer: pinned host tensors in, pinned host output back, every step"
+        d2h = sum(nbytes(o) for o in houts)
 
         for _ in range(3):
             e2e_step()
@@ -387,9 +403,8 @@ def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
         e2e_total, _, _ = time_steps(e2e_step, n_e2e, flush, barrier)
         e2e_ms = max_over_ranks(e2e_total) / n_e2e
         res["e2e"] = {"value": world * tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms, "steps": n_e2e,
-                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                      "call": "lisa_attn_shared_prefill_host per layer: pinned host tensors in, pinned host output back, every step"}
-        del arena, hp, houts
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "call": e2e_call}
+        del arena, hp, houts, scores
     del d, caches, ws
     return res
 

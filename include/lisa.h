@@ -227,6 +227,12 @@ typedef struct lisa_shared_prefill_carry_args {
 } lisa_shared_prefill_carry_args;
 size_t lisa_prefill_scores_bytes(int32_t B, int32_t N, int32_t Hq);
 lisa_status_t lisa_attn_shared_prefill_carry(const lisa_shared_prefill_carry_args* args, lisa_stream_t stream);
+/* The same call with the layer's tensors, weights and `o` in HOST memory, like lisa_attn_shared_prefill_host (dense layout,
+ * strides ignored, workspace fields ignored); `scores` stays DEVICE memory.  q0 and k0 are staged only when `first`.
+ * device_arena: at least lisa_carry_host_arena_bytes() bytes, 256-byte aligned.  Synchronises the stream before returning. */
+lisa_status_t lisa_attn_shared_prefill_carry_host(const lisa_shared_prefill_carry_args* host_args, void* device_arena,
+                                                  size_t arena_bytes, lisa_stream_t stream);
+lisa_status_t lisa_carry_host_arena_bytes(const lisa_shared_prefill_carry_args* host_args, size_t* bytes);
 
 /* The same call with every tensor, weight and `o` in HOST memory (dense [B,N,H,x] layout, strides
  * ignored; workspace fields ignored).  Inputs are staged into `device_arena` (device memory of at least

@@ -27,7 +27,8 @@ ACTS = {"none": ACT_NONE, "relu": ACT_RELU, "silu": ACT_SILU}
 
 # include/lisa.h (the method's entry points and host helpers) and include/lisa_debug.h (test and measurement hooks)
 EXPORTS = ["lisa_attn_anchor", "lisa_attn_shared_prefill", "lisa_attn_shared_prefill_chain", "lisa_attn_shared_prefill_host",
-           "lisa_attn_shared_prefill_carry", "lisa_prefill_scores_bytes",
+           "lisa_attn_shared_prefill_carry", "lisa_prefill_scores_bytes", "lisa_attn_shared_prefill_carry_host",
+           "lisa_carry_host_arena_bytes",
            "lisa_host_arena_bytes", "lisa_attn_shared_decode", "lisa_attn_shared_decode_static", "lisa_kvcache_append",
            "lisa_kvcache_append_layer", "lisa_project", "lisa_kvcache_bytes", "lisa_kvcache_total_bytes", "lisa_kvcache_init",
            "lisa_workspace_bytes", "lisa_check", "lisa_last_cuda_error", "lisa_status_string", "lisa_version",
@@ -130,6 +131,8 @@ def load():
         lib.lisa_attn_shared_prefill_chain.argtypes = [C.POINTER(SharedPrefillChainArgs), C.c_void_p]
         lib.lisa_attn_shared_prefill_chain.restype = C.c_int
         lib.lisa_attn_shared_prefill_carry.argtypes = [C.POINTER(SharedPrefillCarryArgs), C.c_void_p]
+        lib.lisa_attn_shared_prefill_carry_host.argtypes = [C.POINTER(SharedPrefillCarryArgs), C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.lisa_carry_host_arena_bytes.argtypes = [C.POINTER(SharedPrefillCarryArgs), C.POINTER(C.c_size_t)]
         lib.lisa_prefill_scores_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
         lib.lisa_prefill_scores_bytes.restype = C.c_size_t
         lib.lisa_attn_shared_prefill_host.argtypes = [C.POINTER(SharedPrefillArgs), C.c_void_p, C.c_size_t, C.c_void_p]
@@ -466,6 +469,22 @@ def lisa_attn_shared_prefill_host(q0, k0, links: Sequence[Link], v, out, arena: 
     a, keep = _prefill_args(q0, k0, links, v, out)
     _check(load().lisa_attn_shared_prefill_host(C.byref(a), arena.data_ptr(), arena.numel() * arena.element_size(),
                                                 _stream()), "lisa_attn_shared_prefill_host")
+    return out
+
+
+def lisa_carry_host_arena_bytes(q0, k0, link: Link, v, out, scores, *, first: bool) -> int:
+    c, keepalive = _carry_args(q0 if first else None, k0 if first else None, link, v, out, scores, first, True)
+    n = C.c_size_t()
+    _check(load().lisa_carry_host_arena_bytes(C.byref(c), C.byref(n)), "lisa_carry_host_arena_bytes")
+    return n.value
+
+
+def lisa_attn_shared_prefill_carry_host(q0, k0, link: Link, v, out, scores: torch.Tensor, arena: torch.Tensor, *, first: bool,
+                                        keep: bool) -> torch.Tensor:
+    """lisa_attn_shared_prefill_carry with the layer's tensors in (pinned) HOST memory; `scores` and `arena` are device memory."""
+    c, keepalive = _carry_args(q0 if first else None, k0 if first else None, link, v, out, scores, first, keep)
+    _check(load().lisa_attn_shared_prefill_carry_host(C.byref(c), arena.data_ptr(), arena.numel() * arena.element_size(), _stream()),
+           "lisa_attn_shared_prefill_carry_host")
     return out
 
 

@@ -509,8 +509,9 @@ struct Arena {
 // dev receives device-side copies of the descriptors; h2d lists (dst, src, bytes) to copy.
 struct Copy { void* dst; const void* src; size_t bytes; };
 
+// anchor == false: q0 and k0 are not read by the call (a carried layer past the first): nothing is staged for them.
 size_t plan_host_call(const lisa_shared_prefill_args& h, char* base, lisa_shared_prefill_args* dev, lisa_link* dlinks,
-                      Copy* copies, int* n_copies, size_t* o_bytes) {
+                      Copy* copies, int* n_copies, size_t* o_bytes, bool anchor = true) {
     Arena ar{base, 0};
     int nc = 0;
     auto dense = [&](const lisa_tensor& src, int H, int x, lisa_tensor* dst, bool copy_in) {
@@ -522,8 +523,10 @@ size_t plan_host_call(const lisa_shared_prefill_args& h, char* base, lisa_shared
         }
         return bytes;
     };
-    dense(h.q0, h.Hq, h.d, dev ? &dev->q0 : nullptr, true);
-    dense(h.k0, h.Hkv, h.d, dev ? &dev->k0 : nullptr, true);
+    if (anchor) {
+        dense(h.q0, h.Hq, h.d, dev ? &dev->q0 : nullptr, true);
+        dense(h.k0, h.Hkv, h.d, dev ? &dev->k0 : nullptr, true);
+    }
     dense(h.v, h.Hkv, h.d, dev ? &dev->v : nullptr, true);
     const size_t ob = dense(h.o, h.Hq, h.d, dev ? &dev->o : nullptr, false);
     if (o_bytes) *o_bytes = ob;
@@ -623,6 +626,70 @@ lisa_status_t lisa_attn_shared_prefill_host(const lisa_shared_prefill_args* host
             return cuda_fail(e);
     if ((st = lisa_attn_shared_prefill(&dev, stream)) != LISA_OK) return st;
     if ((e = cudaMemcpyAsync(host_args->o.ptr, dev.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
+    return LISA_OK;
+}
+
+
+// ---- carried scores, tensors in host memory ----
+namespace {
+// The device-side form of a carried host call laid out in the arena (base == nullptr: sizes only), validated, with its workspace.
+lisa_status_t plan_carry_host(const lisa_shared_prefill_carry_args& h, char* base, lisa_shared_prefill_carry_args* dev, lisa_link* dlink,
+                              Copy* copies, int* nc, size_t* o_bytes, size_t* total) {
+    if (h.struct_size != sizeof(lisa_shared_prefill_carry_args)) return LISA_ERR_INVALID_ARG;
+    lisa_shared_prefill_args hl = h.layer;
+    if (hl.struct_size != sizeof(lisa_shared_prefill_args) || hl.chain_len != 1 || !hl.links) return LISA_ERR_INVALID_ARG;
+    if (!h.first) { hl.q0 = hl.o; hl.k0 = hl.v; }   // not read: descriptors of the right shape for the common checks
+    lisa_status_t st = validate_host_args(&hl);
+    if (st != LISA_OK) return st;
+    *dev = h;
+    char* lay = base ? base : reinterpret_cast<char*>(uintptr_t(1) << 20);   // strides and alignment are all the size query needs
+    const size_t used = plan_host_call(hl, lay, &dev->layer, dlink, copies, nc, o_bytes, h.first != 0);
+    dev->layer.links = dlink;
+    if (!h.first) { dev->layer.q0 = lisa_tensor{}; dev->layer.k0 = lisa_tensor{}; }
+    size_t ws = 0;
+    if ((st = lisa_workspace_bytes(LISA_OP_SHARED_PREFILL_CARRY, dev, &ws)) != LISA_OK) return st;
+    dev->layer.workspace = ws ? lay + used : nullptr;
+    dev->layer.workspace_bytes = ws;
+    *total = used + ((ws + 255) & ~(size_t)255);
+    return LISA_OK;
+}
+}  // namespace
+
+lisa_status_t lisa_carry_host_arena_bytes(const lisa_shared_prefill_carry_args* host_args, size_t* bytes) {
+    if (!host_args || !bytes) return LISA_ERR_INVALID_ARG;
+    lisa_shared_prefill_carry_args dev;
+    lisa_link dlink[1];
+    Copy copies[3 + 6];
+    int nc = 0;
+    size_t ob = 0;
+    return plan_carry_host(*host_args, nullptr, &dev, dlink, copies, &nc, &ob, bytes);
+}
+
+lisa_status_t lisa_attn_shared_prefill_carry_host(const lisa_shared_prefill_carry_args* host_args, void* device_arena, size_t arena_bytes,
+                                                  lisa_stream_t stream) {
+    if (!host_args) return LISA_ERR_INVALID_ARG;
+    if (!device_arena || (reinterpret_cast<uintptr_t>(device_arena) & 255u)) return LISA_ERR_WORKSPACE;
+    lisa_shared_prefill_carry_args dev;
+    lisa_link dlink[1];
+    Copy copies[3 + 6];
+    int nc = 0;
+    size_t o_bytes = 0, need = 0;
+    lisa_status_t st = plan_carry_host(*host_args, static_cast<char*>(device_arena), &dev, dlink, copies, &nc, &o_bytes, &need);
+    if (st != LISA_OK) return st;
+    if (arena_bytes < need) return LISA_ERR_WORKSPACE;
+    // everything that can refuse the call is checked before the first copy is enqueued
+    lisa_shared_prefill_args checked;
+    if ((st = carried_layer(dev, &checked)) != LISA_OK) return st;
+    if (!dev.scores || (reinterpret_cast<uintptr_t>(dev.scores) & 255u) || dev.scores_bytes < tc_carry_bytes(checked.B, checked.N, checked.Hq))
+        return LISA_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    for (int i = 0; i < nc; ++i)
+        if ((e = cudaMemcpyAsync(copies[i].dst, copies[i].src, copies[i].bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+            return cuda_fail(e);
+    if ((st = lisa_attn_shared_prefill_carry(&dev, stream)) != LISA_OK) return st;
+    if ((e = cudaMemcpyAsync(host_args->layer.o.ptr, dev.layer.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
     return LISA_OK;
 }

@@ -272,3 +272,27 @@ def test_carried_scores_rejects_bad_arguments():
         lb.lisa_attn_shared_prefill_carry(q0, k0, dc[0], v, scores, first=True, keep=True)
     assert ei.value.status == lb.ERR_UNSUPPORTED
     assert lb.lisa_check() == lb.OK
+
+
+def test_carried_scores_from_host_memory():
+    """lisa_attn_shared_prefill_carry_host: the layer's tensors come from host memory and its output goes back there; the scores
+    stay on the device from layer to layer.  Same results as the device-memory calls."""
+    B, N, Hq, Hkv, chain = 1, 300, 32, 8, 3
+    t = link_inputs(B, N, Hq, Hkv, chain, 64, "relu", 2, 21, 37, True)
+    dl, ol = make_links(t, chain, "relu", lb.INTEGRATE_ADD, 2, True)
+    scores = torch.empty(lb.lisa_prefill_scores_bytes(B, N, Hq), dtype=torch.uint8, device="cuda")
+    scores2 = torch.empty_like(scores)
+    for k in range(chain):
+        hl = lb.Link(t[f"qp{k + 1}"], t[f"kp{k + 1}"], t[f"w1_{k + 1}"], t[f"w2_{k + 1}"], t[f"b1_{k + 1}"], t[f"b2_{k + 1}"], act=lb.ACT_RELU)
+        out_h = torch.empty_like(t["q0"])
+        need = lb.lisa_carry_host_arena_bytes(t["q0"], t["k0"], hl, t[f"v{k + 1}"], out_h, scores2, first=k == 0)
+        arena = torch.empty(need, dtype=torch.uint8, device="cuda")
+        lb.lisa_attn_shared_prefill_carry_host(t["q0"], t["k0"], hl, t[f"v{k + 1}"], out_h, scores2, arena, first=k == 0, keep=k + 1 < chain)
+        got = lb.lisa_attn_shared_prefill_carry(dev(t["q0"]), dev(t["k0"]), dl[k], dev(t[f"v{k + 1}"]), scores, first=k == 0, keep=k + 1 < chain)
+        torch.cuda.synchronize()
+        assert torch.equal(out_h, got.cpu())
+        ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1])
+        assert_close(out_h.float().numpy(), ref, "bf16", "carried scores from host memory, layer %d" % (k + 1))
+        if k > 0:   # past the first layer the arena holds no copy of q0, k0
+            assert need < lb.lisa_carry_host_arena_bytes(t["q0"], t["k0"], hl, t[f"v{k + 1}"], out_h, scores2, first=True)
+    assert lb.lisa_check() == lb.OK
