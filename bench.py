@@ -12,6 +12,7 @@ under "cfg2", the LLaMA2-13B-shaped decode step and the library's own standard-a
 Under torchrun (N > 1) every rank runs the same step on its own batch (weak scaling, no data exchange).
 """
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -38,6 +39,11 @@ CFG2_POSITIONS_HEADS = 2098176 * 32
 PREFILL_TRAFFIC_PER_PH = {"emit_scores": (39902464 + 85123840) / CFG2_POSITIONS_HEADS,
                           "align": (142643200 + 83262464) / CFG2_POSITIONS_HEADS,
                           "attention": (186194944 + 5540864) / CFG2_POSITIONS_HEADS}
+# The kernels of a carried layer, captured on the first wave (query rows 0..2815) of the headline chain at B 1, N 4096:
+# the one-link aligner in place on the scores buffer and the attention kernel that writes its logits back.
+CARRY_POSITIONS_HEADS = 2816 * 2817 // 2 * 32
+CARRY_TRAFFIC_PER_PH = {"align": 4.370805e12 * 107.872e-6 / CARRY_POSITIONS_HEADS,
+                        "attention_keep": 3.943844e12 * 133.088e-6 / CARRY_POSITIONS_HEADS}
 DECODE_TRAFFIC_PER_SEQ = (395952128 + 4544512) / 8  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
 PROJECT_TRAFFIC = 220900096 + 163201024             # projection kernel at the benchmark's own size
 
@@ -197,13 +203,15 @@ def mark():
     return ev
 
 
-def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
+def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e, shape=None):
     """The prefill step of workload `name`: per shared layer of the chain, the layer's attention call + lisa_kvcache_append.
     A chain of several layers runs with the scores carried from layer to layer (lisa_attn_shared_prefill_carry: Sec. 5.1's
     A_{n-1} from the layer before); the same layers recomputed from the anchor per layer (lisa_attn_shared_prefill at depth
     1..C) and in one fused call (lisa_attn_shared_prefill_chain) are timed beside it.  A single layer has nothing to carry."""
     flush, barrier, max_over_ranks, peaks, world = env
     w = synth.WORKLOADS[name]
+    if shape:   # profiling aid: the same layers at another batch and prompt length
+        w = dataclasses.replace(w, B=shape[0], N=shape[1])
     C = w.chain
     carried = C > 1
     t = synth.prefill_inputs(w, seed=rank)
@@ -278,7 +286,13 @@ def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
                       "attention": P * (2 * w.Hq * w.r + 2 * w.Hq * w.d)}
             kbytes = {"pack": c * qk_lr * (w.r + 64), "emit_scores": qk_lr * w.d + c * ph * 2, "align": (c + 1) * ph * 2,
                       "attention": ph * 2 + qk_lr * 64 + w.B * w.N * (w.Hkv + w.Hq) * w.d * 2}
-        ktraffic = PREFILL_TRAFFIC_PER_PH if (c == 1 and not carried) else {}   # the captures are of the recomputing layer at depth 1
+        if not carried:
+            ktraffic = PREFILL_TRAFFIC_PER_PH if c == 1 else {}   # the captures are of the recomputing layer at depth 1
+        else:
+            ktraffic = {"align": CARRY_TRAFFIC_PER_PH["align"],
+                        "attention": CARRY_TRAFFIC_PER_PH["attention_keep"] if c < C else PREFILL_TRAFFIC_PER_PH["attention"]}
+            if c == 1:
+                ktraffic["emit_scores"] = PREFILL_TRAFFIC_PER_PH["emit_scores"]
         kernels = {}
         for i, n in enumerate(names):
             sec = phase_ms[c - 1][i] * 1e-3
@@ -292,10 +306,11 @@ def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
         fl = sum(kflops.values())
         tf = fl / (call_ms[c - 1] * 1e-3) / 1e12
         traffic = sum(k["traffic"] for k in kernels.values() if k["traffic"]) if ktraffic else None
+        alg_bytes = prefill_algorithmic_bytes(w, 1 if carried else c) - (0 if (not carried or c == 1) else w.B * w.N * 2 * (w.Hq + w.Hkv) * w.d)
         per_layer.append({"chain_depth": c, "ms": call_ms[c - 1], "flops": fl, "flops_per_position": fl // P,
                           "achieved": tf, "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
-                          "algorithmic_bytes": prefill_algorithmic_bytes(w, 1 if carried else c),
-                          "traffic_over_algorithmic": traffic / prefill_algorithmic_bytes(w, c) if traffic else None,
+                          "algorithmic_bytes": alg_bytes,   # Q0, K0 (unless carried past the first layer), Q', K', V, O
+                          "traffic_over_algorithmic": traffic / alg_bytes if traffic else None,
                           "kernels": kernels})
 
     flops = sum(pl["flops"] for pl in per_layer)                        # executed
@@ -317,10 +332,13 @@ def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
                     if carried else "causal positions B*N*(N+1)/2 x sum over c of (2hd + c(2hr + 4hm) + 2hd)"),
         "frac_by_recompute_formula": formula_flops / (calls_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
         "recompute_formula": "causal positions x sum over c = 1..C of (2hd + c(2hr + 4hm) + 2hd): what layers recomputed from the anchor execute",
-        "traffic": per_layer[0]["kernels"][dom_name]["traffic"],
-        "traffic_note": ("none: the kernels' DRAM counters were captured on the recomputing layer at depth 1 (see cfg2)" if carried else
+        "traffic": (sum(pl["kernels"][dom_name]["traffic"] or 0 for pl in per_layer) or None) if carried else per_layer[0]["kernels"][dom_name]["traffic"],
+        "traffic_note": ("ncu DRAM bytes of the dominant kernel over the launches of a step (all layers), captures of the carried layer's "
+                         "kernels at B 1, N 4096 scaled by causal positions" if carried else
                          "ncu DRAM bytes of the dominant kernel at chain depth 1, the cfg2 capture scaled by causal positions"),
-        "traffic_over_algorithmic": per_layer[0]["traffic_over_algorithmic"],
+        "traffic_over_algorithmic": (sum(pl["traffic_over_algorithmic"] * pl["algorithmic_bytes"] for pl in per_layer) /
+                                     sum(pl["algorithmic_bytes"] for pl in per_layer)) if all(pl["traffic_over_algorithmic"] for pl in per_layer)
+                                    else per_layer[0]["traffic_over_algorithmic"],
         "dominant_kernel": {"name": dom_name, "ms_per_step": dom_ms, "bound": "hbm" if dom_hbm else "tensor",
                             "achieved": dom_bytes / (dom_ms * 1e-3) / 1e9 if dom_hbm else dom_flops / (dom_ms * 1e-3) / 1e12,
                             "unit": "GB/s" if dom_hbm else "TFLOP/s",
@@ -328,7 +346,7 @@ def bench_prefill(lb, name, rank, args, env, with_chain, with_e2e):
                             "tensor_frac": dom_flops / (dom_ms * 1e-3) / 1e12 / peaks["bf16_tflops"]},
         "per_layer": per_layer}
 
-    res = {"workload": w.name, "ms_per_step": ms_per_step, "value": world * tokens / (ms_per_step * 1e-3), "launches": launches,
+    res = {"workload": w.name, "w": w, "ms_per_step": ms_per_step, "value": world * tokens / (ms_per_step * 1e-3), "launches": launches,
            "roofline": roofline, "tokens": tokens, "outs": outs, "inputs": t, "carried": carried,
            "scores_buffer_bytes": scores.numel() if carried else 0}
 
@@ -452,6 +470,7 @@ def main():
                     help="profiling aid: run just that section (prefill: the headline step; cfg2: the LLaMA2-7B-shaped layer; "
                          "neither runs the end-to-end, decode, stack or CPU legs)")
     ap.add_argument("--decode-batch", type=int, default=0, help="profiling aid: decode batch size (default: the workload's 64)")
+    ap.add_argument("--prefill-shape", default=None, help="profiling aid, with --only prefill: 'B,N' instead of the headline workload's 4,8192")
     args = ap.parse_args()
     if args.only is None:
         args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -488,7 +507,8 @@ def main():
     # ---------------- prefill: the headline step, and the LLaMA2-7B-shaped layer beside it ----------------
     head = second = None
     if args.only in (None, "prefill"):
-        head = bench_prefill(lb, HEADLINE, rank, args, env, with_chain=True, with_e2e=args.only is None)
+        shape = tuple(int(x) for x in args.prefill_shape.split(",")) if (args.prefill_shape and args.only == "prefill") else None
+        head = bench_prefill(lb, HEADLINE, rank, args, env, with_chain=True, with_e2e=args.only is None, shape=shape)
         launches += head["launches"]
     if args.only in (None, "cfg2"):
         second = bench_prefill(lb, SECOND, rank, args, env, with_chain=False, with_e2e=args.only is None)
@@ -654,8 +674,7 @@ def main():
             line.update({"value": project["value"], "ms_per_step": project["ms"], "config": {"workload": "projection " + project["outputs"]},
                          "roofline": project["roofline"]})
         if main_res is not None:
-            w = synth.WORKLOADS[main_res["workload"]]
-            cfg = workload_config(w)
+            cfg = workload_config(main_res["w"])
             line.update({"value": main_res["value"], "ms_per_step": main_res["ms_per_step"], "config": cfg,
                          "e2e": main_res.get("e2e"), "roofline": main_res["roofline"], "recompute": main_res.get("recompute"),
                          "chain_call": main_res.get("chain_call")})
