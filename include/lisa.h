@@ -215,8 +215,8 @@ lisa_status_t lisa_attn_shared_prefill_chain(const lisa_shared_prefill_chain_arg
  *           0: last layer of its chain, the contents of `scores` are unspecified afterwards
  * o is exactly what lisa_attn_shared_prefill returns for the whole chain up to this layer, up to the rounding of the
  * carried scores to fp16 (which the recomputing path applies between links as well).
- * Tensor-core shapes only (d = 128, bf16, 32 or 40 heads, adding Integrate or no FFN, r <= 32): others
- * LISA_ERR_UNSUPPORTED.  Workspace: lisa_workspace_bytes(LISA_OP_SHARED_PREFILL_CARRY, args, &n).  `scores` must be
+ * Tensor-core shapes only (d = 128, bf16, r <= 32; 32 heads with any Integrate, 40 heads with the adding ones; hidden
+ * width up to 256): others LISA_ERR_UNSUPPORTED.  Workspace: lisa_workspace_bytes(LISA_OP_SHARED_PREFILL_CARRY, args, &n).  `scores` must be
  * 256-byte aligned.  On error nothing is launched. */
 typedef struct lisa_shared_prefill_carry_args {
     size_t struct_size;

@@ -119,6 +119,9 @@ struct TcAlignLinkArgs {
     const lisa_link* link;
     int dst_next, dst_scaled;
     int row0 = -1;  // first query row the planes hold (-1: qt_begin * 128)
+    // plane_d with a geometry of its own (0 / -1: the same as plane_x): carried scores as plane_x, a wave's plane as plane_d
+    int64_t d_plane_rows = 0, d_plane_cols = 0;
+    int d_row0 = -1;
 };
 bool tc_align_concat_supported(int Hq, const lisa_link* links, int chain);
 bool tc_align_link_supported(int Hq, const lisa_link* links, int chain);

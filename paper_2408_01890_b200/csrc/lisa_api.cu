@@ -213,7 +213,7 @@ lisa_status_t carried_layer(const lisa_shared_prefill_carry_args& a, lisa_shared
     if (!a.first) { p.q0 = p.o; p.k0 = p.v; }
     lisa_status_t st = validate_prefill(&p);
     if (st != LISA_OK) return st;
-    if (p.links[0].integrate == LISA_INTEGRATE_CONCAT || !tc_shared_prefill_supported(p)) return LISA_ERR_UNSUPPORTED;
+    if (!tc_shared_prefill_supported(p)) return LISA_ERR_UNSUPPORTED;
     *out = p;
     return LISA_OK;
 }

@@ -42,6 +42,8 @@ constexpr int kStages = 2;
 struct LinkParams {
     int B, N, row0, qt_begin, qt_count, units_per_batch;
     int64_t plane_cols;
+    int d_row0;                         // geometry of plane_d where it differs from plane_x's
+    int64_t d_plane_cols;
     __half *plane_x, *plane_d;          // plane_d == nullptr: no difference plane (ADD, top link)
     int dst_next, dst_scaled;           // where the next link's input / the attention kernel's plane go: -1 nowhere, 0 plane_x, 1 plane_d
     const void *w1, *b1, *w2, *b2;
@@ -114,6 +116,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) tc_align_link_kernel(const __grid
     // ---- this warp's contiguous range of pieces: (batch, query tile, row, 64-key block, half) ----
     const int pB = p.B, pN = p.N, p_row0 = p.row0, p_qt0 = p.qt_begin, p_qt1 = p.qt_begin + p.qt_count;
     const int p_ncb = (int)(p.plane_cols >> 6);
+    const int p_row0_d = p.d_row0, p_ncb_d = (int)(p.d_plane_cols >> 6);
     constexpr int PPU = UNIT / PP;
     const long long n_pieces = (long long)p.units_per_batch * pB * PPU;
     const long long n_warps = (long long)gridDim.x * (NTHREADS / 32);
@@ -151,10 +154,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) tc_align_link_kernel(const __grid
     // four lanes cover the 64 bytes [head][32 positions] of one head: a warp-wide access moves 8 heads
     constexpr int CPR = PP / 8, HPA = 32 / CPR, NACC = NH / HPA;
     const int l_head = lane / CPR, l_chunk = lane % CPR;
-    auto piece_off = [&](const Cursor& x) {
-        const int r = x.t * UNIT + x.row - p_row0;
+    auto piece_off = [&](const Cursor& x, int which) {   // which: 0 = plane_x's geometry, 1 = plane_d's
+        const int r = x.t * UNIT + x.row - (which ? p_row0_d : p_row0);
         const int col = x.sub * PP;
-        const int64_t blk = (int64_t)(r >> 7) * p_ncb + (x.jb * 2 + (col >> 6));
+        const int64_t blk = (int64_t)(r >> 7) * (which ? p_ncb_d : p_ncb) + (x.jb * 2 + (col >> 6));
         return ((blk * 128 + (r & 127)) * (pB * NH) + (x.b * NH + l_head)) * 64 + (col & 63) + l_chunk * 8;
     };
     auto scr_off = [&](int head, int chunk) { return (uint32_t)(head * (PP * 2) + ((chunk ^ ((head >> 1) & 3)) << 4)); };
@@ -163,10 +166,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) tc_align_link_kernel(const __grid
     __half* const gd = p.plane_d;
     const bool has_d = gd != nullptr;
     auto fetch = [&](const Cursor& x, int buf) {
-        const int64_t off = piece_off(x);
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
             if (k == 1 && !has_d) break;
+            const int64_t off = piece_off(x, k);
             const __half* src = k == 0 ? gx : gd;
 #pragma unroll
             for (int i = 0; i < NACC; ++i) {
@@ -298,10 +301,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) tc_align_link_kernel(const __grid
             }
         }
         __syncwarp();
-        const int64_t here_off = piece_off(here);
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
             if (dst_next != k && dst_scaled != k) continue;
+            const int64_t here_off = piece_off(here, k);
             __half* dst = k == 0 ? gx : gd;
 #pragma unroll
             for (int i = 0; i < NACC; ++i)
@@ -364,6 +367,10 @@ cudaError_t launch_tc_align_link(const TcAlignLinkArgs& a, cudaStream_t stream) 
     p.B = a.B; p.N = a.N; p.row0 = a.row0 >= 0 ? a.row0 : a.qt_begin * UNIT; p.qt_begin = a.qt_begin; p.qt_count = a.qt_count;
     if (p.row0 % UNIT != 0 || p.row0 > a.qt_begin * UNIT) return cudaErrorInvalidValue;
     p.plane_cols = a.plane_cols;
+    p.d_plane_cols = a.d_plane_cols > 0 ? a.d_plane_cols : a.plane_cols;
+    p.d_row0 = a.d_plane_cols > 0 ? (a.d_row0 >= 0 ? a.d_row0 : a.qt_begin * UNIT) : p.row0;
+    if (p.d_plane_cols % 64 != 0 || p.d_row0 % UNIT != 0 || p.d_row0 > a.qt_begin * UNIT || (a.d_plane_cols > 0 && a.d_plane_rows % 128 != 0))
+        return cudaErrorInvalidValue;
     for (int t = a.qt_begin; t < a.qt_begin + a.qt_count; ++t) p.units_per_batch += std::min(UNIT, a.N - t * UNIT) * (t + 1);
     p.plane_x = reinterpret_cast<__half*>(a.plane_x); p.plane_d = reinterpret_cast<__half*>(a.plane_d);
     p.dst_next = a.dst_next; p.dst_scaled = a.dst_scaled;

@@ -120,7 +120,8 @@ struct Layout {
     size_t total;
 };
 
-// carried: the scores live in the caller's buffer, the workspace holds only the packed Q', K'
+// carried: the scores live in the caller's buffer; the workspace holds the packed Q', K' and, for the concatenating
+// Integrate, the wave's plane of the link's difference
 Layout plan_layout(const lisa_shared_prefill_args& a, bool carried = false) {
     Layout l{};
     size_t off = 0;
@@ -131,14 +132,15 @@ Layout plan_layout(const lisa_shared_prefill_args& a, bool carried = false) {
     }
     const int n_qt = (a.N + kTile - 1) / kTile;
     Wave waves[1024];
-    const int nw = plan_waves(a.B, a.N, a.Hq, plane_count(a), waves, 1024);
+    const int nw = plan_waves(a.B, a.N, a.Hq, carried ? 1 : plane_count(a), waves, 1024);
     int max_cnt = 1;
     for (int i = 0; i < std::min(nw, 1024); ++i) max_cnt = std::max(max_cnt, waves[i].count);
     l.plane_rows = (int64_t)max_cnt * kTile;
     l.plane_cols = (int64_t)n_qt * kTile;
     l.sets = std::max(1, std::min(kWaveSets, nw));
-    for (int set = 0; set < l.sets && !carried; ++set)
-        for (int k = 0; k < plane_count(a); ++k) l.plane_off[set][k] = take((size_t)a.B * a.Hq * l.plane_rows * l.plane_cols * 2);
+    for (int set = 0; set < l.sets; ++set)
+        for (int k = 0; k < plane_count(a); ++k)
+            if (!carried || (concat_chain(a) && k == 1)) l.plane_off[set][k] = take((size_t)a.B * a.Hq * l.plane_rows * l.plane_cols * 2);
     l.total = off;
     return l;
 }
@@ -224,12 +226,10 @@ cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws
 cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, const lisa_tensor* vs, const lisa_tensor* os, void* ws,
                                            cudaStream_t s, const TcCarry* cy) {
     const bool all_layers = vs != nullptr;
-    if (cy && (all_layers || a.chain_len != 1 || concat_chain(a) || !cy->scores)) return cudaErrorInvalidValue;
-    Layout l = plan_layout(a, cy != nullptr);
-    if (cy) {
-        l.plane_rows = l.plane_cols = (int64_t)(a.N + kTile - 1) / kTile * kTile;
-        for (int set = 0; set < kWaveSets; ++set) l.plane_off[set][0] = 0;
-    }
+    if (cy && (all_layers || a.chain_len != 1 || !cy->scores)) return cudaErrorInvalidValue;
+    const Layout l = plan_layout(a, cy != nullptr);
+    // geometry of the plane that holds the running scores: the caller's buffer (whole prompt, rows from 0) or a wave's plane
+    const int64_t x_rows = cy ? (int64_t)(a.N + kTile - 1) / kTile * kTile : l.plane_rows, x_cols = cy ? x_rows : l.plane_cols;
     char* const plane_base = cy ? reinterpret_cast<char*>(cy->scores) : nullptr;
     const int row0 = cy ? 0 : -1;
     char* base = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(ws) + 1023) & ~(uintptr_t)1023);
@@ -272,7 +272,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
     };
     const bool concat = concat_chain(a);
     Wave waves[1024];
-    const int nw = plan_waves(a.B, a.N, a.Hq, plane_count(a), waves, 1024);
+    const int nw = plan_waves(a.B, a.N, a.Hq, cy ? 1 : plane_count(a), waves, 1024);
     // Several waves in flight (see kWaveSets): wave w runs on stream w % sets (0 = the caller's) with plane set w % sets.
     // All of it is forked from and joined back into the caller's stream inside this call, under the lock that keeps
     // another host thread's call from interleaving its event records with these waits.
@@ -292,10 +292,12 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         cudaStream_t st = set == 0 ? s : side->wave[set - 1];
         const size_t* po = l.plane_off[set];
         // 1. anchor scores and the differences of the links below the top one
-        TcFlashArgs f{a.B, a.N, a.Hq, a.Hkv, 128, a.q0, a.k0, a.v, a.o, 1.f / sqrtf((float)a.d), nullptr, l.plane_rows, l.plane_cols,
-                      wv.begin, wv.count};
-        f.plane_row0 = row0;
-        f.emit_plane = cy ? plane_base : base + po[0];
+        const TcFlashArgs fw{a.B, a.N, a.Hq, a.Hkv, 128, a.q0, a.k0, a.v, a.o, 1.f / sqrtf((float)a.d), nullptr, l.plane_rows, l.plane_cols,
+                             wv.begin, wv.count};                 // the wave's own planes
+        TcFlashArgs f = fw;                                       // the plane of the running scores
+        f.plane_rows = x_rows; f.plane_cols = x_cols; f.plane_row0 = row0;
+        char* const x_plane = cy ? plane_base : base + po[0];
+        f.emit_plane = x_plane;
         if (!cy || cy->first) {
             PhaseMark mark(1, st);
             if ((e = launch_tc_flash(f, st)) != cudaSuccess) return e;
@@ -303,7 +305,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         for (int k = 0; k + (concat ? 0 : 1) < c; ++k) {   // the concatenating form also needs the top link's difference as a plane
             if ((e = join_pack()) != cudaSuccess) return e;
             PhaseMark mark(1, st);
-            TcFlashArgs fd = f;
+            TcFlashArgs fd = fw;
             fd.kd = kPadRank;
             fd.qa = packed_view(base + l.qp_off[k], a.Hq, a.N);
             fd.ka = packed_view(base + l.kp_off[k], a.Hkv, a.N);
@@ -316,15 +318,16 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             // 2c. link by link: A_k = FFN_k([A_{k-1}; D_k]) over plane 0; log2(e) * A_k over D_k's plane where a layer's
             // attention consumes it (the top link's; every link's when all layers of the chain are computed)
             for (int k = 0; k < c; ++k) {
-                TcAlignLinkArgs ac{a.B, a.N, a.Hq, wv.begin, wv.count, l.plane_rows, l.plane_cols, base + po[0], base + po[k + 1],
-                                   &a.links[k], k + 1 < c ? 0 : -1, (all_layers || k == c - 1) ? 1 : -1};
+                // carried: the one link reads A_{n-1} from the caller's buffer and leaves A_n there when asked
+                TcAlignLinkArgs ac{a.B, a.N, a.Hq, wv.begin, wv.count, x_rows, x_cols, x_plane, base + po[k + 1],
+                                   &a.links[k], (k + 1 < c || (cy && cy->keep)) ? 0 : -1, (all_layers || k == c - 1) ? 1 : -1, row0,
+                                   l.plane_rows, l.plane_cols, -1};
                 PhaseMark mark(2, st);
                 if ((e = launch_tc_align_link(ac, st)) != cudaSuccess) return e;
             }
             // 3c. softmax and .V on the finished scores: the attention kernel's own difference is switched off (scale 0)
             for (int k = all_layers ? 0 : c - 1; k < c; ++k) {
-                TcFlashArgs fv = f;
-                fv.emit_plane = nullptr;
+                TcFlashArgs fv = fw;
                 fv.kd = kPadRank;
                 fv.qa = packed_view(base + l.qp_off[k], a.Hq, a.N);
                 fv.ka = packed_view(base + l.kp_off[k], a.Hkv, a.N);
@@ -343,7 +346,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             // plane k, writes A_k = FFN_k(A_{k-1}) + D_k over plane k + 1 (which held D_k) and, where a layer's attention
             // consumes it, log2(e) * FFN_k(A_{k-1}) over plane k.
             for (int k = 0; k < c; ++k) {
-                TcAlignLinkArgs al{a.B, a.N, a.Hq, wv.begin, wv.count, l.plane_rows, l.plane_cols, cy ? plane_base : base + po[k],
+                TcAlignLinkArgs al{a.B, a.N, a.Hq, wv.begin, wv.count, x_rows, x_cols, cy ? plane_base : base + po[k],
                                    k + 1 < c ? base + po[k + 1] : nullptr, &a.links[k], k + 1 < c ? 1 : -1,
                                    (all_layers || k == c - 1) ? 0 : -1, row0};
                 PhaseMark mark(2, st);
@@ -353,7 +356,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         // 2. the FFN chain over the head axis, in place
         TcAlignArgs al{};
         al.B = a.B; al.N = a.N; al.chain = c; al.qt_begin = wv.begin; al.qt_count = wv.count;
-        al.plane_rows = l.plane_rows; al.plane_cols = l.plane_cols;
+        al.plane_rows = x_rows; al.plane_cols = x_cols;
         for (int k = 0; k < c; ++k) al.planes[k] = cy ? plane_base : base + po[k];
         al.links = a.links;
         al.row0 = row0;

@@ -266,10 +266,10 @@ def test_carried_scores_rejects_bad_arguments():
         lb.lisa_attn_shared_prefill_carry(q0, k0, dl[0], v, small, first=True, keep=True)
     assert ei.value.status == lb.ERR_INVALID_ARG
     scores = torch.empty(need, dtype=torch.uint8, device="cuda")
-    cat = concat_inputs(B, N, Hkv, 1, 64, "relu", 2, 21, 33, False)
-    dc, _ = make_links(cat, 1, "relu", lb.INTEGRATE_CONCAT, 2, False)
-    with pytest.raises(lb.LisaError) as ei:   # the concatenating Integrate has no carried form
-        lb.lisa_attn_shared_prefill_carry(q0, k0, dc[0], v, scores, first=True, keep=True)
+    wide = link_inputs(B, N, Hq, Hkv, 1, 320, "relu", 2, 21, 33, False)
+    dw, _ = make_links(wide, 1, "relu")
+    with pytest.raises(lb.LisaError) as ei:   # hidden width beyond the tensor-core aligners: no carried form
+        lb.lisa_attn_shared_prefill_carry(q0, k0, dw[0], v, scores, first=True, keep=True)
     assert ei.value.status == lb.ERR_UNSUPPORTED
     assert lb.lisa_check() == lb.OK
 
@@ -296,3 +296,26 @@ def test_carried_scores_from_host_memory():
         if k > 0:   # past the first layer the arena holds no copy of q0, k0
             assert need < lb.lisa_carry_host_arena_bytes(t["q0"], t["k0"], hl, t[f"v{k + 1}"], out_h, scores2, first=True)
     assert lb.lisa_check() == lb.OK
+
+
+@pytest.mark.parametrize("B,N,Hkv,chain,m,act,layers,r,bias", [
+    (1, 300, 32, 3, 256, "relu", 2, 20, False),    # a run of three of the paper's complete layers (64 x 256, 256 x 32, ReLU, r = 20)
+    (2, 200, 8, 4, 64, "silu", 2, 21, True),
+    (1, 260, 8, 2, 32, "none", 1, 32, True)])      # one linear 64 x 32 layer
+def test_carried_scores_concatenating_integrate(B, N, Hkv, chain, m, act, layers, r, bias):
+    """The concatenating Integrate with carried scores: the aligner reads A_{n-1} from the scores buffer and the layer's
+    difference from a plane of the wave, leaves A_n in the buffer, and hands the attention kernel its copy through the
+    difference's plane (launches: pack, [A_0,] the difference, align, attention)."""
+    t = concat_inputs(B, N, Hkv, chain, m, act, layers, r, 41, bias)
+    dl, ol = make_links(t, chain, act, lb.INTEGRATE_CONCAT, layers, bias)
+    scores = torch.full((lb.lisa_prefill_scores_bytes(B, N, 32),), 0xFF, dtype=torch.uint8, device="cuda")
+    q0, k0 = dev(t["q0"]), dev(t["k0"])
+    for k in range(chain):
+        n0 = lb.lisa_kernel_launches()
+        got = lb.lisa_attn_shared_prefill_carry(q0 if k == 0 else None, k0 if k == 0 else None, dl[k], dev(t[f"v{k + 1}"]), scores,
+                                                first=k == 0, keep=k + 1 < chain, out=torch.empty_like(q0))
+        torch.cuda.synchronize()
+        assert lb.lisa_kernel_launches() - n0 == (5 if k == 0 else 4)
+        assert lb.lisa_check() == lb.OK
+        ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1])
+        assert_close(got.float().cpu().numpy(), ref, "bf16", "carried scores, concatenating integrate, layer %d of %d" % (k + 1, chain))
