@@ -162,8 +162,9 @@ lisa_status_t lisa_attn_anchor(const lisa_anchor_args* args, lisa_stream_t strea
 
 /* ------------------------------------------------------------------------------------------------
  * lisa_attn_shared_prefill -- a shared layer at chain depth c = chain_len over a whole prompt
- * (Sec. 5.1, Eq. 3-4, then Eq. 1).  The N x N x Hq scores are never stored: they are recomputed tile by
- * tile from the anchor's q0 [B,N,Hq,d], k0 [B,N,Hkv,d] and links[0..c-1] (links[c-1] is this layer's own,
+ * (Sec. 5.1, Eq. 3-4, then Eq. 1).  The N x N x Hq scores of the whole prompt are not kept: they are recomputed
+ * tile by tile (the tensor-core kernels hold a strip of query rows of them in the workspace at a time)
+ * from the anchor's q0 [B,N,Hq,d], k0 [B,N,Hkv,d] and links[0..c-1] (links[c-1] is this layer's own,
  * the earlier ones belong to the shared layers between the anchor and this one), masked causally AFTER
  * the last link, soft-maxed and multiplied by this layer's v [B,N,Hkv,d].  o [B,N,Hq,d].
  * chain_len == 0 degenerates to lisa_attn_anchor on (q0,k0,v). */

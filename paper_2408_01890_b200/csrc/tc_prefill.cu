@@ -6,7 +6,8 @@
 //   1. tc_flash (emit)   A_0 = Q0.K0^T/sqrt(d) per head, and D_k = Q'_k.K'_k^T/sqrt(r) for the links k < c
 //   2. tc_align          per position: the FFN chain over the head axis, Y written over A_0
 //   3. tc_flash (plane)  per head: logits = Y + Q'_c.K'_c^T/sqrt(r), causal softmax, .V
-// The N x N x Hq scores of the whole prompt are never stored; only the wave's strip of rows is.
+// The recomputing calls store only the wave's strip of rows of the N x N x Hq scores; the carried call keeps the whole
+// prompt's scores in the caller's buffer and works in place on it (see launch_tc_shared_prefill_chain).
 #include <algorithm>
 #include <cmath>
 #include <mutex>
