@@ -141,12 +141,19 @@ struct TcCarry {
     void* scores;
     bool first, keep;
 };
+// Output streamed to host memory while the layer runs (the host-memory entry points): after each wave's attention kernel
+// the wave's rows of o (dense [B,N,Hq,d] on both sides) are copied to host_o on a stream of the library's own, joined
+// into the caller's stream at the end.  done is set when the copies were enqueued; otherwise the caller copies o itself.
+struct TcHostOut {
+    void* host_o;
+    bool done;
+};
 size_t tc_carry_bytes(int B, int N, int Hq);
 size_t tc_shared_prefill_carry_workspace(const lisa_shared_prefill_args& a);
 cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws, cudaStream_t s);
 // vs/os: per-layer V and O of a chain of a.chain_len layers (nullptr: only the deepest layer, a.v / a.o)
 cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, const lisa_tensor* vs, const lisa_tensor* os, void* ws,
-                                           cudaStream_t s, const TcCarry* carry = nullptr);
+                                           cudaStream_t s, const TcCarry* carry = nullptr, TcHostOut* host_out = nullptr);
 cudaError_t prefill_phase_timing(bool enable);
 cudaError_t prefill_phase_times(float* ms4);
 

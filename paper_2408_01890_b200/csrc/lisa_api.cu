@@ -223,7 +223,12 @@ size_t lisa_prefill_scores_bytes(int32_t B, int32_t N, int32_t Hq) {
     return (B < 1 || N < 1 || Hq < 1) ? 0 : tc_carry_bytes(B, N, Hq);
 }
 
+static lisa_status_t shared_prefill_carry_impl(const lisa_shared_prefill_carry_args* a, lisa_stream_t stream, TcHostOut* ho);
 lisa_status_t lisa_attn_shared_prefill_carry(const lisa_shared_prefill_carry_args* a, lisa_stream_t stream) {
+    return shared_prefill_carry_impl(a, stream, nullptr);
+}
+// ho: the layer's output is also wanted in host memory (the host-memory entry points)
+static lisa_status_t shared_prefill_carry_impl(const lisa_shared_prefill_carry_args* a, lisa_stream_t stream, TcHostOut* ho) {
     if (!a || a->struct_size != sizeof(lisa_shared_prefill_carry_args)) return LISA_ERR_INVALID_ARG;
     lisa_shared_prefill_args p;
     lisa_status_t st = carried_layer(*a, &p);
@@ -231,7 +236,7 @@ lisa_status_t lisa_attn_shared_prefill_carry(const lisa_shared_prefill_carry_arg
     if (!a->scores || (reinterpret_cast<uintptr_t>(a->scores) & 255u) || a->scores_bytes < tc_carry_bytes(p.B, p.N, p.Hq)) return LISA_ERR_INVALID_ARG;
     if ((st = check_workspace(p.workspace, p.workspace_bytes, tc_shared_prefill_carry_workspace(p))) != LISA_OK) return st;
     const TcCarry cy{a->scores, a->first != 0, a->keep != 0};
-    cudaError_t e = launch_tc_shared_prefill_chain(p, nullptr, nullptr, p.workspace, static_cast<cudaStream_t>(stream), &cy);
+    cudaError_t e = launch_tc_shared_prefill_chain(p, nullptr, nullptr, p.workspace, static_cast<cudaStream_t>(stream), &cy, ho);
     return e == cudaSuccess ? LISA_OK : cuda_fail(e);
 }
 
@@ -284,7 +289,11 @@ lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes) 
     return LISA_ERR_INVALID_ARG;
 }
 
+static lisa_status_t shared_prefill_impl(const lisa_shared_prefill_args* a, lisa_stream_t stream, TcHostOut* ho);
 lisa_status_t lisa_attn_shared_prefill(const lisa_shared_prefill_args* a, lisa_stream_t stream) {
+    return shared_prefill_impl(a, stream, nullptr);
+}
+static lisa_status_t shared_prefill_impl(const lisa_shared_prefill_args* a, lisa_stream_t stream, TcHostOut* ho) {
     lisa_status_t st = validate_prefill(a);
     if (st != LISA_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -299,7 +308,7 @@ lisa_status_t lisa_attn_shared_prefill(const lisa_shared_prefill_args* a, lisa_s
     if (!g_force_general.load() && a->chain_len > 0 && tc_shared_prefill_supported(*a)) {
         const size_t need = tc_shared_prefill_workspace(*a);
         if ((st = check_workspace(a->workspace, a->workspace_bytes, need)) != LISA_OK) return st;
-        cudaError_t e = launch_tc_shared_prefill(*a, a->workspace, s);
+        cudaError_t e = launch_tc_shared_prefill_chain(*a, nullptr, nullptr, a->workspace, s, nullptr, ho);
         return e == cudaSuccess ? LISA_OK : cuda_fail(e);
     }
     cudaError_t e = launch_generic_prefill(*a, s);
@@ -624,8 +633,9 @@ lisa_status_t lisa_attn_shared_prefill_host(const lisa_shared_prefill_args* host
     for (int i = 0; i < nc; ++i)
         if ((e = cudaMemcpyAsync(copies[i].dst, copies[i].src, copies[i].bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
             return cuda_fail(e);
-    if ((st = lisa_attn_shared_prefill(&dev, stream)) != LISA_OK) return st;
-    if ((e = cudaMemcpyAsync(host_args->o.ptr, dev.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    TcHostOut ho{host_args->o.ptr, false};   // rows of o go back while later waves still compute, where the path supports it
+    if ((st = shared_prefill_impl(&dev, stream, &ho)) != LISA_OK) return st;
+    if (!ho.done && (e = cudaMemcpyAsync(host_args->o.ptr, dev.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
     return LISA_OK;
 }
@@ -688,8 +698,9 @@ lisa_status_t lisa_attn_shared_prefill_carry_host(const lisa_shared_prefill_carr
     for (int i = 0; i < nc; ++i)
         if ((e = cudaMemcpyAsync(copies[i].dst, copies[i].src, copies[i].bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
             return cuda_fail(e);
-    if ((st = lisa_attn_shared_prefill_carry(&dev, stream)) != LISA_OK) return st;
-    if ((e = cudaMemcpyAsync(host_args->layer.o.ptr, dev.layer.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    TcHostOut ho{host_args->layer.o.ptr, false};
+    if ((st = shared_prefill_carry_impl(&dev, stream, &ho)) != LISA_OK) return st;
+    if (!ho.done && (e = cudaMemcpyAsync(host_args->layer.o.ptr, dev.layer.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
     return LISA_OK;
 }

@@ -192,6 +192,8 @@ struct SideStream {
     cudaEvent_t fork = nullptr, join = nullptr;
     cudaStream_t wave[kWaveSets - 1] = {};         // waves beside the caller's stream
     cudaEvent_t wave_done[kWaveSets - 1] = {};
+    cudaStream_t copy_out = nullptr;               // device -> host copies of finished rows (host-memory entry points)
+    cudaEvent_t rows_done = nullptr, copy_done = nullptr;
     bool ok = false;
 };
 SideStream g_side[64];
@@ -209,6 +211,9 @@ SideStream* side_stream() {
             if (cudaStreamCreateWithFlags(&ss.wave[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
             if (cudaEventCreateWithFlags(&ss.wave_done[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
         }
+        if (cudaStreamCreateWithFlags(&ss.copy_out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&ss.rows_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&ss.copy_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         ss.ok = true;
     }
     return &ss;
@@ -225,8 +230,9 @@ cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws
 // With cy: one link, in place on the caller's carried scores (rows from 0, N rounded up to whole tiles both ways): no A_0
 // unless this is the first layer of its chain, no wave planes, and the attention kernel leaves A_n behind when asked.
 cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, const lisa_tensor* vs, const lisa_tensor* os, void* ws,
-                                           cudaStream_t s, const TcCarry* cy) {
+                                           cudaStream_t s, const TcCarry* cy, TcHostOut* ho) {
     const bool all_layers = vs != nullptr;
+    if (ho) ho->done = false;
     if (cy && (all_layers || a.chain_len != 1 || !cy->scores)) return cudaErrorInvalidValue;
     const Layout l = plan_layout(a, cy != nullptr);
     // geometry of the plane that holds the running scores: the caller's buffer (whole prompt, rows from 0) or a wave's plane
@@ -278,8 +284,23 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
     // All of it is forked from and joined back into the caller's stream inside this call, under the lock that keeps
     // another host thread's call from interleaving its event records with these waits.
     const int sets = (side && nw >= 2) ? l.sets : 1;
+    // rows of o leave for the host as soon as their wave's attention kernel is done (dense bf16 o only)
+    const bool stream_out = ho && ho->host_o && side && !all_layers && a.o.stride_h == a.d && a.o.stride_n == (int64_t)a.Hq * a.d;
+    auto copy_out = [&](const Wave& wv, cudaStream_t st) -> cudaError_t {
+        cudaError_t ce;
+        if ((ce = cudaEventRecord(side->rows_done, st)) != cudaSuccess) return ce;
+        if ((ce = cudaStreamWaitEvent(side->copy_out, side->rows_done, 0)) != cudaSuccess) return ce;
+        const int64_t r0 = (int64_t)wv.begin * kTile, r1 = std::min<int64_t>(a.N, (int64_t)(wv.begin + wv.count) * kTile);
+        for (int b = 0; b < a.B; ++b) {
+            const int64_t src = (b * a.o.stride_b + r0 * a.o.stride_n) * 2, dst = ((int64_t)b * a.N + r0) * a.Hq * a.d * 2;
+            if ((ce = cudaMemcpyAsync(static_cast<char*>(ho->host_o) + dst, static_cast<const char*>(a.o.ptr) + src,
+                                      (size_t)(r1 - r0) * a.Hq * a.d * 2, cudaMemcpyDeviceToHost, side->copy_out)) != cudaSuccess)
+                return ce;
+        }
+        return cudaSuccess;
+    };
     std::unique_lock<std::mutex> wave_lock(g_side_mutex, std::defer_lock);
-    if (sets > 1) {
+    if (sets > 1 || stream_out) {
         wave_lock.lock();
         if ((e = cudaStreamWaitEvent(s, side->join, 0)) != cudaSuccess) return e;   // every wave stream starts with the packed Q'/K' ready
         joined = true;
@@ -339,6 +360,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
                 PhaseMark mark(3, st);
                 if ((e = launch_tc_flash(fv, st)) != cudaSuccess) return e;
             }
+            if (stream_out && (e = copy_out(wv, st)) != cudaSuccess) return e;
             continue;
         }
         const bool per_link = !tc_align_supported(a.Hq, a.links, c);
@@ -382,6 +404,12 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
             PhaseMark mark(3, st);
             if ((e = launch_tc_flash(fv, st)) != cudaSuccess) return e;
         }
+        if (stream_out && (e = copy_out(wv, st)) != cudaSuccess) return e;
+    }
+    if (stream_out) {
+        if ((e = cudaEventRecord(side->copy_done, side->copy_out)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(s, side->copy_done, 0)) != cudaSuccess) return e;
+        ho->done = true;
     }
     for (int i = 0; i + 1 < sets; ++i) {
         if ((e = cudaEventRecord(side->wave_done[i], side->wave[i])) != cudaSuccess) return e;
