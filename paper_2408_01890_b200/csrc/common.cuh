@@ -141,19 +141,23 @@ struct TcCarry {
     void* scores;
     bool first, keep;
 };
-// Output streamed to host memory while the layer runs (the host-memory entry points): after each wave's attention kernel
-// the wave's rows of o (dense [B,N,Hq,d] on both sides) are copied to host_o on a stream of the library's own, joined
-// into the caller's stream at the end.  done is set when the copies were enqueued; otherwise the caller copies o itself.
-struct TcHostOut {
+// Host-memory entry points: q0, k0, v (each may be null: nothing to bring in) and o live in host memory, dense [B,N,H,d]
+// like their device copies in the arena.  The tensor-core path streams them: before a wave starts, its rows of q0, k0
+// and v are copied in on a stream of the library's own (a wave needs the keys and values up to its last row, and the
+// waves run from row 0 up); after the wave's attention kernel its rows of o are copied out on another; both are joined
+// into the caller's stream at the end.  out_done is set when the output copies were enqueued; otherwise the caller
+// copies o itself.  Whoever launches the layer's kernels brings the inputs in first (whole tensors where not streamed).
+struct TcHostIO {
     void* host_o;
-    bool done;
+    const void *host_q0, *host_k0, *host_v;
+    bool out_done;
 };
 size_t tc_carry_bytes(int B, int N, int Hq);
 size_t tc_shared_prefill_carry_workspace(const lisa_shared_prefill_args& a);
 cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws, cudaStream_t s);
 // vs/os: per-layer V and O of a chain of a.chain_len layers (nullptr: only the deepest layer, a.v / a.o)
 cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, const lisa_tensor* vs, const lisa_tensor* os, void* ws,
-                                           cudaStream_t s, const TcCarry* carry = nullptr, TcHostOut* host_out = nullptr);
+                                           cudaStream_t s, const TcCarry* carry = nullptr, TcHostIO* host_io = nullptr);
 cudaError_t prefill_phase_timing(bool enable);
 cudaError_t prefill_phase_times(float* ms4);
 

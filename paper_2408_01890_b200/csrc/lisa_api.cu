@@ -223,12 +223,12 @@ size_t lisa_prefill_scores_bytes(int32_t B, int32_t N, int32_t Hq) {
     return (B < 1 || N < 1 || Hq < 1) ? 0 : tc_carry_bytes(B, N, Hq);
 }
 
-static lisa_status_t shared_prefill_carry_impl(const lisa_shared_prefill_carry_args* a, lisa_stream_t stream, TcHostOut* ho);
+static lisa_status_t shared_prefill_carry_impl(const lisa_shared_prefill_carry_args* a, lisa_stream_t stream, TcHostIO* ho);
 lisa_status_t lisa_attn_shared_prefill_carry(const lisa_shared_prefill_carry_args* a, lisa_stream_t stream) {
     return shared_prefill_carry_impl(a, stream, nullptr);
 }
 // ho: the layer's output is also wanted in host memory (the host-memory entry points)
-static lisa_status_t shared_prefill_carry_impl(const lisa_shared_prefill_carry_args* a, lisa_stream_t stream, TcHostOut* ho) {
+static lisa_status_t shared_prefill_carry_impl(const lisa_shared_prefill_carry_args* a, lisa_stream_t stream, TcHostIO* ho) {
     if (!a || a->struct_size != sizeof(lisa_shared_prefill_carry_args)) return LISA_ERR_INVALID_ARG;
     lisa_shared_prefill_args p;
     lisa_status_t st = carried_layer(*a, &p);
@@ -289,14 +289,28 @@ lisa_status_t lisa_workspace_bytes(int32_t op, const void* args, size_t* bytes) 
     return LISA_ERR_INVALID_ARG;
 }
 
-static lisa_status_t shared_prefill_impl(const lisa_shared_prefill_args* a, lisa_stream_t stream, TcHostOut* ho);
+static lisa_status_t shared_prefill_impl(const lisa_shared_prefill_args* a, lisa_stream_t stream, TcHostIO* ho);
 lisa_status_t lisa_attn_shared_prefill(const lisa_shared_prefill_args* a, lisa_stream_t stream) {
     return shared_prefill_impl(a, stream, nullptr);
 }
-static lisa_status_t shared_prefill_impl(const lisa_shared_prefill_args* a, lisa_stream_t stream, TcHostOut* ho) {
+// Whole-tensor copies of the inputs a host-memory call left to the launching side (paths that do not stream them).
+static cudaError_t host_inputs_whole(const lisa_shared_prefill_args& a, const TcHostIO& io, cudaStream_t s) {
+    const size_t rows = (size_t)a.B * a.N;
+    cudaError_t e = cudaSuccess;
+    if (io.host_q0) e = cudaMemcpyAsync(a.q0.ptr, io.host_q0, rows * a.Hq * a.d * esize(a.q0.dtype), cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && io.host_k0) e = cudaMemcpyAsync(a.k0.ptr, io.host_k0, rows * a.Hkv * a.d * esize(a.k0.dtype), cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && io.host_v) e = cudaMemcpyAsync(a.v.ptr, io.host_v, rows * a.Hkv * a.d * esize(a.v.dtype), cudaMemcpyHostToDevice, s);
+    return e;
+}
+static lisa_status_t shared_prefill_impl(const lisa_shared_prefill_args* a, lisa_stream_t stream, TcHostIO* ho) {
     lisa_status_t st = validate_prefill(a);
     if (st != LISA_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool orchestrated = !g_force_general.load() && a->chain_len > 0 && tc_shared_prefill_supported(*a);
+    if (ho && !orchestrated) {   // the tensor-core orchestration brings the inputs in itself, wave by wave
+        cudaError_t e = host_inputs_whole(*a, *ho, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
     if (!g_force_general.load() && a->d == 128 && a->chain_len == 0) {
         TcFlashArgs f{a->B, a->N, a->Hq, a->Hkv, 128, a->q0, a->k0, a->v, a->o, 1.0f / sqrtf((float)a->d), nullptr, 0, 0,
                       0, (a->N + 127) / 128};
@@ -305,7 +319,7 @@ static lisa_status_t shared_prefill_impl(const lisa_shared_prefill_args* a, lisa
             return e == cudaSuccess ? LISA_OK : cuda_fail(e);
         }
     }
-    if (!g_force_general.load() && a->chain_len > 0 && tc_shared_prefill_supported(*a)) {
+    if (orchestrated) {
         const size_t need = tc_shared_prefill_workspace(*a);
         if ((st = check_workspace(a->workspace, a->workspace_bytes, need)) != LISA_OK) return st;
         cudaError_t e = launch_tc_shared_prefill_chain(*a, nullptr, nullptr, a->workspace, s, nullptr, ho);
@@ -516,27 +530,27 @@ struct Arena {
 
 // Lays the call's tensors out in the arena. With arena.base == nullptr only the size is computed.
 // dev receives device-side copies of the descriptors; h2d lists (dst, src, bytes) to copy.
-struct Copy { void* dst; const void* src; size_t bytes; };
+struct Copy { void* dst; const void* src; size_t bytes; int streamed; };   // streamed: q0 (1), k0 (2), v (3) -- left to the launching side
 
 // anchor == false: q0 and k0 are not read by the call (a carried layer past the first): nothing is staged for them.
 size_t plan_host_call(const lisa_shared_prefill_args& h, char* base, lisa_shared_prefill_args* dev, lisa_link* dlinks,
                       Copy* copies, int* n_copies, size_t* o_bytes, bool anchor = true) {
     Arena ar{base, 0};
     int nc = 0;
-    auto dense = [&](const lisa_tensor& src, int H, int x, lisa_tensor* dst, bool copy_in) {
+    auto dense = [&](const lisa_tensor& src, int H, int x, lisa_tensor* dst, bool copy_in, int streamed = 0) {
         const size_t bytes = (size_t)h.B * h.N * H * x * esize(src.dtype);
         void* p = ar.take(bytes);
         if (dst) {
             *dst = lisa_tensor{p, src.dtype, 0, (int64_t)h.N * H * x, (int64_t)H * x, (int64_t)x};
-            if (copy_in) copies[nc++] = Copy{p, src.ptr, bytes};
+            if (copy_in) copies[nc++] = Copy{p, src.ptr, bytes, streamed};
         }
         return bytes;
     };
     if (anchor) {
-        dense(h.q0, h.Hq, h.d, dev ? &dev->q0 : nullptr, true);
-        dense(h.k0, h.Hkv, h.d, dev ? &dev->k0 : nullptr, true);
+        dense(h.q0, h.Hq, h.d, dev ? &dev->q0 : nullptr, true, 1);
+        dense(h.k0, h.Hkv, h.d, dev ? &dev->k0 : nullptr, true, 2);
     }
-    dense(h.v, h.Hkv, h.d, dev ? &dev->v : nullptr, true);
+    dense(h.v, h.Hkv, h.d, dev ? &dev->v : nullptr, true, 3);
     const size_t ob = dense(h.o, h.Hq, h.d, dev ? &dev->o : nullptr, false);
     if (o_bytes) *o_bytes = ob;
     for (int k = 0; k < h.chain_len; ++k) {
@@ -551,7 +565,7 @@ size_t plan_host_call(const lisa_shared_prefill_args& h, char* base, lisa_shared
         auto weight = [&](const void* src, size_t n, const void** dst) {
             if (!src) return;
             void* p = ar.take(n * ws);
-            if (dst) { *dst = p; copies[nc++] = Copy{p, src, n * ws}; }
+            if (dst) { *dst = p; copies[nc++] = Copy{p, src, n * ws, 0}; }
         };
         weight(l.w1, (size_t)h_in * l.m, dl ? &dl->w1 : nullptr);
         weight(l.b1, (size_t)l.m, dl ? &dl->b1 : nullptr);
@@ -630,12 +644,17 @@ lisa_status_t lisa_attn_shared_prefill_host(const lisa_shared_prefill_args* host
     if (used + ((ws + 255) & ~(size_t)255) > arena_bytes) return LISA_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    for (int i = 0; i < nc; ++i)
-        if ((e = cudaMemcpyAsync(copies[i].dst, copies[i].src, copies[i].bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+    // q0, k0, v come in and o goes back wave by wave while other waves compute, where the path supports it
+    TcHostIO ho{host_args->o.ptr, nullptr, nullptr, nullptr, false};
+    for (int i = 0; i < nc; ++i) {
+        if (copies[i].streamed == 1) ho.host_q0 = copies[i].src;
+        else if (copies[i].streamed == 2) ho.host_k0 = copies[i].src;
+        else if (copies[i].streamed == 3) ho.host_v = copies[i].src;
+        else if ((e = cudaMemcpyAsync(copies[i].dst, copies[i].src, copies[i].bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
             return cuda_fail(e);
-    TcHostOut ho{host_args->o.ptr, false};   // rows of o go back while later waves still compute, where the path supports it
+    }
     if ((st = shared_prefill_impl(&dev, stream, &ho)) != LISA_OK) return st;
-    if (!ho.done && (e = cudaMemcpyAsync(host_args->o.ptr, dev.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    if (!ho.out_done && (e = cudaMemcpyAsync(host_args->o.ptr, dev.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
     return LISA_OK;
 }
@@ -695,12 +714,16 @@ lisa_status_t lisa_attn_shared_prefill_carry_host(const lisa_shared_prefill_carr
         return LISA_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    for (int i = 0; i < nc; ++i)
-        if ((e = cudaMemcpyAsync(copies[i].dst, copies[i].src, copies[i].bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+    TcHostIO ho{host_args->layer.o.ptr, nullptr, nullptr, nullptr, false};
+    for (int i = 0; i < nc; ++i) {
+        if (copies[i].streamed == 1) ho.host_q0 = copies[i].src;
+        else if (copies[i].streamed == 2) ho.host_k0 = copies[i].src;
+        else if (copies[i].streamed == 3) ho.host_v = copies[i].src;
+        else if ((e = cudaMemcpyAsync(copies[i].dst, copies[i].src, copies[i].bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
             return cuda_fail(e);
-    TcHostOut ho{host_args->layer.o.ptr, false};
+    }
     if ((st = shared_prefill_carry_impl(&dev, stream, &ho)) != LISA_OK) return st;
-    if (!ho.done && (e = cudaMemcpyAsync(host_args->layer.o.ptr, dev.layer.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+    if (!ho.out_done && (e = cudaMemcpyAsync(host_args->layer.o.ptr, dev.layer.o.ptr, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
     return LISA_OK;
 }

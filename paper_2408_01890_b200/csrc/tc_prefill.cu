@@ -192,8 +192,8 @@ struct SideStream {
     cudaEvent_t fork = nullptr, join = nullptr;
     cudaStream_t wave[kWaveSets - 1] = {};         // waves beside the caller's stream
     cudaEvent_t wave_done[kWaveSets - 1] = {};
-    cudaStream_t copy_out = nullptr;               // device -> host copies of finished rows (host-memory entry points)
-    cudaEvent_t rows_done = nullptr, copy_done = nullptr;
+    cudaStream_t copy_out = nullptr, copy_in = nullptr;   // host-memory entry points: finished rows out, the next wave's rows in
+    cudaEvent_t rows_done = nullptr, copy_done = nullptr, rows_in = nullptr;
     bool ok = false;
 };
 SideStream g_side[64];
@@ -214,6 +214,8 @@ SideStream* side_stream() {
         if (cudaStreamCreateWithFlags(&ss.copy_out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
         if (cudaEventCreateWithFlags(&ss.rows_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         if (cudaEventCreateWithFlags(&ss.copy_done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        if (cudaStreamCreateWithFlags(&ss.copy_in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&ss.rows_in, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         ss.ok = true;
     }
     return &ss;
@@ -230,9 +232,9 @@ cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws
 // With cy: one link, in place on the caller's carried scores (rows from 0, N rounded up to whole tiles both ways): no A_0
 // unless this is the first layer of its chain, no wave planes, and the attention kernel leaves A_n behind when asked.
 cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, const lisa_tensor* vs, const lisa_tensor* os, void* ws,
-                                           cudaStream_t s, const TcCarry* cy, TcHostOut* ho) {
+                                           cudaStream_t s, const TcCarry* cy, TcHostIO* ho) {
     const bool all_layers = vs != nullptr;
-    if (ho) ho->done = false;
+    if (ho) ho->out_done = false;
     if (cy && (all_layers || a.chain_len != 1 || !cy->scores)) return cudaErrorInvalidValue;
     const Layout l = plan_layout(a, cy != nullptr);
     // geometry of the plane that holds the running scores: the caller's buffer (whole prompt, rows from 0) or a wave's plane
@@ -286,6 +288,33 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
     const int sets = (side && nw >= 2) ? l.sets : 1;
     // rows of o leave for the host as soon as their wave's attention kernel is done (dense bf16 o only)
     const bool stream_out = ho && ho->host_o && side && !all_layers && a.o.stride_h == a.d && a.o.stride_n == (int64_t)a.Hq * a.d;
+    // rows [r0, r1) of a dense [B,N,H,d] bf16 tensor, one copy per sequence
+    auto copy_rows = [&](void* dst, const void* src, int H, int64_t r0, int64_t r1, cudaMemcpyKind kind, cudaStream_t cs) -> cudaError_t {
+        for (int b = 0; b < a.B; ++b) {
+            const int64_t off = ((int64_t)b * a.N + r0) * H * a.d * 2;
+            cudaError_t ce = cudaMemcpyAsync(static_cast<char*>(dst) + off, static_cast<const char*>(src) + off,
+                                             (size_t)(r1 - r0) * H * a.d * 2, kind, cs);
+            if (ce != cudaSuccess) return ce;
+        }
+        return cudaSuccess;
+    };
+    auto dense = [&](const lisa_tensor& t, int H) { return t.stride_h == a.d && t.stride_n == (int64_t)H * a.d && t.stride_b == (int64_t)a.N * H * a.d; };
+    const bool has_in = ho && (ho->host_q0 || ho->host_k0 || ho->host_v);
+    const bool stream_in = has_in && stream_out && dense(a.q0, a.Hq) && dense(a.k0, a.Hkv) && dense(a.v, a.Hkv) && dense(a.o, a.Hq);
+    if (has_in && !stream_in) {   // whole tensors, before anything reads them
+        if (ho->host_q0 && (e = copy_rows(a.q0.ptr, ho->host_q0, a.Hq, 0, a.N, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
+        if (ho->host_k0 && (e = copy_rows(a.k0.ptr, ho->host_k0, a.Hkv, 0, a.N, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
+        if (ho->host_v && (e = copy_rows(a.v.ptr, ho->host_v, a.Hkv, 0, a.N, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
+    }
+    auto copy_in = [&](const Wave& wv, cudaStream_t st) -> cudaError_t {
+        cudaError_t ce;
+        const int64_t r0 = (int64_t)wv.begin * kTile, r1 = std::min<int64_t>(a.N, (int64_t)(wv.begin + wv.count) * kTile);
+        if (ho->host_q0 && (ce = copy_rows(a.q0.ptr, ho->host_q0, a.Hq, r0, r1, cudaMemcpyHostToDevice, side->copy_in)) != cudaSuccess) return ce;
+        if (ho->host_k0 && (ce = copy_rows(a.k0.ptr, ho->host_k0, a.Hkv, r0, r1, cudaMemcpyHostToDevice, side->copy_in)) != cudaSuccess) return ce;
+        if (ho->host_v && (ce = copy_rows(a.v.ptr, ho->host_v, a.Hkv, r0, r1, cudaMemcpyHostToDevice, side->copy_in)) != cudaSuccess) return ce;
+        if ((ce = cudaEventRecord(side->rows_in, side->copy_in)) != cudaSuccess) return ce;
+        return cudaStreamWaitEvent(st, side->rows_in, 0);   // everything copied so far: the wave's rows and all rows before them
+    };
     auto copy_out = [&](const Wave& wv, cudaStream_t st) -> cudaError_t {
         cudaError_t ce;
         if ((ce = cudaEventRecord(side->rows_done, st)) != cudaSuccess) return ce;
@@ -299,6 +328,11 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         }
         return cudaSuccess;
     };
+    if (stream_in) {   // the copies start once everything enqueued before the call (earlier users of the arena) is done
+        std::lock_guard<std::mutex> lock(g_side_mutex);
+        if ((e = cudaEventRecord(side->fork, s)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(side->copy_in, side->fork, 0)) != cudaSuccess) return e;
+    }
     std::unique_lock<std::mutex> wave_lock(g_side_mutex, std::defer_lock);
     if (sets > 1 || stream_out) {
         wave_lock.lock();
@@ -313,6 +347,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
         const int set = w % sets;
         cudaStream_t st = set == 0 ? s : side->wave[set - 1];
         const size_t* po = l.plane_off[set];
+        if (stream_in && (e = copy_in(wv, st)) != cudaSuccess) return e;
         // 1. anchor scores and the differences of the links below the top one
         const TcFlashArgs fw{a.B, a.N, a.Hq, a.Hkv, 128, a.q0, a.k0, a.v, a.o, 1.f / sqrtf((float)a.d), nullptr, l.plane_rows, l.plane_cols,
                              wv.begin, wv.count};                 // the wave's own planes
@@ -409,7 +444,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
     if (stream_out) {
         if ((e = cudaEventRecord(side->copy_done, side->copy_out)) != cudaSuccess) return e;
         if ((e = cudaStreamWaitEvent(s, side->copy_done, 0)) != cudaSuccess) return e;
-        ho->done = true;
+        ho->out_done = true;
     }
     for (int i = 0; i + 1 < sets; ++i) {
         if ((e = cudaEventRecord(side->wave_done[i], side->wave[i])) != cudaSuccess) return e;
