@@ -238,7 +238,10 @@ lisa_status_t lisa_carry_host_arena_bytes(const lisa_shared_prefill_carry_args* 
 /* The same call with every tensor, weight and `o` in HOST memory (dense [B,N,H,x] layout, strides
  * ignored; workspace fields ignored).  Inputs are staged into `device_arena` (device memory of at least
  * lisa_host_arena_bytes(), 256-byte aligned), the layer runs, `o` is copied back and the stream is
- * synchronised before returning.  Pinned host memory makes the copies faster but is not required. */
+ * synchronised before returning.  On the tensor-core path the copies overlap the layer: q0, k0 and v come in, and o goes
+ * back, one strip of query rows at a time on streams of the library's own (created on first use, joined into `stream`
+ * before the call returns) while other strips compute; this needs pinned host memory to take effect, pageable memory
+ * works but serialises. */
 lisa_status_t lisa_attn_shared_prefill_host(const lisa_shared_prefill_args* host_args, void* device_arena,
                                             size_t arena_bytes, lisa_stream_t stream);
 lisa_status_t lisa_host_arena_bytes(const lisa_shared_prefill_args* host_args, size_t* bytes);
