@@ -127,6 +127,25 @@ bool tc_align_concat_supported(int Hq, const lisa_link* links, int chain);
 bool tc_align_link_supported(int Hq, const lisa_link* links, int chain);
 cudaError_t launch_tc_align_link(const TcAlignLinkArgs& a, cudaStream_t s);
 
+// Programmatic dependent launch for chains of short kernels (the decode step: append, chunk, merge, layer after layer):
+// a kernel launched with launch_chained may start while its predecessor in the stream is still running; it must call
+// chain_wait() before it touches anything an earlier kernel wrote or still reads (what it does before -- staging constant
+// weights -- overlaps the predecessor's tail), and calls chain_release() early so that its own successor can be set up.
+// chain_wait() returns once the predecessor has completed and its writes are visible; as every kernel of such a chain
+// waits before it finishes, completion is transitive.  In a kernel launched the ordinary way both are no-ops.
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename Params>
+cudaError_t launch_chained(void (*kernel)(Params), dim3 grid, dim3 block, size_t smem, cudaStream_t s, const Params& p) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
 // Packs Q' or K' ([B,N,H,r], any strides) into zero-padded bf16 [B][H][N][64] rows for the tensor-core kernels.
 cudaError_t launch_pack_lowrank(const lisa_tensor& src, int B, int N, int H, int r, void* dst, cudaStream_t s);
 

@@ -233,10 +233,8 @@ template <int HQ_C, int M_C, bool RB>
 __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(16) float smem[];
     const int b = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x;
-    const int L = p.seq_lens ? min(p.seq_lens[b], p.L_uniform) : p.L_uniform;   // never beyond the chunks the launch covers
+    chain_release();
     const int j0 = chunk * kChunk;
-    if (j0 >= L) return;
-    const int nrows = min(kChunk, L - j0);
     const int Hq = HQ_C ? HQ_C : p.Hq;
     const int m = M_C ? M_C : (p.integrate == LISA_INTEGRATE_PLUS ? 0 : p.m);
     const int r = p.r, G = Hq / p.Hkv;
@@ -252,10 +250,7 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
     float* b1_s = w2_s + m * w2_ld;         // [m]
     float* b2_s = b1_s + m;                 // [Hq]
 
-    for (int e = tid; e < Hq * r; e += kThreads) {
-        const int h = e / r, x = e % r;
-        qp_s[h * kMaxRank + x] = ld_elem(p.qp.ptr, b * p.qp.sb + h * p.qp.sh + x, p.qp.dtype);
-    }
+    // the aligner's weights are constants of the model: staged while the kernel before this one may still be running
     if (p.integrate != LISA_INTEGRATE_PLUS) {
         for (int e = tid; e < h_in * m; e += kThreads) w1_s[(e / m) * w1_ld + e % m] = ld_elem(p.w1, e, p.w_dtype);
         for (int e = tid; e < m; e += kThreads) b1_s[e] = ldw(p.b1, e, p.w_dtype);
@@ -263,6 +258,14 @@ __global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_ke
             for (int e = tid; e < m * Hq; e += kThreads) w2_s[(e / Hq) * w2_ld + e % Hq] = ld_elem(p.w2, e, p.w_dtype);
             for (int e = tid; e < Hq; e += kThreads) b2_s[e] = ldw(p.b2, e, p.w_dtype);
         }
+    }
+    chain_wait();   // from here on: lengths, Q', the caches and the score row, which earlier kernels of the stream produce
+    const int L = p.seq_lens ? min(p.seq_lens[b], p.L_uniform) : p.L_uniform;   // never beyond the chunks the launch covers
+    if (j0 >= L) return;
+    const int nrows = min(kChunk, L - j0);
+    for (int e = tid; e < Hq * r; e += kThreads) {
+        const int h = e / r, x = e % r;
+        qp_s[h * kMaxRank + x] = ld_elem(p.qp.ptr, b * p.qp.sb + h * p.qp.sh + x, p.qp.dtype);
     }
     __syncthreads();
 
@@ -498,6 +501,8 @@ __device__ __forceinline__ void anchor_qk_full_chunk(const DecodeParams& p, floa
 __global__ void __launch_bounds__(kThreads, 2) anchor_decode_chunk_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(16) float smem[];
     const int b = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    chain_release();
+    chain_wait();
     const int L = p.seq_lens ? min(p.seq_lens[b], p.L_uniform) : p.L_uniform;   // never beyond the chunks the launch covers
     const int j0 = chunk * kChunk;
     if (j0 >= L) return;
@@ -576,6 +581,8 @@ __global__ void __launch_bounds__(kThreads, 2) anchor_decode_chunk_kernel(const 
 __global__ void decode_merge_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ float s_w[];   // per chunk: exp(m_c - M) / sum, the weight of the chunk's partial output
     const int h = blockIdx.x, b = blockIdx.y, x = threadIdx.x;
+    chain_release();
+    chain_wait();
     const int L = p.seq_lens ? min(p.seq_lens[b], p.L_uniform) : p.L_uniform;   // never beyond the chunks the launch covers
     const int nc = (L + kChunk - 1) / kChunk;
     const size_t base = (size_t)b * p.n_chunks * p.Hq + h;
@@ -665,20 +672,20 @@ cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cud
     do {                                                                                                           \
         if (p.row_bf16) {                                                                                          \
             if ((e = set_smem(shared_decode_chunk_kernel<HQ_, M_, true>, smem)) != cudaSuccess) return e;          \
-            shared_decode_chunk_kernel<HQ_, M_, true><<<grid, kThreads, smem, s>>>(p);                             \
+            e = launch_chained(shared_decode_chunk_kernel<HQ_, M_, true>, grid, dim3(kThreads), smem, s, p);        \
         } else {                                                                                                   \
             if ((e = set_smem(shared_decode_chunk_kernel<HQ_, M_, false>, smem)) != cudaSuccess) return e;         \
-            shared_decode_chunk_kernel<HQ_, M_, false><<<grid, kThreads, smem, s>>>(p);                            \
+            e = launch_chained(shared_decode_chunk_kernel<HQ_, M_, false>, grid, dim3(kThreads), smem, s, p);       \
         }                                                                                                          \
     } while (0)
     if (fast && p.Hq == 40 && p.m == 80) LISA_LAUNCH_CHUNK(40, 80);
     else if (fast && p.Hq == 32 && p.m == 64) LISA_LAUNCH_CHUNK(32, 64);
     else LISA_LAUNCH_CHUNK(0, 0);
 #undef LISA_LAUNCH_CHUNK
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, (size_t)p.n_chunks * sizeof(float), s>>>(p);
+    if (e != cudaSuccess) return e;
+    e = launch_chained(decode_merge_kernel, dim3(p.Hq, p.B), dim3(p.d), (size_t)p.n_chunks * sizeof(float), s, p);
     count_launches(2);
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_anchor_decode(const lisa_anchor_args& a, void* ws, cudaStream_t s) {
@@ -696,11 +703,10 @@ cudaError_t launch_anchor_decode(const lisa_anchor_args& a, void* ws, cudaStream
     const size_t smem = sizeof(float) * ((size_t)p.Hq * kChunk + (size_t)p.Hq * p.d);
     cudaError_t e;
     if ((e = set_smem(anchor_decode_chunk_kernel, smem)) != cudaSuccess) return e;
-    anchor_decode_chunk_kernel<<<dim3(p.n_chunks, p.B), kThreads, smem, s>>>(p);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    decode_merge_kernel<<<dim3(p.Hq, p.B), p.d, (size_t)p.n_chunks * sizeof(float), s>>>(p);
+    if ((e = launch_chained(anchor_decode_chunk_kernel, dim3(p.n_chunks, p.B), dim3(kThreads), smem, s, p)) != cudaSuccess) return e;
+    e = launch_chained(decode_merge_kernel, dim3(p.Hq, p.B), dim3(p.d), (size_t)p.n_chunks * sizeof(float), s, p);
     count_launches(2);
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace lisa

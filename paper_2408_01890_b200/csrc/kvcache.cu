@@ -62,6 +62,8 @@ __device__ __forceinline__ void append_kp_transposed(const AppendParams& p) {
 // transposed K_LR columns (SHARED).
 template <typename Vec, int kElems, typename T>
 __global__ void append_kernel(const __grid_constant__ AppendParams p) {
+    chain_release();
+    chain_wait();
     if (blockIdx.y == 0) append_rows<Vec, kElems>(p, p.v, p.vc, true);
     else if (p.kind == LISA_CACHE_STANDARD) append_rows<Vec, kElems>(p, p.k, p.kc, false);
     else append_kp_transposed<T>(p);
@@ -77,10 +79,11 @@ cudaError_t launch_kvcache_append(const lisa_kvcache_layer& c, const lisa_tensor
     const int threads = 256;
     const int64_t rows = (int64_t)c.B * n_new * c.Hkv;
     auto blocks_for = [&](int64_t n) { return (int)std::max<int64_t>(1, std::min<int64_t>((n + threads - 1) / threads, sm_count() * 16)); };
-    if (c.dtype == LISA_BF16) append_kernel<uint4, 8, __nv_bfloat16><<<dim3(blocks_for(rows * (c.d / 8)), 2), threads, 0, s>>>(p);
-    else append_kernel<float4, 4, float><<<dim3(blocks_for(rows * (c.d / 4)), 2), threads, 0, s>>>(p);
+    cudaError_t e;
+    if (c.dtype == LISA_BF16) e = launch_chained(append_kernel<uint4, 8, __nv_bfloat16>, dim3(blocks_for(rows * (c.d / 8)), 2), dim3(threads), 0, s, p);
+    else e = launch_chained(append_kernel<float4, 4, float>, dim3(blocks_for(rows * (c.d / 4)), 2), dim3(threads), 0, s, p);
     count_launches(1);
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace lisa
