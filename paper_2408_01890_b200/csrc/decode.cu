@@ -229,8 +229,10 @@ __device__ __forceinline__ void softmax_pv_chunk(const DecodeParams& p, float* s
 // Shared layer.  HQ_C/M_C > 0: compile-time sizes, aligner on the tensor cores (ADD, two layers, bf16 cache,
 // M_C % 8 == 0, HQ_C % 8 == 0).  HQ_C == 0: any supported mode and size, per-thread scratch arrays.
 // ---------------------------------------------------------------------------------------------
-template <int HQ_C, int M_C, bool RB>
-__global__ void __launch_bounds__(kThreads, HQ_C ? 2 : 1) shared_decode_chunk_kernel(const __grid_constant__ DecodeParams p) {
+// CTAS: CTAs per SM the kernel is compiled for.  Three hide the FFN phase (no loads in flight from the CTA that is in it)
+// better than two, at 80 instead of 128 registers; which one a launch takes depends on how its grid fills the waves.
+template <int HQ_C, int M_C, bool RB, int CTAS = 2>
+__global__ void __launch_bounds__(kThreads, HQ_C ? CTAS : 1) shared_decode_chunk_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(16) float smem[];
     const int b = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x;
     chain_release();
@@ -668,19 +670,24 @@ cudaError_t launch_shared_decode(const lisa_shared_decode_args& a, void* ws, cud
     dim3 grid(p.n_chunks, p.B);
     const bool fast = p.integrate == LISA_INTEGRATE_ADD && p.ffn_layers == 2 && c.dtype == LISA_BF16;
     cudaError_t e;
-#define LISA_LAUNCH_CHUNK(HQ_, M_)                                                                                 \
+#define LISA_LAUNCH_CHUNK(HQ_, M_, CTAS_)                                                                          \
     do {                                                                                                           \
         if (p.row_bf16) {                                                                                          \
-            if ((e = set_smem(shared_decode_chunk_kernel<HQ_, M_, true>, smem)) != cudaSuccess) return e;          \
-            e = launch_chained(shared_decode_chunk_kernel<HQ_, M_, true>, grid, dim3(kThreads), smem, s, p);        \
+            if ((e = set_smem(shared_decode_chunk_kernel<HQ_, M_, true, CTAS_>, smem)) != cudaSuccess) return e;   \
+            e = launch_chained(shared_decode_chunk_kernel<HQ_, M_, true, CTAS_>, grid, dim3(kThreads), smem, s, p); \
         } else {                                                                                                   \
-            if ((e = set_smem(shared_decode_chunk_kernel<HQ_, M_, false>, smem)) != cudaSuccess) return e;         \
-            e = launch_chained(shared_decode_chunk_kernel<HQ_, M_, false>, grid, dim3(kThreads), smem, s, p);       \
+            if ((e = set_smem(shared_decode_chunk_kernel<HQ_, M_, false, CTAS_>, smem)) != cudaSuccess) return e;  \
+            e = launch_chained(shared_decode_chunk_kernel<HQ_, M_, false, CTAS_>, grid, dim3(kThreads), smem, s, p); \
         }                                                                                                          \
     } while (0)
-    if (fast && p.Hq == 40 && p.m == 80) LISA_LAUNCH_CHUNK(40, 80);
-    else if (fast && p.Hq == 32 && p.m == 64) LISA_LAUNCH_CHUNK(32, 64);
-    else LISA_LAUNCH_CHUNK(0, 0);
+    // Two or three CTAs per SM: a CTA of the three-per-SM build takes about 1.3 times as long as one of the two-per-SM
+    // build runs beside one neighbour (measured at B 64, L 4096, 40 heads: 0.534 against 0.566 ms for the whole grid), and the
+    // grid runs in whole waves of CTAs: take the build whose waves cost less.
+    const int64_t n_ctas = (int64_t)p.n_chunks * p.B, sms = sm_count();
+    const bool three = 1.3 * (double)((n_ctas + 3 * sms - 1) / (3 * sms)) < (double)((n_ctas + 2 * sms - 1) / (2 * sms));
+    if (fast && p.Hq == 40 && p.m == 80) { if (three) LISA_LAUNCH_CHUNK(40, 80, 3); else LISA_LAUNCH_CHUNK(40, 80, 2); }
+    else if (fast && p.Hq == 32 && p.m == 64) { if (three) LISA_LAUNCH_CHUNK(32, 64, 3); else LISA_LAUNCH_CHUNK(32, 64, 2); }
+    else LISA_LAUNCH_CHUNK(0, 0, 2);
 #undef LISA_LAUNCH_CHUNK
     if (e != cudaSuccess) return e;
     e = launch_chained(decode_merge_kernel, dim3(p.Hq, p.B), dim3(p.d), (size_t)p.n_chunks * sizeof(float), s, p);

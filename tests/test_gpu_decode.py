@@ -70,6 +70,15 @@ def test_shared_decode_shapes(Hq, Hkv, d, r, m, L):
     run_shared_decode(w, 2, L, lens=None, seed=5, L_cap=(L + 7) // 8 * 8 + 64)
 
 
+@pytest.mark.parametrize("Hq,Hkv,m,B,L", [(32, 8, 64, 10, 4200), (40, 40, 80, 12, 3500)])
+def test_shared_decode_three_ctas_per_sm(Hq, Hkv, m, B, L):
+    """Grids of 297..444 chunk CTAs (on 148 SMs) take the build of the chunk kernel that runs three CTAs per SM; ragged
+    lengths, against the oracle like every other shape."""
+    w = synth.Workload("dthree", "bf16", B, L, Hq, Hkv, 128, 21, m, "relu", 1, True)
+    lens = [L if b % 3 == 0 else (1 + (b * 977) % L) for b in range(B)]
+    run_shared_decode(w, B, L, lens=lens, seed=6)
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("Hq,Hkv,d,L", [(40, 40, 128, 600), (32, 8, 128, 257), (6, 3, 64, 130), (4, 4, 32, 7)])
 def test_anchor_decode(dtype, Hq, Hkv, d, L):
