@@ -44,7 +44,7 @@ PREFILL_TRAFFIC_PER_PH = {"emit_scores": (39902464 + 85123840) / CFG2_POSITIONS_
 CARRY_POSITIONS_HEADS = 2816 * 2817 // 2 * 32
 CARRY_TRAFFIC_PER_PH = {"align": 4.370805e12 * 107.872e-6 / CARRY_POSITIONS_HEADS,
                         "attention_keep": 3.943844e12 * 133.088e-6 / CARRY_POSITIONS_HEADS}
-DECODE_TRAFFIC_PER_SEQ = (395952128 + 4544512) / 8  # shared decode chunk kernel, captured at 8 sequences; scales with the batch
+DECODE_TRAFFIC_PER_SEQ = (593884160 + 4890112) / 12  # shared decode chunk kernel, captured at 12 sequences; scales with the batch
 PROJECT_TRAFFIC = 220900096 + 163201024             # projection kernel at the benchmark's own size
 
 
