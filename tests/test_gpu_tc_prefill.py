@@ -319,3 +319,48 @@ def test_carried_scores_concatenating_integrate(B, N, Hkv, chain, m, act, layers
         assert lb.lisa_check() == lb.OK
         ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1])
         assert_close(got.float().cpu().numpy(), ref, "bf16", "carried scores, concatenating integrate, layer %d of %d" % (k + 1, chain))
+
+
+def test_carried_scores_several_waves_from_device_and_host_memory():
+    """B = 4, N = 1600: the prompt's scores exceed one wave's budget, so the layers run as two waves on two streams; the
+    host-memory call then also brings q0, k0, v in and takes o out wave by wave.  Both must give bit-identical outputs
+    (same kernels on the same data), and sampled rows (first and last tile, 32 random rows per sequence) must match the
+    oracle at every depth."""
+    B, N, Hq, Hkv, chain = 4, 1600, 32, 8, 2
+    t = link_inputs(B, N, Hq, Hkv, chain, 64, "relu", 2, 21, 43, False)
+    dl, ol = make_links(t, chain, "relu")
+    rng = np.random.default_rng(1)
+    rb, ri = [], []
+    for b in range(B):
+        rows = np.concatenate([np.arange(128), np.arange(N - 128, N), rng.integers(128, N - 128, 32)])
+        rb.append(np.full(rows.shape, b)); ri.append(rows)
+    rb, ri = np.concatenate(rb).astype(np.int32), np.concatenate(ri).astype(np.int32)
+    scores_d = torch.empty(lb.lisa_prefill_scores_bytes(B, N, Hq), dtype=torch.uint8, device="cuda")
+    scores_h = torch.empty_like(scores_d)   # device memory too: the scores of the host-memory calls
+    pin = {k: v.pin_memory() for k, v in t.items()}
+    q0, k0 = dev(t["q0"]), dev(t["k0"])
+    for k in range(chain):
+        first, keep = k == 0, k + 1 < chain
+        got = lb.lisa_attn_shared_prefill_carry(q0, k0, dl[k], dev(t[f"v{k + 1}"]), scores_d, first=first, keep=keep)
+        hl = lb.Link(pin[f"qp{k + 1}"], pin[f"kp{k + 1}"], pin[f"w1_{k + 1}"], pin[f"w2_{k + 1}"], act=lb.ACT_RELU)
+        out_h = torch.empty_like(t["q0"]).pin_memory()
+        arena = torch.empty(lb.lisa_carry_host_arena_bytes(pin["q0"], pin["k0"], hl, pin[f"v{k + 1}"], out_h, scores_h, first=first),
+                            dtype=torch.uint8, device="cuda")
+        lb.lisa_attn_shared_prefill_carry_host(pin["q0"], pin["k0"], hl, pin[f"v{k + 1}"], out_h, scores_h, arena, first=first, keep=keep)
+        torch.cuda.synchronize()
+        assert lb.lisa_check() == lb.OK
+        assert torch.equal(out_h, got.cpu())
+        ref = oracle.prefill_rows(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1], rb, ri)
+        sel = got[torch.from_numpy(rb).long().cuda(), torch.from_numpy(ri).long().cuda()].float().cpu().numpy()
+        assert_close(sel, ref, "bf16", "carried scores over two waves, layer %d" % (k + 1))
+    # the recomputing call at depth 2 through the host-memory entry point (inputs and output streamed per wave as well)
+    hlinks = [lb.Link(pin[f"qp{j}"], pin[f"kp{j}"], pin[f"w1_{j}"], pin[f"w2_{j}"], act=lb.ACT_RELU) for j in (1, 2)]
+    out_h = torch.empty_like(t["q0"]).pin_memory()
+    arena = torch.empty(lb.lisa_host_arena_bytes(pin["q0"], pin["k0"], hlinks, pin["v2"], out_h), dtype=torch.uint8, device="cuda")
+    lb.lisa_attn_shared_prefill_host(pin["q0"], pin["k0"], hlinks, pin["v2"], out_h, arena)
+    got2 = lb.lisa_attn_shared_prefill(q0, k0, dl, dev(t["v2"]))
+    torch.cuda.synchronize()
+    assert torch.equal(out_h, got2.cpu())
+    sel = got2[torch.from_numpy(rb).long().cuda(), torch.from_numpy(ri).long().cuda()].float().cpu().numpy()
+    assert_close(sel, ref, "bf16", "recomputed over two waves, depth 2")
+    assert lb.lisa_check() == lb.OK
