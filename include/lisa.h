@@ -203,7 +203,7 @@ lisa_status_t lisa_attn_shared_prefill_chain(const lisa_shared_prefill_chain_arg
 
 /* ------------------------------------------------------------------------------------------------
  * lisa_attn_shared_prefill_carry -- a shared layer over a whole prompt that takes the scores of the layer before it
- * from memory, as Sec. 5.1 states the method (layer n aligns A_{n-1} "from the adjacent front layer"), instead of
+ * from memory, as Sec. 5.1 states the method (layer n aligns the scores A_{n-1} of the layer directly before it), instead of
  * recomputing them from the anchor: the cost of a layer no longer grows with its depth in the chain, so runs of many
  * consecutive shared layers (the appendix's configurations have runs of 15 and 27) cost the same per layer as the first.
  * The price is memory: `scores` holds A_n for the whole prompt, lisa_prefill_scores_bytes(B, N, Hq) =
