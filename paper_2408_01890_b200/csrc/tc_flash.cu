@@ -36,6 +36,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+constexpr int kPrefetchAhead = 2;   // tiles (0: no L2 prefetch)
 constexpr int kThreads = 256;   // warpgroup 0: softmax/epilogue; warpgroup 1: producer, two MMA issuers, one idle warp
 
 struct FlashParams {
@@ -214,6 +215,19 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
             if (more_k) {
                 if (lane < NK) tma_load_4d(sK + ks_next * L::K_BYTES + lane * (BN * 128), &tmK, k_full + ks_next, lane * 64, g, (t + 1) * BN, b);
                 __syncwarp();
+            }
+            // The V and Y stages of a tile cannot be refilled before the P.V of the tile two before it has run, one softmax pass
+            // before they are needed -- less than a trip to HBM under load.  Their tiles are therefore asked into L2 earlier,
+            // kPrefetchAhead tiles ahead of the one just issued.
+            if constexpr (kPrefetchAhead > 0 && !EMIT) {
+                if (t + kPrefetchAhead < nt) {
+                    if (lane < NV) tma_prefetch_l2_4d(&tmV, lane * 64, g, (t + kPrefetchAhead) * BN, b);
+                    __syncwarp();
+                    if constexpr (PLANE) {
+                        if (lane == 0) tma_prefetch_l2_5d(&tmY, 0, b * p.Hq + h, 0, t + kPrefetchAhead, (q0 - p.plane_row0) / BM);
+                        __syncwarp();
+                    }
+                }
             }
             if (++ks_next == KST) { ks_next = 0; kpar_next ^= 1; }
         }
