@@ -84,7 +84,8 @@ struct PhaseMark {
 
 struct Wave { int begin, count; };
 
-int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves) {
+// carried: the scores live in the caller's buffer, a wave has no planes of its own and its size is free
+int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves, bool carried = false) {
     const int min_ctas = kWaveCtasPerSm * sm_count();
     const int n_qt = (N + kTile - 1) / kTile;
     const size_t per_col_tile = (size_t)B * Hq * kTile * kTile * 2 * c;
@@ -95,6 +96,21 @@ int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves) {
         while (qt + cnt < n_qt && (B * Hq * cnt < min_ctas || bytes + per_col_tile * (qt + cnt + 1) <= kWaveBytes)) {
             bytes += per_col_tile * (qt + cnt + 1);
             ++cnt;
+        }
+        // The head-partitioned kernels run one CTA per (batch, head, query tile), two per SM at a time, and the CTAs of a wave
+        // weigh about the same: a wave of 2.2 rounds of CTAs takes as long as one of 3.  Tiles are added (while the planes,
+        // where the wave has any, stay within four times the budget) until the last round is at least nine tenths full, or the best fill found is taken.
+        {
+            const int64_t slots = 2 * (int64_t)sm_count();
+            auto fill = [&](int k) { const int64_t n = (int64_t)B * Hq * k; return (double)n / (double)(((n + slots - 1) / slots) * slots); };
+            int best = cnt;
+            size_t grow = bytes;
+            for (int k = cnt; qt + k <= n_qt && k <= cnt + 16; ++k) {
+                if (k > cnt) { grow += per_col_tile * (qt + k); if (!carried && grow > 4 * kWaveBytes) break; }
+                if (fill(k) > fill(best) + 1e-9) best = k;
+                if (fill(k) >= 0.9) { best = k; break; }
+            }
+            if (qt + best < n_qt || best == cnt) cnt = best; else cnt = n_qt - qt >= best ? best : cnt;
         }
         if (waves && n < max_waves) waves[n] = Wave{qt, cnt};
         ++n;
@@ -133,7 +149,7 @@ Layout plan_layout(const lisa_shared_prefill_args& a, bool carried = false) {
     }
     const int n_qt = (a.N + kTile - 1) / kTile;
     Wave waves[1024];
-    const int nw = plan_waves(a.B, a.N, a.Hq, carried ? 1 : plane_count(a), waves, 1024);
+    const int nw = plan_waves(a.B, a.N, a.Hq, carried ? 1 : plane_count(a), waves, 1024, carried && !concat_chain(a));
     int max_cnt = 1;
     for (int i = 0; i < std::min(nw, 1024); ++i) max_cnt = std::max(max_cnt, waves[i].count);
     l.plane_rows = (int64_t)max_cnt * kTile;
@@ -281,7 +297,7 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
     };
     const bool concat = concat_chain(a);
     Wave waves[1024];
-    const int nw = plan_waves(a.B, a.N, a.Hq, cy ? 1 : plane_count(a), waves, 1024);
+    const int nw = plan_waves(a.B, a.N, a.Hq, cy ? 1 : plane_count(a), waves, 1024, cy != nullptr && !concat);
     // Several waves in flight (see kWaveSets): wave w runs on stream w % sets (0 = the caller's) with plane set w % sets.
     // All of it is forked from and joined back into the caller's stream inside this call, under the lock that keeps
     // another host thread's call from interleaving its event records with these waits.
