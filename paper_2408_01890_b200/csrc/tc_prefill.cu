@@ -110,7 +110,7 @@ int plan_waves(int B, int N, int Hq, int c, Wave* waves, int max_waves, bool car
                 if (fill(k) > fill(best) + 1e-9) best = k;
                 if (fill(k) >= 0.9) { best = k; break; }
             }
-            if (qt + best < n_qt || best == cnt) cnt = best; else cnt = n_qt - qt >= best ? best : cnt;
+            cnt = best;
         }
         if (waves && n < max_waves) waves[n] = Wave{qt, cnt};
         ++n;
