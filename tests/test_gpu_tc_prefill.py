@@ -364,3 +364,24 @@ def test_carried_scores_several_waves_from_device_and_host_memory():
     sel = got2[torch.from_numpy(rb).long().cuda(), torch.from_numpy(ri).long().cuda()].float().cpu().numpy()
     assert_close(sel, ref, "bf16", "recomputed over two waves, depth 2")
     assert lb.lisa_check() == lb.OK
+
+
+@pytest.mark.parametrize("N", [1, 63, 64, 65, 127, 128, 129, 255, 256, 257, 383])
+def test_carried_scores_at_tile_boundaries(N):
+    """Prompt lengths on and around the 64-key and 128-row tile sizes, three sequences, GQA: two carried layers against the
+    oracle, and the second one against the recomputing call of the same depth (the two differ only in where the first
+    layer's scores were rounded to fp16)."""
+    B, Hq, Hkv, chain = 3, 32, 8, 2
+    t = link_inputs(B, N, Hq, Hkv, chain, 64, "relu", 2, 21, 47, True)
+    dl, ol = make_links(t, chain, "relu", lb.INTEGRATE_ADD, 2, True)
+    scores = torch.full((lb.lisa_prefill_scores_bytes(B, N, Hq),), 0xFF, dtype=torch.uint8, device="cuda")
+    q0, k0 = dev(t["q0"]), dev(t["k0"])
+    for k in range(chain):
+        got = lb.lisa_attn_shared_prefill_carry(q0, k0, dl[k], dev(t[f"v{k + 1}"]), scores, first=k == 0, keep=k + 1 < chain)
+        torch.cuda.synchronize()
+        assert lb.lisa_check() == lb.OK
+        ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t[f"v{k + 1}"]), ol[:k + 1])
+        assert_close(got.float().cpu().numpy(), ref, "bf16", "carried scores, N=%d, layer %d" % (N, k + 1))
+    rec = lb.lisa_attn_shared_prefill(q0, k0, dl, dev(t["v2"]))
+    torch.cuda.synchronize()
+    assert_close(got.float().cpu().numpy(), rec.float().cpu().numpy().astype(np.float64), "bf16", "carried against recomputed, N=%d" % N)
