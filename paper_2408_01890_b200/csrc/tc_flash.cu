@@ -47,6 +47,7 @@ struct FlashParams {
     int* status;
     int plane_row0;  // first query row held by the plane workspace (rows are stored relative to it)
     int qt_begin;    // this launch covers query tiles [qt_begin, qt_begin + gridDim.y)
+    int head_major;  // grid is (query tiles, batch x heads) instead of (batch x heads, query tiles)
     int ksteps;      // 16-wide k-steps of the score MMA actually issued (<= KD/16; the rest is zero padding)
     float scale;     // MODE_EMIT: scores are multiplied by this before rounding to fp16
 };
@@ -135,8 +136,12 @@ tc_flash_kernel(const __grid_constant__ FlashParams p, const __grid_constant__ C
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // blockIdx.x (the fastest-dispatched index) runs over (batch, head), blockIdx.y over query tiles from the last one
     // down: every CTA of the heaviest tile is handed out before any lighter one, so the SMs finish close together
-    const int qt = p.qt_begin + (int)gridDim.y - 1 - (int)blockIdx.y;
-    const int h = (int)blockIdx.x % p.Hq, b = (int)blockIdx.x / p.Hq;
+    // With keys and values too large for L2 to hold for all heads at once, the order is turned round: blockIdx.x runs over the
+    // query tiles of one (batch, head), heaviest first, blockIdx.y over (batch, head), so that the CTAs resident at any time
+    // share the K and V tiles of a few heads instead of re-reading every head's for each query tile.
+    const int qt = p.qt_begin + (p.head_major ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)gridDim.y - 1 - (int)blockIdx.y);
+    const int bh = p.head_major ? (int)blockIdx.y : (int)blockIdx.x;
+    const int h = bh % p.Hq, b = bh / p.Hq;
     const int g = h / (p.Hq / p.Hkv);
     const int q0 = qt * BM;
     const int nt = min((q0 + BM) / BN, (p.N + BN - 1) / BN);  // key tiles 0..nt-1 reach the last query row / the last key
@@ -585,7 +590,11 @@ cudaError_t launch_tc_flash(const TcFlashArgs& a, cudaStream_t stream) {
     p.scale = a.scale;
 
     if (a.qt_count < 1 || a.qt_count > 65535) return cudaErrorInvalidValue;
+    // K and V of all (batch, KV head) pairs against half of a 126 MB L2 (the other half for everything else that streams)
+    const int64_t kv_bytes = (int64_t)a.B * a.Hkv * a.N * (a.kd + (a.emit_plane ? 0 : D)) * 2;
+    p.head_major = kv_bytes > ((int64_t)63 << 20) && (int64_t)a.Hq * a.B <= 65535 && a.qt_count > 1;
     dim3 grid(a.Hq * a.B, a.qt_count);
+    if (p.head_major) grid = dim3(a.qt_count, a.Hq * a.B);
     cudaError_t e;
 #define LISA_LAUNCH_FLASH(KD_, PL_)                                                                                       \
     do {                                                                                                                   \
