@@ -236,6 +236,76 @@ SideStream* side_stream() {
     }
     return &ss;
 }
+
+// The host-memory entry points hand q0, k0, v (host, each may be null) and o (host) to the orchestration (TcHostIO).
+// Where the side streams exist and the device copies are dense, the tensors are streamed: before a wave starts, its rows of
+// q0, k0 and v are copied in on the copy-in stream (the waves run from row 0 up, and a wave needs keys and values up to
+// its last row: exactly what has been copied by then) and the wave's stream waits for them; after the wave's attention
+// kernel its rows of o go out on the copy-out stream.  Otherwise the inputs are copied whole on the caller's stream
+// before anything reads them, and the caller copies o afterwards (out_done stays false).
+struct HostIo {
+    const lisa_shared_prefill_args& a;
+    TcHostIO* ho;
+    SideStream* side;
+    cudaStream_t s;
+    bool stream_out = false, stream_in = false;
+
+    HostIo(const lisa_shared_prefill_args& args, TcHostIO* io, SideStream* ss, cudaStream_t caller, bool one_layer)
+        : a(args), ho(io), side(ss), s(caller) {
+        auto dense = [&](const lisa_tensor& t, int H) {
+            return t.stride_h == a.d && t.stride_n == (int64_t)H * a.d && t.stride_b == (int64_t)a.N * H * a.d;
+        };
+        stream_out = ho && ho->host_o && side && one_layer && dense(a.o, a.Hq);
+        stream_in = has_in() && stream_out && dense(a.q0, a.Hq) && dense(a.k0, a.Hkv) && dense(a.v, a.Hkv);
+    }
+    bool has_in() const { return ho && (ho->host_q0 || ho->host_k0 || ho->host_v); }
+    // rows [r0, r1) of a dense [B,N,H,d] bf16 tensor, one copy per sequence
+    cudaError_t copy_rows(void* dst, const void* src, int H, int64_t r0, int64_t r1, cudaMemcpyKind kind, cudaStream_t cs) const {
+        for (int b = 0; b < a.B; ++b) {
+            const int64_t off = ((int64_t)b * a.N + r0) * H * a.d * 2;
+            cudaError_t e = cudaMemcpyAsync(static_cast<char*>(dst) + off, static_cast<const char*>(src) + off,
+                                            (size_t)(r1 - r0) * H * a.d * 2, kind, cs);
+            if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
+    }
+    cudaError_t inputs(int64_t r0, int64_t r1, cudaStream_t cs) const {
+        cudaError_t e;
+        if (ho->host_q0 && (e = copy_rows(a.q0.ptr, ho->host_q0, a.Hq, r0, r1, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return e;
+        if (ho->host_k0 && (e = copy_rows(a.k0.ptr, ho->host_k0, a.Hkv, r0, r1, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return e;
+        if (ho->host_v && (e = copy_rows(a.v.ptr, ho->host_v, a.Hkv, r0, r1, cudaMemcpyHostToDevice, cs)) != cudaSuccess) return e;
+        return cudaSuccess;
+    }
+    // before the first kernel: whole inputs where they are not streamed; the copy-in stream ordered behind everything
+    // enqueued before the call (earlier users of the arena) where they are
+    cudaError_t begin() const {
+        if (has_in() && !stream_in) return inputs(0, a.N, s);
+        if (!stream_in) return cudaSuccess;
+        std::lock_guard<std::mutex> lock(g_side_mutex);
+        cudaError_t e = cudaEventRecord(side->fork, s);
+        return e != cudaSuccess ? e : cudaStreamWaitEvent(side->copy_in, side->fork, 0);
+    }
+    static void rows_of(const Wave& wv, int N, int64_t* r0, int64_t* r1) {
+        *r0 = (int64_t)wv.begin * kTile;
+        *r1 = std::min<int64_t>(N, (int64_t)(wv.begin + wv.count) * kTile);
+    }
+    cudaError_t rows_in(const Wave& wv, cudaStream_t st) const {
+        int64_t r0, r1;
+        rows_of(wv, a.N, &r0, &r1);
+        cudaError_t e = inputs(r0, r1, side->copy_in);
+        if (e != cudaSuccess) return e;
+        if ((e = cudaEventRecord(side->rows_in, side->copy_in)) != cudaSuccess) return e;
+        return cudaStreamWaitEvent(st, side->rows_in, 0);   // everything copied so far: the wave's rows and all rows before them
+    }
+    cudaError_t rows_out(const Wave& wv, cudaStream_t st) const {
+        int64_t r0, r1;
+        rows_of(wv, a.N, &r0, &r1);
+        cudaError_t e = cudaEventRecord(side->rows_done, st);
+        if (e != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(side->copy_out, side->rows_done, 0)) != cudaSuccess) return e;
+        return copy_rows(ho->host_o, a.o.ptr, a.Hq, r0, r1, cudaMemcpyDeviceToHost, side->copy_out);
+    }
+};
 }  // namespace
 
 cudaError_t launch_tc_shared_prefill(const lisa_shared_prefill_args& a, void* ws, cudaStream_t s) {
@@ -302,53 +372,12 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
     // All of it is forked from and joined back into the caller's stream inside this call, under the lock that keeps
     // another host thread's call from interleaving its event records with these waits.
     const int sets = (side && nw >= 2) ? l.sets : 1;
-    // rows of o leave for the host as soon as their wave's attention kernel is done (dense bf16 o only)
-    const bool stream_out = ho && ho->host_o && side && !all_layers && a.o.stride_h == a.d && a.o.stride_n == (int64_t)a.Hq * a.d;
-    // rows [r0, r1) of a dense [B,N,H,d] bf16 tensor, one copy per sequence
-    auto copy_rows = [&](void* dst, const void* src, int H, int64_t r0, int64_t r1, cudaMemcpyKind kind, cudaStream_t cs) -> cudaError_t {
-        for (int b = 0; b < a.B; ++b) {
-            const int64_t off = ((int64_t)b * a.N + r0) * H * a.d * 2;
-            cudaError_t ce = cudaMemcpyAsync(static_cast<char*>(dst) + off, static_cast<const char*>(src) + off,
-                                             (size_t)(r1 - r0) * H * a.d * 2, kind, cs);
-            if (ce != cudaSuccess) return ce;
-        }
-        return cudaSuccess;
-    };
-    auto dense = [&](const lisa_tensor& t, int H) { return t.stride_h == a.d && t.stride_n == (int64_t)H * a.d && t.stride_b == (int64_t)a.N * H * a.d; };
-    const bool has_in = ho && (ho->host_q0 || ho->host_k0 || ho->host_v);
-    const bool stream_in = has_in && stream_out && dense(a.q0, a.Hq) && dense(a.k0, a.Hkv) && dense(a.v, a.Hkv) && dense(a.o, a.Hq);
-    if (has_in && !stream_in) {   // whole tensors, before anything reads them
-        if (ho->host_q0 && (e = copy_rows(a.q0.ptr, ho->host_q0, a.Hq, 0, a.N, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
-        if (ho->host_k0 && (e = copy_rows(a.k0.ptr, ho->host_k0, a.Hkv, 0, a.N, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
-        if (ho->host_v && (e = copy_rows(a.v.ptr, ho->host_v, a.Hkv, 0, a.N, cudaMemcpyHostToDevice, s)) != cudaSuccess) return e;
-    }
-    auto copy_in = [&](const Wave& wv, cudaStream_t st) -> cudaError_t {
-        cudaError_t ce;
-        const int64_t r0 = (int64_t)wv.begin * kTile, r1 = std::min<int64_t>(a.N, (int64_t)(wv.begin + wv.count) * kTile);
-        if (ho->host_q0 && (ce = copy_rows(a.q0.ptr, ho->host_q0, a.Hq, r0, r1, cudaMemcpyHostToDevice, side->copy_in)) != cudaSuccess) return ce;
-        if (ho->host_k0 && (ce = copy_rows(a.k0.ptr, ho->host_k0, a.Hkv, r0, r1, cudaMemcpyHostToDevice, side->copy_in)) != cudaSuccess) return ce;
-        if (ho->host_v && (ce = copy_rows(a.v.ptr, ho->host_v, a.Hkv, r0, r1, cudaMemcpyHostToDevice, side->copy_in)) != cudaSuccess) return ce;
-        if ((ce = cudaEventRecord(side->rows_in, side->copy_in)) != cudaSuccess) return ce;
-        return cudaStreamWaitEvent(st, side->rows_in, 0);   // everything copied so far: the wave's rows and all rows before them
-    };
-    auto copy_out = [&](const Wave& wv, cudaStream_t st) -> cudaError_t {
-        cudaError_t ce;
-        if ((ce = cudaEventRecord(side->rows_done, st)) != cudaSuccess) return ce;
-        if ((ce = cudaStreamWaitEvent(side->copy_out, side->rows_done, 0)) != cudaSuccess) return ce;
-        const int64_t r0 = (int64_t)wv.begin * kTile, r1 = std::min<int64_t>(a.N, (int64_t)(wv.begin + wv.count) * kTile);
-        for (int b = 0; b < a.B; ++b) {
-            const int64_t src = (b * a.o.stride_b + r0 * a.o.stride_n) * 2, dst = ((int64_t)b * a.N + r0) * a.Hq * a.d * 2;
-            if ((ce = cudaMemcpyAsync(static_cast<char*>(ho->host_o) + dst, static_cast<const char*>(a.o.ptr) + src,
-                                      (size_t)(r1 - r0) * a.Hq * a.d * 2, cudaMemcpyDeviceToHost, side->copy_out)) != cudaSuccess)
-                return ce;
-        }
-        return cudaSuccess;
-    };
-    if (stream_in) {   // the copies start once everything enqueued before the call (earlier users of the arena) is done
-        std::lock_guard<std::mutex> lock(g_side_mutex);
-        if ((e = cudaEventRecord(side->fork, s)) != cudaSuccess) return e;
-        if ((e = cudaStreamWaitEvent(side->copy_in, side->fork, 0)) != cudaSuccess) return e;
-    }
+    // host-memory calls: inputs in and output out wave by wave beside the compute (see HostIo), where the path allows it
+    HostIo io{a, ho, side, s, !all_layers};
+    const bool stream_out = io.stream_out, stream_in = io.stream_in;
+    if ((e = io.begin()) != cudaSuccess) return e;
+    auto copy_in = [&](const Wave& wv, cudaStream_t st) { return io.rows_in(wv, st); };
+    auto copy_out = [&](const Wave& wv, cudaStream_t st) { return io.rows_out(wv, st); };
     std::unique_lock<std::mutex> wave_lock(g_side_mutex, std::defer_lock);
     if (sets > 1 || stream_out) {
         wave_lock.lock();
