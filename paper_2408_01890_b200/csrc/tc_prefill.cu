@@ -367,11 +367,21 @@ cudaError_t launch_tc_shared_prefill_chain(const lisa_shared_prefill_args& a, co
     };
     const bool concat = concat_chain(a);
     Wave waves[1024];
-    const int nw = plan_waves(a.B, a.N, a.Hq, cy ? 1 : plane_count(a), waves, 1024, cy != nullptr && !concat);
+    int nw = plan_waves(a.B, a.N, a.Hq, cy ? 1 : plane_count(a), waves, 1024, cy != nullptr && !concat);
+    // A host-memory call whose prompt fits fewer than four waves is cut into four strips of query tiles all the same (they
+    // run one after the other in the planes laid out for the larger waves): its time is the copies', and strips let the
+    // copies in, the compute and the copies out overlap.
+    if (ho && side && !all_layers && nw < 4) {
+        const int n_qt = (a.N + kTile - 1) / kTile, per = (n_qt + 3) / 4;
+        if (n_qt >= 4) {
+            nw = 0;
+            for (int qt = 0; qt < n_qt; qt += per) waves[nw++] = Wave{qt, std::min(per, n_qt - qt)};
+        }
+    }
     // Several waves in flight (see kWaveSets): wave w runs on stream w % sets (0 = the caller's) with plane set w % sets.
     // All of it is forked from and joined back into the caller's stream inside this call, under the lock that keeps
     // another host thread's call from interleaving its event records with these waits.
-    const int sets = (side && nw >= 2) ? l.sets : 1;
+    const int sets = (side && nw >= 2) ? std::min(l.sets, nw) : 1;
     // host-memory calls: inputs in and output out wave by wave beside the compute (see HostIo), where the path allows it
     HostIo io{a, ho, side, s, !all_layers};
     const bool stream_out = io.stream_out, stream_in = io.stream_in;
