@@ -385,3 +385,20 @@ def test_carried_scores_at_tile_boundaries(N):
     rec = lb.lisa_attn_shared_prefill(q0, k0, dl, dev(t["v2"]))
     torch.cuda.synchronize()
     assert_close(got.float().cpu().numpy(), rec.float().cpu().numpy().astype(np.float64), "bf16", "carried against recomputed, N=%d" % N)
+
+
+def test_carried_scores_single_layer_keeps_nothing():
+    """A chain of one layer through the carried call (first and last at once) equals the recomputing call bit for bit: the
+    same kernels run on the same data, only the plane lives in the caller's buffer."""
+    B, N, Hq, Hkv = 2, 300, 32, 8
+    t = link_inputs(B, N, Hq, Hkv, 1, 64, "silu", 2, 21, 53, False)
+    dl, ol = make_links(t, 1, "silu")
+    q0, k0, v = dev(t["q0"]), dev(t["k0"]), dev(t["v1"])
+    scores = torch.empty(lb.lisa_prefill_scores_bytes(B, N, Hq), dtype=torch.uint8, device="cuda")
+    got = lb.lisa_attn_shared_prefill_carry(q0, k0, dl[0], v, scores, first=True, keep=False)
+    rec = lb.lisa_attn_shared_prefill(q0, k0, dl, v)
+    torch.cuda.synchronize()
+    assert lb.lisa_check() == lb.OK
+    assert torch.equal(got, rec)
+    ref = oracle.prefill_full(f64(t["q0"]), f64(t["k0"]), f64(t["v1"]), ol)
+    assert_close(got.float().cpu().numpy(), ref, "bf16", "carried call, single layer")
