@@ -36,14 +36,14 @@ METRIC = "lisa_attention_tokens_per_s"
 # summarised under profiles/ (cold cache); every kernel streams its planes once, so traffic grows in proportion to
 # the causal positions and the figures are scaled by them for other workloads.  None for a kernel that has changed since.
 CFG2_POSITIONS_HEADS = 2098176 * 32
-PREFILL_TRAFFIC_PER_PH = {"emit_scores": (39975424 + 88312832) / CFG2_POSITIONS_HEADS,
-                          "align": (142643968 + 85279744) / CFG2_POSITIONS_HEADS,
-                          "attention": (186744832 + 6408960) / CFG2_POSITIONS_HEADS}
+PREFILL_TRAFFIC_PER_PH = {"emit_scores": (39989248 + 85851392) / CFG2_POSITIONS_HEADS,
+                          "align": (142656000 + 83307520) / CFG2_POSITIONS_HEADS,
+                          "attention": (186732800 + 5543680) / CFG2_POSITIONS_HEADS}
 # The kernels of a carried layer, captured on the first wave (query rows 0..3199) of the headline chain at B 1, N 4096:
 # the one-link aligner in place on the scores buffer and the attention kernel that writes its logits back.
 CARRY_POSITIONS_HEADS = 3200 * 3201 // 2 * 32
-CARRY_TRAFFIC_PER_PH = {"align": (340836864 + 284195584) / CARRY_POSITIONS_HEADS,
-                        "attention_keep": (371413248 + 312834560) / CARRY_POSITIONS_HEADS}
+CARRY_TRAFFIC_PER_PH = {"align": (340822272 + 281756928) / CARRY_POSITIONS_HEADS,
+                        "attention_keep": (371120640 + 313165824) / CARRY_POSITIONS_HEADS}
 DECODE_TRAFFIC_PER_SEQ = (593884160 + 4890112) / 12  # shared decode chunk kernel, captured at 12 sequences; scales with the batch
 PROJECT_TRAFFIC = 220900096 + 163201024             # projection kernel at the benchmark's own size
 
