@@ -178,3 +178,39 @@ def test_host_arena_ignores_host_strides(lib):
     dense, zero = arena(True), arena(False)
     tensors = 4 * 256 * 32 * 128 * 2
     assert dense == zero and dense > tensors + (1 << 20)     # inputs + output + a score-plane workspace
+
+
+def test_carried_scores_sizes_and_host_arena(lib):
+    """The scores buffer of lisa_attn_shared_prefill_carry holds B x Hq x ceil128(N)^2 fp16 values (Sec. 5.2 counts the
+    h x l x l x 2 bytes of a stored score matrix: the same figure with the prompt rounded up to whole tiles); the host-memory
+    form asks for an arena without the anchor's q0, k0 past the first layer and ignores host strides like its sibling."""
+    lib.lisa_prefill_scores_bytes.restype = C.c_size_t
+    lib.lisa_prefill_scores_bytes.argtypes = [C.c_int32, C.c_int32, C.c_int32]
+    assert lib.lisa_prefill_scores_bytes(4, 8192, 32) == 4 * 32 * 8192 * 8192 * 2
+    assert lib.lisa_prefill_scores_bytes(1, 1, 32) == 32 * 128 * 128 * 2
+    assert lib.lisa_prefill_scores_bytes(2, 129, 40) == 2 * 40 * 256 * 256 * 2
+    assert lib.lisa_prefill_scores_bytes(0, 128, 32) == 0 and lib.lisa_prefill_scores_bytes(1, 0, 32) == 0
+
+    def arena(first, strided):
+        t = lambda H, x: lb.Tensor(1 << 20, lb.BF16, 0, (256 * H * x) if strided else 0, (H * x) if strided else 0, x if strided else 0)
+        link = lb.CLink(t(32, 21), t(8, 21), 1 << 20, None, 1 << 20, None, lb.BF16, 21, 64, lb.ACT_RELU, lb.INTEGRATE_ADD, 2)
+        c = lb.SharedPrefillCarryArgs()
+        c.struct_size = C.sizeof(lb.SharedPrefillCarryArgs)
+        a = c.layer
+        a.struct_size = C.sizeof(lb.SharedPrefillArgs)
+        a.B, a.N, a.Hq, a.Hkv, a.d, a.chain_len = 1, 256, 32, 8, 128, 1
+        if first:
+            a.q0, a.k0 = t(32, 128), t(8, 128)
+        a.v, a.o = t(8, 128), t(32, 128)
+        a.links = C.pointer(link)
+        c.scores, c.scores_bytes, c.first, c.keep = 1 << 21, 32 * 256 * 256 * 2, int(first), 1
+        n = C.c_size_t()
+        assert lib.lisa_carry_host_arena_bytes(C.byref(c), C.byref(n)) == lb.OK
+        return n.value
+    q0k0 = 256 * (32 + 8) * 128 * 2
+    assert arena(True, True) == arena(True, False)
+    assert arena(False, True) == arena(False, False) == arena(True, True) - q0k0
+    c = lb.SharedPrefillCarryArgs()
+    c.struct_size = C.sizeof(lb.SharedPrefillCarryArgs) - 8
+    n = C.c_size_t()
+    assert lib.lisa_carry_host_arena_bytes(C.byref(c), C.byref(n)) == lb.ERR_INVALID_ARG
